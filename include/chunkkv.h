@@ -1,0 +1,157 @@
+/*
+ * chunkkv.h - C ABI of the ChunkKV prefill-time KV-cache compression library (CUDA, sm_100a).
+ *
+ * The operation (ChunkKV paper, Algorithm 3 "ChunkKV Implementation", with Algorithm 1 for the
+ * notation and Algorithm 2 for layer-wise index reuse), for one layer and each KV head h:
+ *
+ *   P = L - w                      prefix length; the last w rows are the observation window
+ *   R = w * (Hq / Hkv)             window queries of the Hq/Hkv query heads sharing KV head h
+ *   p[i, j]                        softmax over the keys row i can see of q_i . k_j / sqrt(d);
+ *                                  row (g, r) sits at position P + r and sees key j iff j <= P + r
+ *   t[j]   = sum_i p[i, j]         token score, j in [0, P)
+ *   C      = ceil(P / c)           chunks over the prefix (origin 0, stride c, last one clipped)
+ *   s[ch]  = sum_{j in chunk} t[j] chunk score
+ *   k      = min(floor((budget - w) / c), C)
+ *   keep the k chunks with the largest s (ties: lower chunk id), whole chunks, plus the window
+ *   idx    = kept token positions in ascending order (window last), padded with -1 to
+ *            n_max = k * c + w
+ *   out_K[n] = K[idx[n]], out_V[n] = V[idx[n]]  (bit copies; zero rows where idx is -1)
+ *
+ * Conventions shared by every entry point
+ *   - All tensor pointers are DEVICE pointers (unless a name says host), 16-byte aligned,
+ *     dense row-major, owned by the caller, and must stay valid until the work queued on
+ *     `stream` has finished. bf16 tensors are passed as `const void*`.
+ *       q_obs [Hq, w, d] bf16   queries of the last w positions (after positional encoding);
+ *                               query head g belongs to KV head g / (Hq / Hkv)
+ *       K, V  [Hkv, L, d] bf16  keys / values of the layer, window rows included
+ *       token scores [Hkv, P] f32, chunk scores [Hkv, C] f32
+ *       idx   [Hkv, n_max] int32, out_K / out_V [Hkv, n_max, d] bf16
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream). Calls only
+ *     enqueue work; they never synchronise the device (except where stated).
+ *   - Limits: d in {64, 128}; Hq a multiple of Hkv; R = w * Hq / Hkv <= 256; 1 <= w <= L;
+ *     c >= 1; budget >= w; Hkv * L * d < 2^40.
+ *   - Return value: CHUNKKV_OK (0) or a negative CHUNKKV_E* code. Arguments are checked on
+ *     the host before anything is launched; nothing is thrown and nothing aborts.
+ *   - Scratch memory: scoring needs device scratch (chunkkv_workspace_bytes). Either hand the
+ *     library a buffer with chunkkv_set_workspace, or let it allocate one on first use (one
+ *     cudaMalloc per device, grown when a larger problem arrives; growing synchronises the
+ *     device). Calls that use the scratch of one device must be ordered on the GPU (same
+ *     stream, or otherwise serialised): concurrent calls would share it.
+ */
+#ifndef CHUNKKV_H_
+#define CHUNKKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CHUNKKV_OK              0
+#define CHUNKKV_EINVAL_NULL    -1  /* a required pointer is NULL */
+#define CHUNKKV_EINVAL_SHAPE   -2  /* a size violates the limits above */
+#define CHUNKKV_EINVAL_ALIGN   -3  /* a tensor pointer is not 16-byte aligned */
+#define CHUNKKV_ENOWORKSPACE   -4  /* caller-provided workspace too small / allocation failed */
+#define CHUNKKV_ECUDA          -5  /* a CUDA runtime or driver call failed (see chunkkv_last_cuda_error) */
+#define CHUNKKV_EDEVICE        -6  /* a kernel gave up on a bounded wait (see chunkkv_device_status) */
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* chunkkv_strerror(int status);
+
+/* The cudaError_t (as int) recorded by the most recent CHUNKKV_ECUDA on this thread. */
+int chunkkv_last_cuda_error(void);
+
+/* C = ceil((L - w) / c); 0 when L == w. Negative status on invalid sizes. (Algorithm 3, chunk count.) */
+int chunkkv_num_chunks(int L, int w, int c);
+
+/* k = min(floor((budget - w) / c), C). (Algorithm 3, "Limit k to available chunks".) */
+int chunkkv_num_kept_chunks(int L, int w, int c, int budget);
+
+/* n_max = k * c + w: row count of idx / out_K / out_V per head. */
+int chunkkv_out_len(int L, int w, int c, int budget);
+
+/* Bytes of device scratch that scoring a layer of this shape needs (0 on invalid sizes). */
+size_t chunkkv_workspace_bytes(int L, int Hq, int Hkv, int d, int w, int c);
+
+/*
+ * Use caller-owned device memory (256-byte aligned, on the current device) as scratch for all
+ * later calls on this device. Its first 256 bytes hold the library's device status word and are
+ * cleared by this call (which synchronises the device). Passing (NULL, 0) returns to
+ * library-managed scratch. The caller keeps ownership.
+ */
+int chunkkv_set_workspace(void* dev_ptr, size_t bytes);
+
+/*
+ * Synchronise `stream`, then report whether any kernel of this library on the current device
+ * abandoned a bounded wait since the last call (CHUNKKV_EDEVICE) - a defect report, not an
+ * expected outcome. Clears the status word.
+ */
+int chunkkv_device_status(void* stream);
+
+/*
+ * Steps "observe-window attention scores" and "chunk score calculation" (Algorithm 3; Algorithm 1
+ * "Observe Window Calculation" / "Chunk Attention Score Calculation").
+ *   out_chunk_scores [Hkv, C] f32   required
+ *   out_token_scores [Hkv, P] f32   optional (NULL to skip); computed by a second pass of the
+ *                                   same kernels with chunk size 1, so it costs scratch for
+ *                                   chunk size 1 as well
+ * With P == 0 nothing is written.
+ */
+int chunkkv_score(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w, int c,
+                  float* out_token_scores, float* out_chunk_scores, void* stream);
+
+/*
+ * Step "top-k chunk selection" and the kept-index list (Algorithm 3: Top-K, selection mask,
+ * window forced on, nonzero). chunk_scores [Hkv, C] f32 -> out_idx [Hkv, n_max] int32:
+ * ascending token positions of the k best chunks (ties to the lower chunk id), then P..L-1,
+ * then -1 padding (only when the clipped last chunk is among the kept ones).
+ */
+int chunkkv_select(const float* chunk_scores, int L, int Hkv, int w, int c, int budget,
+                   int32_t* out_idx, void* stream);
+
+/*
+ * Step "compression" (Algorithm 3 / Algorithm 2: index_select on K and on V).
+ * idx [Hkv, n_max] int32 -> out_K, out_V [Hkv, n_max, d]; entries outside [0, L) give zero rows.
+ * out_K/out_V must not overlap K/V.
+ */
+int chunkkv_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
+                   int n_max, void* out_K, void* out_V, void* stream);
+
+/*
+ * The whole layer (Algorithm 3), or - with reuse_idx non-NULL - a layer that reuses another
+ * layer's indices (Algorithm 2, else-branch): scoring and selection are skipped, reuse_idx
+ * [Hkv, n_max] is copied to out_idx (they may be the same buffer) and only the gather runs.
+ */
+int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                           int d, int w, int c, int budget, const int32_t* reuse_idx_or_null,
+                           void* out_K, void* out_V, int32_t* out_idx, void* stream);
+
+/*
+ * End-to-end convenience for callers whose tensors live in (ideally pinned) HOST memory:
+ * copies q_obs, K, V to the given device staging buffers, runs chunkkv_compress_layer and
+ * copies out_K, out_V, out_idx back to the host buffers, all queued on `stream`.
+ * host_* are host pointers; dev_* are device buffers of the same sizes.
+ */
+int chunkkv_compress_layer_host(const void* host_q_obs, const void* host_K, const void* host_V,
+                                int L, int Hq, int Hkv, int d, int w, int c, int budget,
+                                void* dev_q_obs, void* dev_K, void* dev_V,
+                                void* dev_out_K, void* dev_out_V, int32_t* dev_out_idx,
+                                void* host_out_K, void* host_out_V, int32_t* host_out_idx,
+                                void* stream);
+
+/*
+ * Optional per-kernel timing for benchmarks. While enabled, the entry points bracket each
+ * kernel with CUDA events on the launching stream. chunkkv_profile_read synchronises the
+ * device and returns, per kernel slot, accumulated milliseconds and launch counts since the
+ * last read (arrays of CHUNKKV_PROFILE_SLOTS entries), then resets them.
+ * Slots: 0 score, 1 chunk-score finalisation, 2 select, 3 gather.
+ */
+#define CHUNKKV_PROFILE_SLOTS 4
+int chunkkv_profile_enable(int on);
+int chunkkv_profile_read(float* ms_per_slot, int* launches_per_slot);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CHUNKKV_H_ */

@@ -1,0 +1,49 @@
+// Declarations shared by the translation units of libchunkkv (host side).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace chunkkv {
+
+// Geometry of one scoring launch, fixed on the host.
+struct ScorePlan {
+    int c_static;   // chunk size baked into the kernel (0 = run-time chunk size)
+    int n_mt;       // 128-row query tiles per KV head (1 or 2)
+    int n_tile;     // keys per accumulator tile
+    int n_tiles;    // accumulator tiles per head = ceil(L / n_tile)
+    int spt;        // chunk slots per tile in the partial-sum scratch
+    int n_stages;   // shared-memory stages in the K ring (one stage = n_tile keys x 64 dims)
+    int smem_bytes; // dynamic shared memory of the launch
+};
+
+struct ScoreArgs {
+    int L, P, w, c, R, Hkv, d;
+    float sl2;            // log2(e) / sqrt(d)
+    float* stat_m;        // [Hkv, n_tiles, R] tile row maxima (log2 domain)
+    float* stat_l;        // [Hkv, n_tiles, R] tile row sums relative to the tile maximum
+    float* partial;       // [Hkv, n_tiles, spt, R] chunk partial sums relative to the tile maximum
+    int* status;          // device status word
+};
+
+// Chooses kernel variant and tile geometry for a shape. Returns false if unsupported.
+bool make_score_plan(int L, int R, int d, int c, int smem_limit, ScorePlan* plan);
+
+// Scratch floats needed for a plan (tile statistics + partial sums), per layer.
+size_t score_scratch_floats(const ScorePlan& plan, int Hkv, int R);
+
+cudaError_t launch_score(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                         const ScoreArgs& args, int num_sms, cudaStream_t stream);
+
+cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
+                            int num_sms, cudaStream_t stream);
+
+cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int C, int k, int n_max,
+                          int32_t* out_idx, cudaStream_t stream);
+
+cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
+                          int n_max, void* out_K, void* out_V, int32_t* idx_copy_or_null,
+                          int num_sms, cudaStream_t stream);
+
+}  // namespace chunkkv
