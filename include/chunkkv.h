@@ -44,6 +44,12 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#if defined(__GNUC__)
+#define CHUNKKV_API __attribute__((visibility("default")))
+#else
+#define CHUNKKV_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -57,22 +63,22 @@ extern "C" {
 #define CHUNKKV_EDEVICE        -6  /* a kernel gave up on a bounded wait (see chunkkv_device_status) */
 
 /* Human-readable name of a status code (static string, never NULL). */
-const char* chunkkv_strerror(int status);
+CHUNKKV_API const char* chunkkv_strerror(int status);
 
 /* The cudaError_t (as int) recorded by the most recent CHUNKKV_ECUDA on this thread. */
-int chunkkv_last_cuda_error(void);
+CHUNKKV_API int chunkkv_last_cuda_error(void);
 
 /* C = ceil((L - w) / c); 0 when L == w. Negative status on invalid sizes. (Algorithm 3, chunk count.) */
-int chunkkv_num_chunks(int L, int w, int c);
+CHUNKKV_API int chunkkv_num_chunks(int L, int w, int c);
 
 /* k = min(floor((budget - w) / c), C). (Algorithm 3, "Limit k to available chunks".) */
-int chunkkv_num_kept_chunks(int L, int w, int c, int budget);
+CHUNKKV_API int chunkkv_num_kept_chunks(int L, int w, int c, int budget);
 
 /* n_max = k * c + w: row count of idx / out_K / out_V per head. */
-int chunkkv_out_len(int L, int w, int c, int budget);
+CHUNKKV_API int chunkkv_out_len(int L, int w, int c, int budget);
 
 /* Bytes of device scratch that scoring a layer of this shape needs (0 on invalid sizes). */
-size_t chunkkv_workspace_bytes(int L, int Hq, int Hkv, int d, int w, int c);
+CHUNKKV_API size_t chunkkv_workspace_bytes(int L, int Hq, int Hkv, int d, int w, int c);
 
 /*
  * Use caller-owned device memory (256-byte aligned, on the current device) as scratch for all
@@ -80,14 +86,14 @@ size_t chunkkv_workspace_bytes(int L, int Hq, int Hkv, int d, int w, int c);
  * cleared by this call (which synchronises the device). Passing (NULL, 0) returns to
  * library-managed scratch. The caller keeps ownership.
  */
-int chunkkv_set_workspace(void* dev_ptr, size_t bytes);
+CHUNKKV_API int chunkkv_set_workspace(void* dev_ptr, size_t bytes);
 
 /*
  * Synchronise `stream`, then report whether any kernel of this library on the current device
  * abandoned a bounded wait since the last call (CHUNKKV_EDEVICE) - a defect report, not an
  * expected outcome. Clears the status word.
  */
-int chunkkv_device_status(void* stream);
+CHUNKKV_API int chunkkv_device_status(void* stream);
 
 /*
  * Steps "observe-window attention scores" and "chunk score calculation" (Algorithm 3; Algorithm 1
@@ -98,7 +104,7 @@ int chunkkv_device_status(void* stream);
  *                                   chunk size 1 as well
  * With P == 0 nothing is written.
  */
-int chunkkv_score(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w, int c,
+CHUNKKV_API int chunkkv_score(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w, int c,
                   float* out_token_scores, float* out_chunk_scores, void* stream);
 
 /*
@@ -107,7 +113,7 @@ int chunkkv_score(const void* q_obs, const void* K, int L, int Hq, int Hkv, int 
  * ascending token positions of the k best chunks (ties to the lower chunk id), then P..L-1,
  * then -1 padding (only when the clipped last chunk is among the kept ones).
  */
-int chunkkv_select(const float* chunk_scores, int L, int Hkv, int w, int c, int budget,
+CHUNKKV_API int chunkkv_select(const float* chunk_scores, int L, int Hkv, int w, int c, int budget,
                    int32_t* out_idx, void* stream);
 
 /*
@@ -115,7 +121,7 @@ int chunkkv_select(const float* chunk_scores, int L, int Hkv, int w, int c, int 
  * idx [Hkv, n_max] int32 -> out_K, out_V [Hkv, n_max, d]; entries outside [0, L) give zero rows.
  * out_K/out_V must not overlap K/V.
  */
-int chunkkv_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
+CHUNKKV_API int chunkkv_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
                    int n_max, void* out_K, void* out_V, void* stream);
 
 /*
@@ -123,7 +129,7 @@ int chunkkv_gather(const void* K, const void* V, const int32_t* idx, int L, int 
  * layer's indices (Algorithm 2, else-branch): scoring and selection are skipped, reuse_idx
  * [Hkv, n_max] is copied to out_idx (they may be the same buffer) and only the gather runs.
  */
-int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
                            int d, int w, int c, int budget, const int32_t* reuse_idx_or_null,
                            void* out_K, void* out_V, int32_t* out_idx, void* stream);
 
@@ -133,7 +139,7 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
  * copies out_K, out_V, out_idx back to the host buffers, all queued on `stream`.
  * host_* are host pointers; dev_* are device buffers of the same sizes.
  */
-int chunkkv_compress_layer_host(const void* host_q_obs, const void* host_K, const void* host_V,
+CHUNKKV_API int chunkkv_compress_layer_host(const void* host_q_obs, const void* host_K, const void* host_V,
                                 int L, int Hq, int Hkv, int d, int w, int c, int budget,
                                 void* dev_q_obs, void* dev_K, void* dev_V,
                                 void* dev_out_K, void* dev_out_V, int32_t* dev_out_idx,
@@ -148,8 +154,8 @@ int chunkkv_compress_layer_host(const void* host_q_obs, const void* host_K, cons
  * Slots: 0 score, 1 chunk-score finalisation, 2 select, 3 gather.
  */
 #define CHUNKKV_PROFILE_SLOTS 4
-int chunkkv_profile_enable(int on);
-int chunkkv_profile_read(float* ms_per_slot, int* launches_per_slot);
+CHUNKKV_API int chunkkv_profile_enable(int on);
+CHUNKKV_API int chunkkv_profile_read(float* ms_per_slot, int* launches_per_slot);
 
 #ifdef __cplusplus
 }

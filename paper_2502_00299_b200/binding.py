@@ -1,0 +1,230 @@
+"""ctypes binding of the C ABI declared in include/chunkkv.h (argument marshalling only)."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libchunkkv.so")
+
+
+class ChunkKVError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib.chunkkv_strerror(status).decode()
+        extra = f" (cuda error {lib.chunkkv_last_cuda_error()})" if status == -5 else ""
+        super().__init__(f"{where}: {msg}{extra} [status {status}]")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2502_00299_b200.build` "
+            "(needs nvcc). This package has no fallback path.")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    L.chunkkv_strerror.restype = ctypes.c_char_p
+    L.chunkkv_strerror.argtypes = [i32]
+    L.chunkkv_last_cuda_error.restype = i32
+    L.chunkkv_last_cuda_error.argtypes = []
+    for name, n in (("chunkkv_num_chunks", 3), ("chunkkv_num_kept_chunks", 4), ("chunkkv_out_len", 4)):
+        getattr(L, name).restype = i32
+        getattr(L, name).argtypes = [i32] * n
+    L.chunkkv_workspace_bytes.restype = sz
+    L.chunkkv_workspace_bytes.argtypes = [i32] * 6
+    L.chunkkv_set_workspace.restype = i32
+    L.chunkkv_set_workspace.argtypes = [vp, sz]
+    L.chunkkv_device_status.restype = i32
+    L.chunkkv_device_status.argtypes = [vp]
+    L.chunkkv_score.restype = i32
+    L.chunkkv_score.argtypes = [vp, vp] + [i32] * 6 + [vp, vp, vp]
+    L.chunkkv_select.restype = i32
+    L.chunkkv_select.argtypes = [vp] + [i32] * 5 + [vp, vp]
+    L.chunkkv_gather.restype = i32
+    L.chunkkv_gather.argtypes = [vp, vp, vp] + [i32] * 4 + [vp, vp, vp]
+    L.chunkkv_compress_layer.restype = i32
+    L.chunkkv_compress_layer.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, vp, vp, vp]
+    L.chunkkv_compress_layer_host.restype = i32
+    L.chunkkv_compress_layer_host.argtypes = [vp, vp, vp] + [i32] * 7 + [vp] * 10
+    L.chunkkv_profile_enable.restype = i32
+    L.chunkkv_profile_enable.argtypes = [i32]
+    L.chunkkv_profile_read.restype = i32
+    L.chunkkv_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int)]
+    return L
+
+
+lib = _load()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise ChunkKVError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream: Optional[torch.cuda.Stream]) -> Optional[int]:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+def _dev(t: torch.Tensor, dtype: torch.dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor of dtype {dtype}")
+    return t
+
+
+def strerror(status: int) -> str:
+    return lib.chunkkv_strerror(status).decode()
+
+
+def num_chunks(L: int, w: int, c: int) -> int:
+    v = lib.chunkkv_num_chunks(L, w, c)
+    _check(min(v, 0), "chunkkv_num_chunks")
+    return v
+
+
+def num_kept_chunks(L: int, w: int, c: int, budget: int) -> int:
+    v = lib.chunkkv_num_kept_chunks(L, w, c, budget)
+    _check(min(v, 0), "chunkkv_num_kept_chunks")
+    return v
+
+
+def out_len(L: int, w: int, c: int, budget: int) -> int:
+    v = lib.chunkkv_out_len(L, w, c, budget)
+    _check(min(v, 0), "chunkkv_out_len")
+    return v
+
+
+def workspace_bytes(L: int, Hq: int, Hkv: int, d: int, w: int, c: int) -> int:
+    return int(lib.chunkkv_workspace_bytes(L, Hq, Hkv, d, w, c))
+
+
+def set_workspace(buf: Optional[torch.Tensor]) -> None:
+    """Hand the library a caller-owned scratch buffer (uint8 CUDA tensor), or None to undo."""
+    if buf is None:
+        _check(lib.chunkkv_set_workspace(None, 0), "chunkkv_set_workspace")
+    else:
+        _check(lib.chunkkv_set_workspace(buf.data_ptr(), buf.numel() * buf.element_size()),
+               "chunkkv_set_workspace")
+
+
+def device_status(stream: Optional[torch.cuda.Stream] = None) -> int:
+    """Synchronises the stream; returns 0 or CHUNKKV_EDEVICE (-6)."""
+    return lib.chunkkv_device_status(_stream(stream))
+
+
+def score(q_obs: torch.Tensor, K: torch.Tensor, w: int, c: int, want_token_scores: bool = False,
+          stream: Optional[torch.cuda.Stream] = None) -> Tuple[torch.Tensor, Optional[torch.Tensor]]:
+    """chunk scores [Hkv, C] f32 (and token scores [Hkv, P] f32 if asked)."""
+    _dev(q_obs, torch.bfloat16, "q_obs"); _dev(K, torch.bfloat16, "K")
+    Hq, d = q_obs.shape[0], q_obs.shape[2]
+    Hkv, L = K.shape[0], K.shape[1]
+    C = num_chunks(L, w, c)
+    cs = torch.empty((Hkv, C), dtype=torch.float32, device=K.device)
+    ts = torch.empty((Hkv, L - w), dtype=torch.float32, device=K.device) if want_token_scores else None
+    _check(lib.chunkkv_score(q_obs.data_ptr(), K.data_ptr(), L, Hq, Hkv, d, w, c, _ptr(ts),
+                             cs.data_ptr(), _stream(stream)), "chunkkv_score")
+    return cs, ts
+
+
+def select(chunk_scores: torch.Tensor, L: int, w: int, c: int, budget: int,
+           stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """idx [Hkv, n_max] int32 from chunk scores [Hkv, C] f32."""
+    _dev(chunk_scores, torch.float32, "chunk_scores")
+    Hkv = chunk_scores.shape[0]
+    n_max = out_len(L, w, c, budget)
+    idx = torch.empty((Hkv, n_max), dtype=torch.int32, device=chunk_scores.device)
+    _check(lib.chunkkv_select(chunk_scores.data_ptr(), L, Hkv, w, c, budget, idx.data_ptr(),
+                              _stream(stream)), "chunkkv_select")
+    return idx
+
+
+def gather(K: torch.Tensor, V: torch.Tensor, idx: torch.Tensor,
+           out_K: Optional[torch.Tensor] = None, out_V: Optional[torch.Tensor] = None,
+           stream: Optional[torch.cuda.Stream] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """out_K, out_V [Hkv, n_max, d] = K, V rows at idx [Hkv, n_max] (zero rows where idx < 0)."""
+    _dev(K, torch.bfloat16, "K"); _dev(V, torch.bfloat16, "V"); _dev(idx, torch.int32, "idx")
+    Hkv, L, d = K.shape
+    n_max = idx.shape[1]
+    if out_K is None:
+        out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=K.device)
+    if out_V is None:
+        out_V = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=K.device)
+    _check(lib.chunkkv_gather(K.data_ptr(), V.data_ptr(), idx.data_ptr(), L, Hkv, d, n_max,
+                              out_K.data_ptr(), out_V.data_ptr(), _stream(stream)), "chunkkv_gather")
+    return out_K, out_V
+
+
+def compress_layer(q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tensor, Hq: int, w: int,
+                   c: int, budget: int, reuse_idx: Optional[torch.Tensor] = None,
+                   out_K: Optional[torch.Tensor] = None, out_V: Optional[torch.Tensor] = None,
+                   out_idx: Optional[torch.Tensor] = None,
+                   stream: Optional[torch.cuda.Stream] = None,
+                   ) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """One layer: score -> chunk-sum -> top-k -> gather, or gather only with ``reuse_idx``."""
+    _dev(K, torch.bfloat16, "K"); _dev(V, torch.bfloat16, "V")
+    if q_obs is not None:
+        _dev(q_obs, torch.bfloat16, "q_obs")
+    if reuse_idx is not None:
+        _dev(reuse_idx, torch.int32, "reuse_idx")
+    Hkv, L, d = K.shape
+    n_max = out_len(L, w, c, budget)
+    dev = K.device
+    if out_K is None:
+        out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
+    if out_V is None:
+        out_V = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
+    if out_idx is None:
+        out_idx = torch.empty((Hkv, n_max), dtype=torch.int32, device=dev)
+    _check(lib.chunkkv_compress_layer(_ptr(q_obs), K.data_ptr(), V.data_ptr(), L, Hq, Hkv, d, w, c,
+                                      budget, _ptr(reuse_idx), out_K.data_ptr(), out_V.data_ptr(),
+                                      out_idx.data_ptr(), _stream(stream)), "chunkkv_compress_layer")
+    return out_K, out_V, out_idx
+
+
+def compress_layer_host(host_q: torch.Tensor, host_K: torch.Tensor, host_V: torch.Tensor, Hq: int,
+                        w: int, c: int, budget: int, dev_bufs: Sequence[torch.Tensor],
+                        host_outs: Sequence[torch.Tensor],
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Host tensors in, host tensors out; ``dev_bufs`` = (q, K, V, out_K, out_V, out_idx) staging
+    tensors on the GPU, ``host_outs`` = (out_K, out_V, out_idx) host tensors (pinned for speed)."""
+    Hkv, L, d = host_K.shape
+    dq, dK, dV, doK, doV, dI = dev_bufs
+    hK, hV, hI = host_outs
+    _check(lib.chunkkv_compress_layer_host(
+        host_q.data_ptr(), host_K.data_ptr(), host_V.data_ptr(), L, Hq, Hkv, d, w, c, budget,
+        dq.data_ptr(), dK.data_ptr(), dV.data_ptr(), doK.data_ptr(), doV.data_ptr(), dI.data_ptr(),
+        hK.data_ptr(), hV.data_ptr(), hI.data_ptr(), _stream(stream)), "chunkkv_compress_layer_host")
+
+
+def compress_model(layers: Sequence[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]], Hq: int, w: int,
+                   c: int, budget: int, n_reuse: int = 1,
+                   stream: Optional[torch.cuda.Stream] = None,
+                   ) -> List[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]]:
+    """Layer-wise index reuse: layer l computes indices iff l % n_reuse == 0, otherwise it
+    gathers with the indices of layer (l // n_reuse) * n_reuse. Only the call sequence lives
+    here; every layer is one chunkkv_compress_layer call."""
+    outs: List[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = []
+    for l, (q, K, V) in enumerate(layers):
+        if l % n_reuse == 0:
+            outs.append(compress_layer(q, K, V, Hq, w, c, budget, stream=stream))
+        else:
+            src = outs[(l // n_reuse) * n_reuse][2]
+            outs.append(compress_layer(None, K, V, Hq, w, c, budget, reuse_idx=src, stream=stream))
+    return outs
+
+
+def profile_enable(on: bool) -> None:
+    _check(lib.chunkkv_profile_enable(1 if on else 0), "chunkkv_profile_enable")
+
+
+def profile_read() -> Tuple[List[float], List[int]]:
+    ms = (ctypes.c_float * 4)()
+    n = (ctypes.c_int * 4)()
+    _check(lib.chunkkv_profile_read(ms, n), "chunkkv_profile_read")
+    return list(ms), list(n)

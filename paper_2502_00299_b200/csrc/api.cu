@@ -1,0 +1,495 @@
+// C ABI of libchunkkv: argument checks, scratch management, tensor-map encoding and the
+// launch sequence of each entry point. Every step of the method runs in the kernels of
+// score.cu / select.cu / gather.cu; this file only validates and dispatches.
+#include "../../include/chunkkv.h"
+#include "internal.h"
+
+#include <math.h>
+#include <mutex>
+#include <vector>
+
+using namespace chunkkv;
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+constexpr size_t kHeaderBytes = 256;   // device status word lives at the start of the scratch
+
+thread_local int g_last_cuda_error = 0;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+struct ProfileRec {
+    cudaEvent_t start, stop;
+    int slot;
+};
+
+struct DeviceCtx {
+    bool init = false;
+    int num_sms = 0;
+    int smem_optin = 0;
+    void* ws = nullptr;        // current scratch (header + payload)
+    size_t ws_bytes = 0;
+    bool ws_owned = false;     // allocated by the library
+    bool ws_user = false;      // provided by chunkkv_set_workspace
+    std::vector<ProfileRec> recs;
+    float prof_ms[CHUNKKV_PROFILE_SLOTS] = {0, 0, 0, 0};
+    int prof_n[CHUNKKV_PROFILE_SLOTS] = {0, 0, 0, 0};
+};
+
+std::mutex g_mu;
+DeviceCtx g_ctx[kMaxDevices];
+EncodeTiledFn g_encode = nullptr;
+bool g_profile = false;
+
+int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = static_cast<int>(e);
+    return CHUNKKV_ECUDA;
+}
+
+// Caller holds g_mu.
+int get_ctx(DeviceCtx** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxDevices) return CHUNKKV_EINVAL_SHAPE;
+    DeviceCtx& c = g_ctx[dev];
+    if (!c.init) {
+        e = cudaDeviceGetAttribute(&c.num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        e = cudaDeviceGetAttribute(&c.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+        if (e != cudaSuccess) return cuda_fail(e);
+        c.init = true;
+    }
+    if (g_encode == nullptr) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cuda_fail(cudaErrorNotSupported);
+        g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    *out = &c;
+    return CHUNKKV_OK;
+}
+
+// Shared-memory budget for the dynamic part of the score kernel (static control block excluded).
+int smem_budget(const DeviceCtx& c) { return c.smem_optin - 1024; }
+
+int ensure_workspace(DeviceCtx& c, size_t payload_bytes) {
+    const size_t need = kHeaderBytes + payload_bytes;
+    if (c.ws != nullptr && c.ws_bytes >= need) return CHUNKKV_OK;
+    if (c.ws_user) return CHUNKKV_ENOWORKSPACE;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (c.ws_owned && c.ws != nullptr) cudaFree(c.ws);
+    c.ws = nullptr;
+    c.ws_bytes = 0;
+    size_t bytes = need + (need >> 2);
+    bytes = (bytes + 255) & ~static_cast<size_t>(255);
+    e = cudaMalloc(&c.ws, bytes);
+    if (e != cudaSuccess) {
+        c.ws = nullptr;
+        g_last_cuda_error = static_cast<int>(e);
+        cudaGetLastError();
+        return CHUNKKV_ENOWORKSPACE;
+    }
+    e = cudaMemset(c.ws, 0, kHeaderBytes);
+    if (e != cudaSuccess) return cuda_fail(e);
+    c.ws_bytes = bytes;
+    c.ws_owned = true;
+    return CHUNKKV_OK;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_sizes(int L, int w, int c, int budget) {
+    if (w < 1 || c < 1 || L < w || budget < w) return CHUNKKV_EINVAL_SHAPE;
+    return CHUNKKV_OK;
+}
+
+int check_heads(int L, int Hq, int Hkv, int d, int w) {
+    if (Hkv < 1 || Hq < Hkv || Hq % Hkv != 0) return CHUNKKV_EINVAL_SHAPE;
+    if (d != 64 && d != 128) return CHUNKKV_EINVAL_SHAPE;
+    const long long R = static_cast<long long>(w) * (Hq / Hkv);
+    if (R > 256) return CHUNKKV_EINVAL_SHAPE;
+    if (static_cast<long long>(Hkv) * L * d >= (1LL << 40)) return CHUNKKV_EINVAL_SHAPE;
+    if (Hkv > 65535) return CHUNKKV_EINVAL_SHAPE;
+    return CHUNKKV_OK;
+}
+
+int encode_bf16_3d(CUtensorMap* tm, const void* base, int d, long long rows, int heads, int box_rows,
+                   CUtensorMapL2promotion promo) {
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(rows),
+                          static_cast<cuuint64_t>(heads)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(rows) * d * 2};
+    cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
+                          box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, promo,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_last_cuda_error = 100000 + static_cast<int>(r);
+        return CHUNKKV_ECUDA;
+    }
+    return CHUNKKV_OK;
+}
+
+struct Timer {
+    DeviceCtx* c;
+    cudaStream_t s;
+    bool on;
+    ProfileRec rec;
+    Timer(DeviceCtx* ctx, cudaStream_t st, int slot) : c(ctx), s(st), on(g_profile) {
+        if (!on) return;
+        rec.slot = slot;
+        if (cudaEventCreate(&rec.start) != cudaSuccess || cudaEventCreate(&rec.stop) != cudaSuccess) {
+            on = false;
+            return;
+        }
+        cudaEventRecord(rec.start, s);
+    }
+    ~Timer() {
+        if (!on) return;
+        cudaEventRecord(rec.stop, s);
+        c->recs.push_back(rec);
+    }
+};
+
+// Score + finalise for chunk size c. Chunk scores go to `out_scores`, or - when that is NULL -
+// to the first `extra_payload_floats` floats of the scratch payload; `*resolved` receives the
+// address used. Caller holds g_mu and has validated the arguments.
+int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w,
+              int c, float* out_scores, size_t extra_payload_floats, float** resolved,
+              cudaStream_t stream) {
+    const int G = Hq / Hkv, R = w * G, P = L - w;
+    const int C = (P + c - 1) / c;
+    if (C <= 0) return CHUNKKV_OK;
+    ScorePlan plan;
+    if (!make_score_plan(L, R, d, c, smem_budget(ctx), &plan)) return CHUNKKV_EINVAL_SHAPE;
+    const size_t floats = score_scratch_floats(plan, Hkv, R) + extra_payload_floats;
+    int st = ensure_workspace(ctx, floats * sizeof(float));
+    if (st != CHUNKKV_OK) return st;
+    float* payload = reinterpret_cast<float*>(static_cast<char*>(ctx.ws) + kHeaderBytes);
+    if (out_scores == nullptr) out_scores = payload;
+    if (resolved != nullptr) *resolved = out_scores;
+    const size_t tiles = static_cast<size_t>(Hkv) * plan.n_tiles;
+    ScoreArgs a;
+    a.L = L; a.P = P; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
+    a.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
+    a.stat_m = payload + extra_payload_floats;
+    a.stat_l = a.stat_m + tiles * R;
+    a.partial = a.stat_l + tiles * R;
+    a.status = static_cast<int*>(ctx.ws);
+    CUtensorMap tm_q, tm_k;
+    st = encode_bf16_3d(&tm_q, q_obs, d, R, Hkv, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    if (st != CHUNKKV_OK) return st;
+    st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < plan.n_tile ? L : plan.n_tile,
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+    if (st != CHUNKKV_OK) return st;
+    cudaError_t e;
+    {
+        Timer t(&ctx, stream, 0);
+        e = launch_score(plan, tm_q, tm_k, a, ctx.num_sms, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    {
+        Timer t(&ctx, stream, 1);
+        e = launch_finalize(plan, a, C, out_scores, ctx.num_sms, stream);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+size_t scratch_floats_for(const DeviceCtx& ctx, int L, int R, int Hkv, int d, int c) {
+    ScorePlan plan;
+    if (!make_score_plan(L, R, d, c, smem_budget(ctx), &plan)) return 0;
+    return score_scratch_floats(plan, Hkv, R);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* chunkkv_strerror(int status) {
+    switch (status) {
+        case CHUNKKV_OK: return "ok";
+        case CHUNKKV_EINVAL_NULL: return "a required pointer is NULL";
+        case CHUNKKV_EINVAL_SHAPE: return "a size is outside the supported range";
+        case CHUNKKV_EINVAL_ALIGN: return "a tensor pointer is not 16-byte aligned";
+        case CHUNKKV_ENOWORKSPACE: return "scratch workspace too small or could not be allocated";
+        case CHUNKKV_ECUDA: return "a CUDA call failed";
+        case CHUNKKV_EDEVICE: return "a kernel abandoned a bounded wait";
+        default: return "unknown status";
+    }
+}
+
+int chunkkv_last_cuda_error(void) { return g_last_cuda_error; }
+
+int chunkkv_num_chunks(int L, int w, int c) {
+    if (w < 1 || c < 1 || L < w) return CHUNKKV_EINVAL_SHAPE;
+    return (L - w + c - 1) / c;
+}
+
+int chunkkv_num_kept_chunks(int L, int w, int c, int budget) {
+    int st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    const int C = (L - w + c - 1) / c;
+    const int k = (budget - w) / c;
+    return k < C ? k : C;
+}
+
+int chunkkv_out_len(int L, int w, int c, int budget) {
+    const int k = chunkkv_num_kept_chunks(L, w, c, budget);
+    if (k < 0) return k;
+    const long long n = static_cast<long long>(k) * c + w;
+    if (n > 0x7fffffffLL) return CHUNKKV_EINVAL_SHAPE;
+    return static_cast<int>(n);
+}
+
+size_t chunkkv_workspace_bytes(int L, int Hq, int Hkv, int d, int w, int c) {
+    if (w < 1 || c < 1 || L < w) return 0;
+    if (check_heads(L, Hq, Hkv, d, w) != CHUNKKV_OK) return 0;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    if (get_ctx(&ctx) != CHUNKKV_OK) return 0;
+    const int R = w * (Hq / Hkv);
+    const int C = (L - w + c - 1) / c;
+    const size_t floats = scratch_floats_for(*ctx, L, R, Hkv, d, c) +
+                          ((static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63));
+    return kHeaderBytes + floats * sizeof(float);
+}
+
+int chunkkv_set_workspace(void* dev_ptr, size_t bytes) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    int st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev_ptr == nullptr) {
+        if (ctx->ws_user) { ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->ws_user = false; }
+        return CHUNKKV_OK;
+    }
+    if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return CHUNKKV_EINVAL_ALIGN;
+    if (bytes < kHeaderBytes) return CHUNKKV_ENOWORKSPACE;
+    if (ctx->ws_owned && ctx->ws != nullptr) cudaFree(ctx->ws);
+    ctx->ws_owned = false;
+    e = cudaMemset(dev_ptr, 0, kHeaderBytes);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    ctx->ws = dev_ptr;
+    ctx->ws_bytes = bytes;
+    ctx->ws_user = true;
+    return CHUNKKV_OK;
+}
+
+int chunkkv_device_status(void* stream) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    int st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (ctx->ws == nullptr) return CHUNKKV_OK;
+    int flag = 0;
+    e = cudaMemcpy(&flag, ctx->ws, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (flag != 0) {
+        cudaMemset(ctx->ws, 0, sizeof(int));
+        return CHUNKKV_EDEVICE;
+    }
+    return CHUNKKV_OK;
+}
+
+int chunkkv_score(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w, int c,
+                  float* out_token_scores, float* out_chunk_scores, void* stream) {
+    if (w < 1 || c < 1 || L < w) return CHUNKKV_EINVAL_SHAPE;
+    int st = check_heads(L, Hq, Hkv, d, w);
+    if (st != CHUNKKV_OK) return st;
+    if (q_obs == nullptr || K == nullptr || out_chunk_scores == nullptr) return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(q_obs) || !aligned16(K) || !aligned16(out_chunk_scores) ||
+        (out_token_scores != nullptr && !aligned16(out_token_scores)))
+        return CHUNKKV_EINVAL_ALIGN;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, out_chunk_scores, 0, nullptr, s);
+    if (st != CHUNKKV_OK) return st;
+    if (out_token_scores != nullptr)
+        st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, 1, out_token_scores, 0, nullptr, s);
+    return st;
+}
+
+int chunkkv_select(const float* chunk_scores, int L, int Hkv, int w, int c, int budget,
+                   int32_t* out_idx, void* stream) {
+    int st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    if (Hkv < 1 || Hkv > 65535) return CHUNKKV_EINVAL_SHAPE;
+    const int C = chunkkv_num_chunks(L, w, c);
+    const int k = chunkkv_num_kept_chunks(L, w, c, budget);
+    const int n_max = chunkkv_out_len(L, w, c, budget);
+    if (n_max < 0) return n_max;
+    if (out_idx == nullptr || (C > 0 && k > 0 && chunk_scores == nullptr)) return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(out_idx) || !aligned16(chunk_scores)) return CHUNKKV_EINVAL_ALIGN;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    {
+        Timer t(ctx, s, 2);
+        e = launch_select(chunk_scores, L, Hkv, w, c, C, k, n_max, out_idx, s);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+int chunkkv_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
+                   int n_max, void* out_K, void* out_V, void* stream) {
+    if (L < 1 || Hkv < 1 || Hkv > 65535 || n_max < 0 || (d != 64 && d != 128)) return CHUNKKV_EINVAL_SHAPE;
+    if (static_cast<long long>(Hkv) * L * d >= (1LL << 40)) return CHUNKKV_EINVAL_SHAPE;
+    if (K == nullptr || V == nullptr || idx == nullptr || out_K == nullptr || out_V == nullptr)
+        return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(idx) || !aligned16(out_K) || !aligned16(out_V))
+        return CHUNKKV_EINVAL_ALIGN;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    int st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    {
+        Timer t(ctx, s, 3);
+        e = launch_gather(K, V, idx, L, Hkv, d, n_max, out_K, out_V, nullptr, ctx->num_sms, s);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                           int d, int w, int c, int budget, const int32_t* reuse_idx,
+                           void* out_K, void* out_V, int32_t* out_idx, void* stream) {
+    int st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    st = check_heads(L, Hq, Hkv, d, w);
+    if (st != CHUNKKV_OK) return st;
+    if (K == nullptr || V == nullptr || out_K == nullptr || out_V == nullptr || out_idx == nullptr)
+        return CHUNKKV_EINVAL_NULL;
+    if (reuse_idx == nullptr && q_obs == nullptr) return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(q_obs) || !aligned16(K) || !aligned16(V) || !aligned16(out_K) || !aligned16(out_V) ||
+        !aligned16(out_idx) || !aligned16(reuse_idx))
+        return CHUNKKV_EINVAL_ALIGN;
+    const int C = chunkkv_num_chunks(L, w, c);
+    const int k = chunkkv_num_kept_chunks(L, w, c, budget);
+    const int n_max = chunkkv_out_len(L, w, c, budget);
+    if (n_max < 0) return n_max;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (reuse_idx != nullptr) {
+        Timer t(ctx, s, 3);
+        e = launch_gather(K, V, reuse_idx, L, Hkv, d, n_max, out_K, out_V,
+                          reuse_idx == out_idx ? nullptr : out_idx, ctx->num_sms, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        return CHUNKKV_OK;
+    }
+    float* chunk_scores = nullptr;
+    if (C > 0 && k > 0) {
+        // chunk scores sit at the start of the scratch payload, the score kernels' scratch after them
+        const size_t cs_floats = (static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63);
+        st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, cs_floats, &chunk_scores, s);
+        if (st != CHUNKKV_OK) return st;
+    }
+    {
+        Timer t(ctx, s, 2);
+        e = launch_select(chunk_scores, L, Hkv, w, c, C, k, n_max, out_idx, s);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    {
+        Timer t(ctx, s, 3);
+        e = launch_gather(K, V, out_idx, L, Hkv, d, n_max, out_K, out_V, nullptr, ctx->num_sms, s);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+int chunkkv_compress_layer_host(const void* host_q_obs, const void* host_K, const void* host_V,
+                                int L, int Hq, int Hkv, int d, int w, int c, int budget,
+                                void* dev_q_obs, void* dev_K, void* dev_V,
+                                void* dev_out_K, void* dev_out_V, int32_t* dev_out_idx,
+                                void* host_out_K, void* host_out_V, int32_t* host_out_idx,
+                                void* stream) {
+    int st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    st = check_heads(L, Hq, Hkv, d, w);
+    if (st != CHUNKKV_OK) return st;
+    if (!host_q_obs || !host_K || !host_V || !dev_q_obs || !dev_K || !dev_V || !dev_out_K || !dev_out_V ||
+        !dev_out_idx || !host_out_K || !host_out_V || !host_out_idx)
+        return CHUNKKV_EINVAL_NULL;
+    const int n_max = chunkkv_out_len(L, w, c, budget);
+    if (n_max < 0) return n_max;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t q_bytes = static_cast<size_t>(Hq) * w * d * 2;
+    const size_t kv_bytes = static_cast<size_t>(Hkv) * L * d * 2;
+    const size_t o_bytes = static_cast<size_t>(Hkv) * n_max * d * 2;
+    const size_t i_bytes = static_cast<size_t>(Hkv) * n_max * sizeof(int32_t);
+    cudaError_t e;
+    if ((e = cudaMemcpyAsync(dev_q_obs, host_q_obs, q_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dev_K, host_K, kv_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(dev_V, host_V, kv_bytes, cudaMemcpyHostToDevice, s)) != cudaSuccess)
+        return cuda_fail(e);
+    st = chunkkv_compress_layer(dev_q_obs, dev_K, dev_V, L, Hq, Hkv, d, w, c, budget, nullptr, dev_out_K,
+                                dev_out_V, dev_out_idx, stream);
+    if (st != CHUNKKV_OK) return st;
+    if ((e = cudaMemcpyAsync(host_out_K, dev_out_K, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(host_out_V, dev_out_V, o_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(host_out_idx, dev_out_idx, i_bytes, cudaMemcpyDeviceToHost, s)) != cudaSuccess)
+        return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+int chunkkv_profile_enable(int on) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_profile = (on != 0);
+    return CHUNKKV_OK;
+}
+
+int chunkkv_profile_read(float* ms_per_slot, int* launches_per_slot) {
+    if (ms_per_slot == nullptr || launches_per_slot == nullptr) return CHUNKKV_EINVAL_NULL;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    int st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) return cuda_fail(e);
+    for (ProfileRec& r : ctx->recs) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, r.start, r.stop) == cudaSuccess) {
+            ctx->prof_ms[r.slot] += ms;
+            ctx->prof_n[r.slot] += 1;
+        }
+        cudaEventDestroy(r.start);
+        cudaEventDestroy(r.stop);
+    }
+    ctx->recs.clear();
+    for (int i = 0; i < CHUNKKV_PROFILE_SLOTS; ++i) {
+        ms_per_slot[i] = ctx->prof_ms[i];
+        launches_per_slot[i] = ctx->prof_n[i];
+        ctx->prof_ms[i] = 0.f;
+        ctx->prof_n[i] = 0;
+    }
+    return CHUNKKV_OK;
+}
+
+}  // extern "C"

@@ -48,23 +48,36 @@ struct SharedCtl {
 
 // One thread owns one query row of the tile. `taddr` points at the thread's lane quarter and
 // the first column of the accumulator. All reads use 32- or 16-column TMEM loads.
-template <int N_TILE, typename F>
+// UNROLL_BLOCKS: unroll across the 32-column blocks too, so that column numbers are
+// compile-time constants in `f` (the fast path needs that; the general path does not).
+template <int N_TILE, bool UNROLL_BLOCKS, typename F>
 __device__ __forceinline__ void for_each_column(uint32_t taddr, F&& f) {
+    constexpr int FULL = N_TILE / 32;
+    if constexpr (UNROLL_BLOCKS) {
 #pragma unroll
-    for (int cb = 0; cb < N_TILE; cb += 32) {
-        if (cb + 32 <= N_TILE) {
+        for (int b = 0; b < FULL; ++b) {
             float v[32];
-            tmem_ld_x32(taddr + cb, v);
+            tmem_ld_x32(taddr + b * 32, v);
             tmem_ld_wait();
 #pragma unroll
-            for (int u = 0; u < 32; ++u) f(cb + u, v[u]);
-        } else {
-            float v[16];
-            tmem_ld_x16(taddr + cb, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int u = 0; u < 16; ++u) f(cb + u, v[u]);
+            for (int u = 0; u < 32; ++u) f(b * 32 + u, v[u]);
         }
+    } else {
+#pragma unroll 1
+        for (int b = 0; b < FULL; ++b) {
+            float v[32];
+            tmem_ld_x32(taddr + b * 32, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int u = 0; u < 32; ++u) f(b * 32 + u, v[u]);
+        }
+    }
+    if constexpr (N_TILE % 32 != 0) {
+        float v[16];
+        tmem_ld_x16(taddr + FULL * 32, v);
+        tmem_ld_wait();
+#pragma unroll
+        for (int u = 0; u < 16; ++u) f(FULL * 32 + u, v[u]);
     }
 }
 
@@ -92,7 +105,7 @@ __device__ __forceinline__ void tile_fast(uint32_t taddr, float sl2, bool active
     }
     const float neg_m2 = -mx * sl2;
     float l = 0.f, acc = 0.f;
-    for_each_column<N_TILE>(taddr, [&](int j, float x) {
+    for_each_column<N_TILE, true>(taddr, [&](int j, float x) {
         const float e = ex2_approx(fmaf(x, sl2, neg_m2));
         acc += e;
         if ((j + 1) % C == 0) {
@@ -113,7 +126,7 @@ __device__ __forceinline__ void tile_general(uint32_t taddr, float sl2, bool act
                                              float* out_m, float* out_l) {
     const int last_visible = min(P + r, L - 1);   // this row sees keys j <= P + r
     float mx = -CUDART_INF_F;
-    for_each_column<N_TILE>(taddr, [&](int u, float x) {
+    for_each_column<N_TILE, false>(taddr, [&](int u, float x) {
         const bool vis = (j0 + u) <= last_visible;
         mx = vis ? fmaxf(mx, x) : mx;
     });
@@ -121,7 +134,7 @@ __device__ __forceinline__ void tile_general(uint32_t taddr, float sl2, bool act
     float l = 0.f, acc = 0.f;
     int slot = 0;
     int nb = (j0 < P) ? min((j0 / c + 1) * c, P) : 0;   // end (exclusive) of the current chunk
-    for_each_column<N_TILE>(taddr, [&](int u, float x) {
+    for_each_column<N_TILE, false>(taddr, [&](int u, float x) {
         const int j = j0 + u;
         const bool vis = j <= last_visible;
         const float e = vis ? ex2_approx(fmaf(x, sl2, neg_m2)) : 0.f;

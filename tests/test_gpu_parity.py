@@ -1,0 +1,261 @@
+"""GPU-vs-oracle parity through the C ABI (kernels of libchunkkv against oracle/).
+
+Tolerances: token and chunk scores within 1e-3 relative (plus an absolute floor of 1e-6 of the
+mean token score); selected chunk sets identical except swaps among chunks whose oracle score
+is within 1e-4 relative of the k-th best; indices and gathered K/V bit-exact given the set.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import chunkkv_oracle as ora
+from tests.helpers import (assert_gather_exact, assert_scores_close, assert_selection_matches,
+                           bits_of, chunks_of_idx, rand_bits, to_dev)
+from workloads import CONFIGS, iter_layers, make_layer, ragged_lengths, scaled
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ck():
+    import paper_2502_00299_b200 as ck
+    assert torch.cuda.is_available()
+    return ck
+
+
+def _status_ok(ck):
+    assert ck.device_status() == 0, "a kernel reported an abandoned wait"
+
+
+# ------------------------------------------------------------------------------ gather
+@pytest.mark.parametrize("Hkv,L,d,n_max", [(2, 300, 64, 77), (3, 1000, 128, 513), (1, 64, 128, 1),
+                                           (8, 4096, 128, 1311)])
+def test_gather_bit_exact(ck, Hkv, L, d, n_max):
+    rng = np.random.default_rng(L + n_max)
+    K, V = rand_bits(rng, (Hkv, L, d)), rand_bits(rng, (Hkv, L, d))
+    idx = np.stack([np.sort(rng.choice(L, size=n_max, replace=False)) for _ in range(Hkv)]).astype(np.int32)
+    idx[0, n_max // 2:] = -1                      # padding -> zero rows
+    if n_max > 3:
+        idx[-1, 1] = L + 5                        # out of range -> zero row, never dereferenced
+    oK, oV = ck.gather(to_dev(K), to_dev(V), torch.from_numpy(idx).cuda())
+    ref_idx = np.where((idx >= 0) & (idx < L), idx, -1)
+    assert_gather_exact(bits_of(oK), bits_of(oV), ref_idx, K, V)
+
+
+# ------------------------------------------------------------------------------ select
+@pytest.mark.parametrize("L,w,c,budget,Hkv", [
+    (2048, 16, 10, 256, 2), (1003, 8, 10, 203, 3), (500, 4, 7, 4 + 7 * 20, 2), (26, 4, 5, 1000, 1),
+    (26, 4, 5, 8, 1), (4, 4, 5, 4, 2), (9000, 32, 1, 32 + 777, 2), (20000, 32, 3, 32 + 3 * 2500, 1),
+])
+def test_select_bit_exact_on_given_scores(ck, L, w, c, budget, Hkv):
+    rng = np.random.default_rng(L * 7 + c)
+    C = ora.num_chunks(L, w, c)
+    s = rng.random((Hkv, max(C, 1))).astype(np.float32)[:, :C]
+    if C > 0:
+        s[0, C - 1] = 2.0                          # the clipped last chunk is kept in head 0
+    idx = ck.select(torch.from_numpy(np.ascontiguousarray(s)).cuda(), L, w, c, budget).cpu().numpy()
+    ref = ora.select(s.astype(np.float64), L, w, c, budget)
+    assert np.array_equal(idx, ref)
+
+
+def test_select_ties_go_to_lower_chunk_ids(ck):
+    L, w, c, Hkv = 5000, 8, 4, 3
+    C = ora.num_chunks(L, w, c)
+    rng = np.random.default_rng(3)
+    s = rng.integers(0, 6, size=(Hkv, C)).astype(np.float32)       # massive ties
+    s[1] = 1.0                                                      # all equal
+    s[2, ::2] = -0.0                                                # -0 ties with +0
+    s[2, 1::2] = 0.0
+    for budget in (w + c * 1, w + c * 37, w + c * (C // 2), w + c * (C - 1)):
+        idx = ck.select(torch.from_numpy(s).cuda(), L, w, c, budget).cpu().numpy()
+        assert np.array_equal(idx, ora.select(s.astype(np.float64), L, w, c, budget))
+
+
+# ------------------------------------------------------------------------------ score
+SCORE_CASES = [
+    # Hq, Hkv, d, L, w, c    (R = w * Hq / Hkv)
+    (8, 2, 64, 2048, 16, 10),        # R 64, several tiles, tail chunk of 2
+    (32, 8, 128, 1999, 32, 10),      # R 128, ragged everything
+    (4, 1, 128, 960, 32, 10),        # P = 928 < 4 tiles, window straddles the 240-key tile edge
+    (4, 1, 128, 975, 32, 10),        # window crosses a tile boundary (tile edge at 960)
+    (8, 2, 128, 1500, 16, 20),       # static c = 20
+    (8, 2, 128, 1500, 16, 7),        # run-time c, chunks straddle tiles
+    (8, 2, 64, 700, 16, 300),        # chunk longer than a tile
+    (6, 2, 128, 777, 5, 13),         # R = 15, not a multiple of 32
+    (32, 4, 128, 1200, 32, 10),      # R = 256: two query tiles
+    (24, 4, 64, 900, 32, 20),        # R = 192: second query tile half empty
+    (8, 2, 128, 100, 16, 10),        # L smaller than one tile
+    (8, 2, 128, 17, 16, 10),         # P = 1
+]
+
+
+@pytest.mark.parametrize("Hq,Hkv,d,L,w,c", SCORE_CASES)
+def test_score_matches_oracle(ck, Hq, Hkv, d, L, w, c):
+    rng = np.random.default_rng(Hq * 1000 + L + c)
+    q, K = rand_bits(rng, (Hq, w, d), 1.5), rand_bits(rng, (Hkv, L, d), 1.5)
+    cs, ts = ck.score(to_dev(q), to_dev(K), w, c, want_token_scores=True)
+    _status_ok(ck)
+    t = ora.token_scores(q, K, Hq, Hkv, w)
+    s = ora.chunk_scores(t, c)
+    R = w * Hq // Hkv
+    assert_scores_close(ts.cpu().numpy(), t, R, L, "token scores")
+    assert_scores_close(cs.cpu().numpy(), s, R, L, "chunk scores")
+    # invariant at any size: chunk scores carry the whole prefix mass
+    assert np.allclose(cs.sum(dim=1).cpu().numpy(), t.sum(axis=1), rtol=1e-4)
+
+
+def test_score_with_large_logits_and_planted_structure(ck):
+    # logits far from N(0,1): exercises the per-tile maxima and their recombination
+    Hq, Hkv, d, L, w, c = 8, 2, 128, 3000, 16, 10
+    rng = np.random.default_rng(42)
+    q, K = rand_bits(rng, (Hq, w, d), 4.0), rand_bits(rng, (Hkv, L, d), 4.0)
+    cs, ts = ck.score(to_dev(q), to_dev(K), w, c, want_token_scores=True)
+    _status_ok(ck)
+    t = ora.token_scores(q, K, Hq, Hkv, w)
+    assert_scores_close(ts.cpu().numpy(), t, w * Hq // Hkv, L, "token scores")
+    assert_scores_close(cs.cpu().numpy(), ora.chunk_scores(t, c), w * Hq // Hkv, L, "chunk scores")
+
+
+def test_score_is_deterministic(ck):
+    x = make_layer(scaled(CONFIGS[2], L=5000))
+    q, K = to_dev(x.q_obs), to_dev(x.K)
+    a, _ = ck.score(q, K, 32, 10)
+    b, _ = ck.score(q, K, 32, 10)
+    assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------------------ whole layer
+def _run_layer(ck, x, wl, budget=None, L=None):
+    budget = wl.budget if budget is None else budget
+    q, K, V = to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)
+    oK, oV, idx = ck.compress_layer(q, K, V, wl.Hq, wl.w, wl.c, budget)
+    _status_ok(ck)
+    return bits_of(oK), bits_of(oV), idx.cpu().numpy()
+
+
+def _check_layer(x, wl, oK, oV, idx, budget=None):
+    budget = wl.budget if budget is None else budget
+    L = x.K.shape[1]
+    t = ora.token_scores(x.q_obs, x.K, wl.Hq, wl.Hkv, wl.w)
+    s = ora.chunk_scores(t, wl.c)
+    assert idx.shape == (wl.Hkv, ora.out_len(L, wl.w, wl.c, budget))
+    swaps = assert_selection_matches(idx, s, L, wl.w, wl.c, budget)
+    assert_gather_exact(oK, oV, idx, x.K, x.V)
+    return swaps
+
+
+def test_compress_layer_config1(ck):
+    wl = CONFIGS[1]
+    x = make_layer(wl)
+    oK, oV, idx = _run_layer(ck, x, wl)
+    _check_layer(x, wl, oK, oV, idx)
+    for h in range(wl.Hkv):                       # the planted chunks are all kept
+        got, n_kept = chunks_of_idx(idx[h], wl.L, wl.w, wl.c)
+        assert set(x.planted.tolist()) <= set(got.tolist())
+        assert n_kept == 24 * 10 + 16
+
+
+@pytest.mark.parametrize("budget", [16, 25, 26, 2032 + 16 + 10, 100000])
+def test_compress_layer_degenerate_budgets(ck, budget):
+    wl = CONFIGS[1]                               # k = 0, 0, 1, C (identity), C
+    x = make_layer(wl)
+    oK, oV, idx = _run_layer(ck, x, wl, budget=budget)
+    _check_layer(x, wl, oK, oV, idx, budget=budget)
+    if budget >= wl.L + wl.c:
+        assert idx[0][:wl.L].tolist() == list(range(wl.L))
+
+
+def test_compress_layer_window_only_sequence(ck):
+    wl = scaled(CONFIGS[1], L=16)                 # P = 0: nothing to score
+    x = make_layer(wl)
+    oK, oV, idx = _run_layer(ck, x, wl)
+    assert idx.tolist() == [list(range(16))] * wl.Hkv
+    assert_gather_exact(oK, oV, idx, x.K, x.V)
+
+
+@pytest.mark.parametrize("cfg,L", [(2, 4000), (4, 9000)])
+def test_compress_layer_scaled_configs(ck, cfg, L):
+    wl = scaled(CONFIGS[cfg], L=L, budget=max(CONFIGS[cfg].w + 50, L // 10))
+    x = make_layer(wl)
+    oK, oV, idx = _run_layer(ck, x, wl)
+    _check_layer(x, wl, oK, oV, idx)
+
+
+def test_compress_layer_config2_full_size(ck):
+    wl = CONFIGS[2]
+    x = make_layer(wl)
+    q, K = to_dev(x.q_obs), to_dev(x.K)
+    cs, _ = ck.score(q, K, wl.w, wl.c)
+    t = ora.token_scores(x.q_obs, x.K, wl.Hq, wl.Hkv, wl.w)
+    assert_scores_close(cs.cpu().numpy(), ora.chunk_scores(t, wl.c), 128, wl.L, "chunk scores")
+    oK, oV, idx = _run_layer(ck, x, wl)
+    _check_layer(x, wl, oK, oV, idx)
+    for h in range(wl.Hkv):
+        got, _ = chunks_of_idx(idx[h], wl.L, wl.w, wl.c)
+        assert set(x.planted.tolist()) <= set(got.tolist()) and 0 in got   # planted + sink chunk
+
+
+def test_reuse_layers_config3_scaled(ck):
+    wl = scaled(CONFIGS[3], L=3000, budget=300, n_layers=5)
+    layers = list(iter_layers(wl))
+    dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in layers]
+    outs = ck.compress_model(dev, wl.Hq, wl.w, wl.c, wl.budget, n_reuse=wl.reuse_depth)
+    _status_ok(ck)
+    for l, (x, (oK, oV, idx)) in enumerate(zip(layers, outs)):
+        src = (l // wl.reuse_depth) * wl.reuse_depth
+        idx_np = idx.cpu().numpy()
+        assert np.array_equal(idx_np, outs[src][2].cpu().numpy())      # reused indices are copies
+        assert_gather_exact(bits_of(oK), bits_of(oV), idx_np, x.K, x.V)
+        if l == src:
+            _check_layer(x, wl, bits_of(oK), bits_of(oV), idx_np)
+    # aliasing out_idx == reuse_idx is allowed
+    q, K, V = dev[1]
+    idx0 = outs[0][2].clone()
+    oK, oV, idx_same = ck.compress_layer(None, K, V, wl.Hq, wl.w, wl.c, wl.budget, reuse_idx=idx0, out_idx=idx0)
+    assert torch.equal(idx_same, outs[0][2]) and torch.equal(oK, outs[1][0])
+
+
+def test_ragged_batch_config5_scaled(ck):
+    wl = scaled(CONFIGS[5], len_lo=700, len_hi=3000, budget=200, n_layers=4)
+    lens = ragged_lengths(wl)
+    assert len(set(lens)) > 1
+    for seq, L in enumerate(lens[:4]):
+        x = make_layer(wl, layer=0, seq=seq, L=L)
+        oK, oV, idx = _run_layer(ck, x, wl)
+        _check_layer(x, wl, oK, oV, idx)
+
+
+def test_compress_layer_host_round_trip(ck):
+    wl = scaled(CONFIGS[2], L=3000, budget=300)
+    x = make_layer(wl)
+    n_max = ora.out_len(wl.L, wl.w, wl.c, wl.budget)
+    as_t = lambda b: torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).pin_memory()
+    hq, hK, hV = as_t(x.q_obs), as_t(x.K), as_t(x.V)
+    dev = [torch.empty_like(t, device="cuda") for t in (hq, hK, hV)]
+    dev += [torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    dev += [torch.empty((wl.Hkv, n_max), dtype=torch.int32, device="cuda")]
+    outs = [torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
+    outs += [torch.empty((wl.Hkv, n_max), dtype=torch.int32).pin_memory()]
+    ck.compress_layer_host(hq, hK, hV, wl.Hq, wl.w, wl.c, wl.budget, dev, outs)
+    torch.cuda.synchronize()
+    _status_ok(ck)
+    _check_layer(x, wl, bits_of(outs[0]), bits_of(outs[1]), outs[2].numpy())
+
+
+def test_caller_provided_workspace(ck):
+    wl = scaled(CONFIGS[2], L=2500, budget=250)
+    x = make_layer(wl)
+    need = ck.workspace_bytes(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c)
+    assert need > 0
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    ck.set_workspace(small)
+    try:
+        with pytest.raises(ck.ChunkKVError) as e:
+            _run_layer(ck, x, wl)
+        assert e.value.status == -4
+        buf = torch.empty(need, dtype=torch.uint8, device="cuda")
+        ck.set_workspace(buf)
+        oK, oV, idx = _run_layer(ck, x, wl)
+        _check_layer(x, wl, oK, oV, idx)
+    finally:
+        ck.set_workspace(None)
