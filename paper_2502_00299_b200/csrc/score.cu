@@ -395,8 +395,17 @@ template <int C_STATIC, int N_MT, int N_TILE>
 cudaError_t launch_variant(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                            const ScoreArgs& args, int num_sms, cudaStream_t stream) {
     auto kern = score_kernel<C_STATIC, N_MT, N_TILE>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+    // Opt in to large dynamic shared memory once per device and variant (not a stream operation,
+    // so later launches stay free of it, e.g. inside a stream capture).
+    static int smem_set[64] = {0};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64 || smem_set[dev] < plan.smem_bytes) {
+        e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) smem_set[dev] = plan.smem_bytes;
+    }
     KernelGeom g;
     g.n_tiles = plan.n_tiles;
     g.spt = plan.spt;
