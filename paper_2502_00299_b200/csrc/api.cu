@@ -169,20 +169,17 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
     const int C = (P + c - 1) / c;
     if (C <= 0) return CHUNKKV_OK;
     ScorePlan plan;
-    if (!make_score_plan(L, R, d, c, smem_budget(ctx), &plan)) return CHUNKKV_EINVAL_SHAPE;
+    if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), &plan)) return CHUNKKV_EINVAL_SHAPE;
     const size_t floats = score_scratch_floats(plan, Hkv, R) + extra_payload_floats;
     int st = ensure_workspace(ctx, floats * sizeof(float));
     if (st != CHUNKKV_OK) return st;
     float* payload = reinterpret_cast<float*>(static_cast<char*>(ctx.ws) + kHeaderBytes);
     if (out_scores == nullptr) out_scores = payload;
     if (resolved != nullptr) *resolved = out_scores;
-    const size_t tiles = static_cast<size_t>(Hkv) * plan.n_tiles;
     ScoreArgs a;
     a.L = L; a.P = P; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
     a.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
-    a.stat_m = payload + extra_payload_floats;
-    a.stat_l = a.stat_m + tiles * R;
-    a.partial = a.stat_l + tiles * R;
+    score_scratch_layout(plan, Hkv, R, payload + extra_payload_floats, &a);
     a.status = static_cast<int*>(ctx.ws);
     CUtensorMap tm_q, tm_k;
     st = encode_bf16_3d(&tm_q, q_obs, d, R, Hkv, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
@@ -193,7 +190,7 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
     cudaError_t e;
     {
         Timer t(&ctx, stream, 0);
-        e = launch_score(plan, tm_q, tm_k, a, ctx.num_sms, stream);
+        e = launch_score(plan, tm_q, tm_k, a, stream);
     }
     if (e != cudaSuccess) return cuda_fail(e);
     {
@@ -206,7 +203,7 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
 
 size_t scratch_floats_for(const DeviceCtx& ctx, int L, int R, int Hkv, int d, int c) {
     ScorePlan plan;
-    if (!make_score_plan(L, R, d, c, smem_budget(ctx), &plan)) return 0;
+    if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), &plan)) return 0;
     return score_scratch_floats(plan, Hkv, R);
 }
 

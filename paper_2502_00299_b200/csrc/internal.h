@@ -11,9 +11,13 @@ namespace chunkkv {
 struct ScorePlan {
     int c_static;   // chunk size baked into the kernel (0 = run-time chunk size)
     int n_mt;       // 128-row query tiles per KV head (1 or 2)
-    int n_tile;     // keys per accumulator tile
+    int n_tile;     // keys per accumulator tile (one UMMA N)
+    int wp;         // keys per epilogue panel (n_tile / 4 with one query tile, else n_tile / 2)
     int n_tiles;    // accumulator tiles per head = ceil(L / n_tile)
-    int spt;        // chunk slots per tile in the partial-sum scratch
+    int n_panels;   // panels per head
+    int spp;        // chunk slots per panel in the partial-sum scratch
+    int grid;       // CTAs of the scoring launch
+    int hs_max;     // per-CTA head records in the CTA statistics scratch
     int n_stages;   // shared-memory stages in the K ring (one stage = n_tile keys x 64 dims)
     int smem_bytes; // dynamic shared memory of the launch
 };
@@ -21,20 +25,23 @@ struct ScorePlan {
 struct ScoreArgs {
     int L, P, w, c, R, Hkv, d;
     float sl2;            // log2(e) / sqrt(d)
-    float* stat_m;        // [Hkv, n_tiles, R] tile row maxima (log2 domain)
-    float* stat_l;        // [Hkv, n_tiles, R] tile row sums relative to the tile maximum
-    float* partial;       // [Hkv, n_tiles, spt, R] chunk partial sums relative to the tile maximum
+    float* stat_m;        // [Hkv, n_panels, R] panel row maxima (log2 domain)
+    float* cta_stat;      // [grid, hs_max, 2 groups, {max, sum}, 128] per-CTA folded row statistics
+    float* partial;       // [Hkv, n_panels, spp, R] chunk partial sums relative to the panel maximum
     int* status;          // device status word
 };
 
 // Chooses kernel variant and tile geometry for a shape. Returns false if unsupported.
-bool make_score_plan(int L, int R, int d, int c, int smem_limit, ScorePlan* plan);
+bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_limit, ScorePlan* plan);
 
-// Scratch floats needed for a plan (tile statistics + partial sums), per layer.
+// Scratch floats needed for a plan (panel maxima + CTA records + partial sums), per layer.
 size_t score_scratch_floats(const ScorePlan& plan, int Hkv, int R);
 
+// Points the scratch pointers of `args` into `base` (score_scratch_floats floats).
+void score_scratch_layout(const ScorePlan& plan, int Hkv, int R, float* base, ScoreArgs* args);
+
 cudaError_t launch_score(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                         const ScoreArgs& args, int num_sms, cudaStream_t stream);
+                         const ScoreArgs& args, cudaStream_t stream);
 
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
                             int num_sms, cudaStream_t stream);

@@ -1,17 +1,21 @@
 // Observation-window attention scoring with the chunk sums fused into the epilogue
 // (ChunkKV Algorithm 3: "A <- q_observe K^T" and "Vectorized Chunk Score Calculation"),
-// followed by a small finalisation kernel that turns per-tile partial sums into chunk scores.
+// followed by a small finalisation kernel that turns per-panel partial sums into chunk scores.
 //
 // Per KV head the score matrix is S = Q_obs K^T (R rows = window queries of the grouped
-// query heads, L columns = keys). The kernel streams K through shared memory with TMA,
+// query heads, L columns = keys). The kernel streams K through shared memory with TMA and
 // multiplies 128-row x n_tile-key tiles on the tensor cores (tcgen05, fp32 accumulators in
-// tensor memory) and lets one thread per query row reduce its row of the tile:
-//     tile row maximum, exp2 of every visible element relative to it, row sum, and the sum
-//     over each chunk's columns ("partial", one value per row and chunk).
-// Each score element is exponentiated exactly once. Because the softmax normaliser of a row
-// is only known after all tiles, partials are kept per row; the finalisation kernel combines
-// tile statistics into global row maxima / sums and contracts partials over the rows:
-//     score[ch] = sum_i partial[ch, i] * exp2(m_tile[i] - m[i]) / l[i].
+// tensor memory). The accumulator is consumed in "panels" of wp columns: one thread per query
+// row pulls its wp values into registers with one round of TMEM loads (the accumulator buffer
+// goes back to the tensor cores as soon as a thread holds its last panel), then computes
+//     the panel row maximum, exp2 of every visible element relative to it, the row sum, and
+//     the sum over each chunk's columns ("partial", one value per row and chunk).
+// Each score element is read once and exponentiated once. The softmax normaliser of a row is
+// only known after all panels, so partials are kept per row; every CTA also folds the
+// (max, sum) pairs of the panels it processed into one record per head and row. The
+// finalisation kernel merges those records into global row maxima / sums and contracts the
+// partials over the rows:
+//     score[ch] = sum_i partial[ch, i] * exp2(m_panel[i] - m[i]) / l[i].
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -26,15 +30,6 @@ constexpr int kThreads = 320;          // warp 0: TMA, warp 1: UMMA issue, warps
 constexpr int kTmemCols = 512;
 constexpr int kQTileBytes = 128 * 128; // 128 query rows x 64 bf16, swizzled 128-byte rows
 
-struct KernelGeom {
-    int n_tiles;      // tiles per head
-    int spt;          // chunk slots per tile
-    int n_stages;
-    int total_tiles;  // Hkv * n_tiles
-    int q_box_rows;   // rows delivered per Q box (min(128, R))
-    int k_box_rows;   // rows delivered per K box (min(n_tile, L))
-};
-
 struct SharedCtl {
     unsigned long long full[kMaxStages];
     unsigned long long empty[kMaxStages];
@@ -46,115 +41,79 @@ struct SharedCtl {
     int abort_flag;
 };
 
-// One thread owns one query row of the tile. `taddr` points at the thread's lane quarter and
-// the first column of the accumulator. All reads use 32- or 16-column TMEM loads.
-// UNROLL_BLOCKS: unroll across the 32-column blocks too, so that column numbers are
-// compile-time constants in `f` (the fast path needs that; the general path does not).
-template <int N_TILE, bool UNROLL_BLOCKS, typename F>
-__device__ __forceinline__ void for_each_column(uint32_t taddr, F&& f) {
-    constexpr int FULL = N_TILE / 32;
-    if constexpr (UNROLL_BLOCKS) {
+// Pull WP consecutive accumulator columns of this thread's row into registers.
+template <int WP>
+__device__ __forceinline__ void load_panel(uint32_t taddr, float (&v)[WP]) {
+    static_assert(WP % 4 == 0, "panel width must be a multiple of 4 columns");
+    int o = 0;
 #pragma unroll
-        for (int b = 0; b < FULL; ++b) {
-            float v[32];
-            tmem_ld_x32(taddr + b * 32, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int u = 0; u < 32; ++u) f(b * 32 + u, v[u]);
-        }
-    } else {
-#pragma unroll 1
-        for (int b = 0; b < FULL; ++b) {
-            float v[32];
-            tmem_ld_x32(taddr + b * 32, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int u = 0; u < 32; ++u) f(b * 32 + u, v[u]);
-        }
-    }
-    if constexpr (N_TILE % 32 != 0) {
-        float v[16];
-        tmem_ld_x16(taddr + FULL * 32, v);
-        tmem_ld_wait();
-#pragma unroll
-        for (int u = 0; u < 16; ++u) f(FULL * 32 + u, v[u]);
-    }
+    for (int b = 0; b < WP / 32; ++b, o += 32) tmem_ld_x32(taddr + o, &v[o]);
+    if constexpr ((WP & 16) != 0) { tmem_ld_x16(taddr + o, &v[o]); o += 16; }
+    if constexpr ((WP & 8) != 0) { tmem_ld_x8(taddr + o, &v[o]); o += 8; }
+    if constexpr ((WP & 4) != 0) { tmem_ld_x4(taddr + o, &v[o]); o += 4; }
+    tmem_ld_wait();
 }
 
-// Tile that lies wholly inside the prefix and starts on a chunk boundary, chunk size known at
-// compile time: every branch below folds away after unrolling.
-template <int C, int N_TILE>
-__device__ __forceinline__ void tile_fast(uint32_t taddr, float sl2, bool active, float* part,
-                                          int row_stride, float* out_m, float* out_l) {
-    float mx = -CUDART_INF_F;
+// Panel that lies wholly inside the prefix and starts on a chunk boundary, chunk size known at
+// compile time: all control flow below folds away after unrolling.
+template <int C, int WP>
+__device__ __forceinline__ void panel_fast(const float (&v)[WP], float sl2, bool active, float* part,
+                                           int row_stride, float* out_m, float* out_l) {
+    float m0 = v[0], m1 = v[1], m2 = v[2], m3 = v[3];
 #pragma unroll
-    for (int cb = 0; cb < N_TILE; cb += 32) {
-        if (cb + 32 <= N_TILE) {
-            float v[32];
-            tmem_ld_x32(taddr + cb, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int u = 0; u < 32; u += 2) mx = fmax3(mx, v[u], v[u + 1]);
-        } else {
-            float v[16];
-            tmem_ld_x16(taddr + cb, v);
-            tmem_ld_wait();
-#pragma unroll
-            for (int u = 0; u < 16; u += 2) mx = fmax3(mx, v[u], v[u + 1]);
-        }
+    for (int u = 4; u + 3 < WP; u += 4) {
+        m0 = fmaxf(m0, v[u]); m1 = fmaxf(m1, v[u + 1]); m2 = fmaxf(m2, v[u + 2]); m3 = fmaxf(m3, v[u + 3]);
     }
+    const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     const float neg_m2 = -mx * sl2;
     float l = 0.f, acc = 0.f;
-    for_each_column<N_TILE, true>(taddr, [&](int j, float x) {
-        const float e = ex2_approx(fmaf(x, sl2, neg_m2));
-        acc += e;
-        if ((j + 1) % C == 0) {
-            if (active) part[static_cast<size_t>((j + 1) / C - 1) * row_stride] = acc;
+#pragma unroll
+    for (int u = 0; u < WP; ++u) {
+        const float e = ex2_approx(fmaf(v[u], sl2, neg_m2));
+        acc = (u % C == 0) ? e : acc + e;
+        if ((u + 1) % C == 0) {
+            if (active) part[static_cast<size_t>((u + 1) / C - 1) * row_stride] = acc;
             l += acc;
-            acc = 0.f;
         }
-    });
+    }
     *out_m = mx * sl2;
     *out_l = l;
 }
 
-// Any tile: run-time chunk size, chunk grid clipped at P, causal mask inside the window
+// Any panel: run-time chunk size, chunk grid clipped at P, causal mask inside the window
 // columns [P, L), nothing visible at or beyond L. Window columns add to the row sum only.
-template <int N_TILE>
-__device__ __forceinline__ void tile_general(uint32_t taddr, float sl2, bool active, float* part,
-                                             int row_stride, int j0, int P, int L, int c, int r,
-                                             float* out_m, float* out_l) {
-    const int last_visible = min(P + r, L - 1);   // this row sees keys j <= P + r
+template <int WP>
+__device__ __forceinline__ void panel_general(const float (&v)[WP], float sl2, bool active, float* part,
+                                              int row_stride, int j0, int P, int c, int last_visible,
+                                              float* out_m, float* out_l) {
     float mx = -CUDART_INF_F;
-    for_each_column<N_TILE, false>(taddr, [&](int u, float x) {
-        const bool vis = (j0 + u) <= last_visible;
-        mx = vis ? fmaxf(mx, x) : mx;
-    });
+#pragma unroll
+    for (int u = 0; u < WP; ++u) mx = (j0 + u <= last_visible) ? fmaxf(mx, v[u]) : mx;
     const float neg_m2 = (mx == -CUDART_INF_F) ? 0.f : -mx * sl2;
     float l = 0.f, acc = 0.f;
-    int slot = 0;
     int nb = (j0 < P) ? min((j0 / c + 1) * c, P) : 0;   // end (exclusive) of the current chunk
-    for_each_column<N_TILE, false>(taddr, [&](int u, float x) {
+    float* dst = part;
+#pragma unroll
+    for (int u = 0; u < WP; ++u) {
         const int j = j0 + u;
-        const bool vis = j <= last_visible;
-        const float e = vis ? ex2_approx(fmaf(x, sl2, neg_m2)) : 0.f;
+        const float e = (j <= last_visible) ? ex2_approx(fmaf(v[u], sl2, neg_m2)) : 0.f;
         if (j < P) {
             acc += e;
             if (j + 1 == nb) {
-                if (active) part[static_cast<size_t>(slot) * row_stride] = acc;
+                if (active) *dst = acc;
+                dst += row_stride;
                 l += acc;
                 acc = 0.f;
-                ++slot;
                 nb = min(nb + c, P);
             }
         } else {
             l += e;
         }
-    });
+    }
     if (j0 < P) {
-        const int je = min(j0 + N_TILE, P);
-        if (je != P && (je % c) != 0) {   // a chunk continues into the next tile: emit its piece
-            if (active) part[static_cast<size_t>(slot) * row_stride] = acc;
+        const int je = min(j0 + WP, P);
+        if (je != P && (je % c) != 0) {   // a chunk continues into the next panel: emit its piece
+            if (active) *dst = acc;
             l += acc;
         }
     }
@@ -162,15 +121,28 @@ __device__ __forceinline__ void tile_general(uint32_t taddr, float sl2, bool act
     *out_l = l;
 }
 
+struct KernelGeom {
+    int n_tiles;      // accumulator tiles per head
+    int spp;          // chunk slots per panel
+    int n_stages;
+    int total_tiles;  // Hkv * n_tiles
+    int q_box_rows;   // rows delivered per Q box (min(128, R))
+    int k_box_rows;   // rows delivered per K box (min(n_tile, L))
+    int hs_max;       // head records per CTA in cta_stat
+};
+
 template <int C_STATIC, int N_MT, int N_TILE>
 __global__ void __launch_bounds__(kThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
              const ScoreArgs a, const KernelGeom g) {
     static_assert(N_MT == 1 || N_MT == 2, "one or two 128-row query tiles");
     static_assert(N_TILE % 16 == 0 && N_TILE * N_MT <= 256, "accumulator tiles must fit half of TMEM");
-    static_assert(C_STATIC == 0 || N_TILE % C_STATIC == 0, "static chunk size must divide the tile");
     constexpr int NQBUF = (N_MT == 1) ? 2 : 1;
     constexpr int TCOLS = 256 / N_MT;              // TMEM columns reserved per accumulator
+    constexpr int GPT = (N_MT == 1) ? 2 : 1;       // epilogue groups sharing a tile's columns
+    constexpr int PPT = GPT * 2;                   // panels per tile: each group takes two in turn
+    constexpr int WP = N_TILE / PPT;               // panel width in keys
+    static_assert(C_STATIC == 0 || WP % C_STATIC == 0, "static chunk size must divide the panel");
     constexpr uint32_t IDESC = umma_idesc_bf16(128, N_TILE);
 
     extern __shared__ uint8_t smem_raw[];
@@ -196,7 +168,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.tfull[b]), 1);
-            mbar_init(smem_u32(&ctl.tempty[b]), 128 * N_MT);
+            mbar_init(smem_u32(&ctl.tempty[b]), 256);
             mbar_init(smem_u32(&ctl.qfull[b]), 1);
             mbar_init(smem_u32(&ctl.qempty[b]), 1);
         }
@@ -306,37 +278,69 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------------ epilogue
-        const int grp = (warp - 2) >> 2;            // 0 or 1
+        // Two groups of four warps. With one query tile, group g takes the left or right half
+        // of every accumulator tile; with two query tiles, group g takes query tile g. A group
+        // walks its columns as two panels in turn (one panel's worth of registers at a time)
+        // and releases the accumulator buffer once the second panel is in registers.
+        const int grp = (warp - 2) >> 2;
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
         const int mt = (N_MT == 2) ? grp : 0;
+        const int half = (N_MT == 2) ? 0 : grp;
         const int row = mt * 128 + quarter * 32 + lane;
         const bool active = row < a.R;
-        const int r = row % a.w;
-        int ti = 0;
+        const int last_visible = a.P + (row % a.w);  // this row sees keys j <= P + r (all < L)
+        const int n_panels = g.n_tiles * PPT;
+        float run_m = -CUDART_INF_F, run_l = 0.f;    // (max, sum) over this thread's panels of the head
+        int cur_head = -1, hs = -1, ti = 0;
+        auto flush_head = [&]() {
+            if (cur_head >= 0 && hs < g.hs_max) {
+                float* rec = a.cta_stat + ((static_cast<size_t>(blockIdx.x) * g.hs_max + hs) * 2 + grp) * 256;
+                rec[quarter * 32 + lane] = run_m;
+                rec[128 + quarter * 32 + lane] = run_l;
+            }
+        };
         for (int t = t_begin; t < t_end; ++t, ++ti) {
-            if (N_MT == 1 && (ti & 1) != grp) continue;
             const int head = t / g.n_tiles, tile = t - head * g.n_tiles;
+            if (head != cur_head) {
+                flush_head();
+                cur_head = head;
+                ++hs;
+                run_m = -CUDART_INF_F;
+                run_l = 0.f;
+            }
             const int buf = ti & 1, use = ti >> 1;
             if (!mbar_wait(smem_u32(&ctl.tfull[buf]), use & 1, abort_flag)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                   static_cast<uint32_t>(buf * 256 + mt * TCOLS);
-            const size_t tile_id = static_cast<size_t>(head) * g.n_tiles + tile;
-            float* part = a.partial + tile_id * g.spt * a.R + row;
-            const int j0 = tile * N_TILE;
-            float m2, l;
-            if (C_STATIC > 0 && j0 + N_TILE <= a.P) {
-                tile_fast<(C_STATIC > 0 ? C_STATIC : 1), N_TILE>(taddr, a.sl2, active, part, a.R, &m2, &l);
-            } else {
-                tile_general<N_TILE>(taddr, a.sl2, active, part, a.R, j0, a.P, a.L, a.c, r, &m2, &l);
-            }
-            tc_fence_before();
-            mbar_arrive(smem_u32(&ctl.tempty[buf]));
-            if (active) {
-                a.stat_m[tile_id * a.R + row] = m2;
-                a.stat_l[tile_id * a.R + row] = l;
+                                   static_cast<uint32_t>(buf * 256 + mt * TCOLS + half * 2 * WP);
+#pragma unroll
+            for (int sub = 0; sub < 2; ++sub) {
+                float v[WP];
+                load_panel<WP>(taddr + sub * WP, v);
+                if (sub == 1) {                      // last read of this buffer by this thread
+                    tc_fence_before();
+                    mbar_arrive(smem_u32(&ctl.tempty[buf]));
+                }
+                const int panel = tile * PPT + half * 2 + sub;
+                const size_t panel_id = static_cast<size_t>(head) * n_panels + panel;
+                float* part = a.partial + panel_id * g.spp * a.R + row;
+                const int j0 = panel * WP;
+                float m2, l;
+                if (C_STATIC > 0 && j0 + WP <= a.P) {
+                    panel_fast<(C_STATIC > 0 ? C_STATIC : 1), WP>(v, a.sl2, active, part, a.R, &m2, &l);
+                } else {
+                    panel_general<WP>(v, a.sl2, active, part, a.R, j0, a.P, a.c, last_visible, &m2, &l);
+                }
+                if (active) a.stat_m[panel_id * a.R + row] = m2;
+                // fold into the running record: l is relative to m2, run_l to run_m
+                const float nm = fmaxf(run_m, m2);
+                const float s_old = (run_m == -CUDART_INF_F) ? 0.f : ex2_approx(run_m - nm);
+                const float s_new = (m2 == -CUDART_INF_F) ? 0.f : ex2_approx(m2 - nm);
+                run_l = run_l * s_old + l * s_new;
+                run_m = nm;
             }
         }
+        flush_head();
     }
 
     tc_fence_before();
@@ -349,51 +353,113 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 }
 
 // ---------------------------------------------------------------------------------------------
-// Finalisation: global row statistics from tile statistics, then one warp per chunk contracts
-// the chunk's partial sums over the R rows. Fixed reduction order, so results are deterministic.
-constexpr int kFinThreads = 256;
+// Finalisation. grid = (blocks per head, Hkv). Each block
+//   1. merges the per-CTA records of its head into global row maxima m[i] and 1 / l[i],
+//   2. computes the scale f[p][i] = exp2(m_panel[p][i] - m[i]) / l[i] for the panels its chunks
+//      touch (kept in shared memory),
+//   3. lets one warp per chunk contract partial[ch][.] * f over the R rows.
+// All reductions have a fixed order, so results are deterministic.
+constexpr int kFinThreads = 512;
+constexpr int kFinPanelCap = 24;      // panels whose scales fit in shared memory (24 x 256 floats)
+
+struct FinGeom {
+    int n_panels;     // per head
+    int spp;
+    int wp;
+    int n_tiles;
+    int n_mt;
+    int score_grid;   // CTAs of the scoring launch
+    int hs_max;
+    int C;
+};
 
 __global__ void __launch_bounds__(kFinThreads)
-finalize_kernel(const ScoreArgs a, int n_tiles, int spt, int n_tile, int C, float* __restrict__ out) {
+finalize_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
     __shared__ float gm[256];
     __shared__ float ginv[256];
+    __shared__ float fs[kFinPanelCap * 256];
     const int h = blockIdx.y;
-    const size_t stat_base = static_cast<size_t>(h) * n_tiles * a.R;
-    for (int i = threadIdx.x; i < a.R; i += blockDim.x) {
+    const int tid = threadIdx.x;
+
+    // 1. global row statistics from the records of the CTAs that touched head h
+    const long long total = static_cast<long long>(a.Hkv) * g.n_tiles;
+    const long long first_tile = static_cast<long long>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
+    // CTA b owns tiles [total*b/G, total*(b+1)/G): the owner of tile T is floor(((T+1)*G - 1) / total)
+    const int b_lo = static_cast<int>(((first_tile + 1) * g.score_grid - 1) / total);
+    const int b_hi = static_cast<int>(((last_tile + 1) * g.score_grid - 1) / total);
+    if (tid < a.R) {
+        const int grp_lo = (g.n_mt == 2) ? (tid >> 7) : 0;
+        const int grp_hi = (g.n_mt == 2) ? (tid >> 7) : 1;
+        const int rr = tid & 127;
         float m = -CUDART_INF_F;
-        for (int t = 0; t < n_tiles; ++t) m = fmaxf(m, a.stat_m[stat_base + static_cast<size_t>(t) * a.R + i]);
-        float l = 0.f;
-        for (int t = 0; t < n_tiles; ++t) {
-            const size_t o = stat_base + static_cast<size_t>(t) * a.R + i;
-            l += a.stat_l[o] * ex2_approx(a.stat_m[o] - m);
+        for (int b = b_lo; b <= b_hi; ++b) {
+            const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
+            const int hs = h - head0;
+            for (int gq = grp_lo; gq <= grp_hi; ++gq) {
+                const float* rec = a.cta_stat + ((static_cast<size_t>(b) * g.hs_max + hs) * 2 + gq) * 256;
+                m = fmaxf(m, rec[rr]);
+            }
         }
-        gm[i] = m;
-        ginv[i] = 1.0f / l;
+        float l = 0.f;
+        for (int b = b_lo; b <= b_hi; ++b) {
+            const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
+            const int hs = h - head0;
+            for (int gq = grp_lo; gq <= grp_hi; ++gq) {
+                const float* rec = a.cta_stat + ((static_cast<size_t>(b) * g.hs_max + hs) * 2 + gq) * 256;
+                const float rm = rec[rr];
+                l += (rm == -CUDART_INF_F) ? 0.f : rec[128 + rr] * ex2_approx(rm - m);
+            }
+        }
+        gm[tid] = m;
+        ginv[tid] = 1.0f / l;
     }
     __syncthreads();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    const int per_block = (C + gridDim.x - 1) / gridDim.x;
-    const int ch0 = blockIdx.x * per_block, ch1 = min(ch0 + per_block, C);
+
+    // 2. scales of the panels this block's chunks touch
+    const int per_block = (g.C + gridDim.x - 1) / gridDim.x;
+    const int ch0 = blockIdx.x * per_block, ch1 = min(ch0 + per_block, g.C);
+    if (ch0 >= ch1) return;
+    const int p_lo = (ch0 * a.c) / g.wp;
+    const int p_hi = (min(ch1 * a.c, a.P) - 1) / g.wp;
+    const bool staged = (p_hi - p_lo + 1) <= kFinPanelCap;
+    const size_t stat_base = static_cast<size_t>(h) * g.n_panels * a.R;
+    if (staged) {
+        const int n = (p_hi - p_lo + 1) * a.R;
+        for (int e = tid; e < n; e += blockDim.x) {
+            const int pp = e / a.R, i = e - pp * a.R;
+            fs[pp * 256 + i] =
+                ex2_approx(a.stat_m[stat_base + static_cast<size_t>(p_lo + pp) * a.R + i] - gm[i]) * ginv[i];
+        }
+    }
+    __syncthreads();
+
+    // 3. one warp per chunk
+    const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
     for (int ch = ch0 + warp; ch < ch1; ch += nwarps) {
         const int ja = ch * a.c, jb = min(ja + a.c, a.P);
-        const int t0 = ja / n_tile, t1 = (jb - 1) / n_tile;
+        const int pa = ja / g.wp, pb = (jb - 1) / g.wp;
         float acc = 0.f;
-        for (int t = t0; t <= t1; ++t) {
-            const int slot = ch - (t * n_tile) / a.c;
-            const size_t so = stat_base + static_cast<size_t>(t) * a.R;
-            const size_t po = ((static_cast<size_t>(h) * n_tiles + t) * spt + slot) * a.R;
-            for (int i = lane; i < a.R; i += 32)
-                acc += a.partial[po + i] * ex2_approx(a.stat_m[so + i] - gm[i]) * ginv[i];
+        for (int p = pa; p <= pb; ++p) {
+            const int slot = ch - (p * g.wp) / a.c;
+            const size_t po = ((static_cast<size_t>(h) * g.n_panels + p) * g.spp + slot) * a.R;
+            if (staged) {
+                const float* f = &fs[(p - p_lo) * 256];
+                for (int i = lane; i < a.R; i += 32) acc += a.partial[po + i] * f[i];
+            } else {
+                const size_t so = stat_base + static_cast<size_t>(p) * a.R;
+                for (int i = lane; i < a.R; i += 32)
+                    acc += a.partial[po + i] * (ex2_approx(a.stat_m[so + i] - gm[i]) * ginv[i]);
+            }
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (lane == 0) out[static_cast<size_t>(h) * C + ch] = acc;
+        if (lane == 0) out[static_cast<size_t>(h) * g.C + ch] = acc;
     }
 }
 
 template <int C_STATIC, int N_MT, int N_TILE>
 cudaError_t launch_variant(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                           const ScoreArgs& args, int num_sms, cudaStream_t stream) {
+                           const ScoreArgs& args, cudaStream_t stream) {
     auto kern = score_kernel<C_STATIC, N_MT, N_TILE>;
     // Opt in to large dynamic shared memory once per device and variant (not a stream operation,
     // so later launches stay free of it, e.g. inside a stream capture).
@@ -408,30 +474,36 @@ cudaError_t launch_variant(const ScorePlan& plan, const CUtensorMap& tm_q, const
     }
     KernelGeom g;
     g.n_tiles = plan.n_tiles;
-    g.spt = plan.spt;
+    g.spp = plan.spp;
     g.n_stages = plan.n_stages;
     g.total_tiles = args.Hkv * plan.n_tiles;
     g.q_box_rows = args.R < 128 ? args.R : 128;
     g.k_box_rows = args.L < N_TILE ? args.L : N_TILE;
-    const int grid = g.total_tiles < num_sms ? g.total_tiles : num_sms;
-    kern<<<grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_k, args, g);
+    g.hs_max = plan.hs_max;
+    kern<<<plan.grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_k, args, g);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-bool make_score_plan(int L, int R, int d, int c, int smem_limit, ScorePlan* plan) {
-    if (R < 1 || R > 256 || (d != 64 && d != 128) || c < 1 || L < 1) return false;
+bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_limit, ScorePlan* plan) {
+    if (R < 1 || R > 256 || (d != 64 && d != 128) || c < 1 || L < 1 || Hkv < 1 || num_sms < 1) return false;
     ScorePlan p{};
     p.n_mt = (R + 127) / 128;
-    // Chunk sizes with a compiled-in variant use a tile that is a multiple of lcm(c, 16);
+    // Chunk sizes with a compiled-in variant use panels that are a multiple of the chunk size;
     // every other chunk size runs the run-time-c variant on the widest tile.
     p.c_static = 0;
     if (p.n_mt == 1 && (c == 10 || c == 20)) { p.c_static = c; p.n_tile = 240; }
     else if (p.n_mt == 1 && c == 1) { p.c_static = 1; p.n_tile = 256; }
     else p.n_tile = 256 / p.n_mt;
+    p.wp = (p.n_mt == 1) ? p.n_tile / 4 : p.n_tile / 2;
     p.n_tiles = (L + p.n_tile - 1) / p.n_tile;
-    p.spt = p.c_static ? p.n_tile / p.c_static : (p.n_tile + c - 1) / c + 1;
+    p.n_panels = p.n_tiles * (p.n_tile / p.wp);
+    p.spp = p.c_static ? p.wp / p.c_static : (p.wp + c - 1) / c + 1;
+    const long long total = static_cast<long long>(Hkv) * p.n_tiles;
+    p.grid = static_cast<int>(total < num_sms ? total : num_sms);
+    const int tiles_per_cta = static_cast<int>((total + p.grid - 1) / p.grid);
+    p.hs_max = (tiles_per_cta + p.n_tiles - 1) / p.n_tiles + 1;
     const int KB = d / 64;
     const int nqbuf = p.n_mt == 1 ? 2 : 1;
     const int q_bytes = nqbuf * p.n_mt * KB * kQTileBytes;
@@ -446,30 +518,46 @@ bool make_score_plan(int L, int R, int d, int c, int smem_limit, ScorePlan* plan
 }
 
 size_t score_scratch_floats(const ScorePlan& plan, int Hkv, int R) {
-    const size_t tiles = static_cast<size_t>(Hkv) * plan.n_tiles;
-    return tiles * R * 2 + tiles * plan.spt * R;
+    const size_t panels = static_cast<size_t>(Hkv) * plan.n_panels;
+    return panels * R + static_cast<size_t>(plan.grid) * plan.hs_max * 512 + panels * plan.spp * R;
+}
+
+void score_scratch_layout(const ScorePlan& plan, int Hkv, int R, float* base, ScoreArgs* args) {
+    const size_t panels = static_cast<size_t>(Hkv) * plan.n_panels;
+    args->stat_m = base;
+    args->cta_stat = base + panels * R;
+    args->partial = args->cta_stat + static_cast<size_t>(plan.grid) * plan.hs_max * 512;
 }
 
 cudaError_t launch_score(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                         const ScoreArgs& args, int num_sms, cudaStream_t stream) {
+                         const ScoreArgs& args, cudaStream_t stream) {
     if (plan.n_mt == 1) {
-        if (plan.c_static == 10) return launch_variant<10, 1, 240>(plan, tm_q, tm_k, args, num_sms, stream);
-        if (plan.c_static == 20) return launch_variant<20, 1, 240>(plan, tm_q, tm_k, args, num_sms, stream);
-        if (plan.c_static == 1) return launch_variant<1, 1, 256>(plan, tm_q, tm_k, args, num_sms, stream);
-        return launch_variant<0, 1, 256>(plan, tm_q, tm_k, args, num_sms, stream);
+        if (plan.c_static == 10) return launch_variant<10, 1, 240>(plan, tm_q, tm_k, args, stream);
+        if (plan.c_static == 20) return launch_variant<20, 1, 240>(plan, tm_q, tm_k, args, stream);
+        if (plan.c_static == 1) return launch_variant<1, 1, 256>(plan, tm_q, tm_k, args, stream);
+        return launch_variant<0, 1, 256>(plan, tm_q, tm_k, args, stream);
     }
-    return launch_variant<0, 2, 128>(plan, tm_q, tm_k, args, num_sms, stream);
+    return launch_variant<0, 2, 128>(plan, tm_q, tm_k, args, stream);
 }
 
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
                             int num_sms, cudaStream_t stream) {
     if (C <= 0) return cudaSuccess;
     int bx = (2 * num_sms + args.Hkv - 1) / args.Hkv;
-    const int max_bx = (C + 7) / 8;
+    const int max_bx = (C + 15) / 16;
     if (bx > max_bx) bx = max_bx;
     if (bx < 1) bx = 1;
+    FinGeom g;
+    g.n_panels = plan.n_panels;
+    g.spp = plan.spp;
+    g.wp = plan.wp;
+    g.n_tiles = plan.n_tiles;
+    g.n_mt = plan.n_mt;
+    g.score_grid = plan.grid;
+    g.hs_max = plan.hs_max;
+    g.C = C;
     dim3 grid(bx, args.Hkv);
-    finalize_kernel<<<grid, kFinThreads, 0, stream>>>(args, plan.n_tiles, plan.spt, plan.n_tile, C, out_scores);
+    finalize_kernel<<<grid, kFinThreads, 0, stream>>>(args, g, out_scores);
     return cudaGetLastError();
 }
 

@@ -2,9 +2,11 @@
 // the selection mask, "always keep most recent tokens", "nonzero(mask)").
 //
 // One CTA per KV head. The k-th largest score is found by an exact 4-pass radix select on
-// order-preserving 32-bit keys; a single ordered sweep then keeps every chunk above the
-// threshold plus the lowest-numbered chunks equal to it until k are kept, and writes their token
-// positions directly in ascending order - no mask, no sort and no compaction of a mask.
+// order-preserving 32-bit keys (warp-aggregated shared-memory histograms, one warp scanning
+// the 256 bins). Each thread then owns a contiguous run of chunk ids; one block-wide prefix
+// sum over (#above threshold, #equal to threshold) gives every chunk its rank among the kept
+// ones: rank = #above before it + min(#equal before it, ties to keep) - ties go to the lower
+// chunk id. Token positions are written directly in ascending order: no mask, no sort.
 #include "internal.h"
 
 namespace chunkkv {
@@ -12,47 +14,21 @@ namespace chunkkv {
 namespace {
 
 constexpr int kSelThreads = 1024;
+constexpr int kKeyCap = 6912;      // chunk keys staged in shared memory (27 KB); more are re-read
+constexpr int kSelCap = 4096;      // kept-chunk ids staged for coalesced index writes
 
 __device__ __forceinline__ uint32_t order_key(float x) {
     const uint32_t b = __float_as_uint(x + 0.0f);          // -0 and +0 compare equal
-    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);   // larger float <=> larger key
-}
-
-// Exclusive prefix sum of one int per thread across the CTA; also returns the CTA total.
-// warp_sums must hold 33 ints. Ends with a barrier, so warp_sums can be reused at once.
-__device__ __forceinline__ int block_exclusive_scan(int v, int* warp_sums, int* total) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    int inc = v;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const int n = __shfl_up_sync(0xffffffffu, inc, off);
-        if (lane >= off) inc += n;
-    }
-    if (lane == 31) warp_sums[warp] = inc;
-    __syncthreads();
-    if (warp == 0) {
-        const int s = warp_sums[lane];
-        int sinc = s;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int n = __shfl_up_sync(0xffffffffu, sinc, off);
-            if (lane >= off) sinc += n;
-        }
-        warp_sums[lane] = sinc - s;            // exclusive warp offsets
-        if (lane == 31) warp_sums[32] = sinc;  // total
-    }
-    __syncthreads();
-    const int res = warp_sums[warp] + inc - v;
-    *total = warp_sums[32];
-    __syncthreads();
-    return res;
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);     // larger float <=> larger key
 }
 
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int k, int n_max,
               int32_t* __restrict__ out_idx) {
+    __shared__ uint32_t keys_s[kKeyCap];
+    __shared__ int sel_s[kSelCap];
     __shared__ int hist[256];
-    __shared__ int warp_sums[33];
+    __shared__ unsigned long long warp_sums[33];
     __shared__ uint32_t s_prefix;
     __shared__ int s_need;
     __shared__ int s_last_kept;
@@ -60,12 +36,18 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
     const int P = L - w;
     const float* sc = scores + static_cast<size_t>(h) * C;
     int32_t* out = out_idx + static_cast<size_t>(h) * n_max;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool cached = C <= kKeyCap;
+    const bool keep_all = (k >= C);
 
     if (tid == 0) s_last_kept = 0;
+    if (cached && k > 0 && !keep_all)
+        for (int i = tid; i < C; i += kSelThreads) keys_s[i] = order_key(sc[i]);
+    __syncthreads();
+    auto key_at = [&](int i) -> uint32_t { return cached ? keys_s[i] : order_key(sc[i]); };
+
     uint32_t thresh = 0;   // key of the k-th largest score
     int need_eq = 0;       // how many chunks equal to the threshold are kept
-    const bool keep_all = (k >= C);
     if (!keep_all && k > 0) {
         uint32_t prefix = 0;
         int need = k;
@@ -74,16 +56,36 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
             if (tid < 256) hist[tid] = 0;
             __syncthreads();
             const uint32_t himask = (pass == 0) ? 0u : (0xFFFFFFFFu << (shift + 8));
-            for (int i = tid; i < C; i += blockDim.x) {
-                const uint32_t key = order_key(sc[i]);
-                if ((key & himask) == prefix) atomicAdd(&hist[(key >> shift) & 0xFF], 1);
+            for (int base = 0; base < C; base += kSelThreads) {
+                const int i = base + tid;
+                uint32_t key = 0;
+                bool in = false;
+                if (i < C) { key = key_at(i); in = (key & himask) == prefix; }
+                // lanes of a warp that hit the same bin add once
+                const int bin = in ? static_cast<int>((key >> shift) & 0xFF) : -1;
+                const unsigned peers = __match_any_sync(0xffffffffu, bin);
+                if (in && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
             }
             __syncthreads();
-            if (tid == 0) {
-                int b = 255, above = 0;
-                while (b > 0 && above + hist[b] < need) { above += hist[b]; --b; }
-                s_prefix = prefix | (static_cast<uint32_t>(b) << shift);
-                s_need = need - above;
+            if (warp == 0) {
+                // lane t owns bins 255-8t .. 248-8t (descending), so a prefix over lanes counts from the top
+                int cnt[8], sum = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) { cnt[q] = hist[255 - 8 * lane - q]; sum += cnt[q]; }
+                int inc = sum;
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const int n = __shfl_up_sync(0xffffffffu, inc, off);
+                    if (lane >= off) inc += n;
+                }
+                const unsigned reach = __ballot_sync(0xffffffffu, inc >= need);
+                const int owner = reach ? (__ffs(reach) - 1) : 31;
+                if (lane == owner) {
+                    int above = inc - sum, q = 0;
+                    while (q < 7 && above + cnt[q] < need) { above += cnt[q]; ++q; }
+                    s_prefix = prefix | (static_cast<uint32_t>(255 - 8 * lane - q) << shift);
+                    s_need = need - above;
+                }
             }
             __syncthreads();
             prefix = s_prefix;
@@ -92,44 +94,76 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
         thresh = prefix;
         need_eq = need;
     }
-    __syncthreads();
 
-    // Ordered sweep over chunk ids: running counts of kept chunks and of threshold ties.
-    if (k > 0) {
-        int kept_before = 0, eq_before = 0;
-        for (int base = 0; base < C; base += blockDim.x) {
-            const int ch = base + tid;
-            bool gt = false, eq = false;
-            if (ch < C) {
-                if (keep_all) gt = true;
-                else {
-                    const uint32_t key = order_key(sc[ch]);
-                    gt = key > thresh;
-                    eq = key == thresh;
-                }
+    // Ordered sweep: thread t owns chunk ids [t * per, (t + 1) * per).
+    const int kk = min(k, C);
+    const bool stage_sel = kk <= kSelCap;
+    if (kk > 0) {
+        const int per = (C + kSelThreads - 1) / kSelThreads;
+        const int c0 = min(tid * per, C), c1 = min(c0 + per, C);
+        unsigned gt_n = 0, eq_n = 0;
+        if (keep_all) gt_n = c1 - c0;
+        else
+            for (int ch = c0; ch < c1; ++ch) {
+                const uint32_t key = key_at(ch);
+                gt_n += key > thresh;
+                eq_n += key == thresh;
             }
-            int eq_total;
-            const int eq_rank = eq_before + block_exclusive_scan(eq ? 1 : 0, warp_sums, &eq_total);
-            const bool keep = gt || (eq && eq_rank < need_eq);
-            int keep_total;
-            const int rank = kept_before + block_exclusive_scan(keep ? 1 : 0, warp_sums, &keep_total);
-            if (keep) {
-                const int j0 = ch * c;
-                const int len = min(c, P - j0);                        // only chunk C-1 can be short
-                int32_t* dst = out + static_cast<size_t>(rank) * c;    // and it is the last one kept
-                for (int t = 0; t < len; ++t) dst[t] = j0 + t;
+        // block-wide exclusive prefix of the packed pair (eq in the high half, gt in the low half)
+        const unsigned long long mine = (static_cast<unsigned long long>(eq_n) << 32) | gt_n;
+        unsigned long long inc = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += n;
+        }
+        if (lane == 31) warp_sums[warp] = inc;
+        __syncthreads();
+        if (warp == 0) {
+            const unsigned long long s = warp_sums[lane];
+            unsigned long long sinc = s;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned long long n = __shfl_up_sync(0xffffffffu, sinc, off);
+                if (lane >= off) sinc += n;
+            }
+            warp_sums[lane] = sinc - s;
+        }
+        __syncthreads();
+        const unsigned long long excl = warp_sums[warp] + inc - mine;
+        int gt_before = static_cast<int>(excl & 0xffffffffu), eq_before = static_cast<int>(excl >> 32);
+        for (int ch = c0; ch < c1; ++ch) {
+            bool gt = keep_all, eq = false;
+            if (!keep_all) {
+                const uint32_t key = key_at(ch);
+                gt = key > thresh;
+                eq = key == thresh;
+            }
+            if (gt || (eq && eq_before < need_eq)) {
+                const int rank = gt_before + min(eq_before, need_eq);
+                if (stage_sel) sel_s[rank] = ch;
+                else {
+                    const int j0 = ch * c, len = min(c, P - j0);
+                    int32_t* dst = out + static_cast<size_t>(rank) * c;
+                    for (int t = 0; t < len; ++t) dst[t] = j0 + t;
+                }
                 if (ch == C - 1) s_last_kept = 1;
             }
-            kept_before += keep_total;
-            eq_before += eq_total;
+            gt_before += gt;
+            eq_before += eq;
         }
     }
     __syncthreads();
-    const int kk = min(k, C);
-    const int tail = (C > 0) ? (P - (C - 1) * c) : 0;            // length of chunk C-1
+    // Every kept chunk is full except possibly chunk C-1, which can only be the last kept one.
+    const int tail = (C > 0) ? (P - (C - 1) * c) : 0;
     const int n_tok = kk * c - ((s_last_kept && kk > 0) ? (c - tail) : 0);
-    for (int i = tid; i < w; i += blockDim.x) out[n_tok + i] = P + i;
-    for (int i = n_tok + w + tid; i < n_max; i += blockDim.x) out[i] = -1;
+    if (stage_sel)
+        for (int n = tid; n < n_tok; n += kSelThreads) {
+            const int rank = n / c;
+            out[n] = sel_s[rank] * c + (n - rank * c);
+        }
+    for (int i = tid; i < w; i += kSelThreads) out[n_tok + i] = P + i;
+    for (int i = n_tok + w + tid; i < n_max; i += kSelThreads) out[i] = -1;
 }
 
 }  // namespace
