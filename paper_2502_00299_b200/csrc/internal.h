@@ -12,7 +12,7 @@ struct ScorePlan {
     int c_static;   // chunk size baked into the kernel (0 = run-time chunk size)
     int n_mt;       // 128-row query tiles per KV head (1 or 2)
     int n_tile;     // keys per accumulator tile (one UMMA N)
-    int wp;         // keys per epilogue panel (n_tile / 4 with one query tile, else n_tile / 2)
+    int wp;         // keys per epilogue panel (n_tile / 4 with one query tile, n_tile / 2 with two)
     int n_tiles;    // accumulator tiles per head = ceil(L / n_tile)
     int n_panels;   // panels per head
     int spp;        // chunk slots per panel in the partial-sum scratch
@@ -26,7 +26,7 @@ struct ScoreArgs {
     int L, P, w, c, R, Hkv, d;
     float sl2;            // log2(e) / sqrt(d)
     float* stat_m;        // [Hkv, n_panels, R] panel row maxima (log2 domain)
-    float* cta_stat;      // [grid, hs_max, 2 groups, {max, sum}, 128] per-CTA folded row statistics
+    float* cta_stat;      // [grid, hs_max, 4 groups, {max, sum}, 128] per-CTA folded row statistics
     float* partial;       // [Hkv, n_panels, spp, R] chunk partial sums relative to the panel maximum
     int* status;          // device status word
 };

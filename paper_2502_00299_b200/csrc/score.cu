@@ -26,7 +26,8 @@ namespace chunkkv {
 namespace {
 
 constexpr int kMaxStages = 16;
-constexpr int kThreads = 320;          // warp 0: TMA, warp 1: UMMA issue, warps 2..9: epilogue
+constexpr int kThreads = 576;          // warp 0: TMA, warp 1: UMMA issue, warps 2..17: epilogue
+constexpr int kGroups = 4;             // epilogue groups of four warps (one warp per TMEM lane quarter)
 constexpr int kTmemCols = 512;
 constexpr int kQTileBytes = 128 * 128; // 128 query rows x 64 bf16, swizzled 128-byte rows
 
@@ -139,8 +140,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     static_assert(N_TILE % 16 == 0 && N_TILE * N_MT <= 256, "accumulator tiles must fit half of TMEM");
     constexpr int NQBUF = (N_MT == 1) ? 2 : 1;
     constexpr int TCOLS = 256 / N_MT;              // TMEM columns reserved per accumulator
-    constexpr int GPT = (N_MT == 1) ? 2 : 1;       // epilogue groups sharing a tile's columns
-    constexpr int PPT = GPT * 2;                   // panels per tile: each group takes two in turn
+    constexpr int PPT = kGroups / N_MT;            // panels per tile = groups sharing a query tile
     constexpr int WP = N_TILE / PPT;               // panel width in keys
     static_assert(C_STATIC == 0 || WP % C_STATIC == 0, "static chunk size must divide the panel");
     constexpr uint32_t IDESC = umma_idesc_bf16(128, N_TILE);
@@ -168,7 +168,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.tfull[b]), 1);
-            mbar_init(smem_u32(&ctl.tempty[b]), 256);
+            mbar_init(smem_u32(&ctl.tempty[b]), 128 * kGroups);
             mbar_init(smem_u32(&ctl.qfull[b]), 1);
             mbar_init(smem_u32(&ctl.qempty[b]), 1);
         }
@@ -278,14 +278,14 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------------ epilogue
-        // Two groups of four warps. With one query tile, group g takes the left or right half
-        // of every accumulator tile; with two query tiles, group g takes query tile g. A group
-        // walks its columns as two panels in turn (one panel's worth of registers at a time)
-        // and releases the accumulator buffer once the second panel is in registers.
+        // Four groups of four warps; a group's warps cover the four TMEM lane quarters, i.e. the
+        // 128 rows of one query tile. With one query tile the groups split the tile's columns
+        // into four panels; with two query tiles, two groups (two panels) serve each of them.
+        // A thread pulls its panel into registers and releases the accumulator buffer at once.
         const int grp = (warp - 2) >> 2;
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
-        const int mt = (N_MT == 2) ? grp : 0;
-        const int half = (N_MT == 2) ? 0 : grp;
+        const int mt = grp / PPT;
+        const int pit = grp % PPT;                  // panel within the tile
         const int row = mt * 128 + quarter * 32 + lane;
         const bool active = row < a.R;
         const int last_visible = a.P + (row % a.w);  // this row sees keys j <= P + r (all < L)
@@ -294,7 +294,8 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         int cur_head = -1, hs = -1, ti = 0;
         auto flush_head = [&]() {
             if (cur_head >= 0 && hs < g.hs_max) {
-                float* rec = a.cta_stat + ((static_cast<size_t>(blockIdx.x) * g.hs_max + hs) * 2 + grp) * 256;
+                float* rec = a.cta_stat +
+                             ((static_cast<size_t>(blockIdx.x) * g.hs_max + hs) * kGroups + grp) * 256;
                 rec[quarter * 32 + lane] = run_m;
                 rec[128 + quarter * 32 + lane] = run_l;
             }
@@ -312,33 +313,29 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             if (!mbar_wait(smem_u32(&ctl.tfull[buf]), use & 1, abort_flag)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                   static_cast<uint32_t>(buf * 256 + mt * TCOLS + half * 2 * WP);
-#pragma unroll
-            for (int sub = 0; sub < 2; ++sub) {
-                float v[WP];
-                load_panel<WP>(taddr + sub * WP, v);
-                if (sub == 1) {                      // last read of this buffer by this thread
-                    tc_fence_before();
-                    mbar_arrive(smem_u32(&ctl.tempty[buf]));
-                }
-                const int panel = tile * PPT + half * 2 + sub;
-                const size_t panel_id = static_cast<size_t>(head) * n_panels + panel;
-                float* part = a.partial + panel_id * g.spp * a.R + row;
-                const int j0 = panel * WP;
-                float m2, l;
-                if (C_STATIC > 0 && j0 + WP <= a.P) {
-                    panel_fast<(C_STATIC > 0 ? C_STATIC : 1), WP>(v, a.sl2, active, part, a.R, &m2, &l);
-                } else {
-                    panel_general<WP>(v, a.sl2, active, part, a.R, j0, a.P, a.c, last_visible, &m2, &l);
-                }
-                if (active) a.stat_m[panel_id * a.R + row] = m2;
-                // fold into the running record: l is relative to m2, run_l to run_m
-                const float nm = fmaxf(run_m, m2);
-                const float s_old = (run_m == -CUDART_INF_F) ? 0.f : ex2_approx(run_m - nm);
-                const float s_new = (m2 == -CUDART_INF_F) ? 0.f : ex2_approx(m2 - nm);
-                run_l = run_l * s_old + l * s_new;
-                run_m = nm;
+                                   static_cast<uint32_t>(buf * 256 + mt * TCOLS + pit * WP);
+            float v[WP];
+            load_panel<WP>(taddr, v);
+            tc_fence_before();
+            mbar_arrive(smem_u32(&ctl.tempty[buf]));   // the tensor cores may overwrite the buffer now
+
+            const int panel = tile * PPT + pit;
+            const size_t panel_id = static_cast<size_t>(head) * n_panels + panel;
+            float* part = a.partial + panel_id * g.spp * a.R + row;
+            const int j0 = panel * WP;
+            float m2, l;
+            if (C_STATIC > 0 && j0 + WP <= a.P) {
+                panel_fast<(C_STATIC > 0 ? C_STATIC : 1), WP>(v, a.sl2, active, part, a.R, &m2, &l);
+            } else {
+                panel_general<WP>(v, a.sl2, active, part, a.R, j0, a.P, a.c, last_visible, &m2, &l);
             }
+            if (active) a.stat_m[panel_id * a.R + row] = m2;
+            // fold into the running record: l is relative to m2, run_l to run_m
+            const float nm = fmaxf(run_m, m2);
+            const float s_old = (run_m == -CUDART_INF_F) ? 0.f : ex2_approx(run_m - nm);
+            const float s_new = (m2 == -CUDART_INF_F) ? 0.f : ex2_approx(m2 - nm);
+            run_l = run_l * s_old + l * s_new;
+            run_m = nm;
         }
         flush_head();
     }
@@ -354,13 +351,15 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 
 // ---------------------------------------------------------------------------------------------
 // Finalisation. grid = (blocks per head, Hkv). Each block
-//   1. merges the per-CTA records of its head into global row maxima m[i] and 1 / l[i],
+//   1. merges the per-CTA records of its head into global row maxima m[i] and 1 / l[i]
+//      (every thread takes a slice of the records of one row, so the loads overlap),
 //   2. computes the scale f[p][i] = exp2(m_panel[p][i] - m[i]) / l[i] for the panels its chunks
 //      touch (kept in shared memory),
-//   3. lets one warp per chunk contract partial[ch][.] * f over the R rows.
+//   3. contracts partial[ch][.] * f over the R rows, one warp working on four chunks at a time.
 // All reductions have a fixed order, so results are deterministic.
 constexpr int kFinThreads = 512;
 constexpr int kFinPanelCap = 24;      // panels whose scales fit in shared memory (24 x 256 floats)
+constexpr int kFinBatch = 4;          // chunks a warp reduces together
 
 struct FinGeom {
     int n_panels;     // per head
@@ -377,41 +376,63 @@ __global__ void __launch_bounds__(kFinThreads)
 finalize_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
     __shared__ float gm[256];
     __shared__ float ginv[256];
+    __shared__ float red[kFinThreads];
+    __shared__ int rec_base[160];
     __shared__ float fs[kFinPanelCap * 256];
     const int h = blockIdx.y;
     const int tid = threadIdx.x;
 
-    // 1. global row statistics from the records of the CTAs that touched head h
+    // 1. global row statistics from the records of the CTAs that touched head h.
+    // CTA b owns tiles [total*b/G, total*(b+1)/G): the owner of tile T is floor(((T+1)*G - 1) / total).
     const long long total = static_cast<long long>(a.Hkv) * g.n_tiles;
     const long long first_tile = static_cast<long long>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
-    // CTA b owns tiles [total*b/G, total*(b+1)/G): the owner of tile T is floor(((T+1)*G - 1) / total)
     const int b_lo = static_cast<int>(((first_tile + 1) * g.score_grid - 1) / total);
     const int b_hi = static_cast<int>(((last_tile + 1) * g.score_grid - 1) / total);
-    if (tid < a.R) {
-        const int grp_lo = (g.n_mt == 2) ? (tid >> 7) : 0;
-        const int grp_hi = (g.n_mt == 2) ? (tid >> 7) : 1;
-        const int rr = tid & 127;
+    const int nb = b_hi - b_lo + 1;
+    for (int j = tid; j < nb; j += kFinThreads) {
+        const int b = b_lo + j;
+        const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
+        rec_base[j % 160] = (b * g.hs_max + (h - head0)) * (kGroups * 256);
+    }
+    __syncthreads();
+    const int rp = (a.R > 128) ? 256 : 128;         // rows padded to the slice stride
+    const int ns = kFinThreads / rp;                // record slices per row
+    const int gpr = kGroups / g.n_mt;               // groups (records per CTA) that hold a given row
+    {
+        const int i = tid % rp, sl = tid / rp;
+        const int g0 = (g.n_mt == 2) ? (i >> 7) * gpr : 0;
+        const int rr = i & 127;
+        const int nrec = nb * gpr;
         float m = -CUDART_INF_F;
-        for (int b = b_lo; b <= b_hi; ++b) {
-            const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
-            const int hs = h - head0;
-            for (int gq = grp_lo; gq <= grp_hi; ++gq) {
-                const float* rec = a.cta_stat + ((static_cast<size_t>(b) * g.hs_max + hs) * 2 + gq) * 256;
+        if (i < a.R) {
+#pragma unroll 4
+            for (int q = sl; q < nrec; q += ns) {
+                const float* rec = a.cta_stat + rec_base[(q / gpr) % 160] + (g0 + q % gpr) * 256;
                 m = fmaxf(m, rec[rr]);
             }
         }
+        red[tid] = m;
+        __syncthreads();
+        float M = red[i];
+        for (int s2 = 1; s2 < ns; ++s2) M = fmaxf(M, red[s2 * rp + i]);
+        __syncthreads();
         float l = 0.f;
-        for (int b = b_lo; b <= b_hi; ++b) {
-            const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
-            const int hs = h - head0;
-            for (int gq = grp_lo; gq <= grp_hi; ++gq) {
-                const float* rec = a.cta_stat + ((static_cast<size_t>(b) * g.hs_max + hs) * 2 + gq) * 256;
+        if (i < a.R) {
+#pragma unroll 4
+            for (int q = sl; q < nrec; q += ns) {
+                const float* rec = a.cta_stat + rec_base[(q / gpr) % 160] + (g0 + q % gpr) * 256;
                 const float rm = rec[rr];
-                l += (rm == -CUDART_INF_F) ? 0.f : rec[128 + rr] * ex2_approx(rm - m);
+                l += (rm == -CUDART_INF_F) ? 0.f : rec[128 + rr] * ex2_approx(rm - M);
             }
         }
-        gm[tid] = m;
-        ginv[tid] = 1.0f / l;
+        red[tid] = l;
+        __syncthreads();
+        if (sl == 0 && i < a.R) {
+            float lt = red[i];
+            for (int s2 = 1; s2 < ns; ++s2) lt += red[s2 * rp + i];
+            gm[i] = M;
+            ginv[i] = 1.0f / lt;
+        }
     }
     __syncthreads();
 
@@ -425,7 +446,7 @@ finalize_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
     const size_t stat_base = static_cast<size_t>(h) * g.n_panels * a.R;
     if (staged) {
         const int n = (p_hi - p_lo + 1) * a.R;
-        for (int e = tid; e < n; e += blockDim.x) {
+        for (int e = tid; e < n; e += kFinThreads) {
             const int pp = e / a.R, i = e - pp * a.R;
             fs[pp * 256 + i] =
                 ex2_approx(a.stat_m[stat_base + static_cast<size_t>(p_lo + pp) * a.R + i] - gm[i]) * ginv[i];
@@ -433,27 +454,48 @@ finalize_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
     }
     __syncthreads();
 
-    // 3. one warp per chunk
-    const int warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
-    for (int ch = ch0 + warp; ch < ch1; ch += nwarps) {
-        const int ja = ch * a.c, jb = min(ja + a.c, a.P);
-        const int pa = ja / g.wp, pb = (jb - 1) / g.wp;
-        float acc = 0.f;
-        for (int p = pa; p <= pb; ++p) {
-            const int slot = ch - (p * g.wp) / a.c;
-            const size_t po = ((static_cast<size_t>(h) * g.n_panels + p) * g.spp + slot) * a.R;
-            if (staged) {
-                const float* f = &fs[(p - p_lo) * 256];
-                for (int i = lane; i < a.R; i += 32) acc += a.partial[po + i] * f[i];
-            } else {
-                const size_t so = stat_base + static_cast<size_t>(p) * a.R;
-                for (int i = lane; i < a.R; i += 32)
-                    acc += a.partial[po + i] * (ex2_approx(a.stat_m[so + i] - gm[i]) * ginv[i]);
+    // 3. chunks -> scores
+    const int warp = tid >> 5, lane = tid & 31, nwarps = kFinThreads >> 5;
+    const size_t part_base = static_cast<size_t>(h) * g.n_panels * g.spp * a.R;
+    for (int cb = ch0 + warp * kFinBatch; cb < ch1; cb += nwarps * kFinBatch) {
+        float acc[kFinBatch];
+        bool single = staged;
+        int pa[kFinBatch];
+        size_t po[kFinBatch];
+#pragma unroll
+        for (int u = 0; u < kFinBatch; ++u) {
+            const int ch = min(cb + u, ch1 - 1);
+            const int ja = ch * a.c, jb = min(ja + a.c, a.P);
+            pa[u] = ja / g.wp;
+            single = single && (pa[u] == (jb - 1) / g.wp);
+            po[u] = part_base + (static_cast<size_t>(pa[u]) * g.spp + (ch - (pa[u] * g.wp) / a.c)) * a.R;
+            acc[u] = 0.f;
+        }
+        if (single) {       // every chunk of the batch lies in one panel: all loads are independent
+            for (int i = lane; i < a.R; i += 32) {
+#pragma unroll
+                for (int u = 0; u < kFinBatch; ++u) acc[u] += a.partial[po[u] + i] * fs[(pa[u] - p_lo) * 256 + i];
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < kFinBatch; ++u) {
+                const int ch = min(cb + u, ch1 - 1);
+                const int ja = ch * a.c, jb = min(ja + a.c, a.P);
+                for (int p = ja / g.wp; p <= (jb - 1) / g.wp; ++p) {
+                    const size_t o = part_base + (static_cast<size_t>(p) * g.spp + (ch - (p * g.wp) / a.c)) * a.R;
+                    const size_t so = stat_base + static_cast<size_t>(p) * a.R;
+                    for (int i = lane; i < a.R; i += 32)
+                        acc[u] += a.partial[o + i] * (ex2_approx(a.stat_m[so + i] - gm[i]) * ginv[i]);
+                }
             }
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-        if (lane == 0) out[static_cast<size_t>(h) * g.C + ch] = acc;
+        for (int u = 0; u < kFinBatch; ++u) {
+            float v = acc[u];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            if (lane == 0 && cb + u < ch1) out[static_cast<size_t>(h) * g.C + cb + u] = v;
+        }
     }
 }
 
@@ -496,7 +538,7 @@ bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_
     if (p.n_mt == 1 && (c == 10 || c == 20)) { p.c_static = c; p.n_tile = 240; }
     else if (p.n_mt == 1 && c == 1) { p.c_static = 1; p.n_tile = 256; }
     else p.n_tile = 256 / p.n_mt;
-    p.wp = (p.n_mt == 1) ? p.n_tile / 4 : p.n_tile / 2;
+    p.wp = p.n_tile / (kGroups / p.n_mt);
     p.n_tiles = (L + p.n_tile - 1) / p.n_tile;
     p.n_panels = p.n_tiles * (p.n_tile / p.wp);
     p.spp = p.c_static ? p.wp / p.c_static : (p.wp + c - 1) / c + 1;
@@ -519,14 +561,14 @@ bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_
 
 size_t score_scratch_floats(const ScorePlan& plan, int Hkv, int R) {
     const size_t panels = static_cast<size_t>(Hkv) * plan.n_panels;
-    return panels * R + static_cast<size_t>(plan.grid) * plan.hs_max * 512 + panels * plan.spp * R;
+    return panels * R + static_cast<size_t>(plan.grid) * plan.hs_max * (kGroups * 256) + panels * plan.spp * R;
 }
 
 void score_scratch_layout(const ScorePlan& plan, int Hkv, int R, float* base, ScoreArgs* args) {
     const size_t panels = static_cast<size_t>(Hkv) * plan.n_panels;
     args->stat_m = base;
     args->cta_stat = base + panels * R;
-    args->partial = args->cta_stat + static_cast<size_t>(plan.grid) * plan.hs_max * 512;
+    args->partial = args->cta_stat + static_cast<size_t>(plan.grid) * plan.hs_max * (kGroups * 256);
 }
 
 cudaError_t launch_score(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
