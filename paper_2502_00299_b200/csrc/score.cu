@@ -168,7 +168,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.tfull[b]), 1);
-            mbar_init(smem_u32(&ctl.tempty[b]), 128 * kGroups);
+            mbar_init(smem_u32(&ctl.tempty[b]), 4 * kGroups);   // one arrival per epilogue warp
             mbar_init(smem_u32(&ctl.qfull[b]), 1);
             mbar_init(smem_u32(&ctl.qempty[b]), 1);
         }
@@ -310,14 +310,17 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 run_l = 0.f;
             }
             const int buf = ti & 1, use = ti >> 1;
-            if (!mbar_wait(smem_u32(&ctl.tfull[buf]), use & 1, abort_flag)) break;
+            bool ready = true;                       // one lane polls, the warp follows
+            if (lane == 0) ready = mbar_wait(smem_u32(&ctl.tfull[buf]), use & 1, abort_flag);
+            if (!__shfl_sync(0xffffffffu, ready, 0)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(buf * 256 + mt * TCOLS + pit * WP);
             float v[WP];
             load_panel<WP>(taddr, v);
             tc_fence_before();
-            mbar_arrive(smem_u32(&ctl.tempty[buf]));   // the tensor cores may overwrite the buffer now
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[buf]));   // the buffer may be overwritten now
 
             const int panel = tile * PPT + pit;
             const size_t panel_id = static_cast<size_t>(head) * n_panels + panel;

@@ -1,12 +1,13 @@
 // Top-k chunk selection and kept-index emission (ChunkKV Algorithm 3: "Top-K(chunk_scores, k)",
 // the selection mask, "always keep most recent tokens", "nonzero(mask)").
 //
-// One CTA per KV head. The k-th largest score is found by an exact 4-pass radix select on
-// order-preserving 32-bit keys (warp-aggregated shared-memory histograms, one warp scanning
-// the 256 bins). Each thread then owns a contiguous run of chunk ids; one block-wide prefix
-// sum over (#above threshold, #equal to threshold) gives every chunk its rank among the kept
-// ones: rank = #above before it + min(#equal before it, ties to keep) - ties go to the lower
-// chunk id. Token positions are written directly in ascending order: no mask, no sort.
+// One CTA per KV head. Each thread owns a contiguous run of chunk ids and keeps their
+// order-preserving 32-bit keys in registers. The k-th largest key is found by an exact 4-pass
+// radix select; every warp counts into its own 16-bit histogram row (lanes that hit the same
+// bin add once), so no two warps ever touch the same counter. One block-wide prefix sum over
+// (#above threshold, #equal to threshold) then gives every chunk its rank among the kept ones:
+// rank = #above before it + min(#equal before it, ties to keep) - ties go to the lower chunk
+// id. Token positions are written directly in ascending order: no mask, no sort.
 #include "internal.h"
 
 namespace chunkkv {
@@ -14,18 +15,21 @@ namespace chunkkv {
 namespace {
 
 constexpr int kSelThreads = 1024;
-constexpr int kKeyCap = 6912;      // chunk keys staged in shared memory (27 KB); more are re-read
-constexpr int kSelCap = 4096;      // kept-chunk ids staged for coalesced index writes
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kPerThread = 8;                         // chunk keys held in registers per thread
+constexpr int kRegCap = kSelThreads * kPerThread;     // more chunks than this are re-read from memory
+constexpr int kSelCap = 4096;                         // kept-chunk ids staged for coalesced index writes
 
 __device__ __forceinline__ uint32_t order_key(float x) {
     const uint32_t b = __float_as_uint(x + 0.0f);          // -0 and +0 compare equal
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);     // larger float <=> larger key
 }
 
+template <bool IN_REGS>
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int k, int n_max,
               int32_t* __restrict__ out_idx) {
-    __shared__ uint32_t keys_s[kKeyCap];
+    __shared__ unsigned short whist[kSelWarps][256];
     __shared__ int sel_s[kSelCap];
     __shared__ int hist[256];
     __shared__ unsigned long long warp_sums[33];
@@ -37,34 +41,53 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
     const float* sc = scores + static_cast<size_t>(h) * C;
     int32_t* out = out_idx + static_cast<size_t>(h) * n_max;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const bool cached = C <= kKeyCap;
     const bool keep_all = (k >= C);
+    const int kk = min(k, C);
 
+    // thread t owns chunk ids [c0, c1)
+    const int per = (C + kSelThreads - 1) / kSelThreads;
+    const int c0 = min(tid * per, C), c1 = min(c0 + per, C);
+    uint32_t keys[kPerThread];
+    if (IN_REGS && kk > 0 && !keep_all) {
+#pragma unroll
+        for (int u = 0; u < kPerThread; ++u) keys[u] = (c0 + u < c1) ? order_key(sc[c0 + u]) : 0u;
+    }
     if (tid == 0) s_last_kept = 0;
-    if (cached && k > 0 && !keep_all)
-        for (int i = tid; i < C; i += kSelThreads) keys_s[i] = order_key(sc[i]);
-    __syncthreads();
-    auto key_at = [&](int i) -> uint32_t { return cached ? keys_s[i] : order_key(sc[i]); };
 
     uint32_t thresh = 0;   // key of the k-th largest score
     int need_eq = 0;       // how many chunks equal to the threshold are kept
-    if (!keep_all && k > 0) {
+    if (!keep_all && kk > 0) {
         uint32_t prefix = 0;
         int need = k;
         for (int pass = 0; pass < 4; ++pass) {
             const int shift = 24 - 8 * pass;
-            if (tid < 256) hist[tid] = 0;
-            __syncthreads();
+            {   // clear this warp's histogram row (256 x 16 bit = 128 words)
+                uint32_t* row = reinterpret_cast<uint32_t*>(whist[warp]);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) row[lane + 32 * q] = 0u;
+            }
+            __syncwarp();
             const uint32_t himask = (pass == 0) ? 0u : (0xFFFFFFFFu << (shift + 8));
-            for (int base = 0; base < C; base += kSelThreads) {
-                const int i = base + tid;
-                uint32_t key = 0;
-                bool in = false;
-                if (i < C) { key = key_at(i); in = (key & himask) == prefix; }
-                // lanes of a warp that hit the same bin add once
+            auto count_one = [&](bool have, uint32_t key) {
+                const bool in = have && (key & himask) == prefix;
                 const int bin = in ? static_cast<int>((key >> shift) & 0xFF) : -1;
                 const unsigned peers = __match_any_sync(0xffffffffu, bin);
-                if (in && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
+                if (in && lane == __ffs(peers) - 1) whist[warp][bin] += static_cast<unsigned short>(__popc(peers));
+                __syncwarp();
+            };
+            if (IN_REGS) {
+#pragma unroll
+                for (int u = 0; u < kPerThread; ++u)
+                    if (u < per) count_one(c0 + u < c1, keys[u]);      // `per` is uniform: no divergence
+            } else {
+                for (int u = 0; u < per; ++u) count_one(c0 + u < c1, (c0 + u < c1) ? order_key(sc[c0 + u]) : 0u);
+            }
+            __syncthreads();
+            if (tid < 256) {
+                int sum = 0;
+#pragma unroll 8
+                for (int wv = 0; wv < kSelWarps; ++wv) sum += whist[wv][tid];
+                hist[tid] = sum;
             }
             __syncthreads();
             if (warp == 0) {
@@ -95,20 +118,22 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
         need_eq = need;
     }
 
-    // Ordered sweep: thread t owns chunk ids [t * per, (t + 1) * per).
-    const int kk = min(k, C);
+    // Ordered sweep over the chunk ids.
     const bool stage_sel = kk <= kSelCap;
     if (kk > 0) {
-        const int per = (C + kSelThreads - 1) / kSelThreads;
-        const int c0 = min(tid * per, C), c1 = min(c0 + per, C);
         unsigned gt_n = 0, eq_n = 0;
         if (keep_all) gt_n = c1 - c0;
-        else
+        else if (IN_REGS) {
+#pragma unroll
+            for (int u = 0; u < kPerThread; ++u)
+                if (c0 + u < c1) { gt_n += keys[u] > thresh; eq_n += keys[u] == thresh; }
+        } else {
             for (int ch = c0; ch < c1; ++ch) {
-                const uint32_t key = key_at(ch);
+                const uint32_t key = order_key(sc[ch]);
                 gt_n += key > thresh;
                 eq_n += key == thresh;
             }
+        }
         // block-wide exclusive prefix of the packed pair (eq in the high half, gt in the low half)
         const unsigned long long mine = (static_cast<unsigned long long>(eq_n) << 32) | gt_n;
         unsigned long long inc = mine;
@@ -132,13 +157,9 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
         __syncthreads();
         const unsigned long long excl = warp_sums[warp] + inc - mine;
         int gt_before = static_cast<int>(excl & 0xffffffffu), eq_before = static_cast<int>(excl >> 32);
-        for (int ch = c0; ch < c1; ++ch) {
-            bool gt = keep_all, eq = false;
-            if (!keep_all) {
-                const uint32_t key = key_at(ch);
-                gt = key > thresh;
-                eq = key == thresh;
-            }
+        auto visit = [&](int ch, uint32_t key) {
+            const bool gt = keep_all || key > thresh;
+            const bool eq = !keep_all && key == thresh;
             if (gt || (eq && eq_before < need_eq)) {
                 const int rank = gt_before + min(eq_before, need_eq);
                 if (stage_sel) sel_s[rank] = ch;
@@ -151,6 +172,13 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
             }
             gt_before += gt;
             eq_before += eq;
+        };
+        if (IN_REGS && !keep_all) {
+#pragma unroll
+            for (int u = 0; u < kPerThread; ++u)
+                if (c0 + u < c1) visit(c0 + u, keys[u]);
+        } else {
+            for (int ch = c0; ch < c1; ++ch) visit(ch, keep_all ? 0u : order_key(sc[ch]));
         }
     }
     __syncthreads();
@@ -170,7 +198,10 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
 
 cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int C, int k, int n_max,
                           int32_t* out_idx, cudaStream_t stream) {
-    select_kernel<<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx);
+    if (C <= kRegCap)
+        select_kernel<true><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx);
+    else
+        select_kernel<false><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx);
     return cudaGetLastError();
 }
 
