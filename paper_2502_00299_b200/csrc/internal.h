@@ -12,7 +12,7 @@ struct ScorePlan {
     int c_static;   // chunk size baked into the kernel (0 = run-time chunk size)
     int n_mt;       // 128-row query tiles per KV head (1 or 2)
     int n_tile;     // keys per accumulator tile (one UMMA N)
-    int wp;         // keys per epilogue panel (n_tile / 4 with one query tile, n_tile / 2 with two)
+    int wp;         // keys per epilogue panel (a quarter or half tile; 32 for run-time chunk sizes)
     int n_tiles;    // accumulator tiles per head = ceil(L / n_tile)
     int n_panels;   // panels per head
     int spp;        // chunk slots per panel in the partial-sum scratch

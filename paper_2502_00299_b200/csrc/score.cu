@@ -81,6 +81,34 @@ __device__ __forceinline__ void panel_fast(const float (&v)[WP], float sl2, bool
     *out_l = l;
 }
 
+// Panel of a compile-time chunk size that starts on a chunk boundary but reaches past the
+// prefix: chunk positions are still static; columns at or past P only feed the row sum, and
+// columns the row cannot see (causal mask in the window, or past L) contribute nothing.
+template <int C, int WP>
+__device__ __forceinline__ void panel_static_tail(const float (&v)[WP], float sl2, bool active, float* part,
+                                                  int row_stride, int j0, int P, int last_visible,
+                                                  float* out_m, float* out_l) {
+    const int n_vis = last_visible - j0 + 1;     // columns u < n_vis are visible
+    const int n_pre = P - j0;                    // columns u < n_pre belong to the prefix
+    float mx = -CUDART_INF_F;
+#pragma unroll
+    for (int u = 0; u < WP; ++u) mx = (u < n_vis) ? fmaxf(mx, v[u]) : mx;
+    const float neg_m2 = (mx == -CUDART_INF_F) ? 0.f : -mx * sl2;
+    float l = 0.f, acc = 0.f;
+#pragma unroll
+    for (int u = 0; u < WP; ++u) {
+        const float e = (u < n_vis) ? ex2_approx(fmaf(v[u], sl2, neg_m2)) : 0.f;
+        l += e;
+        const float pe = (u < n_pre) ? e : 0.f;
+        acc = (u % C == 0) ? pe : acc + pe;
+        if ((u + 1) % C == 0) {
+            if (active && (u + 1 - C) < n_pre) part[static_cast<size_t>((u + 1) / C - 1) * row_stride] = acc;
+        }
+    }
+    *out_m = (mx == -CUDART_INF_F) ? -CUDART_INF_F : mx * sl2;
+    *out_l = l;
+}
+
 // Any panel: run-time chunk size, chunk grid clipped at P, causal mask inside the window
 // columns [P, L), nothing visible at or beyond L. Window columns add to the row sum only.
 template <int WP>
@@ -141,8 +169,13 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     constexpr int NQBUF = (N_MT == 1) ? 2 : 1;
     constexpr int TCOLS = 256 / N_MT;              // TMEM columns reserved per accumulator
     constexpr int PPT = kGroups / N_MT;            // panels per tile = groups sharing a query tile
-    constexpr int WP = N_TILE / PPT;               // panel width in keys
-    static_assert(C_STATIC == 0 || WP % C_STATIC == 0, "static chunk size must divide the panel");
+    constexpr int WP = N_TILE / PPT;               // columns per group
+    // Compile-time chunk sizes take a group's columns as one panel; the run-time-c path walks
+    // them as 32-column panels to keep its register footprint small.
+    constexpr int WPP = (C_STATIC > 0) ? WP : 32;  // panel width in keys
+    constexpr int SUBS = WP / WPP;                 // panels a thread processes per tile
+    static_assert(WP % WPP == 0, "group columns must split into whole panels");
+    static_assert(C_STATIC == 0 || WPP % C_STATIC == 0, "static chunk size must divide the panel");
     constexpr uint32_t IDESC = umma_idesc_bf16(128, N_TILE);
 
     extern __shared__ uint8_t smem_raw[];
@@ -289,7 +322,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int row = mt * 128 + quarter * 32 + lane;
         const bool active = row < a.R;
         const int last_visible = a.P + (row % a.w);  // this row sees keys j <= P + r (all < L)
-        const int n_panels = g.n_tiles * PPT;
+        const int n_panels = g.n_tiles * PPT * SUBS;
         float run_m = -CUDART_INF_F, run_l = 0.f;    // (max, sum) over this thread's panels of the head
         int cur_head = -1, hs = -1, ti = 0;
         auto flush_head = [&]() {
@@ -316,29 +349,36 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(buf * 256 + mt * TCOLS + pit * WP);
-            float v[WP];
-            load_panel<WP>(taddr, v);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[buf]));   // the buffer may be overwritten now
-
-            const int panel = tile * PPT + pit;
-            const size_t panel_id = static_cast<size_t>(head) * n_panels + panel;
-            float* part = a.partial + panel_id * g.spp * a.R + row;
-            const int j0 = panel * WP;
-            float m2, l;
-            if (C_STATIC > 0 && j0 + WP <= a.P) {
-                panel_fast<(C_STATIC > 0 ? C_STATIC : 1), WP>(v, a.sl2, active, part, a.R, &m2, &l);
-            } else {
-                panel_general<WP>(v, a.sl2, active, part, a.R, j0, a.P, a.c, last_visible, &m2, &l);
+#pragma unroll
+            for (int sub = 0; sub < SUBS; ++sub) {
+                float v[WPP];
+                load_panel<WPP>(taddr + sub * WPP, v);
+                if (sub == SUBS - 1) {               // this thread's last read of the buffer
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[buf]));   // it may be overwritten now
+                }
+                const int panel = (tile * PPT + pit) * SUBS + sub;
+                const size_t panel_id = static_cast<size_t>(head) * n_panels + panel;
+                float* part = a.partial + panel_id * g.spp * a.R + row;
+                const int j0 = panel * WPP;
+                float m2, l;
+                if constexpr (C_STATIC > 0) {
+                    if (j0 + WPP <= a.P)
+                        panel_fast<C_STATIC, WPP>(v, a.sl2, active, part, a.R, &m2, &l);
+                    else
+                        panel_static_tail<C_STATIC, WPP>(v, a.sl2, active, part, a.R, j0, a.P, last_visible, &m2, &l);
+                } else {
+                    panel_general<WPP>(v, a.sl2, active, part, a.R, j0, a.P, a.c, last_visible, &m2, &l);
+                }
+                if (active) a.stat_m[panel_id * a.R + row] = m2;
+                // fold into the running record: l is relative to m2, run_l to run_m
+                const float nm = fmaxf(run_m, m2);
+                const float s_old = (run_m == -CUDART_INF_F) ? 0.f : ex2_approx(run_m - nm);
+                const float s_new = (m2 == -CUDART_INF_F) ? 0.f : ex2_approx(m2 - nm);
+                run_l = run_l * s_old + l * s_new;
+                run_m = nm;
             }
-            if (active) a.stat_m[panel_id * a.R + row] = m2;
-            // fold into the running record: l is relative to m2, run_l to run_m
-            const float nm = fmaxf(run_m, m2);
-            const float s_old = (run_m == -CUDART_INF_F) ? 0.f : ex2_approx(run_m - nm);
-            const float s_new = (m2 == -CUDART_INF_F) ? 0.f : ex2_approx(m2 - nm);
-            run_l = run_l * s_old + l * s_new;
-            run_m = nm;
         }
         flush_head();
     }
@@ -541,7 +581,7 @@ bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_
     if (p.n_mt == 1 && (c == 10 || c == 20)) { p.c_static = c; p.n_tile = 240; }
     else if (p.n_mt == 1 && c == 1) { p.c_static = 1; p.n_tile = 256; }
     else p.n_tile = 256 / p.n_mt;
-    p.wp = p.n_tile / (kGroups / p.n_mt);
+    p.wp = p.c_static ? p.n_tile / (kGroups / p.n_mt) : 32;
     p.n_tiles = (L + p.n_tile - 1) / p.n_tile;
     p.n_panels = p.n_tiles * (p.n_tile / p.wp);
     p.spp = p.c_static ? p.wp / p.c_static : (p.wp + c - 1) / c + 1;
