@@ -27,6 +27,7 @@ struct ScoreArgs {
     float sl2;            // log2(e) / sqrt(d)
     float* stat_m;        // [Hkv, n_panels, R] panel row maxima (log2 domain)
     float* cta_stat;      // [grid, hs_max, 4 groups, {max, sum}, 128] per-CTA folded row statistics
+    float* row_stat;      // [Hkv, {max, 1 / sum}, 256] global row statistics
     float* partial;       // [Hkv, n_panels, spp, R] chunk partial sums relative to the panel maximum
     int* status;          // device status word
 };

@@ -393,12 +393,12 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 }
 
 // ---------------------------------------------------------------------------------------------
-// Finalisation. grid = (blocks per head, Hkv). Each block
-//   1. merges the per-CTA records of its head into global row maxima m[i] and 1 / l[i]
-//      (every thread takes a slice of the records of one row, so the loads overlap),
-//   2. computes the scale f[p][i] = exp2(m_panel[p][i] - m[i]) / l[i] for the panels its chunks
-//      touch (kept in shared memory),
-//   3. contracts partial[ch][.] * f over the R rows, one warp working on four chunks at a time.
+// Finalisation, two small kernels:
+//   rowstats_kernel  merges the per-CTA records of each head into global row maxima m[i] and
+//                    1 / l[i];
+//   finalize_kernel  computes the scale f[p][i] = exp2(m_panel[p][i] - m[i]) / l[i] for the
+//                    panels its chunks touch (kept in shared memory) and contracts
+//                    partial[ch][.] * f over the R rows, one warp working on four chunks at a time.
 // All reductions have a fixed order, so results are deterministic.
 constexpr int kFinThreads = 512;
 constexpr int kFinPanelCap = 24;      // panels whose scales fit in shared memory (24 x 256 floats)
@@ -415,67 +415,78 @@ struct FinGeom {
     int C;
 };
 
+// One block per KV head: merge the records of the CTAs that touched the head into the global
+// row maxima m[i] and 1 / l[i]. Every thread takes a slice of the records of one row, so the
+// loads overlap. Output: row_stat[h][0][i] = m, row_stat[h][1][i] = 1 / l.
 __global__ void __launch_bounds__(kFinThreads)
-finalize_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
-    __shared__ float gm[256];
-    __shared__ float ginv[256];
+rowstats_kernel(const ScoreArgs a, const FinGeom g) {
     __shared__ float red[kFinThreads];
-    __shared__ int rec_base[160];
-    __shared__ float fs[kFinPanelCap * 256];
-    const int h = blockIdx.y;
+    __shared__ int rec_base[256];
+    const int h = blockIdx.x;
     const int tid = threadIdx.x;
-
-    // 1. global row statistics from the records of the CTAs that touched head h.
     // CTA b owns tiles [total*b/G, total*(b+1)/G): the owner of tile T is floor(((T+1)*G - 1) / total).
     const long long total = static_cast<long long>(a.Hkv) * g.n_tiles;
     const long long first_tile = static_cast<long long>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
     const int b_lo = static_cast<int>(((first_tile + 1) * g.score_grid - 1) / total);
     const int b_hi = static_cast<int>(((last_tile + 1) * g.score_grid - 1) / total);
-    const int nb = b_hi - b_lo + 1;
+    const int nb = b_hi - b_lo + 1;                 // <= 256: the scoring grid is capped there
     for (int j = tid; j < nb; j += kFinThreads) {
         const int b = b_lo + j;
         const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
-        rec_base[j % 160] = (b * g.hs_max + (h - head0)) * (kGroups * 256);
+        rec_base[j] = (b * g.hs_max + (h - head0)) * (kGroups * 256);
     }
     __syncthreads();
     const int rp = (a.R > 128) ? 256 : 128;         // rows padded to the slice stride
     const int ns = kFinThreads / rp;                // record slices per row
     const int gpr = kGroups / g.n_mt;               // groups (records per CTA) that hold a given row
-    {
-        const int i = tid % rp, sl = tid / rp;
-        const int g0 = (g.n_mt == 2) ? (i >> 7) * gpr : 0;
-        const int rr = i & 127;
-        const int nrec = nb * gpr;
-        float m = -CUDART_INF_F;
-        if (i < a.R) {
+    const int i = tid % rp, sl = tid / rp;
+    const int g0 = (g.n_mt == 2) ? (i >> 7) * gpr : 0;
+    const int rr = i & 127;
+    float m = -CUDART_INF_F;
+    if (i < a.R) {
+        for (int j = sl; j < nb; j += ns) {
+            const float* rec = a.cta_stat + rec_base[j] + g0 * 256 + rr;
 #pragma unroll 4
-            for (int q = sl; q < nrec; q += ns) {
-                const float* rec = a.cta_stat + rec_base[(q / gpr) % 160] + (g0 + q % gpr) * 256;
-                m = fmaxf(m, rec[rr]);
+            for (int q = 0; q < gpr; ++q) m = fmaxf(m, rec[q * 256]);
+        }
+    }
+    red[tid] = m;
+    __syncthreads();
+    float M = red[i];
+    for (int s2 = 1; s2 < ns; ++s2) M = fmaxf(M, red[s2 * rp + i]);
+    __syncthreads();
+    float l = 0.f;
+    if (i < a.R) {
+        for (int j = sl; j < nb; j += ns) {
+            const float* rec = a.cta_stat + rec_base[j] + g0 * 256 + rr;
+#pragma unroll 4
+            for (int q = 0; q < gpr; ++q) {
+                const float rm = rec[q * 256];
+                l += (rm == -CUDART_INF_F) ? 0.f : rec[q * 256 + 128] * ex2_approx(rm - M);
             }
         }
-        red[tid] = m;
-        __syncthreads();
-        float M = red[i];
-        for (int s2 = 1; s2 < ns; ++s2) M = fmaxf(M, red[s2 * rp + i]);
-        __syncthreads();
-        float l = 0.f;
-        if (i < a.R) {
-#pragma unroll 4
-            for (int q = sl; q < nrec; q += ns) {
-                const float* rec = a.cta_stat + rec_base[(q / gpr) % 160] + (g0 + q % gpr) * 256;
-                const float rm = rec[rr];
-                l += (rm == -CUDART_INF_F) ? 0.f : rec[128 + rr] * ex2_approx(rm - M);
-            }
-        }
-        red[tid] = l;
-        __syncthreads();
-        if (sl == 0 && i < a.R) {
-            float lt = red[i];
-            for (int s2 = 1; s2 < ns; ++s2) lt += red[s2 * rp + i];
-            gm[i] = M;
-            ginv[i] = 1.0f / lt;
-        }
+    }
+    red[tid] = l;
+    __syncthreads();
+    if (sl == 0 && i < a.R) {
+        float lt = red[i];
+        for (int s2 = 1; s2 < ns; ++s2) lt += red[s2 * rp + i];
+        a.row_stat[static_cast<size_t>(h) * 512 + i] = M;
+        a.row_stat[static_cast<size_t>(h) * 512 + 256 + i] = 1.0f / lt;
+    }
+}
+
+// grid = (blocks per head, Hkv): chunk scores from partial sums, see the header of this section.
+__global__ void __launch_bounds__(kFinThreads)
+finalize_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
+    __shared__ float gm[256];
+    __shared__ float ginv[256];
+    __shared__ float fs[kFinPanelCap * 256];
+    const int h = blockIdx.y;
+    const int tid = threadIdx.x;
+    if (tid < a.R) {
+        gm[tid] = a.row_stat[static_cast<size_t>(h) * 512 + tid];
+        ginv[tid] = a.row_stat[static_cast<size_t>(h) * 512 + 256 + tid];
     }
     __syncthreads();
 
@@ -587,6 +598,7 @@ bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_
     p.spp = p.c_static ? p.wp / p.c_static : (p.wp + c - 1) / c + 1;
     const long long total = static_cast<long long>(Hkv) * p.n_tiles;
     p.grid = static_cast<int>(total < num_sms ? total : num_sms);
+    if (p.grid > 256) p.grid = 256;   // rowstats_kernel indexes at most 256 CTA records per head
     const int tiles_per_cta = static_cast<int>((total + p.grid - 1) / p.grid);
     p.hs_max = (tiles_per_cta + p.n_tiles - 1) / p.n_tiles + 1;
     const int KB = d / 64;
@@ -604,14 +616,16 @@ bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_
 
 size_t score_scratch_floats(const ScorePlan& plan, int Hkv, int R) {
     const size_t panels = static_cast<size_t>(Hkv) * plan.n_panels;
-    return panels * R + static_cast<size_t>(plan.grid) * plan.hs_max * (kGroups * 256) + panels * plan.spp * R;
+    return panels * R + static_cast<size_t>(plan.grid) * plan.hs_max * (kGroups * 256) +
+           static_cast<size_t>(Hkv) * 512 + panels * plan.spp * R;
 }
 
 void score_scratch_layout(const ScorePlan& plan, int Hkv, int R, float* base, ScoreArgs* args) {
     const size_t panels = static_cast<size_t>(Hkv) * plan.n_panels;
     args->stat_m = base;
     args->cta_stat = base + panels * R;
-    args->partial = args->cta_stat + static_cast<size_t>(plan.grid) * plan.hs_max * (kGroups * 256);
+    args->row_stat = args->cta_stat + static_cast<size_t>(plan.grid) * plan.hs_max * (kGroups * 256);
+    args->partial = args->row_stat + static_cast<size_t>(Hkv) * 512;
 }
 
 cudaError_t launch_score(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
@@ -641,6 +655,7 @@ cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C,
     g.score_grid = plan.grid;
     g.hs_max = plan.hs_max;
     g.C = C;
+    rowstats_kernel<<<args.Hkv, kFinThreads, 0, stream>>>(args, g);
     dim3 grid(bx, args.Hkv);
     finalize_kernel<<<grid, kFinThreads, 0, stream>>>(args, g, out_scores);
     return cudaGetLastError();
