@@ -61,6 +61,7 @@ extern "C" {
 #define CHUNKKV_ENOWORKSPACE   -4  /* caller-provided workspace too small / allocation failed */
 #define CHUNKKV_ECUDA          -5  /* a CUDA runtime or driver call failed (see chunkkv_last_cuda_error) */
 #define CHUNKKV_EDEVICE        -6  /* a kernel gave up on a bounded wait (see chunkkv_device_status) */
+#define CHUNKKV_ETOOLARGE      -7  /* the problem needs more scratch than a fixed-size variant provides */
 
 /* Human-readable name of a status code (static string, never NULL). */
 CHUNKKV_API const char* chunkkv_strerror(int status);
@@ -106,6 +107,31 @@ CHUNKKV_API int chunkkv_device_status(void* stream);
  */
 CHUNKKV_API int chunkkv_score(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w, int c,
                   float* out_token_scores, float* out_chunk_scores, void* stream);
+
+/*
+ * chunkkv_score for callers that must not allocate. (No counterpart in the paper: this is a
+ * deployment convenience, not a step of the method.)
+ *
+ * Who needs it: serving processes that hand every free byte of HBM to their own cache pool at
+ * start-up, so that a later cudaMalloc either fails or eats into memory they have promised
+ * elsewhere; and callers inside latency-critical loops that cannot accept the device-wide
+ * synchronisation cudaMalloc / cudaFree imply. This entry point calls no cudaMalloc, cudaFree or
+ * any other allocating routine, and ignores chunkkv_set_workspace: its scratch is a fixed
+ * 8 MiB array that lives in the library's device image (every GPU that loads the library holds
+ * those 8 MiB until the process exits).
+ *
+ * Same arguments, layouts and result as chunkkv_score without the token-score output:
+ * out_chunk_scores [Hkv, C] f32. Shapes whose chunkkv_workspace_bytes(L, Hq, Hkv, d, w, c)
+ * exceeds 8 MiB are rejected with CHUNKKV_ETOOLARGE and nothing is launched.
+ *
+ * The first call on each device looks up the device address of the array (with that device
+ * current); make that first call outside any stream capture. All calls on a device share the one
+ * array, which keeps whatever the previous call left in it: the library clears the status word it
+ * needs zeroed on every call, and calls that overlap on the GPU (different streams, no ordering)
+ * race on the scratch - order them.
+ */
+CHUNKKV_API int chunkkv_score_noalloc(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d,
+                                      int w, int c, float* out_chunk_scores, void* stream);
 
 /*
  * Step "top-k chunk selection" and the kept-index list (Algorithm 3: Top-K, selection mask,

@@ -209,6 +209,41 @@ size_t scratch_floats_for(const DeviceCtx& ctx, int L, int R, int Hkv, int d, in
 
 }  // namespace
 
+namespace chunkkv {
+
+// Scoring into caller-supplied scratch (256-byte header + payload). Used by the fixed-scratch
+// entry point; allocates nothing and records no profiling events.
+int score_with_scratch(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w, int c,
+                       float* out_scores, void* scratch, size_t scratch_bytes, cudaStream_t stream) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    int st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    const int R = w * (Hq / Hkv), P = L - w;
+    const int C = (P + c - 1) / c;
+    if (C <= 0) return CHUNKKV_OK;
+    ScorePlan plan;
+    if (!make_score_plan(L, R, Hkv, d, c, ctx->num_sms, smem_budget(*ctx), &plan)) return CHUNKKV_EINVAL_SHAPE;
+    if (kHeaderBytes + score_scratch_floats(plan, Hkv, R) * sizeof(float) > scratch_bytes) return CHUNKKV_ETOOLARGE;
+    ScoreArgs a;
+    a.L = L; a.P = P; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
+    a.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
+    score_scratch_layout(plan, Hkv, R, reinterpret_cast<float*>(static_cast<char*>(scratch) + kHeaderBytes), &a);
+    a.status = static_cast<int*>(scratch);
+    CUtensorMap tm_q, tm_k;
+    st = encode_bf16_3d(&tm_q, q_obs, d, R, Hkv, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    if (st != CHUNKKV_OK) return st;
+    st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < plan.n_tile ? L : plan.n_tile, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+    if (st != CHUNKKV_OK) return st;
+    cudaError_t e = launch_score(plan, tm_q, tm_k, a, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_finalize(plan, a, C, out_scores, ctx->num_sms, stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+}  // namespace chunkkv
+
 extern "C" {
 
 const char* chunkkv_strerror(int status) {
@@ -220,6 +255,7 @@ const char* chunkkv_strerror(int status) {
         case CHUNKKV_ENOWORKSPACE: return "scratch workspace too small or could not be allocated";
         case CHUNKKV_ECUDA: return "a CUDA call failed";
         case CHUNKKV_EDEVICE: return "a kernel abandoned a bounded wait";
+        case CHUNKKV_ETOOLARGE: return "the problem needs more scratch than the fixed-size variant provides";
         default: return "unknown status";
     }
 }

@@ -54,4 +54,10 @@ cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int 
                           int n_max, void* out_K, void* out_V, int32_t* idx_copy_or_null,
                           int num_sms, cudaStream_t stream);
 
+// Scoring (score + finalisation kernels) into caller-supplied scratch: a 256-byte header whose
+// first word is the device status word, then the payload. Returns a CHUNKKV_* status;
+// CHUNKKV_ETOOLARGE if scratch_bytes is too small. Allocates nothing.
+int score_with_scratch(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w, int c,
+                       float* out_scores, void* scratch, size_t scratch_bytes, cudaStream_t stream);
+
 }  // namespace chunkkv
