@@ -177,7 +177,8 @@ CHUNKKV_API int chunkkv_compress_layer_host(const void* host_q_obs, const void* 
  * kernel with CUDA events on the launching stream. chunkkv_profile_read synchronises the
  * device and returns, per kernel slot, accumulated milliseconds and launch counts since the
  * last read (arrays of CHUNKKV_PROFILE_SLOTS entries), then resets them.
- * Slots: 0 score, 1 chunk-score finalisation, 2 select, 3 gather.
+ * Slots: 0 score (or the fused whole-layer kernel of chunkkv_compress_layer), 1 chunk-score
+ * finalisation, 2 select, 3 gather.
  */
 #define CHUNKKV_PROFILE_SLOTS 4
 CHUNKKV_API int chunkkv_profile_enable(int on);

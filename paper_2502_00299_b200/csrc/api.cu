@@ -5,6 +5,7 @@
 #include "internal.h"
 
 #include <math.h>
+#include <stdlib.h>
 #include <mutex>
 #include <vector>
 
@@ -44,6 +45,9 @@ std::mutex g_mu;
 DeviceCtx g_ctx[kMaxDevices];
 EncodeTiledFn g_encode = nullptr;
 bool g_profile = false;
+// CHUNKKV_UNFUSED=1 makes chunkkv_compress_layer use the separate score / finalize / select /
+// gather kernels instead of the single fused launch (for comparison and debugging).
+const bool g_unfused = [] { const char* v = getenv("CHUNKKV_UNFUSED"); return v != nullptr && v[0] == '1'; }();
 
 int cuda_fail(cudaError_t e) {
     g_last_cuda_error = static_cast<int>(e);
@@ -169,7 +173,7 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
     const int C = (P + c - 1) / c;
     if (C <= 0) return CHUNKKV_OK;
     ScorePlan plan;
-    if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), &plan)) return CHUNKKV_EINVAL_SHAPE;
+    if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
     const size_t floats = score_scratch_floats(plan, Hkv, R) + extra_payload_floats;
     int st = ensure_workspace(ctx, floats * sizeof(float));
     if (st != CHUNKKV_OK) return st;
@@ -203,7 +207,7 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
 
 size_t scratch_floats_for(const DeviceCtx& ctx, int L, int R, int Hkv, int d, int c) {
     ScorePlan plan;
-    if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), &plan)) return 0;
+    if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), false, &plan)) return 0;
     return score_scratch_floats(plan, Hkv, R);
 }
 
@@ -223,7 +227,7 @@ int score_with_scratch(const void* q_obs, const void* K, int L, int Hq, int Hkv,
     const int C = (P + c - 1) / c;
     if (C <= 0) return CHUNKKV_OK;
     ScorePlan plan;
-    if (!make_score_plan(L, R, Hkv, d, c, ctx->num_sms, smem_budget(*ctx), &plan)) return CHUNKKV_EINVAL_SHAPE;
+    if (!make_score_plan(L, R, Hkv, d, c, ctx->num_sms, smem_budget(*ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
     if (kHeaderBytes + score_scratch_floats(plan, Hkv, R) * sizeof(float) > scratch_bytes) return CHUNKKV_ETOOLARGE;
     ScoreArgs a;
     a.L = L; a.P = P; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
@@ -333,7 +337,7 @@ int chunkkv_device_status(void* stream) {
     e = cudaMemcpy(&flag, ctx->ws, sizeof(int), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(e);
     if (flag != 0) {
-        cudaMemset(ctx->ws, 0, sizeof(int));
+        cudaMemset(ctx->ws, 0, kHeaderBytes);   // status word and grid-barrier words
         return CHUNKKV_EDEVICE;
     }
     return CHUNKKV_OK;
@@ -439,8 +443,40 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
     }
     float* chunk_scores = nullptr;
     if (C > 0 && k > 0) {
+        const int R = w * (Hq / Hkv);
         // chunk scores sit at the start of the scratch payload, the score kernels' scratch after them
         const size_t cs_floats = (static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63);
+        ScorePlan plan;
+        if (!g_unfused && make_score_plan(L, R, Hkv, d, c, ctx->num_sms, smem_budget(*ctx), true, &plan)) {
+            // One cooperative launch for the whole layer.
+            st = ensure_workspace(*ctx, (cs_floats + score_scratch_floats(plan, Hkv, R)) * sizeof(float));
+            if (st != CHUNKKV_OK) return st;
+            char* base = static_cast<char*>(ctx->ws);
+            float* payload = reinterpret_cast<float*>(base + kHeaderBytes);
+            ScoreArgs a;
+            a.L = L; a.P = L - w; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
+            a.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
+            score_scratch_layout(plan, Hkv, R, payload + cs_floats, &a);
+            a.status = reinterpret_cast<int*>(base);
+            CUtensorMap tm_q, tm_k;
+            st = encode_bf16_3d(&tm_q, q_obs, d, R, Hkv, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+            if (st != CHUNKKV_OK) return st;
+            st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < plan.n_tile ? L : plan.n_tile,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+            if (st != CHUNKKV_OK) return st;
+            FusedLayerIO io;
+            io.K = K; io.V = V; io.out_K = out_K; io.out_V = out_V; io.out_idx = out_idx;
+            io.chunk_scores = payload;
+            io.C = C; io.k = k; io.n_max = n_max;
+            io.bar_count = reinterpret_cast<unsigned*>(base + 64);
+            io.bar_gen = reinterpret_cast<unsigned*>(base + 128);
+            {
+                Timer t(ctx, s, 0);
+                e = launch_layer_fused(plan, tm_q, tm_k, a, io, s);
+            }
+            if (e != cudaSuccess) return cuda_fail(e);
+            return CHUNKKV_OK;
+        }
         st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, cs_floats, &chunk_scores, s);
         if (st != CHUNKKV_OK) return st;
     }

@@ -1,0 +1,63 @@
+// Device-side body of the K/V row gather (ChunkKV Algorithm 3 "index_select(K, indices)" /
+// "index_select(V, indices)"), shared by the stand-alone gather kernel and the fused layer kernel.
+//
+// Rows are d bf16 = 128 or 256 bytes. Each thread moves 16 bytes of a row; a row is covered by
+// d/8 adjacent threads, so every warp request is a set of fully used 128-byte lines. Each
+// thread handles kGatherRowsPerThread rows of K and of V with all loads issued before the stores.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace chunkkv {
+
+constexpr int kGatherRowsPerThread = 4;
+
+__device__ __forceinline__ uint4 gather_ld(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void gather_st(uint4* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+                 "r"(v.w)
+                 : "memory");
+}
+
+// Work item `item` of `n_items` (a CTA-sized slab of rows of one head); threads = nthreads
+// (a multiple of VPR). VPR = 16-byte vectors per row: 8 (d = 64) or 16 (d = 128).
+// FRESH_IDX: the indices were written earlier in the same kernel launch, so they must not be
+// read through the non-coherent path.
+template <int VPR, bool FRESH_IDX>
+__device__ __forceinline__ void gather_rows(const uint4* __restrict__ Kh, const uint4* __restrict__ Vh,
+                                            const int32_t* ih, int L, int n_max, int n0, int tid, int nthreads,
+                                            uint4* __restrict__ oK, uint4* __restrict__ oV, int32_t* idx_copy) {
+    const int rows_per_pass = nthreads / VPR;
+    const int vec = tid % VPR, sub = tid / VPR;
+    int src[kGatherRowsPerThread];
+    uint4 kv[kGatherRowsPerThread], vv[kGatherRowsPerThread];
+#pragma unroll
+    for (int u = 0; u < kGatherRowsPerThread; ++u) {
+        const int n = n0 + u * rows_per_pass + sub;
+        if (n < n_max) src[u] = FRESH_IDX ? __ldcg(ih + n) : ih[n];
+        else src[u] = -1;
+    }
+#pragma unroll
+    for (int u = 0; u < kGatherRowsPerThread; ++u) {
+        const bool ok = static_cast<unsigned>(src[u]) < static_cast<unsigned>(L);
+        kv[u] = ok ? gather_ld(Kh + static_cast<size_t>(src[u]) * VPR + vec) : make_uint4(0, 0, 0, 0);
+        vv[u] = ok ? gather_ld(Vh + static_cast<size_t>(src[u]) * VPR + vec) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int u = 0; u < kGatherRowsPerThread; ++u) {
+        const int n = n0 + u * rows_per_pass + sub;
+        if (n < n_max) {
+            gather_st(oK + static_cast<size_t>(n) * VPR + vec, kv[u]);
+            gather_st(oV + static_cast<size_t>(n) * VPR + vec, vv[u]);
+            if (idx_copy != nullptr && vec == 0) idx_copy[n] = src[u];
+        }
+    }
+}
+
+}  // namespace chunkkv

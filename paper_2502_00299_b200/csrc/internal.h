@@ -33,7 +33,10 @@ struct ScoreArgs {
 };
 
 // Chooses kernel variant and tile geometry for a shape. Returns false if unsupported.
-bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_limit, ScorePlan* plan);
+// full_grid: launch one CTA per SM even if there are fewer tiles (the fused layer kernel wants
+// every SM for its later phases).
+bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_limit, bool full_grid,
+                     ScorePlan* plan);
 
 // Scratch floats needed for a plan (panel maxima + CTA records + partial sums), per layer.
 size_t score_scratch_floats(const ScorePlan& plan, int Hkv, int R);
@@ -43,6 +46,23 @@ void score_scratch_layout(const ScorePlan& plan, int Hkv, int R, float* base, Sc
 
 cudaError_t launch_score(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                          const ScoreArgs& args, cudaStream_t stream);
+
+// Inputs and outputs of the fused layer kernel beyond scoring.
+struct FusedLayerIO {
+    const void* K;
+    const void* V;
+    void* out_K;
+    void* out_V;
+    int32_t* out_idx;
+    float* chunk_scores;   // [Hkv, C] scratch
+    int C, k, n_max;
+    unsigned* bar_count;   // grid barrier words in the scratch header (zero between launches)
+    unsigned* bar_gen;
+};
+
+// The whole layer in one cooperative launch (plan made with full_grid = true, C > 0, k > 0).
+cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                               const ScoreArgs& args, const FusedLayerIO& io, cudaStream_t stream);
 
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
                             int num_sms, cudaStream_t stream);

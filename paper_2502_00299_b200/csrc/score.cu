@@ -16,8 +16,10 @@
 // finalisation kernel merges those records into global row maxima / sums and contracts the
 // partials over the rows:
 //     score[ch] = sum_i partial[ch, i] * exp2(m_panel[i] - m[i]) / l[i].
+#include "gather.cuh"
 #include "internal.h"
 #include "ptx.cuh"
+#include "select.cuh"
 
 #include <math_constants.h>
 
@@ -150,6 +152,187 @@ __device__ __forceinline__ void panel_general(const float (&v)[WP], float sl2, b
     *out_l = l;
 }
 
+constexpr int kFinThreads = 512;
+constexpr int kFinPanelCap = 24;      // panels whose scales fit in the finalize kernel's shared memory
+constexpr int kFinBatch = 4;          // chunks a warp reduces together
+
+struct FinGeom {
+    int n_panels;     // per head
+    int spp;
+    int wp;
+    int n_tiles;
+    int n_mt;
+    int score_grid;   // CTAs of the scoring launch
+    int hs_max;
+    int C;
+};
+
+struct RowStatSmem {
+    float red[kFinThreads];
+    int rec_base[256];
+};
+
+// Merge the records of the CTAs that touched head h into the global row maxima m[i] and
+// 1 / l[i] (written to gm / ginv, which may be shared or global memory). Block-wide: every
+// thread of the CTA must call it; the first kFinThreads threads work, each on a slice of the
+// records of one row so that the loads overlap.
+__device__ __forceinline__ void block_row_stats(const ScoreArgs& a, const FinGeom& g, int h, float* gm,
+                                                float* ginv, RowStatSmem& sm) {
+    const int tid = threadIdx.x;
+    // CTA b owns tiles [total*b/G, total*(b+1)/G): the owner of tile T is floor(((T+1)*G - 1) / total).
+    const long long total = static_cast<long long>(a.Hkv) * g.n_tiles;
+    const long long first_tile = static_cast<long long>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
+    const int b_lo = static_cast<int>(((first_tile + 1) * g.score_grid - 1) / total);
+    const int b_hi = static_cast<int>(((last_tile + 1) * g.score_grid - 1) / total);
+    const int nb = b_hi - b_lo + 1;                 // <= 256: the scoring grid is capped there
+    for (int j = tid; j < nb; j += blockDim.x) {
+        const int b = b_lo + j;
+        const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
+        sm.rec_base[j] = (b * g.hs_max + (h - head0)) * (kGroups * 256);
+    }
+    __syncthreads();
+    const int rp = (a.R > 128) ? 256 : 128;         // rows padded to the slice stride
+    const int ns = kFinThreads / rp;                // record slices per row
+    const int gpr = kGroups / g.n_mt;               // groups (records per CTA) that hold a given row
+    const int i = tid % rp, sl = tid / rp;
+    const bool work = tid < kFinThreads && i < a.R;
+    const int g0 = (g.n_mt == 2) ? (i >> 7) * gpr : 0;
+    const int rr = i & 127;
+    float m = -CUDART_INF_F;
+    if (work) {
+#pragma unroll 2
+        for (int j = sl; j < nb; j += ns) {
+            const float* rec = a.cta_stat + sm.rec_base[j] + g0 * 256 + rr;
+#pragma unroll 4
+            for (int q = 0; q < gpr; ++q) m = fmaxf(m, __ldcg(rec + q * 256));
+        }
+    }
+    if (tid < kFinThreads) sm.red[tid] = m;
+    __syncthreads();
+    float M = -CUDART_INF_F;
+    if (work) {
+        M = sm.red[i];
+        for (int s2 = 1; s2 < ns; ++s2) M = fmaxf(M, sm.red[s2 * rp + i]);
+    }
+    __syncthreads();
+    float l = 0.f;
+    if (work) {
+#pragma unroll 2
+        for (int j = sl; j < nb; j += ns) {
+            const float* rec = a.cta_stat + sm.rec_base[j] + g0 * 256 + rr;
+#pragma unroll 4
+            for (int q = 0; q < gpr; ++q) {
+                const float rm = __ldcg(rec + q * 256);
+                l += (rm == -CUDART_INF_F) ? 0.f : __ldcg(rec + q * 256 + 128) * ex2_approx(rm - M);
+            }
+        }
+    }
+    if (tid < kFinThreads) sm.red[tid] = l;
+    __syncthreads();
+    if (work && sl == 0) {
+        float lt = sm.red[i];
+        for (int s2 = 1; s2 < ns; ++s2) lt += sm.red[s2 * rp + i];
+        gm[i] = M;
+        ginv[i] = 1.0f / lt;
+    }
+    __syncthreads();
+}
+
+// Chunk scores of the chunks that start in panels [p_lo, p_hi) of head h, whose scales
+// f[p - p_lo][i] = exp2(m_panel - m) / l are staged in `fs` (row stride fs_stride). A chunk
+// that continues past p_hi takes the scale of the later panels from global memory. One warp
+// reduces kFinBatch chunks at a time; fixed order, so results are deterministic.
+__device__ __forceinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& g, int h, int p_lo, int p_hi,
+                                                int ch0, int ch1, const float* fs, int fs_stride,
+                                                const float* gm, const float* ginv, float* __restrict__ out) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+    const size_t stat_base = static_cast<size_t>(h) * g.n_panels * a.R;
+    const size_t part_base = static_cast<size_t>(h) * g.n_panels * g.spp * a.R;
+    for (int cb = ch0 + warp * kFinBatch; cb < ch1; cb += nwarps * kFinBatch) {
+        float acc[kFinBatch];
+        bool single = true;
+        int pa[kFinBatch];
+        size_t po[kFinBatch];
+#pragma unroll
+        for (int u = 0; u < kFinBatch; ++u) {
+            const int ch = min(cb + u, ch1 - 1);
+            const int ja = ch * a.c, jb = min(ja + a.c, a.P);
+            pa[u] = ja / g.wp;
+            single = single && (pa[u] == (jb - 1) / g.wp) && pa[u] >= p_lo && pa[u] < p_hi;
+            po[u] = part_base + (static_cast<size_t>(pa[u]) * g.spp + (ch - (pa[u] * g.wp) / a.c)) * a.R;
+            acc[u] = 0.f;
+        }
+        if (single) {       // every chunk of the batch lies in one staged panel: all loads are independent
+            for (int i = lane; i < a.R; i += 32) {
+#pragma unroll
+                for (int u = 0; u < kFinBatch; ++u)
+                    acc[u] += __ldcg(a.partial + po[u] + i) * fs[(pa[u] - p_lo) * fs_stride + i];
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < kFinBatch; ++u) {
+                const int ch = min(cb + u, ch1 - 1);
+                const int ja = ch * a.c, jb = min(ja + a.c, a.P);
+                for (int p = ja / g.wp; p <= (jb - 1) / g.wp; ++p) {
+                    const size_t o = part_base + (static_cast<size_t>(p) * g.spp + (ch - (p * g.wp) / a.c)) * a.R;
+                    const size_t so = stat_base + static_cast<size_t>(p) * a.R;
+                    for (int i = lane; i < a.R; i += 32)
+                        acc[u] += __ldcg(a.partial + o + i) * (ex2_approx(__ldcg(a.stat_m + so + i) - gm[i]) * ginv[i]);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kFinBatch; ++u) {
+            float v = acc[u];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            if (lane == 0 && cb + u < ch1) out[static_cast<size_t>(h) * g.C + cb + u] = v;
+        }
+    }
+}
+
+// Everything the fused layer kernel needs beyond scoring.
+struct LayerArgs {
+    const uint4* K;
+    const uint4* V;
+    uint4* out_K;
+    uint4* out_V;
+    int32_t* out_idx;
+    float* chunk_scores;   // [Hkv, C]
+    int C, k, n_max;
+    unsigned* bar_count;   // grid barrier state (zero between launches)
+    unsigned* bar_gen;
+};
+
+// Grid-wide barrier for a cooperative launch (all CTAs co-resident). Sense is carried by a
+// generation word, so the state needs no reset between launches. The wait is bounded: on
+// expiry the CTA raises its abort flag and the caller leaves the kernel.
+__device__ __forceinline__ bool grid_barrier(unsigned* count, unsigned* gen, unsigned nblocks, int* ok_smem,
+                                             volatile int* abort_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        bool ok = true;
+        const unsigned my_gen = *reinterpret_cast<volatile unsigned*>(gen);
+        __threadfence();
+        if (atomicAdd(count, 1u) == nblocks - 1) {
+            *reinterpret_cast<volatile unsigned*>(count) = 0u;
+            __threadfence();
+            atomicAdd(gen, 1u);
+        } else {
+            const long long t0 = clock64();
+            while (*reinterpret_cast<volatile unsigned*>(gen) == my_gen) {
+                if (clock64() - t0 > kWaitLimitClocks) { ok = false; break; }
+                __nanosleep(20);
+            }
+        }
+        __threadfence();
+        if (!ok) *abort_flag = 1;
+        *ok_smem = ok ? 1 : 0;
+    }
+    __syncthreads();
+    return *ok_smem != 0;
+}
+
 struct KernelGeom {
     int n_tiles;      // accumulator tiles per head
     int spp;          // chunk slots per panel
@@ -158,12 +341,17 @@ struct KernelGeom {
     int q_box_rows;   // rows delivered per Q box (min(128, R))
     int k_box_rows;   // rows delivered per K box (min(n_tile, L))
     int hs_max;       // head records per CTA in cta_stat
+    int dyn_bytes;    // usable dynamic shared memory after 1024-byte alignment
 };
 
-template <int C_STATIC, int N_MT, int N_TILE>
+// FUSED = false: scoring only (chunkkv_score). FUSED = true: the whole layer in one cooperative
+// launch - after scoring, a grid barrier, then every CTA turns the partial sums of its own
+// panels into chunk scores, a second barrier, top-k selection (one CTA per head), a third
+// barrier, and the K/V gather on all CTAs.
+template <int C_STATIC, int N_MT, int N_TILE, bool FUSED>
 __global__ void __launch_bounds__(kThreads, 1)
 score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-             const ScoreArgs a, const KernelGeom g) {
+             const ScoreArgs a, const KernelGeom g, const LayerArgs la) {
     static_assert(N_MT == 1 || N_MT == 2, "one or two 128-row query tiles");
     static_assert(N_TILE % 16 == 0 && N_TILE * N_MT <= 256, "accumulator tiles must fit half of TMEM");
     constexpr int NQBUF = (N_MT == 1) ? 2 : 1;
@@ -389,7 +577,96 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
-    if (threadIdx.x == 0 && ctl.abort_flag) atomicExch(a.status, 1);
+    if (ctl.abort_flag) {
+        if (threadIdx.x == 0) atomicExch(a.status, 1);
+        return;
+    }
+    if constexpr (FUSED) {
+        // The K ring and the Q buffers are idle from here on: reuse the dynamic shared memory.
+        uint8_t* dyn = smem_raw + (smem_base - smem_u32(smem_raw));
+        RowStatSmem& rs = *reinterpret_cast<RowStatSmem*>(dyn);
+        float* gm = reinterpret_cast<float*>(dyn + sizeof(RowStatSmem));
+        float* ginv = gm + 256;
+        float* fs = ginv + 256;
+        const int fs_cap = (g.dyn_bytes - static_cast<int>(sizeof(RowStatSmem)) - 2048) / 4;   // floats
+        SelectSmem& ss = *reinterpret_cast<SelectSmem*>(dyn);
+        int* bar_ok = reinterpret_cast<int*>(&ctl.tmem_base);     // free again after the dealloc
+        FinGeom fg;
+        fg.n_panels = g.n_tiles * PPT * SUBS;
+        fg.spp = g.spp;
+        fg.wp = WPP;
+        fg.n_tiles = g.n_tiles;
+        fg.n_mt = N_MT;
+        fg.score_grid = gridDim.x;
+        fg.hs_max = g.hs_max;
+        fg.C = la.C;
+        constexpr int PPTT = PPT * SUBS;               // panels per tile
+
+        if (!grid_barrier(la.bar_count, la.bar_gen, gridDim.x, bar_ok, abort_flag)) {
+            if (threadIdx.x == 0) atomicExch(a.status, 1);
+            return;
+        }
+        // ---- chunk scores of the panels this CTA scored
+        for (int t = t_begin; t < t_end;) {
+            const int head = t / g.n_tiles;
+            const int seg_end = min(t_end, (head + 1) * g.n_tiles);
+            block_row_stats(a, fg, head, gm, ginv, rs);
+            const int max_tiles = max(1, fs_cap / (PPTT * a.R));
+            const size_t stat_base = static_cast<size_t>(head) * fg.n_panels * a.R;
+            for (int ta = t; ta < seg_end; ta += max_tiles) {
+                const int tb = min(seg_end, ta + max_tiles);
+                const int p_lo = (ta - head * g.n_tiles) * PPTT, p_hi = (tb - head * g.n_tiles) * PPTT;
+                const int n = (p_hi - p_lo) * a.R;
+                for (int e = threadIdx.x; e < n; e += kThreads) {
+                    const int pp = e / a.R, i = e - pp * a.R;
+                    fs[e] = ex2_approx(__ldcg(a.stat_m + stat_base + static_cast<size_t>(p_lo + pp) * a.R + i) - gm[i]) *
+                            ginv[i];
+                }
+                __syncthreads();
+                const int key_a = p_lo * WPP, key_b = min(p_hi * WPP, a.P);
+                if (key_a < key_b)   // chunks whose first key lies in [key_a, key_b)
+                    contract_chunks(a, fg, head, p_lo, p_hi, (key_a + a.c - 1) / a.c, (key_b + a.c - 1) / a.c, fs,
+                                    a.R, gm, ginv, la.chunk_scores);
+                __syncthreads();
+            }
+            t = seg_end;
+        }
+        if (!grid_barrier(la.bar_count, la.bar_gen, gridDim.x, bar_ok, abort_flag)) {
+            if (threadIdx.x == 0) atomicExch(a.status, 1);
+            return;
+        }
+        // ---- top-k selection: one CTA per head
+        for (int h = blockIdx.x; h < a.Hkv; h += gridDim.x) {
+            const float* sc = la.chunk_scores + static_cast<size_t>(h) * la.C;
+            int32_t* out = la.out_idx + static_cast<size_t>(h) * la.n_max;
+            if (la.C <= kThreads * kSelPerThread)
+                select_head<true>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+            else
+                select_head<false>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+        }
+        if (!grid_barrier(la.bar_count, la.bar_gen, gridDim.x, bar_ok, abort_flag)) {
+            if (threadIdx.x == 0) atomicExch(a.status, 1);
+            return;
+        }
+        // ---- gather: slabs of rows of one head, round-robin over the CTAs
+        const int vpr = a.d >> 3;
+        const int rows_per_item = (kThreads / vpr) * kGatherRowsPerThread;
+        const int items_per_head = (la.n_max + rows_per_item - 1) / rows_per_item;
+        for (int it = blockIdx.x; it < items_per_head * a.Hkv; it += gridDim.x) {
+            const int h = it / items_per_head, n0 = (it - h * items_per_head) * rows_per_item;
+            const int32_t* ih = la.out_idx + static_cast<size_t>(h) * la.n_max;
+            if (vpr == 16)
+                gather_rows<16, true>(la.K + static_cast<size_t>(h) * a.L * 16, la.V + static_cast<size_t>(h) * a.L * 16, ih,
+                                      a.L, la.n_max, n0, threadIdx.x, kThreads,
+                                      la.out_K + static_cast<size_t>(h) * la.n_max * 16,
+                                      la.out_V + static_cast<size_t>(h) * la.n_max * 16, nullptr);
+            else
+                gather_rows<8, true>(la.K + static_cast<size_t>(h) * a.L * 8, la.V + static_cast<size_t>(h) * a.L * 8, ih,
+                                     a.L, la.n_max, n0, threadIdx.x, kThreads,
+                                     la.out_K + static_cast<size_t>(h) * la.n_max * 8,
+                                     la.out_V + static_cast<size_t>(h) * la.n_max * 8, nullptr);
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -400,80 +677,11 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 //                    panels its chunks touch (kept in shared memory) and contracts
 //                    partial[ch][.] * f over the R rows, one warp working on four chunks at a time.
 // All reductions have a fixed order, so results are deterministic.
-constexpr int kFinThreads = 512;
-constexpr int kFinPanelCap = 24;      // panels whose scales fit in shared memory (24 x 256 floats)
-constexpr int kFinBatch = 4;          // chunks a warp reduces together
-
-struct FinGeom {
-    int n_panels;     // per head
-    int spp;
-    int wp;
-    int n_tiles;
-    int n_mt;
-    int score_grid;   // CTAs of the scoring launch
-    int hs_max;
-    int C;
-};
-
-// One block per KV head: merge the records of the CTAs that touched the head into the global
-// row maxima m[i] and 1 / l[i]. Every thread takes a slice of the records of one row, so the
-// loads overlap. Output: row_stat[h][0][i] = m, row_stat[h][1][i] = 1 / l.
 __global__ void __launch_bounds__(kFinThreads)
 rowstats_kernel(const ScoreArgs a, const FinGeom g) {
-    __shared__ float red[kFinThreads];
-    __shared__ int rec_base[256];
+    __shared__ RowStatSmem sm;
     const int h = blockIdx.x;
-    const int tid = threadIdx.x;
-    // CTA b owns tiles [total*b/G, total*(b+1)/G): the owner of tile T is floor(((T+1)*G - 1) / total).
-    const long long total = static_cast<long long>(a.Hkv) * g.n_tiles;
-    const long long first_tile = static_cast<long long>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
-    const int b_lo = static_cast<int>(((first_tile + 1) * g.score_grid - 1) / total);
-    const int b_hi = static_cast<int>(((last_tile + 1) * g.score_grid - 1) / total);
-    const int nb = b_hi - b_lo + 1;                 // <= 256: the scoring grid is capped there
-    for (int j = tid; j < nb; j += kFinThreads) {
-        const int b = b_lo + j;
-        const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
-        rec_base[j] = (b * g.hs_max + (h - head0)) * (kGroups * 256);
-    }
-    __syncthreads();
-    const int rp = (a.R > 128) ? 256 : 128;         // rows padded to the slice stride
-    const int ns = kFinThreads / rp;                // record slices per row
-    const int gpr = kGroups / g.n_mt;               // groups (records per CTA) that hold a given row
-    const int i = tid % rp, sl = tid / rp;
-    const int g0 = (g.n_mt == 2) ? (i >> 7) * gpr : 0;
-    const int rr = i & 127;
-    float m = -CUDART_INF_F;
-    if (i < a.R) {
-        for (int j = sl; j < nb; j += ns) {
-            const float* rec = a.cta_stat + rec_base[j] + g0 * 256 + rr;
-#pragma unroll 4
-            for (int q = 0; q < gpr; ++q) m = fmaxf(m, rec[q * 256]);
-        }
-    }
-    red[tid] = m;
-    __syncthreads();
-    float M = red[i];
-    for (int s2 = 1; s2 < ns; ++s2) M = fmaxf(M, red[s2 * rp + i]);
-    __syncthreads();
-    float l = 0.f;
-    if (i < a.R) {
-        for (int j = sl; j < nb; j += ns) {
-            const float* rec = a.cta_stat + rec_base[j] + g0 * 256 + rr;
-#pragma unroll 4
-            for (int q = 0; q < gpr; ++q) {
-                const float rm = rec[q * 256];
-                l += (rm == -CUDART_INF_F) ? 0.f : rec[q * 256 + 128] * ex2_approx(rm - M);
-            }
-        }
-    }
-    red[tid] = l;
-    __syncthreads();
-    if (sl == 0 && i < a.R) {
-        float lt = red[i];
-        for (int s2 = 1; s2 < ns; ++s2) lt += red[s2 * rp + i];
-        a.row_stat[static_cast<size_t>(h) * 512 + i] = M;
-        a.row_stat[static_cast<size_t>(h) * 512 + 256 + i] = 1.0f / lt;
-    }
+    block_row_stats(a, g, h, a.row_stat + static_cast<size_t>(h) * 512, a.row_stat + static_cast<size_t>(h) * 512 + 256, sm);
 }
 
 // grid = (blocks per head, Hkv): chunk scores from partial sums, see the header of this section.
@@ -489,74 +697,26 @@ finalize_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
         ginv[tid] = a.row_stat[static_cast<size_t>(h) * 512 + 256 + tid];
     }
     __syncthreads();
-
-    // 2. scales of the panels this block's chunks touch
     const int per_block = (g.C + gridDim.x - 1) / gridDim.x;
     const int ch0 = blockIdx.x * per_block, ch1 = min(ch0 + per_block, g.C);
     if (ch0 >= ch1) return;
     const int p_lo = (ch0 * a.c) / g.wp;
-    const int p_hi = (min(ch1 * a.c, a.P) - 1) / g.wp;
-    const bool staged = (p_hi - p_lo + 1) <= kFinPanelCap;
+    const int p_hi = min(p_lo + kFinPanelCap, (min(ch1 * a.c, a.P) - 1) / g.wp + 1);
     const size_t stat_base = static_cast<size_t>(h) * g.n_panels * a.R;
-    if (staged) {
-        const int n = (p_hi - p_lo + 1) * a.R;
-        for (int e = tid; e < n; e += kFinThreads) {
-            const int pp = e / a.R, i = e - pp * a.R;
-            fs[pp * 256 + i] =
-                ex2_approx(a.stat_m[stat_base + static_cast<size_t>(p_lo + pp) * a.R + i] - gm[i]) * ginv[i];
-        }
+    const int n = (p_hi - p_lo) * a.R;
+    for (int e = tid; e < n; e += kFinThreads) {
+        const int pp = e / a.R, i = e - pp * a.R;
+        fs[pp * 256 + i] =
+            ex2_approx(a.stat_m[stat_base + static_cast<size_t>(p_lo + pp) * a.R + i] - gm[i]) * ginv[i];
     }
     __syncthreads();
-
-    // 3. chunks -> scores
-    const int warp = tid >> 5, lane = tid & 31, nwarps = kFinThreads >> 5;
-    const size_t part_base = static_cast<size_t>(h) * g.n_panels * g.spp * a.R;
-    for (int cb = ch0 + warp * kFinBatch; cb < ch1; cb += nwarps * kFinBatch) {
-        float acc[kFinBatch];
-        bool single = staged;
-        int pa[kFinBatch];
-        size_t po[kFinBatch];
-#pragma unroll
-        for (int u = 0; u < kFinBatch; ++u) {
-            const int ch = min(cb + u, ch1 - 1);
-            const int ja = ch * a.c, jb = min(ja + a.c, a.P);
-            pa[u] = ja / g.wp;
-            single = single && (pa[u] == (jb - 1) / g.wp);
-            po[u] = part_base + (static_cast<size_t>(pa[u]) * g.spp + (ch - (pa[u] * g.wp) / a.c)) * a.R;
-            acc[u] = 0.f;
-        }
-        if (single) {       // every chunk of the batch lies in one panel: all loads are independent
-            for (int i = lane; i < a.R; i += 32) {
-#pragma unroll
-                for (int u = 0; u < kFinBatch; ++u) acc[u] += a.partial[po[u] + i] * fs[(pa[u] - p_lo) * 256 + i];
-            }
-        } else {
-#pragma unroll
-            for (int u = 0; u < kFinBatch; ++u) {
-                const int ch = min(cb + u, ch1 - 1);
-                const int ja = ch * a.c, jb = min(ja + a.c, a.P);
-                for (int p = ja / g.wp; p <= (jb - 1) / g.wp; ++p) {
-                    const size_t o = part_base + (static_cast<size_t>(p) * g.spp + (ch - (p * g.wp) / a.c)) * a.R;
-                    const size_t so = stat_base + static_cast<size_t>(p) * a.R;
-                    for (int i = lane; i < a.R; i += 32)
-                        acc[u] += a.partial[o + i] * (ex2_approx(a.stat_m[so + i] - gm[i]) * ginv[i]);
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < kFinBatch; ++u) {
-            float v = acc[u];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-            if (lane == 0 && cb + u < ch1) out[static_cast<size_t>(h) * g.C + cb + u] = v;
-        }
-    }
+    contract_chunks(a, g, h, p_lo, p_hi, ch0, ch1, fs, 256, gm, ginv, out);
 }
 
-template <int C_STATIC, int N_MT, int N_TILE>
+template <int C_STATIC, int N_MT, int N_TILE, bool FUSED>
 cudaError_t launch_variant(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                           const ScoreArgs& args, cudaStream_t stream) {
-    auto kern = score_kernel<C_STATIC, N_MT, N_TILE>;
+                           const ScoreArgs& args, const LayerArgs& la, cudaStream_t stream) {
+    auto kern = score_kernel<C_STATIC, N_MT, N_TILE, FUSED>;
     // Opt in to large dynamic shared memory once per device and variant (not a stream operation,
     // so later launches stay free of it, e.g. inside a stream capture).
     static int smem_set[64] = {0};
@@ -576,13 +736,35 @@ cudaError_t launch_variant(const ScorePlan& plan, const CUtensorMap& tm_q, const
     g.q_box_rows = args.R < 128 ? args.R : 128;
     g.k_box_rows = args.L < N_TILE ? args.L : N_TILE;
     g.hs_max = plan.hs_max;
-    kern<<<plan.grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_k, args, g);
-    return cudaGetLastError();
+    g.dyn_bytes = plan.smem_bytes - 1024;
+    if constexpr (FUSED) {
+        // Cooperative launch: the grid barriers need every CTA resident (one per SM).
+        void* params[] = {const_cast<CUtensorMap*>(&tm_q), const_cast<CUtensorMap*>(&tm_k),
+                          const_cast<ScoreArgs*>(&args), &g, const_cast<LayerArgs*>(&la)};
+        return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kern), dim3(plan.grid), dim3(kThreads),
+                                           params, static_cast<size_t>(plan.smem_bytes), stream);
+    } else {
+        kern<<<plan.grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_k, args, g, la);
+        return cudaGetLastError();
+    }
+}
+
+template <bool FUSED>
+cudaError_t dispatch_variant(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                             const ScoreArgs& args, const LayerArgs& la, cudaStream_t stream) {
+    if (plan.n_mt == 1) {
+        if (plan.c_static == 10) return launch_variant<10, 1, 240, FUSED>(plan, tm_q, tm_k, args, la, stream);
+        if (plan.c_static == 20) return launch_variant<20, 1, 240, FUSED>(plan, tm_q, tm_k, args, la, stream);
+        if (plan.c_static == 1) return launch_variant<1, 1, 256, FUSED>(plan, tm_q, tm_k, args, la, stream);
+        return launch_variant<0, 1, 256, FUSED>(plan, tm_q, tm_k, args, la, stream);
+    }
+    return launch_variant<0, 2, 128, FUSED>(plan, tm_q, tm_k, args, la, stream);
 }
 
 }  // namespace
 
-bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_limit, ScorePlan* plan) {
+bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_limit, bool full_grid,
+                     ScorePlan* plan) {
     if (R < 1 || R > 256 || (d != 64 && d != 128) || c < 1 || L < 1 || Hkv < 1 || num_sms < 1) return false;
     ScorePlan p{};
     p.n_mt = (R + 127) / 128;
@@ -597,7 +779,7 @@ bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_
     p.n_panels = p.n_tiles * (p.n_tile / p.wp);
     p.spp = p.c_static ? p.wp / p.c_static : (p.wp + c - 1) / c + 1;
     const long long total = static_cast<long long>(Hkv) * p.n_tiles;
-    p.grid = static_cast<int>(total < num_sms ? total : num_sms);
+    p.grid = static_cast<int>((total < num_sms && !full_grid) ? total : num_sms);
     if (p.grid > 256) p.grid = 256;   // rowstats_kernel indexes at most 256 CTA records per head
     const int tiles_per_cta = static_cast<int>((total + p.grid - 1) / p.grid);
     p.hs_max = (tiles_per_cta + p.n_tiles - 1) / p.n_tiles + 1;
@@ -630,13 +812,25 @@ void score_scratch_layout(const ScorePlan& plan, int Hkv, int R, float* base, Sc
 
 cudaError_t launch_score(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                          const ScoreArgs& args, cudaStream_t stream) {
-    if (plan.n_mt == 1) {
-        if (plan.c_static == 10) return launch_variant<10, 1, 240>(plan, tm_q, tm_k, args, stream);
-        if (plan.c_static == 20) return launch_variant<20, 1, 240>(plan, tm_q, tm_k, args, stream);
-        if (plan.c_static == 1) return launch_variant<1, 1, 256>(plan, tm_q, tm_k, args, stream);
-        return launch_variant<0, 1, 256>(plan, tm_q, tm_k, args, stream);
-    }
-    return launch_variant<0, 2, 128>(plan, tm_q, tm_k, args, stream);
+    LayerArgs none{};
+    return dispatch_variant<false>(plan, tm_q, tm_k, args, none, stream);
+}
+
+cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                               const ScoreArgs& args, const FusedLayerIO& io, cudaStream_t stream) {
+    LayerArgs la;
+    la.K = static_cast<const uint4*>(io.K);
+    la.V = static_cast<const uint4*>(io.V);
+    la.out_K = static_cast<uint4*>(io.out_K);
+    la.out_V = static_cast<uint4*>(io.out_V);
+    la.out_idx = io.out_idx;
+    la.chunk_scores = io.chunk_scores;
+    la.C = io.C;
+    la.k = io.k;
+    la.n_max = io.n_max;
+    la.bar_count = io.bar_count;
+    la.bar_gen = io.bar_gen;
+    return dispatch_variant<true>(plan, tm_q, tm_k, args, la, stream);
 }
 
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
