@@ -187,8 +187,10 @@ __device__ __forceinline__ void block_row_stats(const ScoreArgs& a, const FinGeo
     const int nb = b_hi - b_lo + 1;                 // <= 256: the scoring grid is capped there
     for (int j = tid; j < nb; j += blockDim.x) {
         const int b = b_lo + j;
-        const int head0 = static_cast<int>((total * b / g.score_grid) / g.n_tiles);
-        sm.rec_base[j] = (b * g.hs_max + (h - head0)) * (kGroups * 256);
+        const long long tb0 = total * b / g.score_grid, tb1 = total * (b + 1) / g.score_grid;
+        const int head0 = static_cast<int>(tb0 / g.n_tiles);
+        // a CTA without tiles (more CTAs than tiles) wrote no record
+        sm.rec_base[j] = (tb1 > tb0) ? (b * g.hs_max + (h - head0)) * (kGroups * 256) : -1;
     }
     __syncthreads();
     const int rp = (a.R > 128) ? 256 : 128;         // rows padded to the slice stride
@@ -202,6 +204,7 @@ __device__ __forceinline__ void block_row_stats(const ScoreArgs& a, const FinGeo
     if (work) {
 #pragma unroll 2
         for (int j = sl; j < nb; j += ns) {
+            if (sm.rec_base[j] < 0) continue;
             const float* rec = a.cta_stat + sm.rec_base[j] + g0 * 256 + rr;
 #pragma unroll 4
             for (int q = 0; q < gpr; ++q) m = fmaxf(m, __ldcg(rec + q * 256));
@@ -219,6 +222,7 @@ __device__ __forceinline__ void block_row_stats(const ScoreArgs& a, const FinGeo
     if (work) {
 #pragma unroll 2
         for (int j = sl; j < nb; j += ns) {
+            if (sm.rec_base[j] < 0) continue;
             const float* rec = a.cta_stat + sm.rec_base[j] + g0 * 256 + rr;
 #pragma unroll 4
             for (int q = 0; q < gpr; ++q) {
