@@ -205,10 +205,17 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
     return CHUNKKV_OK;
 }
 
+// Scratch floats of the scoring kernels for a shape: the larger of the score-only launch and the
+// fused layer launch (which always uses one CTA per SM and so may keep more per-CTA records).
 size_t scratch_floats_for(const DeviceCtx& ctx, int L, int R, int Hkv, int d, int c) {
     ScorePlan plan;
-    if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), false, &plan)) return 0;
-    return score_scratch_floats(plan, Hkv, R);
+    size_t n = 0;
+    for (int full = 0; full < 2; ++full) {
+        if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), full != 0, &plan)) return 0;
+        const size_t f = score_scratch_floats(plan, Hkv, R);
+        n = f > n ? f : n;
+    }
+    return n;
 }
 
 }  // namespace
