@@ -169,6 +169,7 @@ struct FinGeom {
 
 struct RowStatSmem {
     float red[kFinThreads];
+    float red2[kFinThreads];
     int rec_base[256];
 };
 
@@ -200,43 +201,52 @@ __device__ __forceinline__ void block_row_stats(const ScoreArgs& a, const FinGeo
     const bool work = tid < kFinThreads && i < a.R;
     const int g0 = (g.n_mt == 2) ? (i >> 7) * gpr : 0;
     const int rr = i & 127;
-    float m = -CUDART_INF_F;
+    // Each thread folds its slice of the records into one (max, sum) pair. Records are fetched
+    // kRecBatch CTAs at a time with every load issued before the first use.
+    constexpr int kRecBatch = 6;
+    float M = -CUDART_INF_F, Lsum = 0.f;
     if (work) {
-#pragma unroll 2
-        for (int j = sl; j < nb; j += ns) {
-            if (sm.rec_base[j] < 0) continue;
-            const float* rec = a.cta_stat + sm.rec_base[j] + g0 * 256 + rr;
-#pragma unroll 4
-            for (int q = 0; q < gpr; ++q) m = fmaxf(m, __ldcg(rec + q * 256));
-        }
-    }
-    if (tid < kFinThreads) sm.red[tid] = m;
-    __syncthreads();
-    float M = -CUDART_INF_F;
-    if (work) {
-        M = sm.red[i];
-        for (int s2 = 1; s2 < ns; ++s2) M = fmaxf(M, sm.red[s2 * rp + i]);
-    }
-    __syncthreads();
-    float l = 0.f;
-    if (work) {
-#pragma unroll 2
-        for (int j = sl; j < nb; j += ns) {
-            if (sm.rec_base[j] < 0) continue;
-            const float* rec = a.cta_stat + sm.rec_base[j] + g0 * 256 + rr;
-#pragma unroll 4
-            for (int q = 0; q < gpr; ++q) {
-                const float rm = __ldcg(rec + q * 256);
-                l += (rm == -CUDART_INF_F) ? 0.f : __ldcg(rec + q * 256 + 128) * ex2_approx(rm - M);
+        for (int j0 = sl; j0 < nb; j0 += ns * kRecBatch) {
+            float rm[kRecBatch][kGroups], rl[kRecBatch][kGroups];
+#pragma unroll
+            for (int t = 0; t < kRecBatch; ++t) {
+                const int j = j0 + t * ns;
+                const int base = (j < nb) ? sm.rec_base[j] : -1;
+#pragma unroll
+                for (int q = 0; q < kGroups; ++q) {
+                    const bool have = base >= 0 && q < gpr;
+                    const float* rec = a.cta_stat + (have ? base : 0) + (g0 + (have ? q : 0)) * 256 + rr;
+                    rm[t][q] = have ? __ldcg(rec) : -CUDART_INF_F;
+                    rl[t][q] = have ? __ldcg(rec + 128) : 0.f;
+                }
             }
+            float bm = M;
+#pragma unroll
+            for (int t = 0; t < kRecBatch; ++t)
+#pragma unroll
+                for (int q = 0; q < kGroups; ++q) bm = fmaxf(bm, rm[t][q]);
+            float acc = (M == -CUDART_INF_F) ? 0.f : Lsum * ex2_approx(M - bm);
+#pragma unroll
+            for (int t = 0; t < kRecBatch; ++t)
+#pragma unroll
+                for (int q = 0; q < kGroups; ++q)
+                    acc += (rm[t][q] == -CUDART_INF_F) ? 0.f : rl[t][q] * ex2_approx(rm[t][q] - bm);
+            M = bm;
+            Lsum = acc;
         }
     }
-    if (tid < kFinThreads) sm.red[tid] = l;
+    float* red_m = sm.red;                           // [kFinThreads] maxima, sums in red2
+    if (tid < kFinThreads) { red_m[tid] = M; sm.red2[tid] = Lsum; }
     __syncthreads();
     if (work && sl == 0) {
-        float lt = sm.red[i];
-        for (int s2 = 1; s2 < ns; ++s2) lt += sm.red[s2 * rp + i];
-        gm[i] = M;
+        float gmax = M;
+        for (int s2 = 1; s2 < ns; ++s2) gmax = fmaxf(gmax, red_m[s2 * rp + i]);
+        float lt = 0.f;
+        for (int s2 = 0; s2 < ns; ++s2) {
+            const float pm = red_m[s2 * rp + i];
+            lt += (pm == -CUDART_INF_F) ? 0.f : sm.red2[s2 * rp + i] * ex2_approx(pm - gmax);
+        }
+        gm[i] = gmax;
         ginv[i] = 1.0f / lt;
     }
     __syncthreads();
@@ -316,20 +326,23 @@ __device__ __forceinline__ bool grid_barrier(unsigned* count, unsigned* gen, uns
     __syncthreads();
     if (threadIdx.x == 0) {
         bool ok = true;
-        const unsigned my_gen = *reinterpret_cast<volatile unsigned*>(gen);
-        __threadfence();
-        if (atomicAdd(count, 1u) == nblocks - 1) {
-            *reinterpret_cast<volatile unsigned*>(count) = 0u;
-            __threadfence();
-            atomicAdd(gen, 1u);
+        unsigned my_gen, old;
+        asm volatile("ld.relaxed.gpu.u32 %0, [%1];" : "=r"(my_gen) : "l"(gen) : "memory");
+        // release: everything this CTA wrote (ordered before by the barrier above) becomes visible
+        asm volatile("atom.add.release.gpu.u32 %0, [%1], 1;" : "=r"(old) : "l"(count) : "memory");
+        if (old == nblocks - 1) {
+            asm volatile("st.relaxed.gpu.u32 [%0], %1;" ::"l"(count), "r"(0u) : "memory");
+            asm volatile("red.release.gpu.add.u32 [%0], 1;" ::"l"(gen) : "memory");
         } else {
             const long long t0 = clock64();
-            while (*reinterpret_cast<volatile unsigned*>(gen) == my_gen) {
+            unsigned cur;
+            for (;;) {
+                asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(cur) : "l"(gen) : "memory");
+                if (cur != my_gen) break;
                 if (clock64() - t0 > kWaitLimitClocks) { ok = false; break; }
-                __nanosleep(20);
             }
         }
-        __threadfence();
+        asm volatile("fence.acq_rel.gpu;" ::: "memory");
         if (!ok) *abort_flag = 1;
         *ok_smem = ok ? 1 : 0;
     }
@@ -614,17 +627,42 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         for (int t = t_begin; t < t_end;) {
             const int head = t / g.n_tiles;
             const int seg_end = min(t_end, (head + 1) * g.n_tiles);
-            block_row_stats(a, fg, head, gm, ginv, rs);
             const int max_tiles = max(1, fs_cap / (PPTT * a.R));
             const size_t stat_base = static_cast<size_t>(head) * fg.n_panels * a.R;
+            // Panel maxima of the first batch of tiles are fetched into registers before the row
+            // statistics are computed, so that the two round trips to L2 overlap.
+            constexpr int kPF = 8;
+            float mp[kPF];
+            const int tb_first = min(seg_end, t + max_tiles);
+            const int p_first = (t - head * g.n_tiles) * PPTT;
+            const int n_first = (tb_first - t) * PPTT * a.R;
+            const bool prefetched = n_first <= kPF * kThreads;
+            if (prefetched) {
+#pragma unroll
+                for (int u = 0; u < kPF; ++u) {
+                    const int e = threadIdx.x + u * kThreads;
+                    mp[u] = (e < n_first) ? __ldcg(a.stat_m + stat_base + static_cast<size_t>(p_first) * a.R + e) : 0.f;
+                }
+            }
+            block_row_stats(a, fg, head, gm, ginv, rs);
             for (int ta = t; ta < seg_end; ta += max_tiles) {
                 const int tb = min(seg_end, ta + max_tiles);
                 const int p_lo = (ta - head * g.n_tiles) * PPTT, p_hi = (tb - head * g.n_tiles) * PPTT;
                 const int n = (p_hi - p_lo) * a.R;
-                for (int e = threadIdx.x; e < n; e += kThreads) {
-                    const int pp = e / a.R, i = e - pp * a.R;
-                    fs[e] = ex2_approx(__ldcg(a.stat_m + stat_base + static_cast<size_t>(p_lo + pp) * a.R + i) - gm[i]) *
-                            ginv[i];
+                if (ta == t && prefetched) {
+#pragma unroll
+                    for (int u = 0; u < kPF; ++u) {
+                        const int e = threadIdx.x + u * kThreads;
+                        if (e < n) {
+                            const int i = e % a.R;
+                            fs[e] = ex2_approx(mp[u] - gm[i]) * ginv[i];
+                        }
+                    }
+                } else {
+                    for (int e = threadIdx.x; e < n; e += kThreads) {
+                        const int i = e % a.R;
+                        fs[e] = ex2_approx(__ldcg(a.stat_m + stat_base + static_cast<size_t>(p_lo) * a.R + e) - gm[i]) * ginv[i];
+                    }
                 }
                 __syncthreads();
                 const int key_a = p_lo * WPP, key_b = min(p_hi * WPP, a.P);
@@ -652,23 +690,30 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             if (threadIdx.x == 0) atomicExch(a.status, 1);
             return;
         }
-        // ---- gather: slabs of rows of one head, round-robin over the CTAs
+        // ---- gather: the Hkv * n_max output rows are split evenly over the CTAs
         const int vpr = a.d >> 3;
-        const int rows_per_item = (kThreads / vpr) * kGatherRowsPerThread;
-        const int items_per_head = (la.n_max + rows_per_item - 1) / rows_per_item;
-        for (int it = blockIdx.x; it < items_per_head * a.Hkv; it += gridDim.x) {
-            const int h = it / items_per_head, n0 = (it - h * items_per_head) * rows_per_item;
+        const int rows_per_pass = (kThreads / vpr) * kGatherRowsPerThread;
+        const long long rows_total = static_cast<long long>(a.Hkv) * la.n_max;
+        const long long r_begin = rows_total * blockIdx.x / gridDim.x, r_end = rows_total * (blockIdx.x + 1) / gridDim.x;
+        for (long long r0 = r_begin; r0 < r_end;) {
+            const int h = static_cast<int>(r0 / la.n_max);
+            const int n0 = static_cast<int>(r0 - static_cast<long long>(h) * la.n_max);
+            // rows [n0, n_hi) of head h in this pass
+            const int n_hi = static_cast<int>(min(static_cast<long long>(la.n_max),
+                                                  min(r_end - static_cast<long long>(h) * la.n_max,
+                                                      static_cast<long long>(n0) + rows_per_pass)));
             const int32_t* ih = la.out_idx + static_cast<size_t>(h) * la.n_max;
             if (vpr == 16)
                 gather_rows<16, true>(la.K + static_cast<size_t>(h) * a.L * 16, la.V + static_cast<size_t>(h) * a.L * 16, ih,
-                                      a.L, la.n_max, n0, threadIdx.x, kThreads,
+                                      a.L, n_hi, n0, threadIdx.x, kThreads,
                                       la.out_K + static_cast<size_t>(h) * la.n_max * 16,
                                       la.out_V + static_cast<size_t>(h) * la.n_max * 16, nullptr);
             else
                 gather_rows<8, true>(la.K + static_cast<size_t>(h) * a.L * 8, la.V + static_cast<size_t>(h) * a.L * 8, ih,
-                                     a.L, la.n_max, n0, threadIdx.x, kThreads,
+                                     a.L, n_hi, n0, threadIdx.x, kThreads,
                                      la.out_K + static_cast<size_t>(h) * la.n_max * 8,
                                      la.out_V + static_cast<size_t>(h) * la.n_max * 8, nullptr);
+            r0 += n_hi - n0;
         }
     }
 }
