@@ -475,8 +475,7 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
             io.K = K; io.V = V; io.out_K = out_K; io.out_V = out_V; io.out_idx = out_idx;
             io.chunk_scores = payload;
             io.C = C; io.k = k; io.n_max = n_max;
-            io.bar_count = reinterpret_cast<unsigned*>(base + 64);
-            io.bar_gen = reinterpret_cast<unsigned*>(base + 128);
+            io.bar_count = reinterpret_cast<unsigned long long*>(base + 64);
             {
                 Timer t(ctx, s, 0);
                 e = launch_layer_fused(plan, tm_q, tm_k, a, io, s);

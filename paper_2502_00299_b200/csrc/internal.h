@@ -56,8 +56,7 @@ struct FusedLayerIO {
     int32_t* out_idx;
     float* chunk_scores;   // [Hkv, C] scratch
     int C, k, n_max;
-    unsigned* bar_count;   // grid barrier words in the scratch header (zero between launches)
-    unsigned* bar_gen;
+    unsigned long long* bar_count;   // grid barrier ticket counter in the scratch header
 };
 
 // The whole layer in one cooperative launch (plan made with full_grid = true, C > 0, k > 0).

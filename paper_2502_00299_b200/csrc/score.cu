@@ -276,11 +276,22 @@ __device__ __forceinline__ void contract_chunks(const ScoreArgs& a, const FinGeo
             po[u] = part_base + (static_cast<size_t>(pa[u]) * g.spp + (ch - (pa[u] * g.wp) / a.c)) * a.R;
             acc[u] = 0.f;
         }
-        if (single) {       // every chunk of the batch lies in one staged panel: all loads are independent
-            for (int i = lane; i < a.R; i += 32) {
+        if (single) {       // every chunk of the batch lies in one staged panel
+            // R <= 256 = 8 x 32 rows: issue every load of the batch before the first use
+            float pv[kFinBatch][8];
 #pragma unroll
-                for (int u = 0; u < kFinBatch; ++u)
-                    acc[u] += __ldcg(a.partial + po[u] + i) * fs[(pa[u] - p_lo) * fs_stride + i];
+            for (int it = 0; it < 8; ++it) {
+                const int i = lane + 32 * it;
+#pragma unroll
+                for (int u = 0; u < kFinBatch; ++u) pv[u][it] = (i < a.R) ? __ldcg(a.partial + po[u] + i) : 0.f;
+            }
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                const int i = lane + 32 * it;
+                if (i < a.R) {
+#pragma unroll
+                    for (int u = 0; u < kFinBatch; ++u) acc[u] += pv[u][it] * fs[(pa[u] - p_lo) * fs_stride + i];
+                }
             }
         } else {
 #pragma unroll
@@ -314,31 +325,30 @@ struct LayerArgs {
     int32_t* out_idx;
     float* chunk_scores;   // [Hkv, C]
     int C, k, n_max;
-    unsigned* bar_count;   // grid barrier state (zero between launches)
-    unsigned* bar_gen;
+    unsigned long long* bar_count;   // grid barrier ticket counter (a multiple of the grid size between launches)
 };
 
-// Grid-wide barrier for a cooperative launch (all CTAs co-resident). Sense is carried by a
-// generation word, so the state needs no reset between launches. The wait is bounded: on
-// expiry the CTA raises its abort flag and the caller leaves the kernel.
-__device__ __forceinline__ bool grid_barrier(unsigned* count, unsigned* gen, unsigned nblocks, int* ok_smem,
+// Grid-wide barrier for a cooperative launch (all CTAs co-resident). One 64-bit counter that
+// only ever grows: a CTA that drew ticket `old` waits until the counter reaches the next
+// multiple of the grid size, so nothing is reset and there is no second flag to publish.
+// Requires the counter to be a multiple of the grid size between launches (it is zeroed with
+// the scratch header and every launch on a device uses the same grid size). The wait is
+// bounded: on expiry the CTA raises its abort flag and the caller leaves the kernel.
+__device__ __forceinline__ bool grid_barrier(unsigned long long* count, unsigned nblocks, int* ok_smem,
                                              volatile int* abort_flag) {
     __syncthreads();
     if (threadIdx.x == 0) {
         bool ok = true;
-        unsigned my_gen, old;
-        asm volatile("ld.relaxed.gpu.u32 %0, [%1];" : "=r"(my_gen) : "l"(gen) : "memory");
+        unsigned long long old;
         // release: everything this CTA wrote (ordered before by the barrier above) becomes visible
-        asm volatile("atom.add.release.gpu.u32 %0, [%1], 1;" : "=r"(old) : "l"(count) : "memory");
-        if (old == nblocks - 1) {
-            asm volatile("st.relaxed.gpu.u32 [%0], %1;" ::"l"(count), "r"(0u) : "memory");
-            asm volatile("red.release.gpu.add.u32 [%0], 1;" ::"l"(gen) : "memory");
-        } else {
+        asm volatile("atom.add.release.gpu.u64 %0, [%1], 1;" : "=l"(old) : "l"(count) : "memory");
+        const unsigned long long target = (old / nblocks + 1ull) * nblocks;
+        if (old + 1ull != target) {
             const long long t0 = clock64();
-            unsigned cur;
+            unsigned long long cur;
             for (;;) {
-                asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(cur) : "l"(gen) : "memory");
-                if (cur != my_gen) break;
+                asm volatile("ld.acquire.gpu.u64 %0, [%1];" : "=l"(cur) : "l"(count) : "memory");
+                if (cur >= target) break;
                 if (clock64() - t0 > kWaitLimitClocks) { ok = false; break; }
             }
         }
@@ -619,7 +629,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         fg.C = la.C;
         constexpr int PPTT = PPT * SUBS;               // panels per tile
 
-        if (!grid_barrier(la.bar_count, la.bar_gen, gridDim.x, bar_ok, abort_flag)) {
+        if (!grid_barrier(la.bar_count, gridDim.x, bar_ok, abort_flag)) {
             if (threadIdx.x == 0) atomicExch(a.status, 1);
             return;
         }
@@ -673,7 +683,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             }
             t = seg_end;
         }
-        if (!grid_barrier(la.bar_count, la.bar_gen, gridDim.x, bar_ok, abort_flag)) {
+        if (!grid_barrier(la.bar_count, gridDim.x, bar_ok, abort_flag)) {
             if (threadIdx.x == 0) atomicExch(a.status, 1);
             return;
         }
@@ -686,7 +696,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             else
                 select_head<false>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
         }
-        if (!grid_barrier(la.bar_count, la.bar_gen, gridDim.x, bar_ok, abort_flag)) {
+        if (!grid_barrier(la.bar_count, gridDim.x, bar_ok, abort_flag)) {
             if (threadIdx.x == 0) atomicExch(a.status, 1);
             return;
         }
@@ -878,7 +888,6 @@ cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, c
     la.k = io.k;
     la.n_max = io.n_max;
     la.bar_count = io.bar_count;
-    la.bar_gen = io.bar_gen;
     return dispatch_variant<true>(plan, tm_q, tm_k, args, la, stream);
 }
 
