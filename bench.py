@@ -47,6 +47,7 @@ def parse_args():
     ap.add_argument("--config", type=int, default=2, help="workload table entry (2 = headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--lanes", type=int, default=4, help="layers in flight (each on 1/lanes of the SMs)")
     return ap.parse_args()
 
 
@@ -217,51 +218,81 @@ def run_ours(args, wl):
         x = make_layer(wl, layer=i, seq=rank)
         hosts.append(x)
         t = [torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16) for b in (x.q_obs, x.K, x.V)]
-        outs = [torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device=dev) for _ in range(2)]
-        outs.append(torch.empty((wl.Hkv, n_max), dtype=torch.int32, device=dev))
-        sets.append((t, outs))
+        sets.append((t,))
 
-    def call_layer(i: int, stream_ptr):
-        (q, K, V), (oK, oV, oI) = sets[i % NSETS]
-        st = lib.chunkkv_compress_layer(q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d,
-                                        wl.w, wl.c, wl.budget, None, oK.data_ptr(), oV.data_ptr(),
-                                        oI.data_ptr(), stream_ptr)
+    # ---- lanes: S layers in flight, each on its own stream with 1/S of the SMs and its own scratch
+    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+    S = max(1, args.lanes)
+    stream = torch.cuda.Stream(device=dev)
+    lanes = []
+    if S > 1:
+        for li in range(S):
+            ln = ck.Lane(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=n_sm // S, device=dev,
+                         stream=stream if li == 0 else None)
+            lanes.append(ln)
+    lane_streams = [ln.stream for ln in lanes] if lanes else [stream]
+    # every lane writes its own output buffers (layers in flight never share an output)
+    lane_outs = []
+    for _ in range(S):
+        o = [torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+        o.append(torch.empty((wl.Hkv, n_max), dtype=torch.int32, device=dev))
+        lane_outs.append(o)
+
+    def call_layer(i: int, reuse: bool = False, single: bool = False):
+        q, K, V = sets[i % NSETS][0]
+        li = 0 if single else i % S
+        oK, oV, oI = lane_outs[li]
+        if S > 1 and not single:
+            ln = lanes[li]
+            st = lib.chunkkv_compress_layer_lane(
+                None if reuse else q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
+                wl.budget, oI.data_ptr() if reuse else None, oK.data_ptr(), oV.data_ptr(), oI.data_ptr(),
+                ln.buf.data_ptr(), ln.bytes, ln.max_ctas, ln.stream.cuda_stream)
+        else:
+            st = lib.chunkkv_compress_layer(
+                None if reuse else q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
+                wl.budget, oI.data_ptr() if reuse else None, oK.data_ptr(), oV.data_ptr(), oI.data_ptr(),
+                stream.cuda_stream)
         if st != 0:
             raise ck.ChunkKVError(st, "chunkkv_compress_layer")
 
-    def call_reuse(i: int, stream_ptr):
-        (q, K, V), (oK, oV, oI) = sets[i % NSETS]
-        st = lib.chunkkv_compress_layer(None, K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d,
-                                        wl.w, wl.c, wl.budget, oI.data_ptr(), oK.data_ptr(), oV.data_ptr(),
-                                        oI.data_ptr(), stream_ptr)
-        if st != 0:
-            raise ck.ChunkKVError(st, "chunkkv_compress_layer(reuse)")
-
-    stream = torch.cuda.Stream(device=dev)
-    sp = stream.cuda_stream
-
-    def step_eager(fn=call_layer):
+    def issue_step(reuse: bool = False, single: bool = False):
+        """One step = LAYERS_PER_STEP layers; lane streams fork from and join back into `stream`."""
+        multi = S > 1 and not single
+        if multi:
+            ev = torch.cuda.Event()
+            ev.record(stream)
+            for st_ in lane_streams[1:]:
+                st_.wait_event(ev)
         for i in range(LAYERS_PER_STEP):
-            fn(i, sp)
+            call_layer(i, reuse, single)
+        if multi:
+            for st_ in lane_streams[1:]:
+                ev = torch.cuda.Event()
+                ev.record(st_)
+                stream.wait_event(ev)
+
+    def step_eager():
+        issue_step()
 
     with torch.cuda.stream(stream):
         for _ in range(max(args.warmup, 3)):
-            step_eager()
+            issue_step()
+            issue_step(single=True)
     torch.cuda.synchronize()
-    if ck.device_status(stream) != 0:
+    if ck.device_status(stream) != 0 or any(ln.status() != 0 for ln in lanes):
         raise RuntimeError("a kernel reported an abandoned wait during warm-up")
 
     # ---- the step as a CUDA graph
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph, stream=stream):
-        cur = torch.cuda.current_stream().cuda_stream
-        for i in range(LAYERS_PER_STEP):
-            call_layer(i, cur)
-    reuse_graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(reuse_graph, stream=stream):
-        cur = torch.cuda.current_stream().cuda_stream
-        for i in range(LAYERS_PER_STEP):
-            call_reuse(i, cur)
+    def capture(**kw):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr, stream=stream):
+            issue_step(**kw)
+        return gr
+
+    graph = capture()
+    reuse_graph = capture(reuse=True)
+    single_graph = capture(single=True)        # one layer at a time on the whole GPU
 
     def timed(fn, steps):
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -278,6 +309,7 @@ def run_ours(args, wl):
         for _ in range(max(args.warmup, 3)):
             graph.replay()
             reuse_graph.replay()
+            single_graph.replay()
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     except Exception:
@@ -291,15 +323,16 @@ def run_ours(args, wl):
     ms_per_step = ms_max / args.steps
     ms_layer = ms_per_step / LAYERS_PER_STEP
 
-    # ---- the same step, call by call (no graph), and gather-only (index reuse) layers
+    # ---- the same step, call by call (no graph); gather-only (index reuse) layers; one layer at a time
     eager_steps = max(3, min(args.steps, 100))
     ms_eager = max_over_ranks(timed(step_eager, eager_steps), dev) / eager_steps
     ms_reuse = max_over_ranks(timed(reuse_graph.replay, eager_steps), dev) / eager_steps / LAYERS_PER_STEP
+    ms_single = max_over_ranks(timed(single_graph.replay, eager_steps), dev) / eager_steps / LAYERS_PER_STEP
 
     # ---- per-kernel durations (CUDA events around every kernel, on the launching stream)
     ck.profile_enable(True)
     prof_steps = max(3, min(args.steps, 30))
-    timed(step_eager, prof_steps)
+    timed(lambda: issue_step(single=True), prof_steps)      # one layer at a time: each kernel has the GPU to itself
     ms_slot, n_slot = ck.profile_read()
     ck.profile_enable(False)
     names = ("score", "finalize", "select", "gather")
@@ -317,12 +350,19 @@ def run_ours(args, wl):
     roofline = {"kernel": "score_kernel<FUSED> (score+chunk-sum+select+gather in one launch)" if fused else "score_kernel",
                 "bound": "hbm", "achieved": achieved, "peak": peak,
                 "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
-                "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_us": score_us}
+                "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_us": score_us,
+                "note": "kernel timed with the GPU to itself (one layer at a time); the step overlaps "
+                        f"{S} such launches on disjoint SM sets"}
     layer_gbs = nbytes["layer"] / (ms_layer * 1e-3) / 1e9
     gather_us = per_kernel["gather"]["avg_us"] or float("nan")   # nan when the layer kernel is fused
     extra_roof = {
-        "layer_call": {"algorithmic_bytes": nbytes["layer"], "us": ms_layer * 1e3, "GB/s": layer_gbs,
-                       "frac_of_measured_peak": layer_gbs / peak, "frac_of_8TBs": layer_gbs / NOMINAL_HBM_GBS},
+        "layer_throughput": {"algorithmic_bytes": nbytes["layer"], "us_per_layer": ms_layer * 1e3, "GB/s": layer_gbs,
+                             "frac_of_measured_peak": layer_gbs / peak, "frac_of_8TBs": layer_gbs / NOMINAL_HBM_GBS,
+                             "lanes": S},
+        "single_layer": {"algorithmic_bytes": nbytes["layer"], "us": ms_single * 1e3,
+                         "GB/s": nbytes["layer"] / (ms_single * 1e-3) / 1e9,
+                         "frac_of_measured_peak": nbytes["layer"] / (ms_single * 1e-3) / 1e9 / peak,
+                         "note": "layers one after another, each on all SMs"},
         "gather_kernel": {"algorithmic_bytes": nbytes["gather"], "us": gather_us,
                           "GB/s": nbytes["gather"] / (gather_us * 1e-6) / 1e9,
                           "frac_of_measured_peak": nbytes["gather"] / (gather_us * 1e-6) / 1e9 / peak},
@@ -343,12 +383,13 @@ def run_ours(args, wl):
 
         def step_e2e():
             for i in range(LAYERS_PER_STEP):
-                (q, K, V), (oK, oV, oI) = sets[i % NSETS]
+                q, K, V = sets[i % NSETS][0]
+                oK, oV, oI = lane_outs[0]
                 hq, hK, hV = pin[i % NSETS]
                 st = lib.chunkkv_compress_layer_host(
                     hq.data_ptr(), hK.data_ptr(), hV.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
                     wl.budget, q.data_ptr(), K.data_ptr(), V.data_ptr(), oK.data_ptr(), oV.data_ptr(),
-                    oI.data_ptr(), h_out[0].data_ptr(), h_out[1].data_ptr(), h_out[2].data_ptr(), sp)
+                    oI.data_ptr(), h_out[0].data_ptr(), h_out[1].data_ptr(), h_out[2].data_ptr(), stream.cuda_stream)
                 if st != 0:
                     raise ck.ChunkKVError(st, "chunkkv_compress_layer_host")
 
@@ -360,7 +401,7 @@ def run_ours(args, wl):
         d2h = LAYERS_PER_STEP * (2 * wl.Hkv * n_max * wl.d * 2 + wl.Hkv * n_max * 4)
         e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "steps": e2e_steps}
-    if ck.device_status(stream) != 0:
+    if ck.device_status(stream) != 0 or any(ln.status() != 0 for ln in lanes):
         raise RuntimeError("a kernel reported an abandoned wait")
 
     cpu_baseline = None
@@ -374,7 +415,10 @@ def run_ours(args, wl):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "Hq": wl.Hq, "Hkv": wl.Hkv, "d": wl.d, "L": wl.L, "w": wl.w,
                        "c": wl.c, "budget": wl.budget, "layers_per_step": LAYERS_PER_STEP,
-                       "launch": "one CUDA graph per step (32 chunkkv_compress_layer calls captured)",
+                       "lanes": S,
+                       "launch": f"one CUDA graph per step: 32 chunkkv_compress_layer calls, {S} in flight "
+                                 f"on {S} streams with {n_sm // S} CTAs each" if S > 1 else
+                                 "one CUDA graph per step (32 chunkkv_compress_layer calls captured)",
                        "l2": f"layers cycle over {NSETS} distinct K/V sets of "
                              f"{2 * wl.Hkv * wl.L * wl.d * 2 / 1e6:.0f} MB each (> L2)"},
             "us_per_layer": ms_layer * 1e3,

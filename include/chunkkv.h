@@ -160,6 +160,35 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
                            void* out_K, void* out_V, int32_t* out_idx, void* stream);
 
 /*
+ * Lanes: several layers in flight at once (Algorithm 2 visits the layers one after another, and
+ * they are independent). A lane is caller-owned scratch plus a CTA budget. Layers submitted to
+ * different lanes on different streams run concurrently, each on its share of the SMs, so the
+ * latency-bound steps of one layer (top-k selection, grid-wide hand-overs) overlap the
+ * bandwidth-bound scoring and gathering of the others.
+ *
+ *   chunkkv_lane_bytes          scratch a lane needs for a shape with a CTA budget (0 = all SMs)
+ *   chunkkv_lane_init           clears the lane's 256-byte header (queued on `stream`); call once
+ *                               before first use, and again before using the lane with a different
+ *                               CTA budget
+ *   chunkkv_compress_layer_lane chunkkv_compress_layer with the lane's scratch and at most
+ *                               max_ctas CTAs (0 = all SMs). Calls on one lane must be ordered
+ *                               (same stream). The budgets of all lanes that may run at the same
+ *                               time must add up to no more than the number of SMs: the layer
+ *                               kernel synchronises its CTAs grid-wide, which needs all of them
+ *                               resident.
+ *   chunkkv_lane_status         synchronises `stream`, then CHUNKKV_OK or CHUNKKV_EDEVICE for the
+ *                               lane (and clears its header)
+ * lane must be 256-byte aligned device memory.
+ */
+CHUNKKV_API size_t chunkkv_lane_bytes(int L, int Hq, int Hkv, int d, int w, int c, int max_ctas);
+CHUNKKV_API int chunkkv_lane_init(void* lane, size_t bytes, void* stream);
+CHUNKKV_API int chunkkv_lane_status(void* lane, void* stream);
+CHUNKKV_API int chunkkv_compress_layer_lane(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                                            int d, int w, int c, int budget, const int32_t* reuse_idx_or_null,
+                                            void* out_K, void* out_V, int32_t* out_idx,
+                                            void* lane, size_t lane_bytes, int max_ctas, void* stream);
+
+/*
  * End-to-end convenience for callers whose tensors live in (ideally pinned) HOST memory:
  * copies q_obs, K, V to the given device staging buffers, runs chunkkv_compress_layer and
  * copies out_K, out_V, out_idx back to the host buffers, all queued on `stream`.

@@ -48,6 +48,16 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_compress_layer.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, vp, vp, vp]
     L.chunkkv_compress_layer_host.restype = i32
     L.chunkkv_compress_layer_host.argtypes = [vp, vp, vp] + [i32] * 7 + [vp] * 10
+    L.chunkkv_lane_bytes.restype = sz
+    L.chunkkv_lane_bytes.argtypes = [i32] * 7
+    L.chunkkv_lane_init.restype = i32
+    L.chunkkv_lane_init.argtypes = [vp, sz, vp]
+    L.chunkkv_lane_status.restype = i32
+    L.chunkkv_lane_status.argtypes = [vp, vp]
+    L.chunkkv_compress_layer_lane.restype = i32
+    L.chunkkv_compress_layer_lane.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, vp, vp, vp, sz, i32, vp]
+    L.chunkkv_score_noalloc.restype = i32
+    L.chunkkv_score_noalloc.argtypes = [vp, vp] + [i32] * 6 + [vp, vp]
     L.chunkkv_profile_enable.restype = i32
     L.chunkkv_profile_enable.argtypes = [i32]
     L.chunkkv_profile_read.restype = i32
@@ -185,6 +195,48 @@ def compress_layer(q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tens
                                       budget, _ptr(reuse_idx), out_K.data_ptr(), out_V.data_ptr(),
                                       out_idx.data_ptr(), _stream(stream)), "chunkkv_compress_layer")
     return out_K, out_V, out_idx
+
+
+class Lane:
+    """Caller-owned scratch plus a CTA budget: layers submitted to different lanes on different
+    streams run concurrently (see chunkkv.h). The budgets of lanes used at the same time must add
+    up to at most the number of SMs."""
+
+    def __init__(self, L: int, Hq: int, Hkv: int, d: int, w: int, c: int, max_ctas: int = 0,
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+        self.max_ctas = int(max_ctas)
+        self.bytes = int(lib.chunkkv_lane_bytes(L, Hq, Hkv, d, w, c, self.max_ctas))
+        if self.bytes == 0:
+            raise ChunkKVError(-2, "chunkkv_lane_bytes")
+        self.buf = torch.empty(self.bytes, dtype=torch.uint8, device=device or "cuda")
+        self.stream = stream if stream is not None else torch.cuda.Stream(device=self.buf.device)
+        _check(lib.chunkkv_lane_init(self.buf.data_ptr(), self.bytes, self.stream.cuda_stream or None),
+               "chunkkv_lane_init")
+
+    def status(self) -> int:
+        return lib.chunkkv_lane_status(self.buf.data_ptr(), self.stream.cuda_stream or None)
+
+    def compress_layer(self, q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tensor, Hq: int, w: int,
+                       c: int, budget: int, reuse_idx: Optional[torch.Tensor] = None,
+                       out_K: Optional[torch.Tensor] = None, out_V: Optional[torch.Tensor] = None,
+                       out_idx: Optional[torch.Tensor] = None,
+                       ) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+        """chunkkv_compress_layer_lane on this lane's stream."""
+        Hkv, L, d = K.shape
+        n_max = out_len(L, w, c, budget)
+        dev = K.device
+        with torch.cuda.stream(self.stream):
+            if out_K is None:
+                out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
+            if out_V is None:
+                out_V = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
+            if out_idx is None:
+                out_idx = torch.empty((Hkv, n_max), dtype=torch.int32, device=dev)
+        _check(lib.chunkkv_compress_layer_lane(
+            _ptr(q_obs), K.data_ptr(), V.data_ptr(), L, Hq, Hkv, d, w, c, budget, _ptr(reuse_idx),
+            out_K.data_ptr(), out_V.data_ptr(), out_idx.data_ptr(), self.buf.data_ptr(), self.bytes,
+            self.max_ctas, self.stream.cuda_stream or None), "chunkkv_compress_layer_lane")
+        return out_K, out_V, out_idx
 
 
 def compress_layer_host(host_q: torch.Tensor, host_K: torch.Tensor, host_V: torch.Tensor, Hq: int,

@@ -418,9 +418,11 @@ int chunkkv_gather(const void* K, const void* V, const int32_t* idx, int L, int 
     return CHUNKKV_OK;
 }
 
-int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
-                           int d, int w, int c, int budget, const int32_t* reuse_idx,
-                           void* out_K, void* out_V, int32_t* out_idx, void* stream) {
+// Shared body of chunkkv_compress_layer and chunkkv_compress_layer_lane. `lane` = caller-owned
+// scratch (NULL: the device-wide scratch), `max_ctas` = CTA budget of the launch (0: every SM).
+static int compress_impl(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv, int d, int w,
+                         int c, int budget, const int32_t* reuse_idx, void* out_K, void* out_V,
+                         int32_t* out_idx, void* lane, size_t lane_bytes, int max_ctas, void* stream) {
     int st = check_sizes(L, w, c, budget);
     if (st != CHUNKKV_OK) return st;
     st = check_heads(L, Hq, Hkv, d, w);
@@ -431,6 +433,7 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
     if (!aligned16(q_obs) || !aligned16(K) || !aligned16(V) || !aligned16(out_K) || !aligned16(out_V) ||
         !aligned16(out_idx) || !aligned16(reuse_idx))
         return CHUNKKV_EINVAL_ALIGN;
+    if (max_ctas < 0) return CHUNKKV_EINVAL_SHAPE;
     const int C = chunkkv_num_chunks(L, w, c);
     const int k = chunkkv_num_kept_chunks(L, w, c, budget);
     const int n_max = chunkkv_out_len(L, w, c, budget);
@@ -439,12 +442,13 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
     DeviceCtx* ctx;
     st = get_ctx(&ctx);
     if (st != CHUNKKV_OK) return st;
+    const int ctas = (max_ctas > 0 && max_ctas < ctx->num_sms) ? max_ctas : ctx->num_sms;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
     if (reuse_idx != nullptr) {
         Timer t(ctx, s, 3);
         e = launch_gather(K, V, reuse_idx, L, Hkv, d, n_max, out_K, out_V,
-                          reuse_idx == out_idx ? nullptr : out_idx, ctx->num_sms, s);
+                          reuse_idx == out_idx ? nullptr : out_idx, ctas, s);
         if (e != cudaSuccess) return cuda_fail(e);
         return CHUNKKV_OK;
     }
@@ -454,11 +458,18 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
         // chunk scores sit at the start of the scratch payload, the score kernels' scratch after them
         const size_t cs_floats = (static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63);
         ScorePlan plan;
-        if (!g_unfused && make_score_plan(L, R, Hkv, d, c, ctx->num_sms, smem_budget(*ctx), true, &plan)) {
+        if ((lane != nullptr || !g_unfused) && make_score_plan(L, R, Hkv, d, c, ctas, smem_budget(*ctx), true, &plan)) {
             // One cooperative launch for the whole layer.
-            st = ensure_workspace(*ctx, (cs_floats + score_scratch_floats(plan, Hkv, R)) * sizeof(float));
-            if (st != CHUNKKV_OK) return st;
-            char* base = static_cast<char*>(ctx->ws);
+            const size_t need = (cs_floats + score_scratch_floats(plan, Hkv, R)) * sizeof(float);
+            char* base;
+            if (lane != nullptr) {
+                if (kHeaderBytes + need > lane_bytes) return CHUNKKV_ENOWORKSPACE;
+                base = static_cast<char*>(lane);
+            } else {
+                st = ensure_workspace(*ctx, need);
+                if (st != CHUNKKV_OK) return st;
+                base = static_cast<char*>(ctx->ws);
+            }
             float* payload = reinterpret_cast<float*>(base + kHeaderBytes);
             ScoreArgs a;
             a.L = L; a.P = L - w; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
@@ -483,6 +494,7 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
             if (e != cudaSuccess) return cuda_fail(e);
             return CHUNKKV_OK;
         }
+        if (lane != nullptr) return CHUNKKV_EINVAL_SHAPE;
         st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, cs_floats, &chunk_scores, s);
         if (st != CHUNKKV_OK) return st;
     }
@@ -493,10 +505,66 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
     if (e != cudaSuccess) return cuda_fail(e);
     {
         Timer t(ctx, s, 3);
-        e = launch_gather(K, V, out_idx, L, Hkv, d, n_max, out_K, out_V, nullptr, ctx->num_sms, s);
+        e = launch_gather(K, V, out_idx, L, Hkv, d, n_max, out_K, out_V, nullptr, ctas, s);
     }
     if (e != cudaSuccess) return cuda_fail(e);
     return CHUNKKV_OK;
+}
+
+int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                           int d, int w, int c, int budget, const int32_t* reuse_idx,
+                           void* out_K, void* out_V, int32_t* out_idx, void* stream) {
+    return compress_impl(q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_idx, out_K, out_V, out_idx, nullptr, 0, 0,
+                         stream);
+}
+
+size_t chunkkv_lane_bytes(int L, int Hq, int Hkv, int d, int w, int c, int max_ctas) {
+    if (w < 1 || c < 1 || L < w || max_ctas < 0) return 0;
+    if (check_heads(L, Hq, Hkv, d, w) != CHUNKKV_OK) return 0;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    if (get_ctx(&ctx) != CHUNKKV_OK) return 0;
+    const int ctas = (max_ctas > 0 && max_ctas < ctx->num_sms) ? max_ctas : ctx->num_sms;
+    const int R = w * (Hq / Hkv);
+    const int C = (L - w + c - 1) / c;
+    ScorePlan plan;
+    if (!make_score_plan(L, R, Hkv, d, c, ctas, smem_budget(*ctx), true, &plan)) return 0;
+    const size_t floats = score_scratch_floats(plan, Hkv, R) + ((static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63));
+    return kHeaderBytes + floats * sizeof(float);
+}
+
+int chunkkv_lane_init(void* lane, size_t bytes, void* stream) {
+    if (lane == nullptr) return CHUNKKV_EINVAL_NULL;
+    if ((reinterpret_cast<uintptr_t>(lane) & 255u) != 0) return CHUNKKV_EINVAL_ALIGN;
+    if (bytes < kHeaderBytes) return CHUNKKV_ENOWORKSPACE;
+    cudaError_t e = cudaMemsetAsync(lane, 0, kHeaderBytes, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+int chunkkv_lane_status(void* lane, void* stream) {
+    if (lane == nullptr) return CHUNKKV_EINVAL_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int flag = 0;
+    e = cudaMemcpy(&flag, lane, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (flag != 0) {
+        cudaMemset(lane, 0, kHeaderBytes);
+        return CHUNKKV_EDEVICE;
+    }
+    return CHUNKKV_OK;
+}
+
+int chunkkv_compress_layer_lane(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                                int d, int w, int c, int budget, const int32_t* reuse_idx,
+                                void* out_K, void* out_V, int32_t* out_idx,
+                                void* lane, size_t lane_bytes, int max_ctas, void* stream) {
+    if (lane == nullptr) return CHUNKKV_EINVAL_NULL;
+    if ((reinterpret_cast<uintptr_t>(lane) & 255u) != 0) return CHUNKKV_EINVAL_ALIGN;
+    return compress_impl(q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_idx, out_K, out_V, out_idx, lane, lane_bytes,
+                         max_ctas, stream);
 }
 
 int chunkkv_compress_layer_host(const void* host_q_obs, const void* host_K, const void* host_V,

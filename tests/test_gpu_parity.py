@@ -259,3 +259,29 @@ def test_caller_provided_workspace(ck):
         _check_layer(x, wl, oK, oV, idx)
     finally:
         ck.set_workspace(None)
+
+
+def test_lanes_run_layers_concurrently_and_match(ck):
+    # four lanes of 37 CTAs, four layers in flight on four streams
+    wl = scaled(CONFIGS[2], L=6000, budget=600)
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    lanes = [ck.Lane(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=n_sm // 4) for _ in range(4)]
+    layers = [make_layer(wl, layer=i) for i in range(4)]
+    dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in layers]
+    torch.cuda.synchronize()
+    outs = []
+    for rep in range(2):                      # second round reuses the lanes' scratch
+        outs = [lanes[i].compress_layer(*dev[i], wl.Hq, wl.w, wl.c, wl.budget) for i in range(4)]
+    for ln in lanes:
+        assert ln.status() == 0
+    for x, (oK, oV, idx) in zip(layers, outs):
+        _check_layer(x, wl, bits_of(oK), bits_of(oV), idx.cpu().numpy())
+    # a lane also serves gather-only (index reuse) layers, and a too-small lane is refused
+    rK, rV, ridx = lanes[1].compress_layer(None, dev[1][1], dev[1][2], wl.Hq, wl.w, wl.c, wl.budget, reuse_idx=outs[1][2])
+    assert lanes[1].status() == 0
+    assert torch.equal(rK, outs[1][0]) and torch.equal(ridx, outs[1][2])
+    st = ck.lib.chunkkv_compress_layer_lane(dev[0][0].data_ptr(), dev[0][1].data_ptr(), dev[0][2].data_ptr(), wl.L,
+                                            wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, wl.budget, None, outs[0][0].data_ptr(),
+                                            outs[0][1].data_ptr(), outs[0][2].data_ptr(), lanes[0].buf.data_ptr(),
+                                            4096, n_sm // 4, None)
+    assert st == -4
