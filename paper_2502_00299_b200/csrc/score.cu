@@ -176,24 +176,22 @@ struct RowStatSmem {
 // Merge the records of the CTAs that touched head h into the global row maxima m[i] and
 // 1 / l[i] (written to gm / ginv, which may be shared or global memory). Block-wide: every
 // thread of the CTA must call it; the first kFinThreads threads work, each on a slice of the
-// records of one row. This code runs once per launch: loops stay rolled to keep it short
-// (instruction fetch, not arithmetic, is what it costs). Tile/CTA arithmetic is 32-bit: the
-// host guarantees total_tiles * grid < 2^31.
-__device__ __noinline__ void block_row_stats(const ScoreArgs& a, const FinGeom& g, int h, float* gm,
-                                             float* ginv, RowStatSmem& sm) {
+// records of one row so that the loads overlap.
+__device__ __forceinline__ void block_row_stats(const ScoreArgs& a, const FinGeom& g, int h, float* gm,
+                                                float* ginv, RowStatSmem& sm) {
     const int tid = threadIdx.x;
     // CTA b owns tiles [total*b/G, total*(b+1)/G): the owner of tile T is floor(((T+1)*G - 1) / total).
-    const unsigned total = static_cast<unsigned>(a.Hkv) * g.n_tiles, G = g.score_grid;
-    const unsigned first_tile = static_cast<unsigned>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
-    const int b_lo = static_cast<int>(((first_tile + 1) * G - 1) / total);
-    const int b_hi = static_cast<int>(((last_tile + 1) * G - 1) / total);
+    const long long total = static_cast<long long>(a.Hkv) * g.n_tiles;
+    const long long first_tile = static_cast<long long>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
+    const int b_lo = static_cast<int>(((first_tile + 1) * g.score_grid - 1) / total);
+    const int b_hi = static_cast<int>(((last_tile + 1) * g.score_grid - 1) / total);
     const int nb = b_hi - b_lo + 1;                 // <= 256: the scoring grid is capped there
     for (int j = tid; j < nb; j += blockDim.x) {
-        const unsigned b = b_lo + j;
-        const unsigned tb0 = total * b / G, tb1 = total * (b + 1) / G;
+        const int b = b_lo + j;
+        const long long tb0 = total * b / g.score_grid, tb1 = total * (b + 1) / g.score_grid;
         const int head0 = static_cast<int>(tb0 / g.n_tiles);
         // a CTA without tiles (more CTAs than tiles) wrote no record
-        sm.rec_base[j] = (tb1 > tb0) ? static_cast<int>((b * g.hs_max + (h - head0)) * (kGroups * 256)) : -1;
+        sm.rec_base[j] = (tb1 > tb0) ? (b * g.hs_max + (h - head0)) * (kGroups * 256) : -1;
     }
     __syncthreads();
     const int rp = (a.R > 128) ? 256 : 128;         // rows padded to the slice stride
@@ -203,38 +201,49 @@ __device__ __noinline__ void block_row_stats(const ScoreArgs& a, const FinGeom& 
     const bool work = tid < kFinThreads && i < a.R;
     const int g0 = (g.n_mt == 2) ? (i >> 7) * gpr : 0;
     const int rr = i & 127;
-    // Each thread folds its slice of the records into one (max, sum) pair.
+    // Each thread folds its slice of the records into one (max, sum) pair. Records are fetched
+    // kRecBatch CTAs at a time with every load issued before the first use.
+    constexpr int kRecBatch = 6;
     float M = -CUDART_INF_F, Lsum = 0.f;
     if (work) {
-#pragma unroll 1
-        for (int j = sl; j < nb; j += ns) {
-            const int base = sm.rec_base[j];
-            if (base < 0) continue;
-            const float* rec = a.cta_stat + base + g0 * 256 + rr;
-            float rm[kGroups], rl[kGroups];
+        for (int j0 = sl; j0 < nb; j0 += ns * kRecBatch) {
+            float rm[kRecBatch][kGroups], rl[kRecBatch][kGroups];
 #pragma unroll
-            for (int q = 0; q < kGroups; ++q) {
-                const bool have = q < gpr;
-                rm[q] = have ? __ldcg(rec + q * 256) : -CUDART_INF_F;
-                rl[q] = have ? __ldcg(rec + q * 256 + 128) : 0.f;
+            for (int t = 0; t < kRecBatch; ++t) {
+                const int j = j0 + t * ns;
+                const int base = (j < nb) ? sm.rec_base[j] : -1;
+#pragma unroll
+                for (int q = 0; q < kGroups; ++q) {
+                    const bool have = base >= 0 && q < gpr;
+                    const float* rec = a.cta_stat + (have ? base : 0) + (g0 + (have ? q : 0)) * 256 + rr;
+                    rm[t][q] = have ? __ldcg(rec) : -CUDART_INF_F;
+                    rl[t][q] = have ? __ldcg(rec + 128) : 0.f;
+                }
             }
-            const float bm = fmaxf(fmaxf(fmaxf(rm[0], rm[1]), fmaxf(rm[2], rm[3])), M);
+            float bm = M;
+#pragma unroll
+            for (int t = 0; t < kRecBatch; ++t)
+#pragma unroll
+                for (int q = 0; q < kGroups; ++q) bm = fmaxf(bm, rm[t][q]);
             float acc = (M == -CUDART_INF_F) ? 0.f : Lsum * ex2_approx(M - bm);
 #pragma unroll
-            for (int q = 0; q < kGroups; ++q)
-                acc += (rm[q] == -CUDART_INF_F) ? 0.f : rl[q] * ex2_approx(rm[q] - bm);
+            for (int t = 0; t < kRecBatch; ++t)
+#pragma unroll
+                for (int q = 0; q < kGroups; ++q)
+                    acc += (rm[t][q] == -CUDART_INF_F) ? 0.f : rl[t][q] * ex2_approx(rm[t][q] - bm);
             M = bm;
             Lsum = acc;
         }
     }
-    if (tid < kFinThreads) { sm.red[tid] = M; sm.red2[tid] = Lsum; }
+    float* red_m = sm.red;                           // [kFinThreads] maxima, sums in red2
+    if (tid < kFinThreads) { red_m[tid] = M; sm.red2[tid] = Lsum; }
     __syncthreads();
     if (work && sl == 0) {
         float gmax = M;
-        for (int s2 = 1; s2 < ns; ++s2) gmax = fmaxf(gmax, sm.red[s2 * rp + i]);
+        for (int s2 = 1; s2 < ns; ++s2) gmax = fmaxf(gmax, red_m[s2 * rp + i]);
         float lt = 0.f;
         for (int s2 = 0; s2 < ns; ++s2) {
-            const float pm = sm.red[s2 * rp + i];
+            const float pm = red_m[s2 * rp + i];
             lt += (pm == -CUDART_INF_F) ? 0.f : sm.red2[s2 * rp + i] * ex2_approx(pm - gmax);
         }
         gm[i] = gmax;
@@ -247,26 +256,24 @@ __device__ __noinline__ void block_row_stats(const ScoreArgs& a, const FinGeom& 
 // f[p - p_lo][i] = exp2(m_panel - m) / l are staged in `fs` (row stride fs_stride). A chunk
 // that continues past p_hi takes the scale of the later panels from global memory. One warp
 // reduces kFinBatch chunks at a time; fixed order, so results are deterministic.
-__device__ __noinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& g, int h, int p_lo, int p_hi,
-                                             int ch0, int ch1, const float* fs, int fs_stride,
-                                             const float* gm, const float* ginv, float* __restrict__ out) {
+__device__ __forceinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& g, int h, int p_lo, int p_hi,
+                                                int ch0, int ch1, const float* fs, int fs_stride,
+                                                const float* gm, const float* ginv, float* __restrict__ out) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
-    const float* stat_h = a.stat_m + static_cast<size_t>(h) * g.n_panels * a.R;
-    const float* part_h = a.partial + static_cast<size_t>(h) * g.n_panels * g.spp * a.R;
-    float* out_h = out + static_cast<size_t>(h) * g.C;
-#pragma unroll 1
+    const size_t stat_base = static_cast<size_t>(h) * g.n_panels * a.R;
+    const size_t part_base = static_cast<size_t>(h) * g.n_panels * g.spp * a.R;
     for (int cb = ch0 + warp * kFinBatch; cb < ch1; cb += nwarps * kFinBatch) {
         float acc[kFinBatch];
         bool single = true;
         int pa[kFinBatch];
-        const float* pp[kFinBatch];
+        size_t po[kFinBatch];
 #pragma unroll
         for (int u = 0; u < kFinBatch; ++u) {
             const int ch = min(cb + u, ch1 - 1);
             const int ja = ch * a.c, jb = min(ja + a.c, a.P);
             pa[u] = ja / g.wp;
             single = single && (pa[u] == (jb - 1) / g.wp) && pa[u] >= p_lo && pa[u] < p_hi;
-            pp[u] = part_h + static_cast<size_t>(pa[u] * g.spp + (ch - (pa[u] * g.wp) / a.c)) * a.R;
+            po[u] = part_base + (static_cast<size_t>(pa[u]) * g.spp + (ch - (pa[u] * g.wp) / a.c)) * a.R;
             acc[u] = 0.f;
         }
         if (single) {       // every chunk of the batch lies in one staged panel
@@ -276,7 +283,7 @@ __device__ __noinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& 
             for (int it = 0; it < 8; ++it) {
                 const int i = lane + 32 * it;
 #pragma unroll
-                for (int u = 0; u < kFinBatch; ++u) pv[u][it] = (i < a.R) ? __ldcg(pp[u] + i) : 0.f;
+                for (int u = 0; u < kFinBatch; ++u) pv[u][it] = (i < a.R) ? __ldcg(a.partial + po[u] + i) : 0.f;
             }
 #pragma unroll
             for (int it = 0; it < 8; ++it) {
@@ -287,22 +294,16 @@ __device__ __noinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& 
                 }
             }
         } else {
-#pragma unroll 1
+#pragma unroll
             for (int u = 0; u < kFinBatch; ++u) {
                 const int ch = min(cb + u, ch1 - 1);
                 const int ja = ch * a.c, jb = min(ja + a.c, a.P);
-                float t = 0.f;
-#pragma unroll 1
                 for (int p = ja / g.wp; p <= (jb - 1) / g.wp; ++p) {
-                    const float* o = part_h + static_cast<size_t>(p * g.spp + (ch - (p * g.wp) / a.c)) * a.R;
-                    const float* so = stat_h + static_cast<size_t>(p) * a.R;
-#pragma unroll 1
+                    const size_t o = part_base + (static_cast<size_t>(p) * g.spp + (ch - (p * g.wp) / a.c)) * a.R;
+                    const size_t so = stat_base + static_cast<size_t>(p) * a.R;
                     for (int i = lane; i < a.R; i += 32)
-                        t += __ldcg(o + i) * (ex2_approx(__ldcg(so + i) - gm[i]) * ginv[i]);
+                        acc[u] += __ldcg(a.partial + o + i) * (ex2_approx(__ldcg(a.stat_m + so + i) - gm[i]) * ginv[i]);
                 }
-                // acc[] is indexed with a run-time u here: move the value with selects
-#pragma unroll
-                for (int v = 0; v < kFinBatch; ++v) acc[v] = (v == u) ? t : acc[v];
             }
         }
 #pragma unroll
@@ -310,7 +311,7 @@ __device__ __noinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& 
             float v = acc[u];
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-            if (lane == 0 && cb + u < ch1) out_h[cb + u] = v;
+            if (lane == 0 && cb + u < ch1) out[static_cast<size_t>(h) * g.C + cb + u] = v;
         }
     }
 }
@@ -616,8 +617,6 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         float* fs = ginv + 256;
         const int fs_cap = (g.dyn_bytes - static_cast<int>(sizeof(RowStatSmem)) - 2048) / 4;   // floats
         SelectSmem& ss = *reinterpret_cast<SelectSmem*>(dyn);
-        uint32_t* sel_keys = reinterpret_cast<uint32_t*>(dyn + ((sizeof(SelectSmem) + 15) & ~size_t(15)));
-        const int sel_key_cap = (g.dyn_bytes - static_cast<int>((sizeof(SelectSmem) + 15) & ~size_t(15))) / 4;
         int* bar_ok = reinterpret_cast<int*>(&ctl.tmem_base);     // free again after the dealloc
         FinGeom fg;
         fg.n_panels = g.n_tiles * PPT * SUBS;
@@ -692,7 +691,10 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         for (int h = blockIdx.x; h < a.Hkv; h += gridDim.x) {
             const float* sc = la.chunk_scores + static_cast<size_t>(h) * la.C;
             int32_t* out = la.out_idx + static_cast<size_t>(h) * la.n_max;
-            select_head(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss, sel_keys, sel_key_cap);
+            if (la.C <= kThreads * kSelPerThread)
+                select_head<true>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+            else
+                select_head<false>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
         }
         if (!grid_barrier(la.bar_count, gridDim.x, bar_ok, abort_flag)) {
             if (threadIdx.x == 0) atomicExch(a.status, 1);

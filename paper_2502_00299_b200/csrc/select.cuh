@@ -2,17 +2,13 @@
 // the selection mask, "always keep most recent tokens", "nonzero(mask)"), shared by the
 // stand-alone select kernel and the fused layer kernel.
 //
-// One CTA works on one KV head. Order-preserving 32-bit keys of the chunk scores are staged in
-// shared memory (or re-read from global memory when there are too many). The k-th largest key
-// is found by an exact 4-pass radix select; every warp counts into its own 16-bit histogram row
-// (lanes that hit the same bin add once), so no two warps ever touch the same counter. Each
-// thread then owns a contiguous run of chunk ids; one block-wide prefix sum over
-// (#above threshold, #equal to threshold) gives every chunk its rank among the kept ones:
+// One CTA works on one KV head. Each thread owns a contiguous run of chunk ids and keeps their
+// order-preserving 32-bit keys in registers. The k-th largest key is found by an exact 4-pass
+// radix select; every warp counts into its own 16-bit histogram row (lanes that hit the same
+// bin add once), so no two warps ever touch the same counter. One block-wide prefix sum over
+// (#above threshold, #equal to threshold) then gives every chunk its rank among the kept ones:
 // rank = #above before it + min(#equal before it, ties to keep) - ties go to the lower chunk
 // id. Token positions are written directly in ascending order: no mask, no sort.
-//
-// The code runs once per launch, so it is written with rolled loops: on a path this short the
-// instruction fetch of unrolled code costs more than the loop overhead saves.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -20,6 +16,7 @@
 namespace chunkkv {
 
 constexpr int kSelMaxWarps = 32;
+constexpr int kSelPerThread = 16;     // chunk keys held in registers per thread
 constexpr int kSelCap = 4096;         // kept-chunk ids staged for coalesced index writes
 
 struct SelectSmem {
@@ -38,34 +35,31 @@ __device__ __forceinline__ uint32_t select_order_key(float x) {
 }
 
 // All threads of the CTA must call this (it uses __syncthreads); blockDim.x must be a multiple
-// of 32 and at most 1024. `keys` is shared memory for key_cap keys; if C > key_cap the keys are
-// recomputed from `sc` on every use instead.
-static __device__ __noinline__ void select_head(const float* __restrict__ sc, int L, int w, int c, int C, int k,
-                                         int n_max, int32_t* __restrict__ out, SelectSmem& sm, uint32_t* keys,
-                                         int key_cap) {
+// of 32 and at most 1024. IN_REGS requires C <= blockDim.x * kSelPerThread.
+template <bool IN_REGS>
+__device__ __forceinline__ void select_head(const float* __restrict__ sc, int L, int w, int c, int C, int k,
+                                            int n_max, int32_t* __restrict__ out, SelectSmem& sm) {
     const int P = L - w;
     const int nt = blockDim.x, nwarps = nt >> 5;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool keep_all = (k >= C);
     const int kk = min(k, C);
-    const bool staged = C <= key_cap;
-    const bool search = !keep_all && kk > 0;
 
-    if (staged && search)
-        for (int i = tid; i < C; i += nt) keys[i] = select_order_key(__ldcg(sc + i));
-    if (tid == 0) sm.last_kept = 0;
-    __syncthreads();
-
-    // thread t owns chunk ids [c0, c1) (lanes of a warp own adjacent runs)
+    // thread t owns chunk ids [c0, c1)
     const int per = (C + nt - 1) / nt;
     const int c0 = min(tid * per, C), c1 = min(c0 + per, C);
+    uint32_t keys[kSelPerThread];
+    if (IN_REGS && kk > 0 && !keep_all) {
+#pragma unroll
+        for (int u = 0; u < kSelPerThread; ++u) keys[u] = (c0 + u < c1) ? select_order_key(sc[c0 + u]) : 0u;
+    }
+    if (tid == 0) sm.last_kept = 0;
 
     uint32_t thresh = 0;   // key of the k-th largest score
     int need_eq = 0;       // how many chunks equal to the threshold are kept
-    if (search) {
+    if (!keep_all && kk > 0) {
         uint32_t prefix = 0;
         int need = k;
-#pragma unroll 1
         for (int pass = 0; pass < 4; ++pass) {
             const int shift = 24 - 8 * pass;
             {   // clear this warp's histogram row (256 x 16 bit = 128 words)
@@ -75,22 +69,25 @@ static __device__ __noinline__ void select_head(const float* __restrict__ sc, in
             }
             __syncwarp();
             const uint32_t himask = (pass == 0) ? 0u : (0xFFFFFFFFu << (shift + 8));
-#pragma unroll 1
-            for (int u = 0; u < per; ++u) {              // `per` is uniform: no divergence
-                const int ch = c0 + u;
-                const bool have = ch < c1;
-                const uint32_t key = have ? (staged ? keys[ch] : select_order_key(__ldcg(sc + ch))) : 0u;
+            auto count_one = [&](bool have, uint32_t key) {
                 const bool in = have && (key & himask) == prefix;
                 const int bin = in ? static_cast<int>((key >> shift) & 0xFF) : -1;
                 const unsigned peers = __match_any_sync(0xffffffffu, bin);
                 if (in && lane == __ffs(peers) - 1)
                     sm.whist[warp][bin] += static_cast<unsigned short>(__popc(peers));
                 __syncwarp();
+            };
+            if (IN_REGS) {
+#pragma unroll
+                for (int u = 0; u < kSelPerThread; ++u)
+                    if (u < per) count_one(c0 + u < c1, keys[u]);      // `per` is uniform: no divergence
+            } else {
+                for (int u = 0; u < per; ++u)
+                    count_one(c0 + u < c1, (c0 + u < c1) ? select_order_key(sc[c0 + u]) : 0u);
             }
             __syncthreads();
             if (tid < 256) {
                 int sum = 0;
-#pragma unroll 4
                 for (int wv = 0; wv < nwarps; ++wv) sum += sm.whist[wv][tid];
                 sm.hist[tid] = sum;
             }
@@ -110,9 +107,7 @@ static __device__ __noinline__ void select_head(const float* __restrict__ sc, in
                 const int owner = reach ? (__ffs(reach) - 1) : 31;
                 if (lane == owner) {
                     int above = inc - sum, q = 0;
-#pragma unroll
-                    for (int qq = 0; qq < 7; ++qq)
-                        if (q == qq && above + cnt[qq] < need) { above += cnt[qq]; ++q; }
+                    while (q < 7 && above + cnt[q] < need) { above += cnt[q]; ++q; }
                     sm.prefix = prefix | (static_cast<uint32_t>(255 - 8 * lane - q) << shift);
                     sm.need = need - above;
                 }
@@ -130,10 +125,13 @@ static __device__ __noinline__ void select_head(const float* __restrict__ sc, in
     if (kk > 0) {
         unsigned gt_n = 0, eq_n = 0;
         if (keep_all) gt_n = c1 - c0;
-        else {
-#pragma unroll 1
+        else if (IN_REGS) {
+#pragma unroll
+            for (int u = 0; u < kSelPerThread; ++u)
+                if (c0 + u < c1) { gt_n += keys[u] > thresh; eq_n += keys[u] == thresh; }
+        } else {
             for (int ch = c0; ch < c1; ++ch) {
-                const uint32_t key = staged ? keys[ch] : select_order_key(__ldcg(sc + ch));
+                const uint32_t key = select_order_key(sc[ch]);
                 gt_n += key > thresh;
                 eq_n += key == thresh;
             }
@@ -161,9 +159,7 @@ static __device__ __noinline__ void select_head(const float* __restrict__ sc, in
         __syncthreads();
         const unsigned long long excl = sm.warp_sums[warp] + inc - mine;
         int gt_before = static_cast<int>(excl & 0xffffffffu), eq_before = static_cast<int>(excl >> 32);
-#pragma unroll 1
-        for (int ch = c0; ch < c1; ++ch) {
-            const uint32_t key = keep_all ? 0u : (staged ? keys[ch] : select_order_key(__ldcg(sc + ch)));
+        auto visit = [&](int ch, uint32_t key) {
             const bool gt = keep_all || key > thresh;
             const bool eq = !keep_all && key == thresh;
             if (gt || (eq && eq_before < need_eq)) {
@@ -178,19 +174,24 @@ static __device__ __noinline__ void select_head(const float* __restrict__ sc, in
             }
             gt_before += gt;
             eq_before += eq;
+        };
+        if (IN_REGS && !keep_all) {
+#pragma unroll
+            for (int u = 0; u < kSelPerThread; ++u)
+                if (c0 + u < c1) visit(c0 + u, keys[u]);
+        } else {
+            for (int ch = c0; ch < c1; ++ch) visit(ch, keep_all ? 0u : select_order_key(sc[ch]));
         }
     }
     __syncthreads();
     // Every kept chunk is full except possibly chunk C-1, which can only be the last kept one.
     const int tail = (C > 0) ? (P - (C - 1) * c) : 0;
     const int n_tok = kk * c - ((sm.last_kept && kk > 0) ? (c - tail) : 0);
-    if (stage_sel) {
-#pragma unroll 1
+    if (stage_sel)
         for (int n = tid; n < n_tok; n += nt) {
             const int rank = n / c;
             out[n] = sm.sel[rank] * c + (n - rank * c);
         }
-    }
     for (int i = tid; i < w; i += nt) out[n_tok + i] = P + i;
     for (int i = n_tok + w + tid; i < n_max; i += nt) out[i] = -1;
     __syncthreads();     // shared state may be reused by the caller
