@@ -691,10 +691,12 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         for (int h = blockIdx.x; h < a.Hkv; h += gridDim.x) {
             const float* sc = la.chunk_scores + static_cast<size_t>(h) * la.C;
             int32_t* out = la.out_idx + static_cast<size_t>(h) * la.n_max;
-            if (la.C <= kThreads * kSelPerThread)
-                select_head<true>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+            if (la.C <= kThreads * 6)
+                select_head<6>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+            else if (la.C <= kThreads * kSelPerThread)
+                select_head<kSelPerThread>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
             else
-                select_head<false>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+                select_head<0>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
         }
         if (!grid_barrier(la.bar_count, gridDim.x, bar_ok, abort_flag)) {
             if (threadIdx.x == 0) atomicExch(a.status, 1);

@@ -16,7 +16,7 @@
 namespace chunkkv {
 
 constexpr int kSelMaxWarps = 32;
-constexpr int kSelPerThread = 16;     // chunk keys held in registers per thread
+constexpr int kSelPerThread = 16;     // most chunk keys a thread can hold in registers
 constexpr int kSelCap = 4096;         // kept-chunk ids staged for coalesced index writes
 
 struct SelectSmem {
@@ -35,8 +35,9 @@ __device__ __forceinline__ uint32_t select_order_key(float x) {
 }
 
 // All threads of the CTA must call this (it uses __syncthreads); blockDim.x must be a multiple
-// of 32 and at most 1024. IN_REGS requires C <= blockDim.x * kSelPerThread.
-template <bool IN_REGS>
+// of 32 and at most 1024. KPT > 0: every thread keeps up to KPT keys in registers, which needs
+// C <= blockDim.x * KPT; KPT = 0: keys are re-read from memory on every use.
+template <int KPT>
 __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L, int w, int c, int C, int k,
                                             int n_max, int32_t* __restrict__ out, SelectSmem& sm) {
     const int P = L - w;
@@ -48,10 +49,12 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
     // thread t owns chunk ids [c0, c1)
     const int per = (C + nt - 1) / nt;
     const int c0 = min(tid * per, C), c1 = min(c0 + per, C);
-    uint32_t keys[kSelPerThread];
+    constexpr bool IN_REGS = KPT > 0;
+    constexpr int KR = IN_REGS ? KPT : 1;
+    uint32_t keys[KR];
     if (IN_REGS && kk > 0 && !keep_all) {
 #pragma unroll
-        for (int u = 0; u < kSelPerThread; ++u) keys[u] = (c0 + u < c1) ? select_order_key(sc[c0 + u]) : 0u;
+        for (int u = 0; u < KR; ++u) keys[u] = (c0 + u < c1) ? select_order_key(sc[c0 + u]) : 0u;
     }
     if (tid == 0) sm.last_kept = 0;
 
@@ -79,7 +82,7 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
             };
             if (IN_REGS) {
 #pragma unroll
-                for (int u = 0; u < kSelPerThread; ++u)
+                for (int u = 0; u < KR; ++u)
                     if (u < per) count_one(c0 + u < c1, keys[u]);      // `per` is uniform: no divergence
             } else {
                 for (int u = 0; u < per; ++u)
@@ -127,7 +130,7 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
         if (keep_all) gt_n = c1 - c0;
         else if (IN_REGS) {
 #pragma unroll
-            for (int u = 0; u < kSelPerThread; ++u)
+            for (int u = 0; u < KR; ++u)
                 if (c0 + u < c1) { gt_n += keys[u] > thresh; eq_n += keys[u] == thresh; }
         } else {
             for (int ch = c0; ch < c1; ++ch) {
@@ -177,7 +180,7 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
         };
         if (IN_REGS && !keep_all) {
 #pragma unroll
-            for (int u = 0; u < kSelPerThread; ++u)
+            for (int u = 0; u < KR; ++u)
                 if (c0 + u < c1) visit(c0 + u, keys[u]);
         } else {
             for (int ch = c0; ch < c1; ++ch) visit(ch, keep_all ? 0u : select_order_key(sc[ch]));
