@@ -47,7 +47,7 @@ def parse_args():
     ap.add_argument("--config", type=int, default=2, help="workload table entry (2 = headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--lanes", type=int, default=4, help="layers in flight (each on 1/lanes of the SMs)")
+    ap.add_argument("--lanes", type=int, default=8, help="layers in flight (each on 1/lanes of the SMs)")
     return ap.parse_args()
 
 
