@@ -354,7 +354,7 @@ def run_ours(args, wl):
                 "note": "kernel timed with the GPU to itself (one layer at a time); the step overlaps "
                         f"{S} such launches on disjoint SM sets"}
     layer_gbs = nbytes["layer"] / (ms_layer * 1e-3) / 1e9
-    gather_us = per_kernel["gather"]["avg_us"] or float("nan")   # nan when the layer kernel is fused
+    gather_us = per_kernel["gather"]["avg_us"]                    # None when the layer kernel is fused
     extra_roof = {
         "layer_throughput": {"algorithmic_bytes": nbytes["layer"], "us_per_layer": ms_layer * 1e3, "GB/s": layer_gbs,
                              "frac_of_measured_peak": layer_gbs / peak, "frac_of_8TBs": layer_gbs / NOMINAL_HBM_GBS,
@@ -363,9 +363,10 @@ def run_ours(args, wl):
                          "GB/s": nbytes["layer"] / (ms_single * 1e-3) / 1e9,
                          "frac_of_measured_peak": nbytes["layer"] / (ms_single * 1e-3) / 1e9 / peak,
                          "note": "layers one after another, each on all SMs"},
-        "gather_kernel": {"algorithmic_bytes": nbytes["gather"], "us": gather_us,
-                          "GB/s": nbytes["gather"] / (gather_us * 1e-6) / 1e9,
-                          "frac_of_measured_peak": nbytes["gather"] / (gather_us * 1e-6) / 1e9 / peak},
+        "gather_kernel": None if not gather_us else {
+            "algorithmic_bytes": nbytes["gather"], "us": gather_us,
+            "GB/s": nbytes["gather"] / (gather_us * 1e-6) / 1e9,
+            "frac_of_measured_peak": nbytes["gather"] / (gather_us * 1e-6) / 1e9 / peak},
         "reuse_layer": {"algorithmic_bytes": nbytes["gather"], "us": ms_reuse * 1e3,
                         "GB/s": nbytes["gather"] / (ms_reuse * 1e-3) / 1e9,
                         "frac_of_measured_peak": nbytes["gather"] / (ms_reuse * 1e-3) / 1e9 / peak},
