@@ -29,7 +29,7 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream). Calls only
  *     enqueue work; they never synchronise the device (except where stated).
  *   - Limits: d in {64, 128}; Hq a multiple of Hkv; R = w * Hq / Hkv <= 256; 1 <= w <= L;
- *     c >= 1; budget >= w; Hkv * L * d < 2^40.
+ *     c >= 1; budget >= w; Hkv * L < 2^23 (8 M keys per layer).
  *   - Return value: CHUNKKV_OK (0) or a negative CHUNKKV_E* code. Arguments are checked on
  *     the host before anything is launched; nothing is thrown and nothing aborts.
  *   - Scratch memory: scoring needs device scratch (chunkkv_workspace_bytes). Either hand the

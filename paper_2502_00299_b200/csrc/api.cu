@@ -122,6 +122,7 @@ int check_heads(int L, int Hq, int Hkv, int d, int w) {
     if (R > 256) return CHUNKKV_EINVAL_SHAPE;
     if (static_cast<long long>(Hkv) * L * d >= (1LL << 40)) return CHUNKKV_EINVAL_SHAPE;
     if (Hkv > 65535) return CHUNKKV_EINVAL_SHAPE;
+    if (static_cast<long long>(Hkv) * L >= (1LL << 23)) return CHUNKKV_EINVAL_SHAPE;   // 32-bit row arithmetic in the kernels
     return CHUNKKV_OK;
 }
 

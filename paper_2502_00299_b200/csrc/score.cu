@@ -154,7 +154,6 @@ __device__ __forceinline__ void panel_general(const float (&v)[WP], float sl2, b
 
 constexpr int kFinThreads = 512;
 constexpr int kFinPanelCap = 24;      // panels whose scales fit in the finalize kernel's shared memory
-constexpr int kFinBatch = 4;          // chunks a warp reduces together
 
 struct FinGeom {
     int n_panels;     // per head
@@ -181,17 +180,18 @@ __device__ __forceinline__ void block_row_stats(const ScoreArgs& a, const FinGeo
                                                 float* ginv, RowStatSmem& sm) {
     const int tid = threadIdx.x;
     // CTA b owns tiles [total*b/G, total*(b+1)/G): the owner of tile T is floor(((T+1)*G - 1) / total).
-    const long long total = static_cast<long long>(a.Hkv) * g.n_tiles;
-    const long long first_tile = static_cast<long long>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
-    const int b_lo = static_cast<int>(((first_tile + 1) * g.score_grid - 1) / total);
-    const int b_hi = static_cast<int>(((last_tile + 1) * g.score_grid - 1) / total);
+    // (32-bit arithmetic: the host checks that total_tiles * (grid + 1) fits)
+    const unsigned total = static_cast<unsigned>(a.Hkv) * g.n_tiles, G = g.score_grid;
+    const unsigned first_tile = static_cast<unsigned>(h) * g.n_tiles, last_tile = first_tile + g.n_tiles - 1;
+    const int b_lo = static_cast<int>(((first_tile + 1) * G - 1) / total);
+    const int b_hi = static_cast<int>(((last_tile + 1) * G - 1) / total);
     const int nb = b_hi - b_lo + 1;                 // <= 256: the scoring grid is capped there
     for (int j = tid; j < nb; j += blockDim.x) {
-        const int b = b_lo + j;
-        const long long tb0 = total * b / g.score_grid, tb1 = total * (b + 1) / g.score_grid;
+        const unsigned b = b_lo + j;
+        const unsigned tb0 = total * b / G, tb1 = total * (b + 1) / G;
         const int head0 = static_cast<int>(tb0 / g.n_tiles);
         // a CTA without tiles (more CTAs than tiles) wrote no record
-        sm.rec_base[j] = (tb1 > tb0) ? (b * g.hs_max + (h - head0)) * (kGroups * 256) : -1;
+        sm.rec_base[j] = (tb1 > tb0) ? static_cast<int>((b * g.hs_max + (h - head0)) * (kGroups * 256)) : -1;
     }
     __syncthreads();
     const int rp = (a.R > 128) ? 256 : 128;         // rows padded to the slice stride
@@ -255,65 +255,97 @@ __device__ __forceinline__ void block_row_stats(const ScoreArgs& a, const FinGeo
 // Chunk scores of the chunks that start in panels [p_lo, p_hi) of head h, whose scales
 // f[p - p_lo][i] = exp2(m_panel - m) / l are staged in `fs` (row stride fs_stride). A chunk
 // that continues past p_hi takes the scale of the later panels from global memory. One warp
-// reduces kFinBatch chunks at a time; fixed order, so results are deterministic.
-__device__ __forceinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& g, int h, int p_lo, int p_hi,
-                                                int ch0, int ch1, const float* fs, int fs_stride,
-                                                const float* gm, const float* ginv, float* __restrict__ out) {
+// reduces BATCH chunks at a time with all of their NIT * 32 rows' loads issued before the first
+// use (the step is bound by L2 latency, so loads in flight are what counts); fixed order, so
+// results are deterministic. Requires R <= 32 * NIT.
+template <int NIT, int BATCH>
+__device__ __forceinline__ void contract_chunks_t(const ScoreArgs& a, const FinGeom& g, int h, int p_lo, int p_hi,
+                                                  int ch0, int ch1, const float* fs, int fs_stride,
+                                                  const float* gm, const float* ginv, float* __restrict__ out) {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
-    const size_t stat_base = static_cast<size_t>(h) * g.n_panels * a.R;
-    const size_t part_base = static_cast<size_t>(h) * g.n_panels * g.spp * a.R;
-    for (int cb = ch0 + warp * kFinBatch; cb < ch1; cb += nwarps * kFinBatch) {
-        float acc[kFinBatch];
+    const float* stat_h = a.stat_m + static_cast<size_t>(h) * g.n_panels * a.R;
+    const float* part_h = a.partial + static_cast<size_t>(h) * g.n_panels * g.spp * a.R;
+    float* out_h = out + static_cast<size_t>(h) * g.C;
+    // When the chunk size divides the panel width, slots are exactly the chunks in order: chunk ch
+    // sits at offset ch * R and never straddles panels, so no division is needed per chunk.
+    const bool aligned = (g.wp % a.c) == 0 && g.spp * a.c == g.wp;
+    for (int cb = ch0 + warp * BATCH; cb < ch1; cb += nwarps * BATCH) {
+        float acc[BATCH];
         bool single = true;
-        int pa[kFinBatch];
-        size_t po[kFinBatch];
+        int pa[BATCH], po[BATCH];
+        if (aligned) {
+            int p_ = cb / g.spp, s_ = cb - p_ * g.spp;
+            single = p_ >= p_lo;
 #pragma unroll
-        for (int u = 0; u < kFinBatch; ++u) {
-            const int ch = min(cb + u, ch1 - 1);
-            const int ja = ch * a.c, jb = min(ja + a.c, a.P);
-            pa[u] = ja / g.wp;
-            single = single && (pa[u] == (jb - 1) / g.wp) && pa[u] >= p_lo && pa[u] < p_hi;
-            po[u] = part_base + (static_cast<size_t>(pa[u]) * g.spp + (ch - (pa[u] * g.wp) / a.c)) * a.R;
-            acc[u] = 0.f;
+            for (int u = 0; u < BATCH; ++u) {
+                if (u == 0 || cb + u < ch1) {
+                    pa[u] = p_;
+                    po[u] = (cb + u) * a.R;
+                    if (++s_ == g.spp) { s_ = 0; ++p_; }
+                } else {
+                    pa[u] = pa[u > 0 ? u - 1 : 0];
+                    po[u] = po[u > 0 ? u - 1 : 0];
+                }
+                single = single && pa[u] < p_hi;
+                acc[u] = 0.f;
+            }
+        } else {
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                const int ch = min(cb + u, ch1 - 1);
+                const int ja = ch * a.c, jb = min(ja + a.c, a.P);
+                pa[u] = ja / g.wp;
+                single = single && (pa[u] == (jb - 1) / g.wp) && pa[u] >= p_lo && pa[u] < p_hi;
+                po[u] = (pa[u] * g.spp + (ch - (pa[u] * g.wp) / a.c)) * a.R;
+                acc[u] = 0.f;
+            }
         }
         if (single) {       // every chunk of the batch lies in one staged panel
-            // R <= 256 = 8 x 32 rows: issue every load of the batch before the first use
-            float pv[kFinBatch][8];
+            float pv[BATCH][NIT];
 #pragma unroll
-            for (int it = 0; it < 8; ++it) {
+            for (int it = 0; it < NIT; ++it) {
                 const int i = lane + 32 * it;
 #pragma unroll
-                for (int u = 0; u < kFinBatch; ++u) pv[u][it] = (i < a.R) ? __ldcg(a.partial + po[u] + i) : 0.f;
+                for (int u = 0; u < BATCH; ++u) pv[u][it] = (i < a.R) ? __ldcg(part_h + po[u] + i) : 0.f;
             }
 #pragma unroll
-            for (int it = 0; it < 8; ++it) {
+            for (int it = 0; it < NIT; ++it) {
                 const int i = lane + 32 * it;
                 if (i < a.R) {
 #pragma unroll
-                    for (int u = 0; u < kFinBatch; ++u) acc[u] += pv[u][it] * fs[(pa[u] - p_lo) * fs_stride + i];
+                    for (int u = 0; u < BATCH; ++u) acc[u] += pv[u][it] * fs[(pa[u] - p_lo) * fs_stride + i];
                 }
             }
         } else {
 #pragma unroll
-            for (int u = 0; u < kFinBatch; ++u) {
+            for (int u = 0; u < BATCH; ++u) {
                 const int ch = min(cb + u, ch1 - 1);
                 const int ja = ch * a.c, jb = min(ja + a.c, a.P);
                 for (int p = ja / g.wp; p <= (jb - 1) / g.wp; ++p) {
-                    const size_t o = part_base + (static_cast<size_t>(p) * g.spp + (ch - (p * g.wp) / a.c)) * a.R;
-                    const size_t so = stat_base + static_cast<size_t>(p) * a.R;
+                    const float* o = part_h + static_cast<size_t>(p * g.spp + (ch - (p * g.wp) / a.c)) * a.R;
+                    const float* so = stat_h + static_cast<size_t>(p) * a.R;
                     for (int i = lane; i < a.R; i += 32)
-                        acc[u] += __ldcg(a.partial + o + i) * (ex2_approx(__ldcg(a.stat_m + so + i) - gm[i]) * ginv[i]);
+                        acc[u] += __ldcg(o + i) * (ex2_approx(__ldcg(so + i) - gm[i]) * ginv[i]);
                 }
             }
         }
 #pragma unroll
-        for (int u = 0; u < kFinBatch; ++u) {
+        for (int u = 0; u < BATCH; ++u) {
             float v = acc[u];
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-            if (lane == 0 && cb + u < ch1) out[static_cast<size_t>(h) * g.C + cb + u] = v;
+            if (lane == 0 && cb + u < ch1) out_h[cb + u] = v;
         }
     }
+}
+
+__device__ __forceinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& g, int h, int p_lo, int p_hi,
+                                                int ch0, int ch1, const float* fs, int fs_stride,
+                                                const float* gm, const float* ginv, float* __restrict__ out) {
+    if (a.R <= 128)
+        contract_chunks_t<4, 8>(a, g, h, p_lo, p_hi, ch0, ch1, fs, fs_stride, gm, ginv, out);
+    else
+        contract_chunks_t<8, 4>(a, g, h, p_lo, p_hi, ch0, ch1, fs, fs_stride, gm, ginv, out);
 }
 
 // Everything the fused layer kernel needs beyond scoring.
@@ -405,9 +437,12 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     const uint32_t k_base = q_base + static_cast<uint32_t>(NQBUF * N_MT * KB) * kQTileBytes;
     volatile int* abort_flag = &ctl.abort_flag;
 
-    const long long total = g.total_tiles;
+    // CTA b owns tiles [total*b/G, total*(b+1)/G) in (head, tile) order; 32-bit arithmetic (the
+    // host checks that total_tiles * (grid + 1) fits).
+    const unsigned total = g.total_tiles;
     const int t_begin = static_cast<int>(total * blockIdx.x / gridDim.x);
     const int t_end = static_cast<int>(total * (blockIdx.x + 1) / gridDim.x);
+    const int head_begin = t_begin / g.n_tiles, tile_begin = t_begin - head_begin * g.n_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < g.n_stages; ++s) {
@@ -442,8 +477,9 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const uint32_t k_bytes = static_cast<uint32_t>(g.k_box_rows) * 128u;
             int ctr = 0, hs = -1, cur_head = -1;
             bool ok = true;
-            for (int t = t_begin; t < t_end && ok; ++t) {
-                const int head = t / g.n_tiles, tile = t - head * g.n_tiles;
+            int head = head_begin, tile = tile_begin;
+            for (int t = t_begin; t < t_end && ok; ++t, ++tile) {
+                if (tile == g.n_tiles) { tile = 0; ++head; }
                 if (head != cur_head) {
                     cur_head = head;
                     ++hs;
@@ -486,8 +522,9 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         if (elect_one()) {
             int ctr = 0, hs = -1, cur_head = -1, ti = 0, qb = 0;
             bool ok = true;
-            for (int t = t_begin; t < t_end && ok; ++t, ++ti) {
-                const int head = t / g.n_tiles;
+            int head = head_begin, tile = tile_begin;
+            for (int t = t_begin; t < t_end && ok; ++t, ++ti, ++tile) {
+                if (tile == g.n_tiles) { tile = 0; ++head; }
                 if (head != cur_head) {
                     if (cur_head >= 0) umma_commit(smem_u32(&ctl.qempty[qb]));
                     cur_head = head;
@@ -548,8 +585,9 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 rec[128 + quarter * 32 + lane] = run_l;
             }
         };
-        for (int t = t_begin; t < t_end; ++t, ++ti) {
-            const int head = t / g.n_tiles, tile = t - head * g.n_tiles;
+        int head = head_begin, tile = tile_begin;
+        for (int t = t_begin; t < t_end; ++t, ++ti, ++tile) {
+            if (tile == g.n_tiles) { tile = 0; ++head; }
             if (head != cur_head) {
                 flush_head();
                 cur_head = head;
@@ -660,18 +698,32 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 const int p_lo = (ta - head * g.n_tiles) * PPTT, p_hi = (tb - head * g.n_tiles) * PPTT;
                 const int n = (p_hi - p_lo) * a.R;
                 if (ta == t && prefetched) {
+                    int i = threadIdx.x % a.R;                 // row of element e, advanced without dividing
+                    const int step = kThreads % a.R;
 #pragma unroll
                     for (int u = 0; u < kPF; ++u) {
                         const int e = threadIdx.x + u * kThreads;
-                        if (e < n) {
-                            const int i = e % a.R;
-                            fs[e] = ex2_approx(mp[u] - gm[i]) * ginv[i];
-                        }
+                        if (e < n) fs[e] = ex2_approx(mp[u] - gm[i]) * ginv[i];
+                        i += step;
+                        i -= (i >= a.R) ? a.R : 0;
                     }
                 } else {
-                    for (int e = threadIdx.x; e < n; e += kThreads) {
-                        const int i = e % a.R;
-                        fs[e] = ex2_approx(__ldcg(a.stat_m + stat_base + static_cast<size_t>(p_lo) * a.R + e) - gm[i]) * ginv[i];
+                    const float* src = a.stat_m + stat_base + static_cast<size_t>(p_lo) * a.R;
+                    for (int e0 = threadIdx.x; e0 < n; e0 += 8 * kThreads) {   // eight loads in flight per thread
+                        float t8[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int e = e0 + u * kThreads;
+                            t8[u] = (e < n) ? __ldcg(src + e) : 0.f;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const int e = e0 + u * kThreads;
+                            if (e < n) {
+                                const int i = e % a.R;
+                                fs[e] = ex2_approx(t8[u] - gm[i]) * ginv[i];
+                            }
+                        }
                     }
                 }
                 __syncthreads();
@@ -705,15 +757,15 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         // ---- gather: the Hkv * n_max output rows are split evenly over the CTAs
         const int vpr = a.d >> 3;
         const int rows_per_pass = (kThreads / vpr) * kGatherRowsPerThread;
-        const long long rows_total = static_cast<long long>(a.Hkv) * la.n_max;
-        const long long r_begin = rows_total * blockIdx.x / gridDim.x, r_end = rows_total * (blockIdx.x + 1) / gridDim.x;
-        for (long long r0 = r_begin; r0 < r_end;) {
-            const int h = static_cast<int>(r0 / la.n_max);
-            const int n0 = static_cast<int>(r0 - static_cast<long long>(h) * la.n_max);
+        // (32-bit arithmetic: the host checks that Hkv * n_max * (grid + 1) fits)
+        const unsigned rows_total = static_cast<unsigned>(a.Hkv) * la.n_max;
+        const int r_begin = static_cast<int>(rows_total * blockIdx.x / gridDim.x);
+        const int r_end = static_cast<int>(rows_total * (blockIdx.x + 1) / gridDim.x);
+        for (int r0 = r_begin; r0 < r_end;) {
+            const int h = r0 / la.n_max;
+            const int n0 = r0 - h * la.n_max;
             // rows [n0, n_hi) of head h in this pass
-            const int n_hi = static_cast<int>(min(static_cast<long long>(la.n_max),
-                                                  min(r_end - static_cast<long long>(h) * la.n_max,
-                                                      static_cast<long long>(n0) + rows_per_pass)));
+            const int n_hi = min(la.n_max, min(r_end - h * la.n_max, n0 + rows_per_pass));
             const int32_t* ih = la.out_idx + static_cast<size_t>(h) * la.n_max;
             if (vpr == 16)
                 gather_rows<16, true>(la.K + static_cast<size_t>(h) * a.L * 16, la.V + static_cast<size_t>(h) * a.L * 16, ih,
@@ -841,6 +893,7 @@ bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_
     p.spp = p.c_static ? p.wp / p.c_static : (p.wp + c - 1) / c + 1;
     const long long total = static_cast<long long>(Hkv) * p.n_tiles;
     p.grid = static_cast<int>((total < num_sms && !full_grid) ? total : num_sms);
+    if (total * (static_cast<long long>(num_sms) + 1) >= (1LL << 32)) return false;   // kernels use 32-bit tile arithmetic
     if (p.grid > 256) p.grid = 256;   // rowstats_kernel indexes at most 256 CTA records per head
     const int tiles_per_cta = static_cast<int>((total + p.grid - 1) / p.grid);
     p.hs_max = (tiles_per_cta + p.n_tiles - 1) / p.n_tiles + 1;
