@@ -422,6 +422,12 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     constexpr int WPP = (C_STATIC > 0) ? WP : 32;  // panel width in keys
     constexpr int SUBS = WP / WPP;                 // panels a thread processes per tile
     static_assert(WP % WPP == 0, "group columns must split into whole panels");
+    // ALT: the four groups form two pairs that take alternate accumulator tiles (pair p reads
+    // buffer p only); inside a pair each group walks one half of the tile as two panels. The
+    // pairs run half a tile period apart, so one pair's waits (accumulator ready, TMEM load)
+    // fall into the other pair's arithmetic.
+    constexpr bool ALT = (N_MT == 1 && C_STATIC > 0);
+    constexpr int ASUBS = ALT ? 2 : SUBS;          // panels a thread processes per tile it takes
     static_assert(C_STATIC == 0 || WPP % C_STATIC == 0, "static chunk size must divide the panel");
     constexpr uint32_t IDESC = umma_idesc_bf16(128, N_TILE);
 
@@ -451,7 +457,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.tfull[b]), 1);
-            mbar_init(smem_u32(&ctl.tempty[b]), 4 * kGroups);   // one arrival per epilogue warp
+            mbar_init(smem_u32(&ctl.tempty[b]), ALT ? 2 * kGroups : 4 * kGroups);   // one arrival per reading warp
             mbar_init(smem_u32(&ctl.qfull[b]), 1);
             mbar_init(smem_u32(&ctl.qempty[b]), 1);
         }
@@ -571,6 +577,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int quarter = warp & 3;               // TMEM lane quarter this warp may read
         const int mt = grp / PPT;
         const int pit = grp % PPT;                  // panel within the tile
+        const int pair = grp >> 1, half = grp & 1;  // ALT only
         const int row = mt * 128 + quarter * 32 + lane;
         const bool active = row < a.R;
         const int last_visible = a.P + (row % a.w);  // this row sees keys j <= P + r (all < L)
@@ -595,23 +602,24 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 run_m = -CUDART_INF_F;
                 run_l = 0.f;
             }
+            if (ALT && (ti & 1) != pair) continue;   // the other pair's tile
             const int buf = ti & 1, use = ti >> 1;
             bool ready = true;                       // one lane polls, the warp follows
             if (lane == 0) ready = mbar_wait(smem_u32(&ctl.tfull[buf]), use & 1, abort_flag);
             if (!__shfl_sync(0xffffffffu, ready, 0)) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                   static_cast<uint32_t>(buf * 256 + mt * TCOLS + pit * WP);
+                                   static_cast<uint32_t>(buf * 256 + mt * TCOLS + (ALT ? half * 2 * WPP : pit * WP));
 #pragma unroll
-            for (int sub = 0; sub < SUBS; ++sub) {
+            for (int sub = 0; sub < ASUBS; ++sub) {
                 float v[WPP];
                 load_panel<WPP>(taddr + sub * WPP, v);
-                if (sub == SUBS - 1) {               // this thread's last read of the buffer
+                if (sub == ASUBS - 1) {              // this thread's last read of the buffer
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[buf]));   // it may be overwritten now
                 }
-                const int panel = (tile * PPT + pit) * SUBS + sub;
+                const int panel = ALT ? tile * (PPT * SUBS) + half * 2 + sub : (tile * PPT + pit) * SUBS + sub;
                 const size_t panel_id = static_cast<size_t>(head) * n_panels + panel;
                 float* part = a.partial + panel_id * g.spp * a.R + row;
                 const int j0 = panel * WPP;
