@@ -60,7 +60,7 @@ __device__ __forceinline__ void load_panel(uint32_t taddr, float (&v)[WP]) {
 // Panel that lies wholly inside the prefix and starts on a chunk boundary, chunk size known at
 // compile time: all control flow below folds away after unrolling.
 template <int C, int WP>
-__device__ __forceinline__ void panel_fast(const float (&v)[WP], float sl2, bool active, float* part,
+__device__ __forceinline__ void panel_fast(float (&v)[WP], float sl2, bool active, float* part,
                                            int row_stride, float* out_m, float* out_l) {
     float m0 = v[0], m1 = v[1], m2 = v[2], m3 = v[3];
 #pragma unroll
@@ -69,15 +69,22 @@ __device__ __forceinline__ void panel_fast(const float (&v)[WP], float sl2, bool
     }
     const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
     const float neg_m2 = -mx * sl2;
-    float l = 0.f, acc = 0.f;
+    // exponentials first, in place: WP independent operations the scheduler can overlap freely
 #pragma unroll
-    for (int u = 0; u < WP; ++u) {
-        const float e = ex2_approx(fmaf(v[u], sl2, neg_m2));
-        acc = (u % C == 0) ? e : acc + e;
-        if ((u + 1) % C == 0) {
-            if (active) part[static_cast<size_t>((u + 1) / C - 1) * row_stride] = acc;
-            l += acc;
+    for (int u = 0; u < WP; ++u) v[u] = ex2_approx(fmaf(v[u], sl2, neg_m2));
+    // chunk sums as balanced trees (short dependency chains), one store per chunk
+    float l = 0.f;
+#pragma unroll
+    for (int ch = 0; ch < WP / C; ++ch) {
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+        for (int t = 0; t < C; t += 2) {
+            s0 += v[ch * C + t];
+            if (t + 1 < C) s1 += v[ch * C + t + 1];
         }
+        const float acc = s0 + s1;
+        if (active) part[static_cast<size_t>(ch) * row_stride] = acc;
+        l += acc;
     }
     *out_m = mx * sl2;
     *out_l = l;
