@@ -462,6 +462,8 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     const uint32_t stage_bytes = static_cast<uint32_t>(N_TILE) * 128u;
     const uint32_t k_base = q_base + static_cast<uint32_t>(NQBUF * N_MT * KB) * kQTileBytes;
     volatile int* abort_flag = &ctl.abort_flag;
+    const uint32_t full0_bar = smem_u32(&ctl.full[0]);   // full[s] at +8*s, empty[s] at +8*(kMaxStages + s)
+    const uint32_t n_stages = static_cast<uint32_t>(g.n_stages);
 
     // CTA b owns tiles [total*b/G, total*(b+1)/G) in (head, tile) order; 32-bit arithmetic (the
     // host checks that total_tiles * (grid + 1) fits).
@@ -502,6 +504,9 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const uint32_t q_bytes = static_cast<uint32_t>(N_MT * KB * g.q_box_rows) * 128u;
             const uint32_t k_bytes = static_cast<uint32_t>(g.k_box_rows) * 128u;
             int ctr = 0, hs = -1, cur_head = -1;
+            // ring position and the parity of the phase to wait for, advanced without dividing
+            // (this thread's serial instruction stream bounds how far the loads run ahead)
+            uint32_t st = 0, st_par = 1;
             bool ok = true;
             int head = head_begin, tile = tile_begin;
             for (int t = t_begin; t < t_end && ok; ++t, ++tile) {
@@ -521,14 +526,13 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                                         &tm_q, bar, kb * 64, mt * 128, head);
                 }
                 for (int kb = 0; kb < KB; ++kb) {
-                    const int s = ctr % g.n_stages;
-                    ok = mbar_wait(smem_u32(&ctl.empty[s]), ((ctr / g.n_stages) & 1) ^ 1, abort_flag);
+                    ok = mbar_wait(full0_bar + 8u * (kMaxStages + st), st_par, abort_flag);   // empty[st]
                     if (!ok) break;
-                    const uint32_t bar = smem_u32(&ctl.full[s]);
+                    const uint32_t bar = full0_bar + 8u * st;
                     mbar_arrive_expect_tx(bar, k_bytes);
-                    tma_load_3d(k_base + static_cast<uint32_t>(s) * stage_bytes, &tm_k, bar, kb * 64,
-                                tile * N_TILE, head);
+                    tma_load_3d(k_base + st * stage_bytes, &tm_k, bar, kb * 64, tile * N_TILE, head);
                     ++ctr;
+                    if (++st == n_stages) { st = 0; st_par ^= 1u; }
                 }
             }
             if (!ok) {
@@ -546,7 +550,11 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     } else if (warp == 1) {
         // ------------------------------------------------------------------ UMMA issuer
         if (elect_one()) {
-            int ctr = 0, hs = -1, cur_head = -1, ti = 0, qb = 0;
+            int hs = -1, cur_head = -1, ti = 0, qb = 0;
+            // The tensor pipe is fed by this one thread: its serial instruction stream sets the
+            // floor of the tile period, so the ring position and phase parity advance without
+            // dividing and the descriptors of a stage differ only by an added constant.
+            uint32_t st = 0, st_par = 0;
             bool ok = true;
             int head = head_begin, tile = tile_begin;
             for (int t = t_begin; t < t_end && ok; ++t, ++ti, ++tile) {
@@ -563,26 +571,25 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 ok = mbar_wait(smem_u32(&ctl.tempty[buf]), (use & 1) ^ 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                for (int kb = 0; kb < KB && ok; ++kb) {
-                    const int s = ctr % g.n_stages;
-                    ok = mbar_wait(smem_u32(&ctl.full[s]), (ctr / g.n_stages) & 1, abort_flag);
+#pragma unroll
+                for (int kb = 0; kb < 2; ++kb) {         // d is 64 or 128: one or two 64-element blocks
+                    if (kb >= KB || !ok) break;
+                    ok = mbar_wait(full0_bar + 8u * st, st_par, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t b_addr = k_base + static_cast<uint32_t>(s) * stage_bytes;
+                    // k-steps advance the start-address field (16-byte units) by 32 bytes
+                    const uint64_t b_desc = umma_desc_sw128(k_base + st * stage_bytes);
 #pragma unroll
                     for (int mt = 0; mt < N_MT; ++mt) {
-                        const uint32_t a_addr =
-                            q_base + static_cast<uint32_t>((qb * N_MT + mt) * KB + kb) * kQTileBytes;
+                        const uint64_t a_desc = umma_desc_sw128(
+                            q_base + static_cast<uint32_t>((qb * N_MT + mt) * KB + kb) * kQTileBytes);
                         const uint32_t d_addr = tmem_base + static_cast<uint32_t>(buf * 256 + mt * TCOLS);
 #pragma unroll
-                        for (int k4 = 0; k4 < 4; ++k4) {
-                            umma_bf16(d_addr, umma_desc_sw128(a_addr + k4 * 32),
-                                      umma_desc_sw128(b_addr + k4 * 32), IDESC,
-                                      (kb > 0 || k4 > 0) ? 1u : 0u);
-                        }
+                        for (int k4 = 0; k4 < 4; ++k4)
+                            umma_bf16(d_addr, a_desc + 2u * k4, b_desc + 2u * k4, IDESC, (kb > 0 || k4 > 0) ? 1u : 0u);
                     }
-                    umma_commit(smem_u32(&ctl.empty[s]));
-                    ++ctr;
+                    umma_commit(full0_bar + 8u * (kMaxStages + st));   // empty[st]
+                    if (++st == n_stages) { st = 0; st_par ^= 1u; }
                 }
                 if (ok) umma_commit(smem_u32(&ctl.tfull[buf]));
             }
