@@ -346,6 +346,93 @@ __device__ __forceinline__ void contract_chunks_t(const ScoreArgs& a, const FinG
     }
 }
 
+// Chunk scores of panels [p_lo, p_hi) of head h when chunks never straddle panels (the chunk
+// size divides the panel width, so panel p holds chunks p * spp .. p * spp + spp - 1 in its slots)
+// and R is a multiple of 4. One warp takes one panel at a time: each lane owns four consecutive
+// rows (eight when R > 128), fetches the panel maxima and up to kSlotBatch chunk slots of those
+// rows with 16-byte loads that are all issued before the first use, forms the row factors
+// exp2(m_panel - m) / l in registers and reduces over the rows with shuffles. Nothing is staged in
+// shared memory and no block-wide synchronisation is needed. Fixed order: deterministic.
+// gm / ginv: row maxima and reciprocal sums, 16-byte aligned (shared or global memory).
+constexpr int kSlotBatch = 6;
+template <int RV>   // float4 row groups per lane: 1 for R <= 128, 2 for R <= 256
+__device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, const FinGeom& g, int h, int p_lo,
+                                                        int p_hi, const float* gm, const float* ginv,
+                                                        float* __restrict__ out) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    const int r4 = a.R >> 2;                                       // float4 per row vector
+    const float4* stat_h = reinterpret_cast<const float4*>(a.stat_m + static_cast<size_t>(h) * g.n_panels * a.R);
+    const float4* part_h =
+        reinterpret_cast<const float4*>(a.partial + static_cast<size_t>(h) * g.n_panels * g.spp * a.R);
+    float* out_h = out + static_cast<size_t>(h) * g.C;
+    float4 m4[RV], li4[RV];
+    bool have[RV];
+#pragma unroll
+    for (int it = 0; it < RV; ++it) {
+        const int i4 = lane + 32 * it;
+        have[it] = i4 < r4;
+        m4[it] = have[it] ? reinterpret_cast<const float4*>(gm)[i4] : make_float4(0.f, 0.f, 0.f, 0.f);
+        li4[it] = have[it] ? reinterpret_cast<const float4*>(ginv)[i4] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (int p = p_lo + warp; p < p_hi; p += nwarps) {
+        const int ch_base = p * g.spp;
+        const int n_slots = min(g.spp, g.C - ch_base);             // chunks of this panel that exist
+        if (n_slots <= 0) break;                                   // panels past the prefix hold no chunk
+        float4 pm[RV];
+#pragma unroll
+        for (int it = 0; it < RV; ++it)
+            pm[it] = have[it] ? __ldcg(stat_h + static_cast<size_t>(p) * r4 + lane + 32 * it)
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 f[RV];
+        bool f_ready = false;
+        for (int s0 = 0; s0 < n_slots; s0 += kSlotBatch) {
+            float4 pv[kSlotBatch][RV];
+#pragma unroll
+            for (int u = 0; u < kSlotBatch; ++u) {
+                const bool slot = s0 + u < n_slots;
+#pragma unroll
+                for (int it = 0; it < RV; ++it)
+                    pv[u][it] = (slot && have[it])
+                                    ? __ldcg(part_h + static_cast<size_t>(ch_base + s0 + u) * r4 + lane + 32 * it)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            if (!f_ready) {
+#pragma unroll
+                for (int it = 0; it < RV; ++it) {
+                    f[it].x = ex2_approx(pm[it].x - m4[it].x) * li4[it].x;
+                    f[it].y = ex2_approx(pm[it].y - m4[it].y) * li4[it].y;
+                    f[it].z = ex2_approx(pm[it].z - m4[it].z) * li4[it].z;
+                    f[it].w = ex2_approx(pm[it].w - m4[it].w) * li4[it].w;
+                }
+                f_ready = true;
+            }
+            float acc[kSlotBatch];
+#pragma unroll
+            for (int u = 0; u < kSlotBatch; ++u) {
+                float v = 0.f;
+#pragma unroll
+                for (int it = 0; it < RV; ++it) {
+                    v = fmaf(pv[u][it].x, f[it].x, v);
+                    v = fmaf(pv[u][it].y, f[it].y, v);
+                    v = fmaf(pv[u][it].z, f[it].z, v);
+                    v = fmaf(pv[u][it].w, f[it].w, v);
+                }
+                acc[u] = v;
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+                for (int u = 0; u < kSlotBatch; ++u) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int u = 0; u < kSlotBatch; ++u)
+                    if (s0 + u < n_slots) out_h[ch_base + s0 + u] = acc[u];
+            }
+        }
+    }
+}
+
 __device__ __forceinline__ void contract_chunks(const ScoreArgs& a, const FinGeom& g, int h, int p_lo, int p_hi,
                                                 int ch0, int ch1, const float* fs, int fs_stride,
                                                 const float* gm, const float* ginv, float* __restrict__ out) {
@@ -707,6 +794,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             return;
         }
         // ---- chunk scores of the panels this CTA scored
+        const bool direct = C_STATIC > 0 && (a.R & 3) == 0;
         for (int t = t_begin; t < t_end;) {
             const int head = t / g.n_tiles;
             const int seg_end = min(t_end, (head + 1) * g.n_tiles);
@@ -719,7 +807,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const int tb_first = min(seg_end, t + max_tiles);
             const int p_first = (t - head * g.n_tiles) * PPTT;
             const int n_first = (tb_first - t) * PPTT * a.R;
-            const bool prefetched = n_first <= kPF * kThreads;
+            const bool prefetched = !direct && n_first <= kPF * kThreads;
             if (prefetched) {
 #pragma unroll
                 for (int u = 0; u < kPF; ++u) {
@@ -728,6 +816,16 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 }
             }
             block_row_stats(a, fg, head, gm, ginv, rs);
+            if (direct) {   // chunks never straddle panels: straight from the partial sums, no staging
+                const int p_lo = (t - head * g.n_tiles) * PPTT, p_hi = (seg_end - head * g.n_tiles) * PPTT;
+                if (a.R <= 128)
+                    contract_panels_aligned<1>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                else
+                    contract_panels_aligned<2>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                __syncthreads();            // gm / ginv are rewritten for the next head
+                t = seg_end;
+                continue;
+            }
             for (int ta = t; ta < seg_end; ta += max_tiles) {
                 const int tb = min(seg_end, ta + max_tiles);
                 const int p_lo = (ta - head * g.n_tiles) * PPTT, p_hi = (tb - head * g.n_tiles) * PPTT;
