@@ -348,14 +348,14 @@ __device__ __forceinline__ void contract_chunks_t(const ScoreArgs& a, const FinG
 
 // Chunk scores of panels [p_lo, p_hi) of head h when chunks never straddle panels (the chunk
 // size divides the panel width, so panel p holds chunks p * spp .. p * spp + spp - 1 in its slots)
-// and R is a multiple of 4. One warp takes one panel at a time: each lane owns four consecutive
+// and R is a multiple of 4. One warp takes PP panels at a time: each lane owns four consecutive
 // rows (eight when R > 128), fetches the panel maxima and up to kSlotBatch chunk slots of those
 // rows with 16-byte loads that are all issued before the first use, forms the row factors
 // exp2(m_panel - m) / l in registers and reduces over the rows with shuffles. Nothing is staged in
 // shared memory and no block-wide synchronisation is needed. Fixed order: deterministic.
 // gm / ginv: row maxima and reciprocal sums, 16-byte aligned (shared or global memory).
 constexpr int kSlotBatch = 6;
-template <int RV>   // float4 row groups per lane: 1 for R <= 128, 2 for R <= 256
+template <int RV, int PP>   // RV float4 row groups per lane (1: R <= 128, 2: R <= 256); PP panels in flight per warp
 __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, const FinGeom& g, int h, int p_lo,
                                                         int p_hi, const float* gm, const float* ginv,
                                                         float* __restrict__ out) {
@@ -365,69 +365,85 @@ __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, cons
     const float4* part_h =
         reinterpret_cast<const float4*>(a.partial + static_cast<size_t>(h) * g.n_panels * g.spp * a.R);
     float* out_h = out + static_cast<size_t>(h) * g.C;
+    const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
     float4 m4[RV], li4[RV];
     bool have[RV];
 #pragma unroll
     for (int it = 0; it < RV; ++it) {
         const int i4 = lane + 32 * it;
         have[it] = i4 < r4;
-        m4[it] = have[it] ? reinterpret_cast<const float4*>(gm)[i4] : make_float4(0.f, 0.f, 0.f, 0.f);
-        li4[it] = have[it] ? reinterpret_cast<const float4*>(ginv)[i4] : make_float4(0.f, 0.f, 0.f, 0.f);
+        m4[it] = have[it] ? reinterpret_cast<const float4*>(gm)[i4] : zero4;
+        li4[it] = have[it] ? reinterpret_cast<const float4*>(ginv)[i4] : zero4;
     }
-    for (int p = p_lo + warp; p < p_hi; p += nwarps) {
-        const int ch_base = p * g.spp;
-        const int n_slots = min(g.spp, g.C - ch_base);             // chunks of this panel that exist
-        if (n_slots <= 0) break;                                   // panels past the prefix hold no chunk
-        float4 pm[RV];
+    for (int pb = p_lo + warp; pb < p_hi; pb += nwarps * PP) {
+        int n_slots[PP], max_slots = 0;
+        float4 pm[PP][RV];
 #pragma unroll
-        for (int it = 0; it < RV; ++it)
-            pm[it] = have[it] ? __ldcg(stat_h + static_cast<size_t>(p) * r4 + lane + 32 * it)
-                              : make_float4(0.f, 0.f, 0.f, 0.f);
-        float4 f[RV];
-        bool f_ready = false;
-        for (int s0 = 0; s0 < n_slots; s0 += kSlotBatch) {
-            float4 pv[kSlotBatch][RV];
+        for (int q = 0; q < PP; ++q) {
+            const int p = pb + q * nwarps;
+            n_slots[q] = (p < p_hi) ? max(0, min(g.spp, g.C - p * g.spp)) : 0;   // chunks of the panel that exist
+            max_slots = max(max_slots, n_slots[q]);
 #pragma unroll
-            for (int u = 0; u < kSlotBatch; ++u) {
-                const bool slot = s0 + u < n_slots;
+            for (int it = 0; it < RV; ++it)
+                pm[q][it] = (n_slots[q] > 0 && have[it]) ? __ldcg(stat_h + static_cast<size_t>(p) * r4 + lane + 32 * it)
+                                                         : zero4;
+        }
+        if (max_slots == 0) break;                                 // panels past the prefix hold no chunk
+        float4 f[PP][RV];
+        for (int s0 = 0; s0 < max_slots; s0 += kSlotBatch) {
+            float4 pv[PP][kSlotBatch][RV];
 #pragma unroll
-                for (int it = 0; it < RV; ++it)
-                    pv[u][it] = (slot && have[it])
-                                    ? __ldcg(part_h + static_cast<size_t>(ch_base + s0 + u) * r4 + lane + 32 * it)
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-            if (!f_ready) {
+            for (int q = 0; q < PP; ++q) {
+                const int ch_base = (pb + q * nwarps) * g.spp;
 #pragma unroll
-                for (int it = 0; it < RV; ++it) {
-                    f[it].x = ex2_approx(pm[it].x - m4[it].x) * li4[it].x;
-                    f[it].y = ex2_approx(pm[it].y - m4[it].y) * li4[it].y;
-                    f[it].z = ex2_approx(pm[it].z - m4[it].z) * li4[it].z;
-                    f[it].w = ex2_approx(pm[it].w - m4[it].w) * li4[it].w;
+                for (int u = 0; u < kSlotBatch; ++u) {
+                    const bool slot = s0 + u < n_slots[q];
+#pragma unroll
+                    for (int it = 0; it < RV; ++it)
+                        pv[q][u][it] = (slot && have[it])
+                                           ? __ldcg(part_h + static_cast<size_t>(ch_base + s0 + u) * r4 + lane + 32 * it)
+                                           : zero4;
                 }
-                f_ready = true;
             }
-            float acc[kSlotBatch];
+            if (s0 == 0) {
 #pragma unroll
-            for (int u = 0; u < kSlotBatch; ++u) {
-                float v = 0.f;
+                for (int q = 0; q < PP; ++q)
 #pragma unroll
-                for (int it = 0; it < RV; ++it) {
-                    v = fmaf(pv[u][it].x, f[it].x, v);
-                    v = fmaf(pv[u][it].y, f[it].y, v);
-                    v = fmaf(pv[u][it].z, f[it].z, v);
-                    v = fmaf(pv[u][it].w, f[it].w, v);
+                    for (int it = 0; it < RV; ++it) {
+                        f[q][it].x = ex2_approx(pm[q][it].x - m4[it].x) * li4[it].x;
+                        f[q][it].y = ex2_approx(pm[q][it].y - m4[it].y) * li4[it].y;
+                        f[q][it].z = ex2_approx(pm[q][it].z - m4[it].z) * li4[it].z;
+                        f[q][it].w = ex2_approx(pm[q][it].w - m4[it].w) * li4[it].w;
+                    }
+            }
+            float acc[PP][kSlotBatch];
+#pragma unroll
+            for (int q = 0; q < PP; ++q)
+#pragma unroll
+                for (int u = 0; u < kSlotBatch; ++u) {
+                    float v = 0.f;
+#pragma unroll
+                    for (int it = 0; it < RV; ++it) {
+                        v = fmaf(pv[q][u][it].x, f[q][it].x, v);
+                        v = fmaf(pv[q][u][it].y, f[q][it].y, v);
+                        v = fmaf(pv[q][u][it].z, f[q][it].z, v);
+                        v = fmaf(pv[q][u][it].w, f[q][it].w, v);
+                    }
+                    acc[q][u] = v;
                 }
-                acc[u] = v;
-            }
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) {
 #pragma unroll
-                for (int u = 0; u < kSlotBatch; ++u) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
+                for (int q = 0; q < PP; ++q)
+#pragma unroll
+                    for (int u = 0; u < kSlotBatch; ++u) acc[q][u] += __shfl_xor_sync(0xffffffffu, acc[q][u], off);
             }
             if (lane == 0) {
 #pragma unroll
-                for (int u = 0; u < kSlotBatch; ++u)
-                    if (s0 + u < n_slots) out_h[ch_base + s0 + u] = acc[u];
+                for (int q = 0; q < PP; ++q)
+#pragma unroll
+                    for (int u = 0; u < kSlotBatch; ++u)
+                        if (s0 + u < n_slots[q]) out_h[(pb + q * nwarps) * g.spp + s0 + u] = acc[q][u];
             }
         }
     }
@@ -819,9 +835,9 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             if (direct) {   // chunks never straddle panels: straight from the partial sums, no staging
                 const int p_lo = (t - head * g.n_tiles) * PPTT, p_hi = (seg_end - head * g.n_tiles) * PPTT;
                 if (a.R <= 128)
-                    contract_panels_aligned<1>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                    contract_panels_aligned<1, 2>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
                 else
-                    contract_panels_aligned<2>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                    contract_panels_aligned<2, 1>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
                 __syncthreads();            // gm / ginv are rewritten for the next head
                 t = seg_end;
                 continue;
