@@ -911,13 +911,34 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const unsigned rows_total = static_cast<unsigned>(a.Hkv) * la.n_max;
         const int r_begin = static_cast<int>(rows_total * blockIdx.x / gridDim.x);
         const int r_end = static_cast<int>(rows_total * (blockIdx.x + 1) / gridDim.x);
+        // The indices of this CTA's rows (contiguous in [Hkv, n_max] order) go to shared memory
+        // first, so that each pass below waits for one round trip (the rows) instead of two.
+        int32_t* sidx = reinterpret_cast<int32_t*>(dyn);
+        const bool staged = (r_end - r_begin) * 4 <= g.dyn_bytes - 2048;
+        if (staged) {
+            __syncthreads();                                   // the selection scratch is no longer read
+            for (int i = threadIdx.x; i < r_end - r_begin; i += kThreads) sidx[i] = __ldcg(la.out_idx + r_begin + i);
+            __syncthreads();
+        }
         for (int r0 = r_begin; r0 < r_end;) {
             const int h = r0 / la.n_max;
             const int n0 = r0 - h * la.n_max;
             // rows [n0, n_hi) of head h in this pass
             const int n_hi = min(la.n_max, min(r_end - h * la.n_max, n0 + rows_per_pass));
             const int32_t* ih = la.out_idx + static_cast<size_t>(h) * la.n_max;
-            if (vpr == 16)
+            if (staged) {
+                const int32_t* sh = sidx + (h * la.n_max - r_begin);   // sh[n] = index of row n of head h
+                if (vpr == 16)
+                    gather_rows<16, false>(la.K + static_cast<size_t>(h) * a.L * 16, la.V + static_cast<size_t>(h) * a.L * 16,
+                                           sh, a.L, n_hi, n0, threadIdx.x, kThreads,
+                                           la.out_K + static_cast<size_t>(h) * la.n_max * 16,
+                                           la.out_V + static_cast<size_t>(h) * la.n_max * 16, nullptr);
+                else
+                    gather_rows<8, false>(la.K + static_cast<size_t>(h) * a.L * 8, la.V + static_cast<size_t>(h) * a.L * 8,
+                                          sh, a.L, n_hi, n0, threadIdx.x, kThreads,
+                                          la.out_K + static_cast<size_t>(h) * la.n_max * 8,
+                                          la.out_V + static_cast<size_t>(h) * la.n_max * 8, nullptr);
+            } else if (vpr == 16)
                 gather_rows<16, true>(la.K + static_cast<size_t>(h) * a.L * 16, la.V + static_cast<size_t>(h) * a.L * 16, ih,
                                       a.L, n_hi, n0, threadIdx.x, kThreads,
                                       la.out_K + static_cast<size_t>(h) * la.n_max * 16,
