@@ -65,20 +65,32 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
         int need = k;
         for (int pass = 0; pass < 4; ++pass) {
             const int shift = 24 - 8 * pass;
-            {   // clear this warp's histogram row (256 x 16 bit = 128 words)
+            // Pass 0 sees the sign and exponent bits, which are nearly the same for all scores:
+            // lanes that hit the same bin are grouped with a match and add once to the warp's own
+            // histogram row. Later passes see spread-out digits of the few keys that still carry
+            // the prefix: there one atomic add per key into the shared histogram is cheaper.
+            const bool grouped = (pass == 0);
+            if (grouped) {   // clear this warp's histogram row (256 x 16 bit = 128 words)
                 uint32_t* row = reinterpret_cast<uint32_t*>(sm.whist[warp]);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) row[lane + 32 * q] = 0u;
+                __syncwarp();
+            } else {
+                if (tid < 256) sm.hist[tid] = 0;
+                __syncthreads();
             }
-            __syncwarp();
             const uint32_t himask = (pass == 0) ? 0u : (0xFFFFFFFFu << (shift + 8));
             auto count_one = [&](bool have, uint32_t key) {
                 const bool in = have && (key & himask) == prefix;
                 const int bin = in ? static_cast<int>((key >> shift) & 0xFF) : -1;
-                const unsigned peers = __match_any_sync(0xffffffffu, bin);
-                if (in && lane == __ffs(peers) - 1)
-                    sm.whist[warp][bin] += static_cast<unsigned short>(__popc(peers));
-                __syncwarp();
+                if (grouped) {
+                    const unsigned peers = __match_any_sync(0xffffffffu, bin);
+                    if (in && lane == __ffs(peers) - 1)
+                        sm.whist[warp][bin] += static_cast<unsigned short>(__popc(peers));
+                    __syncwarp();
+                } else if (in) {
+                    atomicAdd(&sm.hist[bin], 1);
+                }
             };
             if (IN_REGS) {
 #pragma unroll
@@ -89,12 +101,14 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
                     count_one(c0 + u < c1, (c0 + u < c1) ? select_order_key(sc[c0 + u]) : 0u);
             }
             __syncthreads();
-            if (tid < 256) {
-                int sum = 0;
-                for (int wv = 0; wv < nwarps; ++wv) sum += sm.whist[wv][tid];
-                sm.hist[tid] = sum;
+            if (grouped) {
+                if (tid < 256) {
+                    int sum = 0;
+                    for (int wv = 0; wv < nwarps; ++wv) sum += sm.whist[wv][tid];
+                    sm.hist[tid] = sum;
+                }
+                __syncthreads();
             }
-            __syncthreads();
             if (warp == 0) {
                 // lane t owns bins 255-8t .. 248-8t (descending), so a prefix over lanes counts from the top
                 int cnt[8], sum = 0;
