@@ -426,7 +426,7 @@ def run_ours(args, wl):
             "eager": {"value": LAYERS_PER_STEP * wl.L * world / (ms_eager * 1e-3), "unit": UNIT,
                       "us_per_layer": ms_eager / LAYERS_PER_STEP * 1e3,
                       "note": "same step, 32 direct C-ABI calls, no graph"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * LAYERS_PER_STEP * (1 if fused else 5),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * LAYERS_PER_STEP * ((2 if (S > 1 and 2 * (n_sm // S) <= n_sm) else 1) if fused else 5),
             "roofline": roofline, "roofline_more": extra_roof, "per_kernel": per_kernel,
             "cpu_baseline": cpu_baseline,
         }

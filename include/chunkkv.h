@@ -175,7 +175,9 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
  *                               (same stream). The budgets of all lanes that may run at the same
  *                               time must add up to no more than the number of SMs: the layer
  *                               kernel synchronises its CTAs grid-wide, which needs all of them
- *                               resident.
+ *                               resident. With a budget of at most half the SMs the rows are
+ *                               gathered by a second launch on the same stream whose small CTAs
+ *                               run on every SM beside the other lanes' resident CTAs.
  *   chunkkv_lane_status         synchronises `stream`, then CHUNKKV_OK or CHUNKKV_EDEVICE for the
  *                               lane (and clears its header)
  * lane must be 256-byte aligned device memory.

@@ -484,7 +484,11 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
             if (st != CHUNKKV_OK) return st;
             FusedLayerIO io;
-            io.K = K; io.V = V; io.out_K = out_K; io.out_V = out_V; io.out_idx = out_idx;
+            // A lane that owns at most half of the SMs leaves the row gather to a second launch of
+            // small CTAs that spread over every SM (they fit beside the other lanes' resident
+            // CTAs), instead of moving the rows through its own few SMs.
+            const bool split = lane != nullptr && 2 * ctas <= ctx->num_sms;
+            io.K = K; io.V = V; io.out_K = split ? nullptr : out_K; io.out_V = out_V; io.out_idx = out_idx;
             io.chunk_scores = payload;
             io.C = C; io.k = k; io.n_max = n_max;
             io.bar_count = reinterpret_cast<unsigned long long*>(base + 64);
@@ -493,6 +497,10 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
                 e = launch_layer_fused(plan, tm_q, tm_k, a, io, s);
             }
             if (e != cudaSuccess) return cuda_fail(e);
+            if (split) {
+                e = launch_gather_shared_sms(K, V, out_idx, L, Hkv, d, n_max, out_K, out_V, ctx->num_sms, s);
+                if (e != cudaSuccess) return cuda_fail(e);
+            }
             return CHUNKKV_OK;
         }
         if (lane != nullptr) return CHUNKKV_EINVAL_SHAPE;

@@ -72,6 +72,9 @@ cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int
 cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
                           int n_max, void* out_K, void* out_V, int32_t* idx_copy_or_null,
                           int num_sms, cudaStream_t stream);
+// The gather in small CTAs that can share SMs with resident layer-kernel CTAs (lanes).
+cudaError_t launch_gather_shared_sms(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
+                                     int n_max, void* out_K, void* out_V, int num_sms, cudaStream_t stream);
 
 // Scoring (score + finalisation kernels) into caller-supplied scratch: a 256-byte header whose
 // first word is the device status word, then the payload. Returns a CHUNKKV_* status;

@@ -904,6 +904,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             return;
         }
         grid_barrier_finish(la.bar_count, la.bar_count + 8, gridDim.x);   // exit counter sits 64 bytes on
+        if (la.out_K == nullptr) return;             // the rows are gathered by a separate launch
         // ---- gather: the Hkv * n_max output rows are split evenly over the CTAs
         const int vpr = a.d >> 3;
         const int rows_per_pass = (kThreads / vpr) * kGatherRowsPerThread;
