@@ -285,3 +285,19 @@ def test_lanes_run_layers_concurrently_and_match(ck):
                                             outs[0][1].data_ptr(), outs[0][2].data_ptr(), lanes[0].buf.data_ptr(),
                                             4096, n_sm // 4, None)
     assert st == -4
+
+
+@pytest.mark.parametrize("cfg,L,budget,ctas", [(1, 2048, 256, 18), (4, 9000, 900, 18), (5, 5000, 500, 16),
+                                               (2, 32768, 3276, 18), (2, 3001, 47, 5)])
+def test_lane_with_few_ctas_matches_oracle(ck, cfg, L, budget, ctas):
+    # a lane with a small share of the SMs (rows gathered by the second launch), shapes with
+    # d = 64, R = 256, c = 20, a ragged last chunk and a budget just above the window
+    wl = scaled(CONFIGS[cfg], L=L, budget=budget)
+    lane = ck.Lane(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=ctas)
+    x = make_layer(wl)
+    dev = (to_dev(x.q_obs), to_dev(x.K), to_dev(x.V))
+    for rep in range(2):
+        oK, oV, idx = lane.compress_layer(*dev, wl.Hq, wl.w, wl.c, wl.budget)
+    assert lane.status() == 0
+    _check_layer(x, wl, bits_of(oK), bits_of(oV), idx.cpu().numpy())
+
