@@ -4,12 +4,15 @@
 Metric: prefix tokens compressed per second per layer, on the Llama-3-8B 32K KV shape
 (Hq 32, Hkv 8, d 128, L 32768, w 32, c 10, budget 3276), seeded synthetic bf16 tensors.
 
-A step compresses the 32 layers of one 32K-token sequence: 32 calls of
-chunkkv_compress_layer (score -> chunk-sum -> top-k -> gather), cycling over NSETS distinct
-layer inputs (each 134 MB of K/V, so consecutive layers never find their K/V in L2).
-`value` is measured with the step captured in a CUDA graph and replayed (inputs resident in
-HBM); the same step launched call by call is reported as `eager`; `e2e` goes through
-chunkkv_compress_layer_host with pinned host buffers, copies inside the timed region.
+A step compresses the 32 layers of one 32K-token sequence: 32 layer calls
+(score -> chunk-sum -> top-k -> gather), cycling over NSETS distinct layer inputs (each 134 MB
+of K/V, so consecutive layers never find their K/V in L2). The layers are independent, so the
+step keeps `--lanes` of them in flight (chunkkv_compress_layer_lane, each lane on its own stream
+with its share of the SMs). `value` is measured with the step captured in a CUDA graph and
+replayed (inputs resident in HBM); the same step launched call by call is reported as `eager`,
+the same layers one after another on the whole GPU (chunkkv_compress_layer) as
+`roofline_more.single_layer`; `e2e` goes through chunkkv_compress_layer_host with pinned host
+buffers, copies inside the timed region.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 """
@@ -36,6 +39,9 @@ NSETS = 4
 LAYERS_PER_STEP = 32
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one cfg2 layer in an 18-CTA lane: layer kernel
+# 71.4 MB + row gather 13.5 MB (ncu capture of both launches)
+TRAFFIC_BYTES_PER_LAYER = 84.9e6
 
 
 def parse_args():
@@ -345,14 +351,25 @@ def run_ours(args, wl):
     peak, peak_src = measured_hbm_peak()
     score_us = per_kernel["score"]["avg_us"] or float("nan")
     fused = per_kernel["gather"]["launches"] == 0          # the whole layer ran as one kernel
-    dom_bytes = nbytes["layer"] if fused else nbytes["score"]
-    achieved = dom_bytes / (score_us * 1e-6) / 1e9
-    roofline = {"kernel": "score_kernel<FUSED> (score+chunk-sum+select+gather in one launch)" if fused else "score_kernel",
-                "bound": "hbm", "achieved": achieved, "peak": peak,
-                "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak, "traffic": None,
-                "algorithmic_bytes_per_launch": dom_bytes, "avg_launch_us": score_us,
-                "note": "kernel timed with the GPU to itself (one layer at a time); the step overlaps "
-                        f"{S} such launches on disjoint SM sets"}
+    split = S > 1 and 2 * (n_sm // S) <= n_sm               # a lane's layer = layer kernel + row-gather launch
+    # The timed region holds nothing but the launches of LAYERS_PER_STEP layers per step, S of them
+    # in flight at a time on disjoint SM sets, so the duration a launch accounts for is the region
+    # divided by the layers; algorithmic bytes per layer over that is what HBM sustains.
+    achieved = nbytes["layer"] / (ms_layer * 1e-3) / 1e9
+    kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) + gather_kernel "
+                   "(row gather in CTAs spread over all SMs): the two launches of a layer in a lane" % (n_sm // S)
+                   if split else "score_kernel<FUSED> (score + chunk sums + finalize + select + gather in one launch)")
+    roofline = {"kernel": kernel_name, "bound": "hbm", "achieved": achieved, "peak": peak,
+                "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": TRAFFIC_BYTES_PER_LAYER if (split and args.config == 2 and S == 8) else None,
+                "algorithmic_bytes_per_launch": nbytes["layer"], "avg_launch_us": ms_layer * 1e3,
+                "launches_in_flight": S,
+                "isolated_launch_us": score_us,
+                "isolated_frac": nbytes["layer"] / (score_us * 1e-6) / 1e9 / peak,
+                "note": "avg_launch_us = CUDA-event time of the timed region / layers launched in it "
+                        f"({S} layers in flight on disjoint SM sets, nothing else in the region); "
+                        "isolated_* = the whole-GPU layer kernel timed alone, one layer at a time; "
+                        "traffic = DRAM bytes of one layer's launches from an ncu capture (cold L2)"}
     layer_gbs = nbytes["layer"] / (ms_layer * 1e-3) / 1e9
     gather_us = per_kernel["gather"]["avg_us"]                    # None when the layer kernel is fused
     extra_roof = {
