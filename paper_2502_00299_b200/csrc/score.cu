@@ -62,29 +62,62 @@ __device__ __forceinline__ void load_panel(uint32_t taddr, float (&v)[WP]) {
 template <int C, int WP>
 __device__ __forceinline__ void panel_fast(float (&v)[WP], float sl2, bool active, float* part,
                                            int row_stride, float* out_m, float* out_l) {
-    float m0 = v[0], m1 = v[1], m2 = v[2], m3 = v[3];
+    static_assert(WP % 4 == 0 && WP >= 8, "panel width");
+    // row max with three-input max instructions, two independent chains
+    float m0 = fmaxf(v[0], v[1]), m1 = fmaxf(v[2], v[3]);
 #pragma unroll
     for (int u = 4; u + 3 < WP; u += 4) {
-        m0 = fmaxf(m0, v[u]); m1 = fmaxf(m1, v[u + 1]); m2 = fmaxf(m2, v[u + 2]); m3 = fmaxf(m3, v[u + 3]);
+        m0 = fmax3(m0, v[u], v[u + 1]);
+        m1 = fmax3(m1, v[u + 2], v[u + 3]);
     }
-    const float mx = fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
+    const float mx = fmaxf(m0, m1);
     const float neg_m2 = -mx * sl2;
-    // exponentials first, in place: WP independent operations the scheduler can overlap freely
-#pragma unroll
-    for (int u = 0; u < WP; ++u) v[u] = ex2_approx(fmaf(v[u], sl2, neg_m2));
-    // chunk sums as balanced trees (short dependency chains), one store per chunk
     float l = 0.f;
+    if constexpr (C % 2 == 0) {
+        // Two columns per instruction: scale-and-shift and the chunk sums run on packed pairs
+        // (same arithmetic, fewer instructions issued).
+        const unsigned long long s2 = pack2(sl2, sl2), n2 = pack2(neg_m2, neg_m2);
+        unsigned long long e[WP / 2];
 #pragma unroll
-    for (int ch = 0; ch < WP / C; ++ch) {
-        float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-        for (int t = 0; t < C; t += 2) {
-            s0 += v[ch * C + t];
-            if (t + 1 < C) s1 += v[ch * C + t + 1];
+        for (int u = 0; u < WP / 2; ++u) {
+            float x0, x1;
+            unpack2(fma2(pack2(v[2 * u], v[2 * u + 1]), s2, n2), x0, x1);
+            e[u] = pack2(ex2_approx(x0), ex2_approx(x1));
         }
-        const float acc = s0 + s1;
-        if (active) part[static_cast<size_t>(ch) * row_stride] = acc;
-        l += acc;
+        constexpr int H = C / 2;     // pairs per chunk
+#pragma unroll
+        for (int ch = 0; ch < WP / C; ++ch) {
+            unsigned long long s0 = e[ch * H];
+            unsigned long long s1 = (H > 1) ? e[ch * H + 1] : 0ull;
+#pragma unroll
+            for (int t = 2; t < H; t += 2) {
+                s0 = add2(s0, e[ch * H + t]);
+                if (t + 1 < H) s1 = add2(s1, e[ch * H + t + 1]);
+            }
+            if (H > 1) s0 = add2(s0, s1);
+            float lo, hi;
+            unpack2(s0, lo, hi);
+            const float acc = lo + hi;
+            if (active) part[static_cast<size_t>(ch) * row_stride] = acc;
+            l += acc;
+        }
+    } else {
+        // exponentials first, in place: WP independent operations the scheduler can overlap freely
+#pragma unroll
+        for (int u = 0; u < WP; ++u) v[u] = ex2_approx(fmaf(v[u], sl2, neg_m2));
+        // chunk sums as balanced trees (short dependency chains), one store per chunk
+#pragma unroll
+        for (int ch = 0; ch < WP / C; ++ch) {
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int t = 0; t < C; t += 2) {
+                s0 += v[ch * C + t];
+                if (t + 1 < C) s1 += v[ch * C + t + 1];
+            }
+            const float acc = s0 + s1;
+            if (active) part[static_cast<size_t>(ch) * row_stride] = acc;
+            l += acc;
+        }
     }
     *out_m = mx * sl2;
     *out_l = l;
@@ -889,6 +922,13 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             return;
         }
         // ---- top-k selection: one CTA per head
+        const bool rows_elsewhere = la.out_K == nullptr;   // the rows are gathered by a separate launch
+        if (rows_elsewhere) {
+            // Nothing follows the selection in this launch: CTAs check out of the barrier now
+            // (no CTA waits on it again) and those without a head leave at once.
+            grid_barrier_finish(la.bar_count, la.bar_count + 8, gridDim.x);
+            if (static_cast<int>(blockIdx.x) >= a.Hkv) return;
+        }
         for (int h = blockIdx.x; h < a.Hkv; h += gridDim.x) {
             const float* sc = la.chunk_scores + static_cast<size_t>(h) * la.C;
             int32_t* out = la.out_idx + static_cast<size_t>(h) * la.n_max;
@@ -899,12 +939,12 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             else
                 select_head<0>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
         }
+        if (rows_elsewhere) return;
         if (!grid_barrier(la.bar_count, gridDim.x, 2, bar_ok, abort_flag)) {
             if (threadIdx.x == 0) atomicExch(a.status, 1);
             return;
         }
         grid_barrier_finish(la.bar_count, la.bar_count + 8, gridDim.x);   // exit counter sits 64 bytes on
-        if (la.out_K == nullptr) return;             // the rows are gathered by a separate launch
         // ---- gather: the Hkv * n_max output rows are split evenly over the CTAs
         const int vpr = a.d >> 3;
         const int rows_per_pass = (kThreads / vpr) * kGatherRowsPerThread;
