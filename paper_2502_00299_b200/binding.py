@@ -56,6 +56,18 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_lane_status.argtypes = [vp, vp]
     L.chunkkv_compress_layer_lane.restype = i32
     L.chunkkv_compress_layer_lane.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, vp, vp, vp, sz, i32, vp]
+    L.chunkkv_pipe_bytes.restype = sz
+    L.chunkkv_pipe_bytes.argtypes = [i32] * 7
+    L.chunkkv_pipe_open.restype = i32
+    L.chunkkv_pipe_open.argtypes = [vp, sz, i32, ctypes.POINTER(vp)]
+    L.chunkkv_pipe_layer.restype = i32
+    L.chunkkv_pipe_layer.argtypes = [vp, vp, vp, vp] + [i32] * 7 + [vp, vp, vp, vp]
+    L.chunkkv_pipe_join.restype = i32
+    L.chunkkv_pipe_join.argtypes = [vp, vp]
+    L.chunkkv_pipe_status.restype = i32
+    L.chunkkv_pipe_status.argtypes = [vp, vp]
+    L.chunkkv_pipe_close.restype = i32
+    L.chunkkv_pipe_close.argtypes = [vp]
     L.chunkkv_score_noalloc.restype = i32
     L.chunkkv_score_noalloc.argtypes = [vp, vp] + [i32] * 6 + [vp, vp]
     L.chunkkv_profile_enable.restype = i32
@@ -237,6 +249,60 @@ class Lane:
             out_K.data_ptr(), out_V.data_ptr(), out_idx.data_ptr(), self.buf.data_ptr(), self.bytes,
             self.max_ctas, self.stream.cuda_stream or None), "chunkkv_compress_layer_lane")
         return out_K, out_V, out_idx
+
+
+class Pipe:
+    """A lane whose layers overlap each other (see chunkkv.h): scoring kernels back to back on
+    `stream`, everything after scoring on the pipe's own stream. Call join() before using outputs."""
+
+    def __init__(self, L: int, Hq: int, Hkv: int, d: int, w: int, c: int, max_ctas: int = 0,
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+        self.max_ctas = int(max_ctas)
+        self.bytes = int(lib.chunkkv_pipe_bytes(L, Hq, Hkv, d, w, c, self.max_ctas))
+        if self.bytes == 0:
+            raise ChunkKVError(-2, "chunkkv_pipe_bytes")
+        self.buf = torch.empty(self.bytes, dtype=torch.uint8, device=device or "cuda")
+        self.stream = stream if stream is not None else torch.cuda.Stream(device=self.buf.device)
+        handle = ctypes.c_void_p()
+        _check(lib.chunkkv_pipe_open(self.buf.data_ptr(), self.bytes, self.max_ctas, ctypes.byref(handle)),
+               "chunkkv_pipe_open")
+        self.handle = handle
+
+    def layer(self, q_obs: torch.Tensor, K: torch.Tensor, V: torch.Tensor, Hq: int, w: int, c: int, budget: int,
+              out_K: Optional[torch.Tensor] = None, out_V: Optional[torch.Tensor] = None,
+              out_idx: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+        """chunkkv_pipe_layer; the outputs are complete after join()."""
+        Hkv, L, d = K.shape
+        n_max = out_len(L, w, c, budget)
+        dev = K.device
+        with torch.cuda.stream(self.stream):
+            if out_K is None:
+                out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
+            if out_V is None:
+                out_V = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
+            if out_idx is None:
+                out_idx = torch.empty((Hkv, n_max), dtype=torch.int32, device=dev)
+        _check(lib.chunkkv_pipe_layer(self.handle, q_obs.data_ptr(), K.data_ptr(), V.data_ptr(), L, Hq, Hkv, d, w, c,
+                                      budget, out_K.data_ptr(), out_V.data_ptr(), out_idx.data_ptr(),
+                                      self.stream.cuda_stream or None), "chunkkv_pipe_layer")
+        return out_K, out_V, out_idx
+
+    def join(self) -> None:
+        _check(lib.chunkkv_pipe_join(self.handle, self.stream.cuda_stream or None), "chunkkv_pipe_join")
+
+    def status(self) -> int:
+        return lib.chunkkv_pipe_status(self.handle, self.stream.cuda_stream or None)
+
+    def close(self) -> None:
+        if self.handle is not None:
+            _check(lib.chunkkv_pipe_close(self.handle), "chunkkv_pipe_close")
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def compress_layer_host(host_q: torch.Tensor, host_K: torch.Tensor, host_V: torch.Tensor, Hq: int,

@@ -1162,6 +1162,23 @@ cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, c
     return dispatch_variant<true>(plan, tm_q, tm_k, args, la, stream);
 }
 
+// Chunk scores for compile-time chunk sizes (chunks never straddle panels) and R % 4 == 0, in CTAs
+// of two warps: small enough (64 threads) to run on an SM beside a resident CTA of the scoring
+// kernel, so the L2-latency-bound contraction of one layer spreads over every SM while other
+// layers are being scored. grid = (blocks per head, Hkv); a block takes a contiguous panel range.
+constexpr int kFinSmallThreads = 64;
+template <int RV, int PP>
+__global__ void __launch_bounds__(kFinSmallThreads)
+finalize_panels_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
+    const int h = blockIdx.y;
+    const int n_p = (a.P + g.wp - 1) / g.wp;                       // panels that hold chunks
+    const int per = (n_p + gridDim.x - 1) / gridDim.x;
+    const int p_lo = blockIdx.x * per, p_hi = min(p_lo + per, n_p);
+    if (p_lo >= p_hi) return;
+    const float* rs = a.row_stat + static_cast<size_t>(h) * 512;
+    contract_panels_aligned<RV, PP>(a, g, h, p_lo, p_hi, rs, rs + 256, out);
+}
+
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
                             int num_sms, cudaStream_t stream) {
     if (C <= 0) return cudaSuccess;
@@ -1179,6 +1196,19 @@ cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C,
     g.hs_max = plan.hs_max;
     g.C = C;
     rowstats_kernel<<<args.Hkv, kFinThreads, 0, stream>>>(args, g);
+    if (plan.c_static > 0 && (args.R & 3) == 0) {
+        const int n_p = (args.P + plan.wp - 1) / plan.wp;
+        int px = (4 * num_sms + args.Hkv - 1) / args.Hkv;          // about four small CTAs per SM
+        const int max_px = (n_p + 3) / 4;                          // at least four panels per CTA
+        if (px > max_px) px = max_px;
+        if (px < 1) px = 1;
+        dim3 pgrid(px, args.Hkv);
+        if (args.R <= 128)
+            finalize_panels_kernel<1, 2><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+        else
+            finalize_panels_kernel<2, 1><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+        return cudaGetLastError();
+    }
     dim3 grid(bx, args.Hkv);
     finalize_kernel<<<grid, kFinThreads, 0, stream>>>(args, g, out_scores);
     return cudaGetLastError();

@@ -301,3 +301,44 @@ def test_lane_with_few_ctas_matches_oracle(ck, cfg, L, budget, ctas):
     assert lane.status() == 0
     _check_layer(x, wl, bits_of(oK), bits_of(oV), idx.cpu().numpy())
 
+
+@pytest.mark.parametrize("cfg,L,budget,ctas", [(2, 6000, 600, 18), (1, 2048, 256, 9), (5, 5000, 500, 16),
+                                               (4, 9000, 900, 0), (2, 3001, 47, 5), (2, 40, 36, 18)])
+def test_pipe_overlapped_layers_match_oracle(ck, cfg, L, budget, ctas):
+    # five layers through one pipe (scoring back to back, the rest on the pipe's own stream, two
+    # scratch halves taking turns), then the same pipe again after a join
+    wl = scaled(CONFIGS[cfg], L=L, budget=budget)
+    pipe = ck.Pipe(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=ctas)
+    layers = [make_layer(wl, layer=i) for i in range(5)]
+    dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in layers]
+    torch.cuda.synchronize()
+    for rep in range(2):
+        outs = [pipe.layer(*dev[i], wl.Hq, wl.w, wl.c, wl.budget) for i in range(5)]
+        pipe.join()
+    assert pipe.status() == 0
+    for x, (oK, oV, idx) in zip(layers, outs):
+        _check_layer(x, wl, bits_of(oK), bits_of(oV), idx.cpu().numpy())
+    pipe.close()
+
+
+def test_pipe_refuses_small_scratch_and_bad_arguments(ck):
+    wl = scaled(CONFIGS[2], L=6000, budget=600)
+    x = make_layer(wl)
+    q, K, V = to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)
+    n_max = ck.out_len(wl.L, wl.w, wl.c, wl.budget)
+    oK = torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device="cuda")
+    oV = torch.empty_like(oK)
+    oI = torch.empty((wl.Hkv, n_max), dtype=torch.int32, device="cuda")
+    small = torch.empty(8192, dtype=torch.uint8, device="cuda")
+    import ctypes
+    h = ctypes.c_void_p()
+    assert ck.lib.chunkkv_pipe_open(small.data_ptr(), 8192, 18, ctypes.byref(h)) == 0
+    args = (q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, wl.budget,
+            oK.data_ptr(), oV.data_ptr(), oI.data_ptr(), None)
+    assert ck.lib.chunkkv_pipe_layer(h, *args) == -4
+    assert ck.lib.chunkkv_pipe_layer(h, None, *args[1:]) == -1
+    assert ck.lib.chunkkv_pipe_layer(None, *args) == -1
+    assert ck.lib.chunkkv_pipe_status(h, None) == 0
+    assert ck.lib.chunkkv_pipe_close(h) == 0
+    assert ck.lib.chunkkv_pipe_open(small.data_ptr() + 16, 8192, 18, ctypes.byref(h)) == -3
+
