@@ -54,6 +54,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--lanes", type=int, default=8, help="layers in flight (each on 1/lanes of the SMs)")
+    ap.add_argument("--mode", choices=("pipe", "lane"), default="pipe",
+                    help="pipe: chunkkv_pipe_layer (scoring back to back, the rest on side streams); "
+                         "lane: chunkkv_compress_layer_lane (one layer at a time per lane)")
     return ap.parse_args()
 
 
@@ -231,15 +234,17 @@ def run_ours(args, wl):
     S = max(1, args.lanes)
     stream = torch.cuda.Stream(device=dev)
     lanes = []
+    piped = args.mode == "pipe" and S > 1
     if S > 1:
         for li in range(S):
-            ln = ck.Lane(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=n_sm // S, device=dev,
-                         stream=stream if li == 0 else None)
+            cls = ck.Pipe if piped else ck.Lane
+            ln = cls(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=n_sm // S, device=dev,
+                     stream=stream if li == 0 else None)
             lanes.append(ln)
     lane_streams = [ln.stream for ln in lanes] if lanes else [stream]
-    # every lane writes its own output buffers (layers in flight never share an output)
+    # every layer of a step writes its own output buffers
     lane_outs = []
-    for _ in range(S):
+    for _ in range(LAYERS_PER_STEP):
         o = [torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device=dev) for _ in range(2)]
         o.append(torch.empty((wl.Hkv, n_max), dtype=torch.int32, device=dev))
         lane_outs.append(o)
@@ -247,8 +252,17 @@ def run_ours(args, wl):
     def call_layer(i: int, reuse: bool = False, single: bool = False):
         q, K, V = sets[i % NSETS][0]
         li = 0 if single else i % S
-        oK, oV, oI = lane_outs[li]
-        if S > 1 and not single:
+        oK, oV, oI = lane_outs[i]
+        if piped and not single and not reuse:
+            ln = lanes[li]
+            st = lib.chunkkv_pipe_layer(
+                ln.handle, q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, wl.budget,
+                oK.data_ptr(), oV.data_ptr(), oI.data_ptr(), ln.stream.cuda_stream)
+        elif piped and not single:
+            st = lib.chunkkv_compress_layer(       # gather-only layers need no pipe: spread over the lane streams
+                None, K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, wl.budget, oI.data_ptr(),
+                oK.data_ptr(), oV.data_ptr(), oI.data_ptr(), lanes[li].stream.cuda_stream)
+        elif S > 1 and not single:
             ln = lanes[li]
             st = lib.chunkkv_compress_layer_lane(
                 None if reuse else q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
@@ -273,6 +287,9 @@ def run_ours(args, wl):
         for i in range(LAYERS_PER_STEP):
             call_layer(i, reuse, single)
         if multi:
+            if piped and not reuse:
+                for ln in lanes:
+                    ln.join()
             for st_ in lane_streams[1:]:
                 ev = torch.cuda.Event()
                 ev.record(st_)
@@ -352,6 +369,7 @@ def run_ours(args, wl):
     score_us = per_kernel["score"]["avg_us"] or float("nan")
     fused = per_kernel["gather"]["launches"] == 0          # the whole layer ran as one kernel
     split = S > 1 and 2 * (n_sm // S) <= n_sm               # a lane's layer = layer kernel + row-gather launch
+    launches_per_layer = 5 if piped else (2 if split else 1)    # pipe: score, row stats, finalize, select, gather
     # The timed region holds nothing but the launches of LAYERS_PER_STEP layers per step, S of them
     # in flight at a time on disjoint SM sets, so the duration a launch accounts for is the region
     # divided by the layers; algorithmic bytes per layer over that is what HBM sustains.
@@ -443,7 +461,7 @@ def run_ours(args, wl):
             "eager": {"value": LAYERS_PER_STEP * wl.L * world / (ms_eager * 1e-3), "unit": UNIT,
                       "us_per_layer": ms_eager / LAYERS_PER_STEP * 1e3,
                       "note": "same step, 32 direct C-ABI calls, no graph"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * LAYERS_PER_STEP * ((2 if (S > 1 and 2 * (n_sm // S) <= n_sm) else 1) if fused else 5),
+            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * LAYERS_PER_STEP * (launches_per_layer if fused else 5),
             "roofline": roofline, "roofline_more": extra_roof, "per_kernel": per_kernel,
             "cpu_baseline": cpu_baseline,
         }

@@ -61,7 +61,7 @@ __device__ __forceinline__ void load_panel(uint32_t taddr, float (&v)[WP]) {
 // compile time: all control flow below folds away after unrolling.
 template <int C, int WP>
 __device__ __forceinline__ void panel_fast(float (&v)[WP], float sl2, bool active, float* part,
-                                           int row_stride, float* out_m, float* out_l) {
+                                           int row_stride, uint64_t keep, float* out_m, float* out_l) {
     static_assert(WP % 4 == 0 && WP >= 8, "panel width");
     // row max with three-input max instructions, two independent chains
     float m0 = fmaxf(v[0], v[1]), m1 = fmaxf(v[2], v[3]);
@@ -98,7 +98,7 @@ __device__ __forceinline__ void panel_fast(float (&v)[WP], float sl2, bool activ
             float lo, hi;
             unpack2(s0, lo, hi);
             const float acc = lo + hi;
-            if (active) part[static_cast<size_t>(ch) * row_stride] = acc;
+            if (active) st_keep(part + static_cast<size_t>(ch) * row_stride, acc, keep);
             l += acc;
         }
     } else {
@@ -115,7 +115,7 @@ __device__ __forceinline__ void panel_fast(float (&v)[WP], float sl2, bool activ
                 if (t + 1 < C) s1 += v[ch * C + t + 1];
             }
             const float acc = s0 + s1;
-            if (active) part[static_cast<size_t>(ch) * row_stride] = acc;
+            if (active) st_keep(part + static_cast<size_t>(ch) * row_stride, acc, keep);
             l += acc;
         }
     }
@@ -128,7 +128,7 @@ __device__ __forceinline__ void panel_fast(float (&v)[WP], float sl2, bool activ
 // columns the row cannot see (causal mask in the window, or past L) contribute nothing.
 template <int C, int WP>
 __device__ __forceinline__ void panel_static_tail(const float (&v)[WP], float sl2, bool active, float* part,
-                                                  int row_stride, int j0, int P, int last_visible,
+                                                  int row_stride, uint64_t keep, int j0, int P, int last_visible,
                                                   float* out_m, float* out_l) {
     const int n_vis = last_visible - j0 + 1;     // columns u < n_vis are visible
     const int n_pre = P - j0;                    // columns u < n_pre belong to the prefix
@@ -144,7 +144,7 @@ __device__ __forceinline__ void panel_static_tail(const float (&v)[WP], float sl
         const float pe = (u < n_pre) ? e : 0.f;
         acc = (u % C == 0) ? pe : acc + pe;
         if ((u + 1) % C == 0) {
-            if (active && (u + 1 - C) < n_pre) part[static_cast<size_t>((u + 1) / C - 1) * row_stride] = acc;
+            if (active && (u + 1 - C) < n_pre) st_keep(part + static_cast<size_t>((u + 1) / C - 1) * row_stride, acc, keep);
         }
     }
     *out_m = (mx == -CUDART_INF_F) ? -CUDART_INF_F : mx * sl2;
@@ -399,6 +399,7 @@ __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, cons
         reinterpret_cast<const float4*>(a.partial + static_cast<size_t>(h) * g.n_panels * g.spp * a.R);
     float* out_h = out + static_cast<size_t>(h) * g.C;
     const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+    const uint64_t drop = l2_policy_evict_first();    // the partial sums are dead once read
     float4 m4[RV], li4[RV];
     bool have[RV];
 #pragma unroll
@@ -418,7 +419,7 @@ __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, cons
             max_slots = max(max_slots, n_slots[q]);
 #pragma unroll
             for (int it = 0; it < RV; ++it)
-                pm[q][it] = (n_slots[q] > 0 && have[it]) ? __ldcg(stat_h + static_cast<size_t>(p) * r4 + lane + 32 * it)
+                pm[q][it] = (n_slots[q] > 0 && have[it]) ? ld_last_use(stat_h + static_cast<size_t>(p) * r4 + lane + 32 * it, drop)
                                                          : zero4;
         }
         if (max_slots == 0) break;                                 // panels past the prefix hold no chunk
@@ -434,7 +435,7 @@ __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, cons
 #pragma unroll
                     for (int it = 0; it < RV; ++it)
                         pv[q][u][it] = (slot && have[it])
-                                           ? __ldcg(part_h + static_cast<size_t>(ch_base + s0 + u) * r4 + lane + 32 * it)
+                                           ? ld_last_use(part_h + static_cast<size_t>(ch_base + s0 + u) * r4 + lane + 32 * it, drop)
                                            : zero4;
                 }
             }
@@ -746,6 +747,8 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int last_visible = a.P + (row % a.w);  // this row sees keys j <= P + r (all < L)
         const int n_panels = g.n_tiles * PPT * SUBS;
         float run_m = -CUDART_INF_F, run_l = 0.f;    // (max, sum) over this thread's panels of the head
+        // the partial sums and panel maxima are read back once, shortly: hold them in L2 ahead of streamed data
+        const uint64_t keep = l2_policy_evict_last();
         int cur_head = -1, hs = -1, ti = 0;
         auto flush_head = [&]() {
             if (cur_head >= 0 && hs < g.hs_max) {
@@ -789,13 +792,13 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 float m2, l;
                 if constexpr (C_STATIC > 0) {
                     if (j0 + WPP <= a.P)
-                        panel_fast<C_STATIC, WPP>(v, a.sl2, active, part, a.R, &m2, &l);
+                        panel_fast<C_STATIC, WPP>(v, a.sl2, active, part, a.R, keep, &m2, &l);
                     else
-                        panel_static_tail<C_STATIC, WPP>(v, a.sl2, active, part, a.R, j0, a.P, last_visible, &m2, &l);
+                        panel_static_tail<C_STATIC, WPP>(v, a.sl2, active, part, a.R, keep, j0, a.P, last_visible, &m2, &l);
                 } else {
                     panel_general<WPP>(v, a.sl2, active, part, a.R, j0, a.P, a.c, last_visible, &m2, &l);
                 }
-                if (active) a.stat_m[panel_id * a.R + row] = m2;
+                if (active) st_keep(a.stat_m + panel_id * a.R + row, m2, keep);
                 // fold into the running record: l is relative to m2, run_l to run_m
                 const float nm = fmaxf(run_m, m2);
                 const float s_old = (run_m == -CUDART_INF_F) ? 0.f : ex2_approx(run_m - nm);
