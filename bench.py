@@ -54,7 +54,7 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--lanes", type=int, default=8, help="layers in flight (each on 1/lanes of the SMs)")
-    ap.add_argument("--mode", choices=("pipe", "lane"), default="pipe",
+    ap.add_argument("--mode", choices=("pipe", "lane"), default="lane",
                     help="pipe: chunkkv_pipe_layer (scoring back to back, the rest on side streams); "
                          "lane: chunkkv_compress_layer_lane (one layer at a time per lane)")
     return ap.parse_args()
@@ -374,12 +374,17 @@ def run_ours(args, wl):
     # in flight at a time on disjoint SM sets, so the duration a launch accounts for is the region
     # divided by the layers; algorithmic bytes per layer over that is what HBM sustains.
     achieved = nbytes["layer"] / (ms_layer * 1e-3) / 1e9
-    kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) + gather_kernel "
-                   "(row gather in CTAs spread over all SMs): the two launches of a layer in a lane" % (n_sm // S)
-                   if split else "score_kernel<FUSED> (score + chunk sums + finalize + select + gather in one launch)")
+    if piped:
+        kernel_name = ("score_kernel on %d CTAs + rowstats/finalize/select/gather kernels on the pipe's side stream: "
+                       "the five launches of a layer in a pipe" % (n_sm // S))
+    elif split:
+        kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) + gather_kernel "
+                       "(row gather in CTAs spread over all SMs): the two launches of a layer in a lane" % (n_sm // S))
+    else:
+        kernel_name = "score_kernel<FUSED> (score + chunk sums + finalize + select + gather in one launch)"
     roofline = {"kernel": kernel_name, "bound": "hbm", "achieved": achieved, "peak": peak,
                 "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": TRAFFIC_BYTES_PER_LAYER if (split and args.config == 2 and S == 8) else None,
+                "traffic": TRAFFIC_BYTES_PER_LAYER if (split and not piped and args.config == 2 and S == 8) else None,
                 "algorithmic_bytes_per_launch": nbytes["layer"], "avg_launch_us": ms_layer * 1e3,
                 "launches_in_flight": S,
                 "isolated_launch_us": score_us,
@@ -452,7 +457,8 @@ def run_ours(args, wl):
             "config": {"workload": wl.name, "Hq": wl.Hq, "Hkv": wl.Hkv, "d": wl.d, "L": wl.L, "w": wl.w,
                        "c": wl.c, "budget": wl.budget, "layers_per_step": LAYERS_PER_STEP,
                        "lanes": S,
-                       "launch": f"one CUDA graph per step: 32 chunkkv_compress_layer calls, {S} in flight "
+                       "mode": args.mode if S > 1 else "single",
+                       "launch": f"one CUDA graph per step: 32 layer calls ({'chunkkv_pipe_layer' if piped else 'chunkkv_compress_layer_lane'}), {S} in flight "
                                  f"on {S} streams with {n_sm // S} CTAs each" if S > 1 else
                                  "one CUDA graph per step (32 chunkkv_compress_layer calls captured)",
                        "l2": f"layers cycle over {NSETS} distinct K/V sets of "
