@@ -12,11 +12,17 @@ namespace chunkkv {
 
 constexpr int kGatherRowsPerThread = 4;
 
-__device__ __forceinline__ uint4 gather_ld(const uint4* p) {
+// Rows are read once: no L1 allocation, first in line for eviction from L2.
+__device__ __forceinline__ unsigned long long gather_policy() {
+    unsigned long long p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint4 gather_ld(const uint4* p, unsigned long long policy) {
     uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
+                 : "l"(p), "l"(policy));
     return v;
 }
 __device__ __forceinline__ void gather_st(uint4* p, const uint4& v) {
@@ -35,6 +41,7 @@ __device__ __forceinline__ void gather_rows(const uint4* __restrict__ Kh, const 
                                             uint4* __restrict__ oK, uint4* __restrict__ oV, int32_t* idx_copy) {
     const int rows_per_pass = nthreads / VPR;
     const int vec = tid % VPR, sub = tid / VPR;
+    const unsigned long long policy = gather_policy();
     int src[kGatherRowsPerThread];
     uint4 kv[kGatherRowsPerThread], vv[kGatherRowsPerThread];
 #pragma unroll
@@ -46,8 +53,8 @@ __device__ __forceinline__ void gather_rows(const uint4* __restrict__ Kh, const 
 #pragma unroll
     for (int u = 0; u < kGatherRowsPerThread; ++u) {
         const bool ok = static_cast<unsigned>(src[u]) < static_cast<unsigned>(L);
-        kv[u] = ok ? gather_ld(Kh + static_cast<size_t>(src[u]) * VPR + vec) : make_uint4(0, 0, 0, 0);
-        vv[u] = ok ? gather_ld(Vh + static_cast<size_t>(src[u]) * VPR + vec) : make_uint4(0, 0, 0, 0);
+        kv[u] = ok ? gather_ld(Kh + static_cast<size_t>(src[u]) * VPR + vec, policy) : make_uint4(0, 0, 0, 0);
+        vv[u] = ok ? gather_ld(Vh + static_cast<size_t>(src[u]) * VPR + vec, policy) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
     for (int u = 0; u < kGatherRowsPerThread; ++u) {
