@@ -342,3 +342,46 @@ def test_pipe_refuses_small_scratch_and_bad_arguments(ck):
     assert ck.lib.chunkkv_pipe_close(h) == 0
     assert ck.lib.chunkkv_pipe_open(small.data_ptr() + 16, 8192, 18, ctypes.byref(h)) == -3
 
+
+def _random_shapes(n, seed):
+    """Seeded shapes over the supported ranges (R <= 256, d in {64, 128}), with L and the budget
+    near the interesting edges as often as in the bulk."""
+    rng = np.random.Generator(np.random.Philox(key=seed))
+    out = []
+    while len(out) < n:
+        Hkv = int(rng.choice([1, 2, 3, 8]))
+        G = int(rng.choice([1, 2, 4, 8]))
+        w = int(rng.choice([1, 4, 16, 32, 64]))
+        if w * G > 256:
+            continue
+        d = int(rng.choice([64, 128]))
+        c = int(rng.choice([1, 3, 10, 16, 20]))
+        L = int(rng.choice([w, w + 1, w + c, int(rng.integers(w, 600)), int(rng.integers(600, 4000))]))
+        budget = int(rng.choice([w, w + c - 1, w + c, max(w, L // 10), max(w, L // 3), L, L + 7]))
+        out.append((Hkv, G, w, d, c, L, budget))
+    return out
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_random_shapes_through_all_three_layer_calls(ck, case):
+    # the same layer through chunkkv_compress_layer, a lane with few CTAs and a pipe with few CTAs
+    Hkv, G, w, d, c, L, budget = _random_shapes(24, 1234)[case]
+    wl = scaled(CONFIGS[1], Hq=Hkv * G, Hkv=Hkv, d=d, L=L, w=w, c=c, budget=budget, seed=100 + case,
+                planted_count=2, sink_tokens=0)
+    x = make_layer(wl)
+    dev = (to_dev(x.q_obs), to_dev(x.K), to_dev(x.V))
+    oK, oV, idx = _run_layer(ck, x, wl)
+    _check_layer(x, wl, oK, oV, idx)
+    ctas = 1 + case % 7
+    lane = ck.Lane(L, wl.Hq, Hkv, d, w, c, max_ctas=ctas)
+    lK, lV, lidx = lane.compress_layer(*dev, wl.Hq, w, c, budget)
+    assert lane.status() == 0
+    _check_layer(x, wl, bits_of(lK), bits_of(lV), lidx.cpu().numpy())
+    pipe = ck.Pipe(L, wl.Hq, Hkv, d, w, c, max_ctas=ctas)
+    outs = [pipe.layer(*dev, wl.Hq, w, c, budget) for _ in range(3)]
+    pipe.join()
+    assert pipe.status() == 0
+    for pK, pV, pidx in outs:
+        _check_layer(x, wl, bits_of(pK), bits_of(pV), pidx.cpu().numpy())
+    pipe.close()
+
