@@ -356,16 +356,20 @@ def _random_shapes(n, seed):
             continue
         d = int(rng.choice([64, 128]))
         c = int(rng.choice([1, 3, 10, 16, 20]))
-        L = int(rng.choice([w, w + 1, w + c, int(rng.integers(w, 600)), int(rng.integers(600, 4000))]))
-        budget = int(rng.choice([w, w + c - 1, w + c, max(w, L // 10), max(w, L // 3), L, L + 7]))
+        if len(out) % 2 == 0:     # edges
+            L = int(rng.choice([w, w + 1, w + c, int(rng.integers(w, 600)), int(rng.integers(600, 4000))]))
+            budget = int(rng.choice([w, w + c - 1, w + c, max(w, L // 10), max(w, L // 3), L, L + 7]))
+        else:                     # bulk: several tiles, a ragged last chunk more often than not
+            L = int(rng.integers(max(600, w + c), 6000))
+            budget = int(rng.integers(w + c, max(w + c + 1, L // 2)))
         out.append((Hkv, G, w, d, c, L, budget))
     return out
 
 
-@pytest.mark.parametrize("case", range(24))
+@pytest.mark.parametrize("case", range(32))
 def test_random_shapes_through_all_three_layer_calls(ck, case):
     # the same layer through chunkkv_compress_layer, a lane with few CTAs and a pipe with few CTAs
-    Hkv, G, w, d, c, L, budget = _random_shapes(24, 1234)[case]
+    Hkv, G, w, d, c, L, budget = _random_shapes(32, 1234)[case]
     wl = scaled(CONFIGS[1], Hq=Hkv * G, Hkv=Hkv, d=d, L=L, w=w, c=c, budget=budget, seed=100 + case,
                 planted_count=2, sink_tokens=0)
     x = make_layer(wl)
