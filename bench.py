@@ -7,8 +7,9 @@ Metric: prefix tokens compressed per second per layer, on the Llama-3-8B 32K KV 
 A step compresses the 32 layers of one 32K-token sequence: 32 layer calls
 (score -> chunk-sum -> top-k -> gather), cycling over NSETS distinct layer inputs (each 134 MB
 of K/V, so consecutive layers never find their K/V in L2). The layers are independent, so the
-step keeps `--lanes` of them in flight (chunkkv_compress_layer_lane, each lane on its own stream
-with its share of the SMs). `value` is measured with the step captured in a CUDA graph and
+step keeps `--lanes` of them in flight (chunkkv_pipe_layer, each pipe on its own stream with
+its share of the SMs and its row gathers on a side stream; `--mode lane` uses
+chunkkv_compress_layer_lane instead). `value` is measured with the step captured in a CUDA graph and
 replayed (inputs resident in HBM); the same step launched call by call is reported as `eager`,
 the same layers one after another on the whole GPU (chunkkv_compress_layer) as
 `roofline_more.single_layer`; `e2e` goes through chunkkv_compress_layer_host with pinned host
@@ -54,8 +55,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--lanes", type=int, default=8, help="layers in flight (each on 1/lanes of the SMs)")
-    ap.add_argument("--mode", choices=("pipe", "lane"), default="lane",
-                    help="pipe: chunkkv_pipe_layer (scoring back to back, the rest on side streams); "
+    ap.add_argument("--mode", choices=("pipe", "lane"), default="pipe",
+                    help="pipe: chunkkv_pipe_layer (layer kernels back to back, row gathers on side streams); "
                          "lane: chunkkv_compress_layer_lane (one layer at a time per lane)")
     return ap.parse_args()
 
@@ -369,14 +370,15 @@ def run_ours(args, wl):
     score_us = per_kernel["score"]["avg_us"] or float("nan")
     fused = per_kernel["gather"]["launches"] == 0          # the whole layer ran as one kernel
     split = S > 1 and 2 * (n_sm // S) <= n_sm               # a lane's layer = layer kernel + row-gather launch
-    launches_per_layer = 5 if piped else (2 if split else 1)    # pipe: score, row stats, finalize, select, gather
+    launches_per_layer = 2 if (piped or split) else 1           # layer kernel + row gather
     # The timed region holds nothing but the launches of LAYERS_PER_STEP layers per step, S of them
     # in flight at a time on disjoint SM sets, so the duration a launch accounts for is the region
     # divided by the layers; algorithmic bytes per layer over that is what HBM sustains.
     achieved = nbytes["layer"] / (ms_layer * 1e-3) / 1e9
     if piped:
-        kernel_name = ("score_kernel on %d CTAs + rowstats/finalize/select/gather kernels on the pipe's side stream: "
-                       "the five launches of a layer in a pipe" % (n_sm // S))
+        kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) on the pipe's main stream + "
+                       "gather_kernel (row gather in CTAs spread over all SMs) on its side stream: the two launches of a "
+                       "layer in a pipe" % (n_sm // S))
     elif split:
         kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) + gather_kernel "
                        "(row gather in CTAs spread over all SMs): the two launches of a layer in a lane" % (n_sm // S))
@@ -384,7 +386,7 @@ def run_ours(args, wl):
         kernel_name = "score_kernel<FUSED> (score + chunk sums + finalize + select + gather in one launch)"
     roofline = {"kernel": kernel_name, "bound": "hbm", "achieved": achieved, "peak": peak,
                 "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": TRAFFIC_BYTES_PER_LAYER if (split and not piped and args.config == 2 and S == 8) else None,
+                "traffic": TRAFFIC_BYTES_PER_LAYER if ((split or piped) and args.config == 2 and S == 8) else None,
                 "algorithmic_bytes_per_launch": nbytes["layer"], "avg_launch_us": ms_layer * 1e3,
                 "launches_in_flight": S,
                 "isolated_launch_us": score_us,

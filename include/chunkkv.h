@@ -191,26 +191,29 @@ CHUNKKV_API int chunkkv_compress_layer_lane(const void* q_obs, const void* K, co
                                             void* lane, size_t lane_bytes, int max_ctas, void* stream);
 
 /*
- * Pipes: a lane whose layers overlap each other. Scoring a layer (Algorithm 3's attention scores
- * and chunk sums) is bound by arithmetic on the lane's SMs; what follows it (normalisation,
- * top-k, gather) is bound by latency and by memory traffic. A pipe therefore runs the scoring
- * kernels of successive layers back to back on the caller's stream, with at most max_ctas CTAs,
- * and everything after scoring on a stream of its own, in small CTAs that share SMs with
- * resident scoring CTAs of this and other pipes. Two scratch halves alternate between layers.
+ * Pipes: a lane whose row gathers overlap the next layer. Scoring and selecting a layer
+ * (Algorithm 3 up to the indices) is bound by arithmetic on the lane's SMs; gathering its rows
+ * is bound by memory traffic and needs none of the lane's scratch. A pipe therefore runs the
+ * lane's layer kernels of successive layers back to back on the caller's stream, with at most
+ * max_ctas CTAs, and each layer's row gather on a stream of its own, in small CTAs that share SMs
+ * with resident layer-kernel CTAs of this and other pipes.
  *
- *   chunkkv_pipe_bytes   device scratch a pipe needs for a shape and CTA budget (0 = all SMs)
- *   chunkkv_pipe_open    makes the host object (a side stream and four events) over caller-owned
- *                        scratch (256-byte aligned device memory, cleared here); synchronous.
+ *   chunkkv_pipe_bytes   device scratch a pipe needs for a shape and CTA budget (0 = all SMs);
+ *                        the same as chunkkv_lane_bytes
+ *   chunkkv_pipe_open    makes the host object (a side stream and two events) over caller-owned
+ *                        scratch (256-byte aligned device memory, header cleared here); synchronous.
  *   chunkkv_pipe_layer   chunkkv_compress_layer (compute path, q_obs required) through the pipe:
- *                        scoring is queued on `stream`, the rest on the pipe's stream. Calls on
- *                        one pipe must come from one thread and use one stream. The outputs of a
- *                        layer are complete only for work queued after chunkkv_pipe_join; layers
- *                        queued before the join must not share output buffers with each other.
+ *                        the layer kernel is queued on `stream`, the gather on the pipe's stream.
+ *                        Calls on one pipe must come from one thread and use one stream. The
+ *                        outputs of a layer are complete only for work queued after
+ *                        chunkkv_pipe_join; layers queued before the join must not share output
+ *                        buffers with each other. The CTA budgets of pipes (and lanes) that may
+ *                        run at the same time must add up to no more than the number of SMs.
  *   chunkkv_pipe_join    makes `stream` wait for everything the pipe has queued (device-side
  *                        wait, no host synchronisation). Required before the outputs are used
  *                        and before a stream capture that contains pipe calls ends.
  *   chunkkv_pipe_status  join + synchronise `stream`; CHUNKKV_OK or CHUNKKV_EDEVICE (an abandoned
- *                        wait in a scoring kernel; the status words are cleared)
+ *                        wait in a layer kernel; the status word is cleared)
  *   chunkkv_pipe_close   waits for the pipe's stream and frees the host object (not the scratch)
  * Errors: CHUNKKV_ENOWORKSPACE when the scratch is too small for the shape; otherwise as
  * chunkkv_compress_layer. The paper runs its layers one after another (Algorithm 2); overlapping

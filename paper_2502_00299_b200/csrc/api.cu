@@ -43,19 +43,17 @@ struct DeviceCtx {
 
 std::mutex g_mu;
 
-// Host side of a pipe (chunkkv_pipe_*): two scratch halves used by alternate layers, a side stream
-// for everything that follows scoring, and the events that order the two streams.
+// Host side of a pipe (chunkkv_pipe_*): caller-owned lane scratch, a side stream for the row gathers
+// and the two events that order it against the caller's stream.
 struct Pipe {
     int device = 0;
     char* scratch = nullptr;
-    size_t half_bytes = 0;
+    size_t bytes = 0;
     int max_ctas = 0;
     cudaStream_t side = nullptr;
-    cudaEvent_t scored[2] = {nullptr, nullptr};
-    cudaEvent_t posted[2] = {nullptr, nullptr};
-    bool pending[2] = {false, false};   // the half's last post-processing was queued since the last join
-    int last = -1;                      // half whose post-processing was queued last (-1: none pending)
-    int next = 0;
+    cudaEvent_t scored = nullptr;    // the layer kernel of the latest layer, on the caller's stream
+    cudaEvent_t posted = nullptr;    // the row gather of the latest layer, on the side stream
+    bool pending = false;            // a gather was queued since the last join
 };
 DeviceCtx g_ctx[kMaxDevices];
 EncodeTiledFn g_encode = nullptr;
@@ -436,9 +434,12 @@ int chunkkv_gather(const void* K, const void* V, const int32_t* idx, int L, int 
 
 // Shared body of chunkkv_compress_layer and chunkkv_compress_layer_lane. `lane` = caller-owned
 // scratch (NULL: the device-wide scratch), `max_ctas` = CTA budget of the launch (0: every SM).
+// rows_elsewhere != NULL (pipes): the caller gathers the rows itself after this call, so the layer
+// kernel always runs without its gather phase and no gather is launched here.
 static int compress_impl(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv, int d, int w,
                          int c, int budget, const int32_t* reuse_idx, void* out_K, void* out_V,
-                         int32_t* out_idx, void* lane, size_t lane_bytes, int max_ctas, void* stream) {
+                         int32_t* out_idx, void* lane, size_t lane_bytes, int max_ctas, void* stream,
+                         const void* rows_elsewhere = nullptr) {
     int st = check_sizes(L, w, c, budget);
     if (st != CHUNKKV_OK) return st;
     st = check_heads(L, Hq, Hkv, d, w);
@@ -502,7 +503,7 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
             // A lane that owns at most half of the SMs leaves the row gather to a second launch of
             // small CTAs that spread over every SM (they fit beside the other lanes' resident
             // CTAs), instead of moving the rows through its own few SMs.
-            const bool split = lane != nullptr && 2 * ctas <= ctx->num_sms;
+            const bool split = rows_elsewhere != nullptr || (lane != nullptr && 2 * ctas <= ctx->num_sms);
             io.K = K; io.V = V; io.out_K = split ? nullptr : out_K; io.out_V = out_V; io.out_idx = out_idx;
             io.chunk_scores = payload;
             io.C = C; io.k = k; io.n_max = n_max;
@@ -512,7 +513,7 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
                 e = launch_layer_fused(plan, tm_q, tm_k, a, io, s);
             }
             if (e != cudaSuccess) return cuda_fail(e);
-            if (split) {
+            if (split && rows_elsewhere == nullptr) {
                 e = launch_gather_shared_sms(K, V, out_idx, L, Hkv, d, n_max, out_K, out_V, ctx->num_sms, s);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
@@ -527,7 +528,7 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
         e = launch_select(chunk_scores, L, Hkv, w, c, C, k, n_max, out_idx, s);
     }
     if (e != cudaSuccess) return cuda_fail(e);
-    {
+    if (rows_elsewhere == nullptr) {
         Timer t(ctx, s, 3);
         e = launch_gather(K, V, out_idx, L, Hkv, d, n_max, out_K, out_V, nullptr, ctas, s);
     }
@@ -592,22 +593,7 @@ int chunkkv_compress_layer_lane(const void* q_obs, const void* K, const void* V,
 }
 
 size_t chunkkv_pipe_bytes(int L, int Hq, int Hkv, int d, int w, int c, int max_ctas) {
-    if (w < 1 || c < 1 || L < w || max_ctas < 0) return 0;
-    if (check_heads(L, Hq, Hkv, d, w) != CHUNKKV_OK) return 0;
-    std::lock_guard<std::mutex> lk(g_mu);
-    DeviceCtx* ctx;
-    if (get_ctx(&ctx) != CHUNKKV_OK) return 0;
-    const int ctas = (max_ctas > 0 && max_ctas < ctx->num_sms) ? max_ctas : ctx->num_sms;
-    const int R = w * (Hq / Hkv);
-    const int C = (L - w + c - 1) / c;
-    size_t floats = (static_cast<size_t>(Hkv) * (C > 0 ? C : 0) + 63) & ~static_cast<size_t>(63);
-    if (C > 0) {
-        ScorePlan plan;
-        if (!make_score_plan(L, R, Hkv, d, c, ctas, smem_budget(*ctx), false, &plan)) return 0;
-        floats += score_scratch_floats(plan, Hkv, R);
-    }
-    const size_t half = (kHeaderBytes + floats * sizeof(float) + 255) & ~static_cast<size_t>(255);
-    return 2 * half;
+    return chunkkv_lane_bytes(L, Hq, Hkv, d, w, c, max_ctas);
 }
 
 int chunkkv_pipe_open(void* scratch, size_t bytes, int max_ctas, void** pipe_out) {
@@ -615,27 +601,22 @@ int chunkkv_pipe_open(void* scratch, size_t bytes, int max_ctas, void** pipe_out
     *pipe_out = nullptr;
     if ((reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return CHUNKKV_EINVAL_ALIGN;
     if (max_ctas < 0) return CHUNKKV_EINVAL_SHAPE;
-    const size_t half = (bytes / 2) & ~static_cast<size_t>(255);
-    if (half < kHeaderBytes) return CHUNKKV_ENOWORKSPACE;
+    if (bytes < kHeaderBytes) return CHUNKKV_ENOWORKSPACE;
     Pipe* p = new Pipe();
     cudaError_t e = cudaGetDevice(&p->device);
     if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&p->side, cudaStreamNonBlocking);
-    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
-        e = cudaEventCreateWithFlags(&p->scored[i], cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->posted[i], cudaEventDisableTiming);
-        if (e == cudaSuccess) e = cudaMemset(static_cast<char*>(scratch) + i * half, 0, kHeaderBytes);
-    }
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->scored, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&p->posted, cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaMemset(scratch, 0, kHeaderBytes);
     if (e != cudaSuccess) {
-        for (int i = 0; i < 2; ++i) {
-            if (p->scored[i]) cudaEventDestroy(p->scored[i]);
-            if (p->posted[i]) cudaEventDestroy(p->posted[i]);
-        }
+        if (p->scored) cudaEventDestroy(p->scored);
+        if (p->posted) cudaEventDestroy(p->posted);
         if (p->side) cudaStreamDestroy(p->side);
         delete p;
         return cuda_fail(e);
     }
     p->scratch = static_cast<char*>(scratch);
-    p->half_bytes = half;
+    p->bytes = bytes;
     p->max_ctas = max_ctas;
     *pipe_out = p;
     return CHUNKKV_OK;
@@ -646,76 +627,28 @@ int chunkkv_pipe_layer(void* pipe, const void* q_obs, const void* K, const void*
                        void* stream) {
     if (pipe == nullptr) return CHUNKKV_EINVAL_NULL;
     Pipe* p = static_cast<Pipe*>(pipe);
-    int st = check_sizes(L, w, c, budget);
+    if (q_obs == nullptr) return CHUNKKV_EINVAL_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // scoring, chunk scores and selection on the caller's stream (the lane's layer kernel without
+    // its gather phase), ...
+    int st = compress_impl(q_obs, K, V, L, Hq, Hkv, d, w, c, budget, nullptr, out_K, out_V, out_idx, p->scratch,
+                           p->bytes, p->max_ctas, stream, /*rows_on=*/&p->side);
     if (st != CHUNKKV_OK) return st;
-    st = check_heads(L, Hq, Hkv, d, w);
-    if (st != CHUNKKV_OK) return st;
-    if (q_obs == nullptr || K == nullptr || V == nullptr || out_K == nullptr || out_V == nullptr ||
-        out_idx == nullptr)
-        return CHUNKKV_EINVAL_NULL;
-    if (!aligned16(q_obs) || !aligned16(K) || !aligned16(V) || !aligned16(out_K) || !aligned16(out_V) ||
-        !aligned16(out_idx))
-        return CHUNKKV_EINVAL_ALIGN;
-    const int C = chunkkv_num_chunks(L, w, c);
-    const int k = chunkkv_num_kept_chunks(L, w, c, budget);
-    const int n_max = chunkkv_out_len(L, w, c, budget);
-    if (n_max < 0) return n_max;
     std::lock_guard<std::mutex> lk(g_mu);
+    // ... the row gather on the pipe's stream, after it
+    cudaError_t e = cudaEventRecord(p->scored, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaStreamWaitEvent(p->side, p->scored, 0);
+    if (e != cudaSuccess) return cuda_fail(e);
     DeviceCtx* ctx;
     st = get_ctx(&ctx);
     if (st != CHUNKKV_OK) return st;
-    const int ctas = (p->max_ctas > 0 && p->max_ctas < ctx->num_sms) ? p->max_ctas : ctx->num_sms;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int half = p->next;
-    char* base = p->scratch + half * p->half_bytes;
-    float* payload = reinterpret_cast<float*>(base + kHeaderBytes);
-    float* chunk_scores = nullptr;
-    cudaError_t e;
-    ScorePlan plan;
-    ScoreArgs a;
-    const bool scoring = C > 0 && k > 0;
-    if (scoring) {
-        const int R = w * (Hq / Hkv);
-        const size_t cs_floats = (static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63);
-        if (!make_score_plan(L, R, Hkv, d, c, ctas, smem_budget(*ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
-        if (kHeaderBytes + (cs_floats + score_scratch_floats(plan, Hkv, R)) * sizeof(float) > p->half_bytes)
-            return CHUNKKV_ENOWORKSPACE;
-        a.L = L; a.P = L - w; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
-        a.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
-        score_scratch_layout(plan, Hkv, R, payload + cs_floats, &a);
-        a.status = reinterpret_cast<int*>(base);
-        CUtensorMap tm_q, tm_k;
-        st = encode_bf16_3d(&tm_q, q_obs, d, R, Hkv, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
-        if (st != CHUNKKV_OK) return st;
-        st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < plan.n_tile ? L : plan.n_tile,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
-        if (st != CHUNKKV_OK) return st;
-        // the half is free once the post-processing of the layer that used it last has finished
-        if (p->pending[half]) {
-            e = cudaStreamWaitEvent(s, p->posted[half], 0);
-            if (e != cudaSuccess) return cuda_fail(e);
-        }
-        e = launch_score(plan, tm_q, tm_k, a, s);
-        if (e != cudaSuccess) return cuda_fail(e);
-        chunk_scores = payload;
-    }
-    e = cudaEventRecord(p->scored[half], s);
-    if (e != cudaSuccess) return cuda_fail(e);
-    e = cudaStreamWaitEvent(p->side, p->scored[half], 0);
-    if (e != cudaSuccess) return cuda_fail(e);
-    if (scoring) {
-        e = launch_finalize(plan, a, C, chunk_scores, ctx->num_sms, p->side);
-        if (e != cudaSuccess) return cuda_fail(e);
-    }
-    e = launch_select(chunk_scores, L, Hkv, w, c, C, k, n_max, out_idx, p->side);
-    if (e != cudaSuccess) return cuda_fail(e);
+    const int n_max = chunkkv_out_len(L, w, c, budget);
     e = launch_gather_shared_sms(K, V, out_idx, L, Hkv, d, n_max, out_K, out_V, ctx->num_sms, p->side);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = cudaEventRecord(p->posted[half], p->side);
+    e = cudaEventRecord(p->posted, p->side);
     if (e != cudaSuccess) return cuda_fail(e);
-    p->pending[half] = true;
-    p->last = half;
-    p->next = half ^ 1;
+    p->pending = true;
     return CHUNKKV_OK;
 }
 
@@ -723,32 +656,18 @@ int chunkkv_pipe_join(void* pipe, void* stream) {
     if (pipe == nullptr) return CHUNKKV_EINVAL_NULL;
     Pipe* p = static_cast<Pipe*>(pipe);
     std::lock_guard<std::mutex> lk(g_mu);
-    if (p->last >= 0) {
-        cudaError_t e = cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), p->posted[p->last], 0);
+    if (p->pending) {
+        cudaError_t e = cudaStreamWaitEvent(static_cast<cudaStream_t>(stream), p->posted, 0);
         if (e != cudaSuccess) return cuda_fail(e);
     }
-    p->pending[0] = p->pending[1] = false;
-    p->last = -1;
+    p->pending = false;
     return CHUNKKV_OK;
 }
 
 int chunkkv_pipe_status(void* pipe, void* stream) {
     int st = chunkkv_pipe_join(pipe, stream);
     if (st != CHUNKKV_OK) return st;
-    Pipe* p = static_cast<Pipe*>(pipe);
-    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
-    if (e != cudaSuccess) return cuda_fail(e);
-    int bad = 0;
-    for (int i = 0; i < 2; ++i) {
-        int flag = 0;
-        e = cudaMemcpy(&flag, p->scratch + i * p->half_bytes, sizeof(int), cudaMemcpyDeviceToHost);
-        if (e != cudaSuccess) return cuda_fail(e);
-        if (flag != 0) {
-            cudaMemset(p->scratch + i * p->half_bytes, 0, kHeaderBytes);
-            bad = 1;
-        }
-    }
-    return bad ? CHUNKKV_EDEVICE : CHUNKKV_OK;
+    return chunkkv_lane_status(static_cast<Pipe*>(pipe)->scratch, stream);
 }
 
 int chunkkv_pipe_close(void* pipe) {
@@ -756,10 +675,8 @@ int chunkkv_pipe_close(void* pipe) {
     Pipe* p = static_cast<Pipe*>(pipe);
     std::lock_guard<std::mutex> lk(g_mu);
     cudaError_t e = cudaStreamSynchronize(p->side);
-    for (int i = 0; i < 2; ++i) {
-        cudaEventDestroy(p->scored[i]);
-        cudaEventDestroy(p->posted[i]);
-    }
+    cudaEventDestroy(p->scored);
+    cudaEventDestroy(p->posted);
     cudaStreamDestroy(p->side);
     delete p;
     if (e != cudaSuccess) return cuda_fail(e);
