@@ -40,9 +40,9 @@ NSETS = 4
 LAYERS_PER_STEP = 32
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one cfg2 layer in an 18-CTA lane: layer kernel
-# 71.4 MB + row gather 13.5 MB (ncu capture of both launches)
-TRAFFIC_BYTES_PER_LAYER = 84.9e6
+# dram__bytes_read.sum + dram__bytes_write.sum of one cfg2 layer through a lane, from ncu captures
+# of both launches (layer kernel + row gather): 8 CTAs 69.5 + 13.5 MB, 18 CTAs 71.4 + 13.5 MB
+TRAFFIC_BYTES_PER_LAYER = {8: 83.1e6, 18: 84.9e6}
 
 
 def parse_args():
@@ -54,7 +54,8 @@ def parse_args():
     ap.add_argument("--config", type=int, default=2, help="workload table entry (2 = headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--lanes", type=int, default=8, help="layers in flight (each on 1/lanes of the SMs)")
+    ap.add_argument("--lanes", type=int, default=18, help="layers in flight (each on 1/lanes of the SMs)")
+    ap.add_argument("--lane-ctas", type=int, default=0, help="CTA budget of a lane (0: SMs // lanes)")
     ap.add_argument("--mode", choices=("pipe", "lane"), default="pipe",
                     help="pipe: chunkkv_pipe_layer (layer kernels back to back, row gathers on side streams); "
                          "lane: chunkkv_compress_layer_lane (one layer at a time per lane)")
@@ -233,13 +234,14 @@ def run_ours(args, wl):
     # ---- lanes: S layers in flight, each on its own stream with 1/S of the SMs and its own scratch
     n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
     S = max(1, args.lanes)
+    lane_ctas = args.lane_ctas if args.lane_ctas > 0 else n_sm // S
     stream = torch.cuda.Stream(device=dev)
     lanes = []
     piped = args.mode == "pipe" and S > 1
     if S > 1:
         for li in range(S):
             cls = ck.Pipe if piped else ck.Lane
-            ln = cls(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=n_sm // S, device=dev,
+            ln = cls(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=lane_ctas, device=dev,
                      stream=stream if li == 0 else None)
             lanes.append(ln)
     lane_streams = [ln.stream for ln in lanes] if lanes else [stream]
@@ -369,7 +371,7 @@ def run_ours(args, wl):
     peak, peak_src = measured_hbm_peak()
     score_us = per_kernel["score"]["avg_us"] or float("nan")
     fused = per_kernel["gather"]["launches"] == 0          # the whole layer ran as one kernel
-    split = S > 1 and 2 * (n_sm // S) <= n_sm               # a lane's layer = layer kernel + row-gather launch
+    split = S > 1 and 2 * lane_ctas <= n_sm               # a lane's layer = layer kernel + row-gather launch
     launches_per_layer = 2 if (piped or split) else 1           # layer kernel + row gather
     # The timed region holds nothing but the launches of LAYERS_PER_STEP layers per step, S of them
     # in flight at a time on disjoint SM sets, so the duration a launch accounts for is the region
@@ -378,15 +380,15 @@ def run_ours(args, wl):
     if piped:
         kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) on the pipe's main stream + "
                        "gather_kernel (row gather in CTAs spread over all SMs) on its side stream: the two launches of a "
-                       "layer in a pipe" % (n_sm // S))
+                       "layer in a pipe" % lane_ctas)
     elif split:
         kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) + gather_kernel "
-                       "(row gather in CTAs spread over all SMs): the two launches of a layer in a lane" % (n_sm // S))
+                       "(row gather in CTAs spread over all SMs): the two launches of a layer in a lane" % lane_ctas)
     else:
         kernel_name = "score_kernel<FUSED> (score + chunk sums + finalize + select + gather in one launch)"
     roofline = {"kernel": kernel_name, "bound": "hbm", "achieved": achieved, "peak": peak,
                 "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": TRAFFIC_BYTES_PER_LAYER if ((split or piped) and args.config == 2 and S == 8) else None,
+                "traffic": TRAFFIC_BYTES_PER_LAYER.get(lane_ctas) if ((split or piped) and args.config == 2) else None,
                 "algorithmic_bytes_per_launch": nbytes["layer"], "avg_launch_us": ms_layer * 1e3,
                 "launches_in_flight": S,
                 "isolated_launch_us": score_us,
@@ -461,7 +463,7 @@ def run_ours(args, wl):
                        "lanes": S,
                        "mode": args.mode if S > 1 else "single",
                        "launch": f"one CUDA graph per step: 32 layer calls ({'chunkkv_pipe_layer' if piped else 'chunkkv_compress_layer_lane'}), {S} in flight "
-                                 f"on {S} streams with {n_sm // S} CTAs each" if S > 1 else
+                                 f"on {S} streams with {lane_ctas} CTAs each" if S > 1 else
                                  "one CUDA graph per step (32 chunkkv_compress_layer calls captured)",
                        "l2": f"layers cycle over {NSETS} distinct K/V sets of "
                              f"{2 * wl.Hkv * wl.L * wl.d * 2 / 1e6:.0f} MB each (> L2)"},
