@@ -160,6 +160,18 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
                            void* out_K, void* out_V, int32_t* out_idx, void* stream);
 
 /*
+ * Index similarity between two layers (the paper's section on layer-wise index reuse reports the
+ * Jaccard similarity of the preserved indices of adjacent layers; Algorithm 2 shares indices
+ * because it is high). Per KV head h: out_ratio[h] = |A n B| / |A u B| (1 when both are empty),
+ * A and B the valid (non-negative) entries of row h of idx_a [Hkv, n_a] and idx_b [Hkv, n_b].
+ * Rows must be as chunkkv_select / chunkkv_compress_layer write them: ascending, no repeats,
+ * -1 padding last. out_counts [Hkv, 3] int32 (optional, may be NULL) receives |A n B|, |A|, |B|.
+ * All pointers are device memory; the call is queued on `stream`.
+ */
+CHUNKKV_API int chunkkv_jaccard(const int32_t* idx_a, const int32_t* idx_b, int Hkv, int n_a, int n_b,
+                                float* out_ratio, int32_t* out_counts, void* stream);
+
+/*
  * Lanes: several layers in flight at once (Algorithm 2 visits the layers one after another, and
  * they are independent). A lane is caller-owned scratch plus a CTA budget. Layers submitted to
  * different lanes on different streams run concurrently, each on its share of the SMs, so the

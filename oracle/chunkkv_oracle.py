@@ -214,23 +214,30 @@ def compress_layer(q_obs: np.ndarray, K: np.ndarray, V: np.ndarray, Hq: int, Hkv
 
 # --------------------------------------------------------------------------- many layers
 def compress_model(layers: Sequence[Tuple[np.ndarray, np.ndarray, np.ndarray]], Hq: int,
-                   Hkv: int, w: int, c: int, budget: int, n_reuse: int = 1,
+                   Hkv: int, w: int, c, budget: int, n_reuse: int = 1,
                    ) -> List[Dict[str, np.ndarray]]:
     """Layer-wise index reuse (Algorithm 2).
 
     Layer l computes its own indices iff l mod n_reuse == 0; otherwise it takes the
     indices stored for layer floor(l / n_reuse) * n_reuse. Every layer gathers.
     ``layers`` is a sequence of (q_obs, K, V).
+
+    ``c`` is one chunk size for all layers or one per layer (the hybrid of the paper's section on
+    chunk- and token-level layers: chunks in the first layers, c = 1 in the rest). A layer that
+    reuses indices has no chunk size of its own: it takes its source layer's.
     """
+    cs = [int(c)] * len(layers) if np.isscalar(c) else [int(v) for v in c]
+    if len(cs) != len(layers):
+        raise ValueError("one chunk size per layer expected")
     store: Dict[int, np.ndarray] = {}
     out = []
     for l, (q_obs, K, V) in enumerate(layers):
         if l % n_reuse == 0:
-            res = compress_layer(q_obs, K, V, Hq, Hkv, w, c, budget)
+            res = compress_layer(q_obs, K, V, Hq, Hkv, w, cs[l], budget)
             store[l] = res["idx"]
         else:
-            res = compress_layer(q_obs, K, V, Hq, Hkv, w, c, budget,
-                                 reuse_idx=store[(l // n_reuse) * n_reuse])
+            src = (l // n_reuse) * n_reuse
+            res = compress_layer(q_obs, K, V, Hq, Hkv, w, cs[src], budget, reuse_idx=store[src])
         out.append(res)
     return out
 

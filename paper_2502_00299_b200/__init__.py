@@ -8,7 +8,7 @@ so that the build module itself can be imported before the library exists.
 """
 _EXPORTS = (
     "ChunkKVError", "LIB_PATH", "Lane", "Pipe", "compress_layer", "compress_layer_host", "compress_model",
-    "device_status", "gather", "lib", "num_chunks", "num_kept_chunks", "out_len", "profile_enable",
+    "device_status", "gather", "jaccard", "lib", "num_chunks", "num_kept_chunks", "out_len", "profile_enable",
     "profile_read", "score", "select", "set_workspace", "strerror", "workspace_bytes",
 )
 __all__ = list(_EXPORTS)

@@ -68,6 +68,8 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_pipe_status.argtypes = [vp, vp]
     L.chunkkv_pipe_close.restype = i32
     L.chunkkv_pipe_close.argtypes = [vp]
+    L.chunkkv_jaccard.restype = i32
+    L.chunkkv_jaccard.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     L.chunkkv_score_noalloc.restype = i32
     L.chunkkv_score_noalloc.argtypes = [vp, vp] + [i32] * 6 + [vp, vp]
     L.chunkkv_profile_enable.restype = i32
@@ -209,6 +211,21 @@ def compress_layer(q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tens
     return out_K, out_V, out_idx
 
 
+def jaccard(idx_a: torch.Tensor, idx_b: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,
+            ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """chunkkv_jaccard: per-head similarity [Hkv] f32 and counts [Hkv, 3] int32 (|A n B|, |A|, |B|)."""
+    idx_a = _dev(idx_a, torch.int32, "idx_a")
+    idx_b = _dev(idx_b, torch.int32, "idx_b")
+    Hkv = idx_a.shape[0]
+    if idx_b.shape[0] != Hkv:
+        raise ValueError("idx_a and idx_b must have the same number of heads")
+    ratio = torch.empty(Hkv, dtype=torch.float32, device=idx_a.device)
+    counts = torch.empty((Hkv, 3), dtype=torch.int32, device=idx_a.device)
+    _check(lib.chunkkv_jaccard(idx_a.data_ptr(), idx_b.data_ptr(), Hkv, idx_a.shape[1], idx_b.shape[1],
+                               ratio.data_ptr(), counts.data_ptr(), _stream(stream)), "chunkkv_jaccard")
+    return ratio, counts
+
+
 class Lane:
     """Caller-owned scratch plus a CTA budget: layers submitted to different lanes on different
     streams run concurrently (see chunkkv.h). The budgets of lanes used at the same time must add
@@ -321,19 +338,24 @@ def compress_layer_host(host_q: torch.Tensor, host_K: torch.Tensor, host_V: torc
 
 
 def compress_model(layers: Sequence[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]], Hq: int, w: int,
-                   c: int, budget: int, n_reuse: int = 1,
+                   c, budget: int, n_reuse: int = 1,
                    stream: Optional[torch.cuda.Stream] = None,
                    ) -> List[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]]:
     """Layer-wise index reuse: layer l computes indices iff l % n_reuse == 0, otherwise it
     gathers with the indices of layer (l // n_reuse) * n_reuse. Only the call sequence lives
-    here; every layer is one chunkkv_compress_layer call."""
+    here; every layer is one chunkkv_compress_layer call. ``c`` is one chunk size or one per
+    layer (chunk-level layers followed by token-level ones, c = 1); a layer that reuses indices
+    takes its source layer's chunk size."""
+    cs = [int(c)] * len(layers) if isinstance(c, int) else [int(v) for v in c]
+    if len(cs) != len(layers):
+        raise ValueError("one chunk size per layer expected")
     outs: List[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = []
     for l, (q, K, V) in enumerate(layers):
         if l % n_reuse == 0:
-            outs.append(compress_layer(q, K, V, Hq, w, c, budget, stream=stream))
+            outs.append(compress_layer(q, K, V, Hq, w, cs[l], budget, stream=stream))
         else:
-            src = outs[(l // n_reuse) * n_reuse][2]
-            outs.append(compress_layer(None, K, V, Hq, w, c, budget, reuse_idx=src, stream=stream))
+            s_l = (l // n_reuse) * n_reuse
+            outs.append(compress_layer(None, K, V, Hq, w, cs[s_l], budget, reuse_idx=outs[s_l][2], stream=stream))
     return outs
 
 

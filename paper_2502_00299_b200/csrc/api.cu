@@ -536,6 +536,15 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
     return CHUNKKV_OK;
 }
 
+int chunkkv_jaccard(const int32_t* idx_a, const int32_t* idx_b, int Hkv, int n_a, int n_b,
+                    float* out_ratio, int32_t* out_counts, void* stream) {
+    if (Hkv < 1 || Hkv > 65535 || n_a < 0 || n_b < 0) return CHUNKKV_EINVAL_SHAPE;
+    if (idx_a == nullptr || idx_b == nullptr || out_ratio == nullptr) return CHUNKKV_EINVAL_NULL;
+    cudaError_t e = launch_jaccard(idx_a, idx_b, Hkv, n_a, n_b, out_ratio, out_counts, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
 int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
                            int d, int w, int c, int budget, const int32_t* reuse_idx,
                            void* out_K, void* out_V, int32_t* out_idx, void* stream) {

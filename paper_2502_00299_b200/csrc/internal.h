@@ -72,6 +72,10 @@ cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int
 cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
                           int n_max, void* out_K, void* out_V, int32_t* idx_copy_or_null,
                           int num_sms, cudaStream_t stream);
+// Jaccard similarity of two kept-index matrices, one CTA per head (diagnostics.cu).
+cudaError_t launch_jaccard(const int32_t* idx_a, const int32_t* idx_b, int Hkv, int n_a, int n_b,
+                           float* out_ratio, int32_t* out_counts_or_null, cudaStream_t stream);
+
 // The gather in small CTAs that can share SMs with resident layer-kernel CTAs (lanes).
 cudaError_t launch_gather_shared_sms(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
                                      int n_max, void* out_K, void* out_V, int num_sms, cudaStream_t stream);

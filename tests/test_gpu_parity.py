@@ -389,3 +389,53 @@ def test_random_shapes_through_all_three_layer_calls(ck, case):
         _check_layer(x, wl, bits_of(pK), bits_of(pV), pidx.cpu().numpy())
     pipe.close()
 
+
+def test_hybrid_model_chunk_layers_then_token_layers(ck):
+    # chunk-level selection in the first layers, token-level (c = 1) in the rest, with and without
+    # index reuse; every layer against the oracle's own run of the same schedule
+    wl = scaled(CONFIGS[3], L=2500, budget=260, n_layers=6)
+    layers = list(iter_layers(wl))
+    cs = [10, 10, 10, 1, 1, 1]
+    dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in layers]
+    for n_reuse in (1, 2):
+        outs = ck.compress_model(dev, wl.Hq, wl.w, cs, wl.budget, n_reuse=n_reuse)
+        _status_ok(ck)
+        ref = ora.compress_model([(x.q_obs, x.K, x.V) for x in layers], wl.Hq, wl.Hkv, wl.w, cs, wl.budget,
+                                 n_reuse=n_reuse)
+        for l, (x, (oK, oV, idx)) in enumerate(zip(layers, outs)):
+            idx_np = idx.cpu().numpy()
+            assert idx_np.shape == ref[l]["idx"].shape
+            if l % n_reuse == 0:
+                t = ora.token_scores(x.q_obs, x.K, wl.Hq, wl.Hkv, wl.w)
+                assert_selection_matches(idx_np, ora.chunk_scores(t, cs[l]), wl.L, wl.w, cs[l], wl.budget)
+            else:
+                assert np.array_equal(idx_np, outs[(l // n_reuse) * n_reuse][2].cpu().numpy())
+            assert_gather_exact(bits_of(oK), bits_of(oV), idx_np, x.K, x.V)
+
+
+def test_jaccard_of_kept_indices_matches_oracle(ck):
+    # adjacent correlated layers, chunk- and token-level, plus rows with padding and an empty row
+    wl = scaled(CONFIGS[3], L=3000, budget=300, n_layers=3)
+    layers = list(iter_layers(wl))
+    idx = []
+    for x in layers:
+        _, _, i = ck.compress_layer(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V), wl.Hq, wl.w, wl.c, wl.budget)
+        idx.append(i)
+    pairs = [(idx[0], idx[1]), (idx[1], idx[2]), (idx[0], idx[0])]
+    a = torch.full((wl.Hkv, 7), -1, dtype=torch.int32, device="cuda")
+    b = torch.full((wl.Hkv, 5), -1, dtype=torch.int32, device="cuda")
+    a[0, :4] = torch.tensor([1, 5, 9, 11], dtype=torch.int32)
+    b[0, :3] = torch.tensor([5, 6, 11], dtype=torch.int32)
+    b[1, :2] = torch.tensor([0, 2], dtype=torch.int32)
+    pairs.append((a, b))
+    for ia, ib in pairs:
+        ratio, counts = ck.jaccard(ia, ib)
+        ra, rb = ia.cpu().numpy(), ib.cpu().numpy()
+        for h in range(wl.Hkv):
+            sa, sb = set(ra[h][ra[h] >= 0].tolist()), set(rb[h][rb[h] >= 0].tolist())
+            assert counts[h].tolist() == [len(sa & sb), len(sa), len(sb)]
+            assert abs(float(ratio[h]) - ora.jaccard(ra[h], rb[h])) < 1e-6
+    r, c3 = ck.jaccard(a, b)
+    assert c3[0].tolist() == [2, 4, 3] and abs(float(r[0]) - 2 / 5) < 1e-6     # worked by hand
+    assert float(r[2]) == 1.0                                                  # two empty rows
+

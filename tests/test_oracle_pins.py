@@ -12,7 +12,7 @@ import pytest
 import torch
 
 from oracle import chunkkv_oracle as ora
-from workloads import f32_to_bf16_bits, bf16_bits_to_f32
+from workloads import CONFIGS, bf16_bits_to_f32, f32_to_bf16_bits, make_layer, scaled
 
 
 def _rand_bits(rng, shape, scale=1.0):
@@ -269,3 +269,26 @@ def test_layerwise_reuse_follows_algorithm_2():
 def test_jaccard():
     assert ora.jaccard(np.array([0, 1, 2, -1]), np.array([1, 2, 3, -1])) == pytest.approx(2 / 4)
     assert ora.jaccard(np.array([5]), np.array([5])) == 1.0
+
+
+def test_per_layer_chunk_sizes_equal_separate_layer_calls():
+    # the hybrid schedule is nothing but per-layer calls with that layer's chunk size
+    wl = scaled(CONFIGS[1], L=400, budget=60)
+    xs = [make_layer(wl, layer=i) for i in range(4)]
+    cs = [10, 10, 1, 1]
+    out = ora.compress_model([(x.q_obs, x.K, x.V) for x in xs], wl.Hq, wl.Hkv, wl.w, cs, wl.budget, n_reuse=1)
+    for x, c, o in zip(xs, cs, out):
+        one = ora.compress_layer(x.q_obs, x.K, x.V, wl.Hq, wl.Hkv, wl.w, c, wl.budget)
+        assert np.array_equal(o["idx"], one["idx"])
+    # with reuse depth 2, layer 3 takes layer 2's token-level indices and layer 1 takes layer 0's
+    out2 = ora.compress_model([(x.q_obs, x.K, x.V) for x in xs], wl.Hq, wl.Hkv, wl.w, cs, wl.budget, n_reuse=2)
+    assert np.array_equal(out2[1]["idx"], out2[0]["idx"]) and np.array_equal(out2[3]["idx"], out2[2]["idx"])
+    assert out2[2]["idx"].shape[1] == ora.out_len(wl.L, wl.w, 1, wl.budget)
+
+
+def test_jaccard_hand_worked():
+    assert ora.jaccard(np.array([1, 5, 9, 11, -1]), np.array([5, 6, 11])) == 2 / 5
+    assert ora.jaccard(np.array([-1, -1]), np.array([-1])) == 1.0
+    assert ora.jaccard(np.array([3, 4]), np.array([3, 4, -1])) == 1.0
+    assert ora.jaccard(np.array([3, 4]), np.array([5, 6])) == 0.0
+
