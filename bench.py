@@ -416,6 +416,38 @@ def run_ours(args, wl):
                         "frac_of_measured_peak": nbytes["gather"] / (ms_reuse * 1e-3) / 1e9 / peak},
     }
 
+    # ---- variants next to the hot path: token-level selection (c = 1) and the index-similarity diagnostic
+    def time_calls(fn, n=30):
+        for _ in range(3):
+            fn()
+        return timed(lambda: [fn() for _ in range(n)], 1) / n * 1e3      # us per call
+
+    n_max1 = ck.out_len(wl.L, wl.w, 1, wl.budget)
+    o1 = [torch.empty((wl.Hkv, n_max1, wl.d), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    o1.append(torch.empty((wl.Hkv, n_max1), dtype=torch.int32, device=dev))
+    calls = [0]
+
+    def token_level_layer():
+        q, K, V = sets[calls[0] % NSETS][0]
+        calls[0] += 1
+        st = lib.chunkkv_compress_layer(q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, 1,
+                                        wl.budget, None, o1[0].data_ptr(), o1[1].data_ptr(), o1[2].data_ptr(),
+                                        stream.cuda_stream)
+        if st != 0:
+            raise ck.ChunkKVError(st, "chunkkv_compress_layer (c = 1)")
+
+    with torch.cuda.stream(stream):
+        us_token = time_calls(token_level_layer)
+        ia, ib = lane_outs[0][2], lane_outs[1][2]
+        us_jac = time_calls(lambda: ck.jaccard(ia, ib, stream=stream))
+    bytes1 = layer_bytes(wl, n_max1)["layer"]
+    extra_roof["token_level_layer"] = {"c": 1, "algorithmic_bytes": bytes1, "us": us_token,
+                                       "GB/s": bytes1 / (us_token * 1e-6) / 1e9,
+                                       "frac_of_measured_peak": bytes1 / (us_token * 1e-6) / 1e9 / peak,
+                                       "note": "chunkkv_compress_layer with c = 1, one layer at a time on all SMs"}
+    extra_roof["jaccard"] = {"us": us_jac, "note": "chunkkv_jaccard on the kept indices of two layers "
+                                                   f"([{wl.Hkv}, {n_max}] int32 each; latency-bound, includes the binding's two small allocations)"}
+
     # ---- end to end: pinned host buffers in, host buffers out, copies inside the timed region
     e2e = None
     if not args.no_e2e:
