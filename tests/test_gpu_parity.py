@@ -439,3 +439,17 @@ def test_jaccard_of_kept_indices_matches_oracle(ck):
     assert c3[0].tolist() == [2, 4, 3] and abs(float(r[0]) - 2 / 5) < 1e-6     # worked by hand
     assert float(r[2]) == 1.0                                                  # two empty rows
 
+
+@pytest.mark.parametrize("cfg", [4, 5])
+def test_compress_layer_full_size_long_contexts(ck, cfg):
+    # the 128K-token workload (w = 64, c = 20) and the longest sequence of the batched workload
+    # (64K tokens, 64 query heads: two query tiles per KV head), whole layer against the oracle
+    wl = CONFIGS[cfg]
+    x = make_layer(wl)
+    oK, oV, idx = _run_layer(ck, x, wl)
+    _check_layer(x, wl, oK, oV, idx)
+    lane = ck.Lane(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=8)
+    lK, lV, lidx = lane.compress_layer(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V), wl.Hq, wl.w, wl.c, wl.budget)
+    assert lane.status() == 0
+    assert np.array_equal(lidx.cpu().numpy(), idx) and np.array_equal(bits_of(lK), oK)
+
