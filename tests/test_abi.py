@@ -58,6 +58,16 @@ def test_invalid_sizes_are_rejected_on_the_host(ck):
                                       None, None) == -2
     assert lib.chunkkv_compress_layer(None, None, None, 1024, 8, 2, 128, 16, 10, 256, None, None, None,
                                       None, None) == -1
+    # the largest supported head set is Hkv * L < 2^23 keys; one key more is refused
+    assert lib.chunkkv_compress_layer(None, None, None, (1 << 20) - 1, 8, 8, 128, 16, 10, 256, None, None, None,
+                                      None, None) == -1        # sizes accepted, then the NULL pointers are seen
+    assert lib.chunkkv_compress_layer(None, None, None, 1 << 20, 8, 8, 128, 16, 10, 256, None, None, None,
+                                      None, None) == -2
+    # the new entry points check their arguments the same way
+    assert lib.chunkkv_jaccard(None, None, 2, 10, 10, None, None, None) == -1
+    assert lib.chunkkv_jaccard(None, None, 0, 10, 10, None, None, None) == -2
+    assert lib.chunkkv_pipe_layer(None, None, None, None, 1024, 8, 2, 128, 16, 10, 256, None, None, None, None) == -1
+    assert lib.chunkkv_pipe_join(None, None) == -1 and lib.chunkkv_pipe_close(None) == -1
     for code in range(-6, 1):
         assert ck.strerror(code) and ck.strerror(code) != "unknown status"
     assert ck.strerror(-99) == "unknown status"
