@@ -453,3 +453,15 @@ def test_compress_layer_full_size_long_contexts(ck, cfg):
     assert lane.status() == 0
     assert np.array_equal(lidx.cpu().numpy(), idx) and np.array_equal(bits_of(lK), oK)
 
+
+def test_compress_layer_at_the_largest_supported_length(ck):
+    # Hkv * L just under 2^23 keys (the library's limit): 8.4 M tokens of one head
+    import psutil
+    if psutil.virtual_memory().available < 48 * 2**30:
+        pytest.skip("needs about 20 GB of host memory for the inputs and the fp64 oracle")
+    L = (1 << 23) - 64
+    wl = scaled(CONFIGS[1], Hq=2, Hkv=1, d=64, L=L, w=8, c=10, budget=5000, seed=11, planted_count=0)
+    x = make_layer(wl)
+    oK, oV, idx = _run_layer(ck, x, wl)
+    _check_layer(x, wl, oK, oV, idx)
+
