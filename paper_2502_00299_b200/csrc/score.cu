@@ -387,8 +387,10 @@ __device__ __forceinline__ void contract_chunks_t(const ScoreArgs& a, const FinG
 // exp2(m_panel - m) / l in registers and reduces over the rows with shuffles. Nothing is staged in
 // shared memory and no block-wide synchronisation is needed. Fixed order: deterministic.
 // gm / ginv: row maxima and reciprocal sums, 16-byte aligned (shared or global memory).
-constexpr int kSlotBatch = 6;
-template <int RV, int PP>   // RV float4 row groups per lane (1: R <= 128, 2: R <= 256); PP panels in flight per warp
+constexpr int kSlotBatch = 6;        // chunk slots in flight per panel (a 60-key panel of 10-key chunks has six)
+constexpr int kSlotBatchWide = 16;   // for panels with many slots (token-level: one slot per key)
+// RV float4 row groups per lane (1: R <= 128, 2: R <= 256); PP panels in flight per warp; SB slots per panel in flight
+template <int RV, int PP, int SB = kSlotBatch>
 __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, const FinGeom& g, int h, int p_lo,
                                                         int p_hi, const float* gm, const float* ginv,
                                                         float* __restrict__ out) {
@@ -424,13 +426,13 @@ __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, cons
         }
         if (max_slots == 0) break;                                 // panels past the prefix hold no chunk
         float4 f[PP][RV];
-        for (int s0 = 0; s0 < max_slots; s0 += kSlotBatch) {
-            float4 pv[PP][kSlotBatch][RV];
+        for (int s0 = 0; s0 < max_slots; s0 += SB) {
+            float4 pv[PP][SB][RV];
 #pragma unroll
             for (int q = 0; q < PP; ++q) {
                 const int ch_base = (pb + q * nwarps) * g.spp;
 #pragma unroll
-                for (int u = 0; u < kSlotBatch; ++u) {
+                for (int u = 0; u < SB; ++u) {
                     const bool slot = s0 + u < n_slots[q];
 #pragma unroll
                     for (int it = 0; it < RV; ++it)
@@ -450,11 +452,11 @@ __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, cons
                         f[q][it].w = ex2_approx(pm[q][it].w - m4[it].w) * li4[it].w;
                     }
             }
-            float acc[PP][kSlotBatch];
+            float acc[PP][SB];
 #pragma unroll
             for (int q = 0; q < PP; ++q)
 #pragma unroll
-                for (int u = 0; u < kSlotBatch; ++u) {
+                for (int u = 0; u < SB; ++u) {
                     float v = 0.f;
 #pragma unroll
                     for (int it = 0; it < RV; ++it) {
@@ -470,13 +472,13 @@ __device__ __forceinline__ void contract_panels_aligned(const ScoreArgs& a, cons
 #pragma unroll
                 for (int q = 0; q < PP; ++q)
 #pragma unroll
-                    for (int u = 0; u < kSlotBatch; ++u) acc[q][u] += __shfl_xor_sync(0xffffffffu, acc[q][u], off);
+                    for (int u = 0; u < SB; ++u) acc[q][u] += __shfl_xor_sync(0xffffffffu, acc[q][u], off);
             }
             if (lane == 0) {
 #pragma unroll
                 for (int q = 0; q < PP; ++q)
 #pragma unroll
-                    for (int u = 0; u < kSlotBatch; ++u)
+                    for (int u = 0; u < SB; ++u)
                         if (s0 + u < n_slots[q]) out_h[(pb + q * nwarps) * g.spp + s0 + u] = acc[q][u];
             }
         }
@@ -873,7 +875,9 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             block_row_stats(a, fg, head, gm, ginv, rs);
             if (direct) {   // chunks never straddle panels: straight from the partial sums, no staging
                 const int p_lo = (t - head * g.n_tiles) * PPTT, p_hi = (seg_end - head * g.n_tiles) * PPTT;
-                if (a.R <= 128)
+                if (C_STATIC == 1)
+                    contract_panels_aligned<1, 1, kSlotBatchWide>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                else if (a.R <= 128)
                     contract_panels_aligned<1, 2>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
                 else
                     contract_panels_aligned<2, 1>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
@@ -942,7 +946,12 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 select_head<6>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
             else if (la.C <= kThreads * kSelPerThread)
                 select_head<kSelPerThread>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
-            else
+            else if (C_STATIC == 1 && la.C <= kThreads * kSelPerThreadMax) {
+                // token-level selection: tens of thousands of keys per head (compiled only into the
+                // c = 1 variant; its register spills stay out of the chunk-level kernels)
+                if constexpr (C_STATIC == 1)
+                    select_head<kSelPerThreadMax>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+            } else
                 select_head<0>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
         }
         if (rows_elsewhere) return;
@@ -1177,7 +1186,7 @@ cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, c
 // kernel, so the L2-latency-bound contraction of one layer spreads over every SM while other
 // layers are being scored. grid = (blocks per head, Hkv); a block takes a contiguous panel range.
 constexpr int kFinSmallThreads = 64;
-template <int RV, int PP>
+template <int RV, int PP, int SB>
 __global__ void __launch_bounds__(kFinSmallThreads)
 finalize_panels_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ out) {
     const int h = blockIdx.y;
@@ -1186,7 +1195,7 @@ finalize_panels_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ o
     const int p_lo = blockIdx.x * per, p_hi = min(p_lo + per, n_p);
     if (p_lo >= p_hi) return;
     const float* rs = a.row_stat + static_cast<size_t>(h) * 512;
-    contract_panels_aligned<RV, PP>(a, g, h, p_lo, p_hi, rs, rs + 256, out);
+    contract_panels_aligned<RV, PP, SB>(a, g, h, p_lo, p_hi, rs, rs + 256, out);
 }
 
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
@@ -1213,10 +1222,12 @@ cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C,
         if (px > max_px) px = max_px;
         if (px < 1) px = 1;
         dim3 pgrid(px, args.Hkv);
-        if (args.R <= 128)
-            finalize_panels_kernel<1, 2><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+        if (plan.spp >= kSlotBatchWide)
+            finalize_panels_kernel<1, 1, kSlotBatchWide><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+        else if (args.R <= 128)
+            finalize_panels_kernel<1, 2, kSlotBatch><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
         else
-            finalize_panels_kernel<2, 1><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+            finalize_panels_kernel<2, 1, kSlotBatch><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
         return cudaGetLastError();
     }
     dim3 grid(bx, args.Hkv);

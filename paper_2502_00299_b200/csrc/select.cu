@@ -29,6 +29,8 @@ cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int
         select_kernel<8><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx);
     else if (C <= kSelThreads * kSelPerThread)
         select_kernel<kSelPerThread><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx);
+    else if (C <= kSelThreads * kSelPerThreadMax)
+        select_kernel<kSelPerThreadMax><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx);
     else
         select_kernel<0><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx);
     return cudaGetLastError();

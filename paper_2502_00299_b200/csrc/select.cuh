@@ -16,7 +16,8 @@
 namespace chunkkv {
 
 constexpr int kSelMaxWarps = 32;
-constexpr int kSelPerThread = 16;     // most chunk keys a thread can hold in registers
+constexpr int kSelPerThread = 16;     // chunk keys per thread of the usual register variant
+constexpr int kSelPerThreadMax = 64;  // the largest register variant (token-level selection: tens of thousands of keys per head)
 constexpr int kSelCap = 4096;         // kept-chunk ids staged for coalesced index writes
 
 struct SelectSmem {
