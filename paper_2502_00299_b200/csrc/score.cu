@@ -1102,6 +1102,8 @@ cudaError_t dispatch_variant(const ScorePlan& plan, const CUtensorMap& tm_q, con
         if (plan.c_static == 1) return launch_variant<1, 1, 256, FUSED>(plan, tm_q, tm_k, args, la, stream);
         return launch_variant<0, 1, 256, FUSED>(plan, tm_q, tm_k, args, la, stream);
     }
+    if (plan.c_static == 10) return launch_variant<10, 2, 80, FUSED>(plan, tm_q, tm_k, args, la, stream);
+    if (plan.c_static == 20) return launch_variant<20, 2, 80, FUSED>(plan, tm_q, tm_k, args, la, stream);
     return launch_variant<0, 2, 128, FUSED>(plan, tm_q, tm_k, args, la, stream);
 }
 
@@ -1115,7 +1117,8 @@ bool make_score_plan(int L, int R, int Hkv, int d, int c, int num_sms, int smem_
     // Chunk sizes with a compiled-in variant use panels that are a multiple of the chunk size;
     // every other chunk size runs the run-time-c variant on the widest tile.
     p.c_static = 0;
-    if (p.n_mt == 1 && (c == 10 || c == 20)) { p.c_static = c; p.n_tile = 240; }
+    // (two query tiles share the accumulator columns: 80 keys per tile, 40 per epilogue panel)
+    if (c == 10 || c == 20) { p.c_static = c; p.n_tile = p.n_mt == 1 ? 240 : 80; }
     else if (p.n_mt == 1 && c == 1) { p.c_static = 1; p.n_tile = 256; }
     else p.n_tile = 256 / p.n_mt;
     p.wp = p.c_static ? p.n_tile / (kGroups / p.n_mt) : 32;
