@@ -875,12 +875,22 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             block_row_stats(a, fg, head, gm, ginv, rs);
             if (direct) {   // chunks never straddle panels: straight from the partial sums, no staging
                 const int p_lo = (t - head * g.n_tiles) * PPTT, p_hi = (seg_end - head * g.n_tiles) * PPTT;
-                if (C_STATIC == 1)
-                    contract_panels_aligned<1, 1, kSlotBatchWide>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
-                else if (a.R <= 128)
-                    contract_panels_aligned<1, 2>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
-                else
-                    contract_panels_aligned<2, 1>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                // panels and slots in flight per warp: about a dozen 16-byte loads per lane, whatever
+                // the number of chunk slots per panel
+                constexpr int SPP = C_STATIC > 0 ? WPP / C_STATIC : 1;
+                if constexpr (N_MT == 1) {
+                    if constexpr (SPP >= kSlotBatchWide)
+                        contract_panels_aligned<1, 1, kSlotBatchWide>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                    else if constexpr (SPP <= 3)
+                        contract_panels_aligned<1, 4, 3>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                    else
+                        contract_panels_aligned<1, 2>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                } else {
+                    if constexpr (SPP <= 2)
+                        contract_panels_aligned<2, 2, 2>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                    else
+                        contract_panels_aligned<2, 1>(a, fg, head, p_lo, p_hi, gm, ginv, la.chunk_scores);
+                }
                 __syncthreads();            // gm / ginv are rewritten for the next head
                 t = seg_end;
                 continue;
@@ -1225,12 +1235,22 @@ cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C,
         if (px > max_px) px = max_px;
         if (px < 1) px = 1;
         dim3 pgrid(px, args.Hkv);
-        if (plan.spp >= kSlotBatchWide)
-            finalize_panels_kernel<1, 1, kSlotBatchWide><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
-        else if (args.R <= 128)
-            finalize_panels_kernel<1, 2, kSlotBatch><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
-        else
-            finalize_panels_kernel<2, 1, kSlotBatch><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+        // panels x slots in flight per warp chosen so that a lane has a dozen or more 16-byte loads out
+        if (args.R <= 128) {
+            if (plan.spp >= kSlotBatchWide)
+                finalize_panels_kernel<1, 1, kSlotBatchWide><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+            else if (plan.spp <= 3)
+                finalize_panels_kernel<1, 4, 3><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+            else
+                finalize_panels_kernel<1, 2, kSlotBatch><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+        } else {
+            if (plan.spp <= 2)
+                finalize_panels_kernel<2, 4, 2><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+            else if (plan.spp <= 4)
+                finalize_panels_kernel<2, 2, 4><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+            else
+                finalize_panels_kernel<2, 1, kSlotBatch><<<pgrid, kFinSmallThreads, 0, stream>>>(args, g, out_scores);
+        }
         return cudaGetLastError();
     }
     dim3 grid(bx, args.Hkv);
