@@ -121,6 +121,23 @@ int ensure_workspace(DeviceCtx& c, size_t payload_bytes) {
     return CHUNKKV_OK;
 }
 
+// How the R = w * Hq / Hkv window rows of a KV head are scored. Rows are independent (each has its
+// own softmax) and chunk scores are sums over rows, so more than 128 rows of an even number of
+// query heads are scored as two heads of R / 2 rows each that read the same keys: every scoring
+// head then fits one 128-row query tile and takes the faster single-tile kernel; its two chunk
+// score vectors are added before the selection.
+struct ScoreShape {
+    int Hs;      // scoring heads
+    int Rs;      // rows per scoring head
+    int shift;   // scoring head v belongs to KV head v >> shift
+};
+ScoreShape score_shape(int Hq, int Hkv, int w) {
+    const int G = Hq / Hkv, R = w * G;
+    if (R > 128 && G % 2 == 0) return {2 * Hkv, R / 2, 1};
+    return {Hkv, R, 0};
+}
+size_t round64(size_t n) { return (n + 63) & ~static_cast<size_t>(63); }
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_sizes(int L, int w, int c, int budget) {
@@ -183,24 +200,29 @@ struct Timer {
 int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w,
               int c, float* out_scores, size_t extra_payload_floats, float** resolved,
               cudaStream_t stream) {
-    const int G = Hq / Hkv, R = w * G, P = L - w;
+    const int P = L - w;
     const int C = (P + c - 1) / c;
     if (C <= 0) return CHUNKKV_OK;
+    const ScoreShape sh = score_shape(Hq, Hkv, w);
+    const int R = sh.Rs;
     ScorePlan plan;
-    if (!make_score_plan(L, R, Hkv, d, c, ctx.num_sms, smem_budget(ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
-    const size_t floats = score_scratch_floats(plan, Hkv, R) + extra_payload_floats;
+    if (!make_score_plan(L, R, sh.Hs, d, c, ctx.num_sms, smem_budget(ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
+    // with two scoring heads per KV head their chunk scores go to scratch first and are added into the output
+    const size_t pair_floats = sh.shift ? round64(static_cast<size_t>(sh.Hs) * C) : 0;
+    const size_t floats = score_scratch_floats(plan, sh.Hs, R) + extra_payload_floats + pair_floats;
     int st = ensure_workspace(ctx, floats * sizeof(float));
     if (st != CHUNKKV_OK) return st;
     float* payload = reinterpret_cast<float*>(static_cast<char*>(ctx.ws) + kHeaderBytes);
     if (out_scores == nullptr) out_scores = payload;
     if (resolved != nullptr) *resolved = out_scores;
+    float* head_scores = sh.shift ? payload + extra_payload_floats : out_scores;
     ScoreArgs a;
-    a.L = L; a.P = P; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
+    a.L = L; a.P = P; a.w = w; a.c = c; a.R = R; a.Hkv = sh.Hs; a.d = d; a.kv_shift = sh.shift;
     a.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
-    score_scratch_layout(plan, Hkv, R, payload + extra_payload_floats, &a);
+    score_scratch_layout(plan, sh.Hs, R, payload + extra_payload_floats + pair_floats, &a);
     a.status = static_cast<int*>(ctx.ws);
     CUtensorMap tm_q, tm_k;
-    st = encode_bf16_3d(&tm_q, q_obs, d, R, Hkv, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    st = encode_bf16_3d(&tm_q, q_obs, d, R, sh.Hs, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (st != CHUNKKV_OK) return st;
     st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < plan.n_tile ? L : plan.n_tile,
                         CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
@@ -213,7 +235,8 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
     if (e != cudaSuccess) return cuda_fail(e);
     {
         Timer t(&ctx, stream, 1);
-        e = launch_finalize(plan, a, C, out_scores, ctx.num_sms, stream);
+        e = launch_finalize(plan, a, C, head_scores, ctx.num_sms, stream);
+        if (e == cudaSuccess && sh.shift) e = launch_pair_sum(head_scores, out_scores, Hkv, C, stream);
     }
     if (e != cudaSuccess) return cuda_fail(e);
     return CHUNKKV_OK;
@@ -244,25 +267,32 @@ int score_with_scratch(const void* q_obs, const void* K, int L, int Hq, int Hkv,
     DeviceCtx* ctx;
     int st = get_ctx(&ctx);
     if (st != CHUNKKV_OK) return st;
-    const int R = w * (Hq / Hkv), P = L - w;
+    const int P = L - w;
     const int C = (P + c - 1) / c;
     if (C <= 0) return CHUNKKV_OK;
+    const ScoreShape sh = score_shape(Hq, Hkv, w);
+    const int R = sh.Rs;
     ScorePlan plan;
-    if (!make_score_plan(L, R, Hkv, d, c, ctx->num_sms, smem_budget(*ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
-    if (kHeaderBytes + score_scratch_floats(plan, Hkv, R) * sizeof(float) > scratch_bytes) return CHUNKKV_ETOOLARGE;
+    if (!make_score_plan(L, R, sh.Hs, d, c, ctx->num_sms, smem_budget(*ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
+    const size_t pair_floats = sh.shift ? round64(static_cast<size_t>(sh.Hs) * C) : 0;
+    if (kHeaderBytes + (score_scratch_floats(plan, sh.Hs, R) + pair_floats) * sizeof(float) > scratch_bytes)
+        return CHUNKKV_ETOOLARGE;
+    float* payload = reinterpret_cast<float*>(static_cast<char*>(scratch) + kHeaderBytes);
+    float* head_scores = sh.shift ? payload : out_scores;
     ScoreArgs a;
-    a.L = L; a.P = P; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
+    a.L = L; a.P = P; a.w = w; a.c = c; a.R = R; a.Hkv = sh.Hs; a.d = d; a.kv_shift = sh.shift;
     a.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
-    score_scratch_layout(plan, Hkv, R, reinterpret_cast<float*>(static_cast<char*>(scratch) + kHeaderBytes), &a);
+    score_scratch_layout(plan, sh.Hs, R, payload + pair_floats, &a);
     a.status = static_cast<int*>(scratch);
     CUtensorMap tm_q, tm_k;
-    st = encode_bf16_3d(&tm_q, q_obs, d, R, Hkv, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+    st = encode_bf16_3d(&tm_q, q_obs, d, R, sh.Hs, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (st != CHUNKKV_OK) return st;
     st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < plan.n_tile ? L : plan.n_tile, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
     if (st != CHUNKKV_OK) return st;
     cudaError_t e = launch_score(plan, tm_q, tm_k, a, stream);
     if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_finalize(plan, a, C, out_scores, ctx->num_sms, stream);
+    e = launch_finalize(plan, a, C, head_scores, ctx->num_sms, stream);
+    if (e == cudaSuccess && sh.shift) e = launch_pair_sum(head_scores, out_scores, Hkv, C, stream);
     if (e != cudaSuccess) return cuda_fail(e);
     return CHUNKKV_OK;
 }
@@ -314,10 +344,11 @@ size_t chunkkv_workspace_bytes(int L, int Hq, int Hkv, int d, int w, int c) {
     std::lock_guard<std::mutex> lk(g_mu);
     DeviceCtx* ctx;
     if (get_ctx(&ctx) != CHUNKKV_OK) return 0;
-    const int R = w * (Hq / Hkv);
+    const ScoreShape sh = score_shape(Hq, Hkv, w);
     const int C = (L - w + c - 1) / c;
-    const size_t floats = scratch_floats_for(*ctx, L, R, Hkv, d, c) +
-                          ((static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63));
+    // chunk scores of the KV heads, those of the scoring heads, and the scoring kernels' scratch
+    const size_t floats = scratch_floats_for(*ctx, L, sh.Rs, sh.Hs, d, c) + round64(static_cast<size_t>(Hkv) * C) +
+                          round64(static_cast<size_t>(sh.Hs) * C);
     return kHeaderBytes + floats * sizeof(float);
 }
 
@@ -471,13 +502,15 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
     }
     float* chunk_scores = nullptr;
     if (C > 0 && k > 0) {
-        const int R = w * (Hq / Hkv);
-        // chunk scores sit at the start of the scratch payload, the score kernels' scratch after them
-        const size_t cs_floats = (static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63);
+        const ScoreShape sh = score_shape(Hq, Hkv, w);
+        const int R = sh.Rs;
+        // chunk scores (of the scoring heads) sit at the start of the scratch payload, the score
+        // kernels' scratch after them
+        const size_t cs_floats = round64(static_cast<size_t>(sh.Hs) * C);
         ScorePlan plan;
-        if ((lane != nullptr || !g_unfused) && make_score_plan(L, R, Hkv, d, c, ctas, smem_budget(*ctx), true, &plan)) {
+        if ((lane != nullptr || !g_unfused) && make_score_plan(L, R, sh.Hs, d, c, ctas, smem_budget(*ctx), true, &plan)) {
             // One cooperative launch for the whole layer.
-            const size_t need = (cs_floats + score_scratch_floats(plan, Hkv, R)) * sizeof(float);
+            const size_t need = (cs_floats + score_scratch_floats(plan, sh.Hs, R)) * sizeof(float);
             char* base;
             if (lane != nullptr) {
                 if (kHeaderBytes + need > lane_bytes) return CHUNKKV_ENOWORKSPACE;
@@ -489,12 +522,12 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
             }
             float* payload = reinterpret_cast<float*>(base + kHeaderBytes);
             ScoreArgs a;
-            a.L = L; a.P = L - w; a.w = w; a.c = c; a.R = R; a.Hkv = Hkv; a.d = d;
+            a.L = L; a.P = L - w; a.w = w; a.c = c; a.R = R; a.Hkv = sh.Hs; a.d = d; a.kv_shift = sh.shift;
             a.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
-            score_scratch_layout(plan, Hkv, R, payload + cs_floats, &a);
+            score_scratch_layout(plan, sh.Hs, R, payload + cs_floats, &a);
             a.status = reinterpret_cast<int*>(base);
             CUtensorMap tm_q, tm_k;
-            st = encode_bf16_3d(&tm_q, q_obs, d, R, Hkv, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+            st = encode_bf16_3d(&tm_q, q_obs, d, R, sh.Hs, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
             if (st != CHUNKKV_OK) return st;
             st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < plan.n_tile ? L : plan.n_tile,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
@@ -506,7 +539,7 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
             const bool split = rows_elsewhere != nullptr || (lane != nullptr && 2 * ctas <= ctx->num_sms);
             io.K = K; io.V = V; io.out_K = split ? nullptr : out_K; io.out_V = out_V; io.out_idx = out_idx;
             io.chunk_scores = payload;
-            io.C = C; io.k = k; io.n_max = n_max;
+            io.C = C; io.k = k; io.n_max = n_max; io.Hkv_out = Hkv;
             io.bar_count = reinterpret_cast<unsigned long long*>(base + 64);
             {
                 Timer t(ctx, s, 0);
@@ -520,7 +553,7 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
             return CHUNKKV_OK;
         }
         if (lane != nullptr) return CHUNKKV_EINVAL_SHAPE;
-        st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, cs_floats, &chunk_scores, s);
+        st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, round64(static_cast<size_t>(Hkv) * C), &chunk_scores, s);
         if (st != CHUNKKV_OK) return st;
     }
     {
@@ -559,11 +592,11 @@ size_t chunkkv_lane_bytes(int L, int Hq, int Hkv, int d, int w, int c, int max_c
     DeviceCtx* ctx;
     if (get_ctx(&ctx) != CHUNKKV_OK) return 0;
     const int ctas = (max_ctas > 0 && max_ctas < ctx->num_sms) ? max_ctas : ctx->num_sms;
-    const int R = w * (Hq / Hkv);
+    const ScoreShape sh = score_shape(Hq, Hkv, w);
     const int C = (L - w + c - 1) / c;
     ScorePlan plan;
-    if (!make_score_plan(L, R, Hkv, d, c, ctas, smem_budget(*ctx), true, &plan)) return 0;
-    const size_t floats = score_scratch_floats(plan, Hkv, R) + ((static_cast<size_t>(Hkv) * C + 63) & ~static_cast<size_t>(63));
+    if (!make_score_plan(L, sh.Rs, sh.Hs, d, c, ctas, smem_budget(*ctx), true, &plan)) return 0;
+    const size_t floats = score_scratch_floats(plan, sh.Hs, sh.Rs) + round64(static_cast<size_t>(sh.Hs) * C);
     return kHeaderBytes + floats * sizeof(float);
 }
 

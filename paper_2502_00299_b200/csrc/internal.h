@@ -23,7 +23,9 @@ struct ScorePlan {
 };
 
 struct ScoreArgs {
-    int L, P, w, c, R, Hkv, d;
+    int L, P, w, c, R, Hkv, d;   // R rows per scoring head, Hkv scoring heads (see kv_shift)
+    int kv_shift;         // scoring head v reads the keys of KV head v >> kv_shift: 1 when the rows of a KV head
+                          // are scored as two heads of half the rows (rows are independent, sums add up)
     float sl2;            // log2(e) / sqrt(d)
     float* stat_m;        // [Hkv, n_panels, R] panel row maxima (log2 domain)
     float* cta_stat;      // [grid, hs_max, 4 groups, {max, sum}, 128] per-CTA folded row statistics
@@ -54,8 +56,9 @@ struct FusedLayerIO {
     void* out_K;
     void* out_V;
     int32_t* out_idx;
-    float* chunk_scores;   // [Hkv, C] scratch
+    float* chunk_scores;   // [scoring heads, C] scratch
     int C, k, n_max;
+    int Hkv_out;           // KV heads (selection and gather), = scoring heads >> kv_shift
     unsigned long long* bar_count;   // grid barrier ticket counter in the scratch header
 };
 
@@ -75,6 +78,9 @@ cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int 
 // Jaccard similarity of two kept-index matrices, one CTA per head (diagnostics.cu).
 cudaError_t launch_jaccard(const int32_t* idx_a, const int32_t* idx_b, int Hkv, int n_a, int n_b,
                            float* out_ratio, int32_t* out_counts_or_null, cudaStream_t stream);
+
+// out[h][ch] = in[2h][ch] + in[2h + 1][ch]: chunk scores of KV heads from their two scoring heads.
+cudaError_t launch_pair_sum(const float* in, float* out, int Hkv, int C, cudaStream_t stream);
 
 // The gather in small CTAs that can share SMs with resident layer-kernel CTAs (lanes).
 cudaError_t launch_gather_shared_sms(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,

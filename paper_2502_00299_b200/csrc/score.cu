@@ -503,6 +503,7 @@ struct LayerArgs {
     int32_t* out_idx;
     float* chunk_scores;   // [Hkv, C]
     int C, k, n_max;
+    int Hkv_out;           // KV heads: selection and gather (scoring heads >> kv_shift)
     unsigned long long* bar_count;   // grid barrier counter (zero between launches); its exit counter 64 bytes on
 };
 
@@ -669,7 +670,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                     if (!ok) break;
                     const uint32_t bar = full0_bar + 8u * st;
                     mbar_arrive_expect_tx(bar, k_bytes);
-                    tma_load_3d(k_base + st * stage_bytes, &tm_k, bar, kb * 64, tile * N_TILE, head);
+                    tma_load_3d(k_base + st * stage_bytes, &tm_k, bar, kb * 64, tile * N_TILE, head >> a.kv_shift);
                     ++ctr;
                     if (++st == n_stages) { st = 0; st_par ^= 1u; }
                 }
@@ -845,7 +846,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
 
         // One CTA per head (grid = Hkv): tiles, row statistics, chunk scores, selection and output
         // rows of a head all belong to the same CTA, so no CTA ever waits for another one.
-        const bool solo = static_cast<int>(gridDim.x) == a.Hkv;
+        const bool solo = static_cast<int>(gridDim.x) == a.Hkv && a.kv_shift == 0;
         if (!solo && !grid_barrier(la.bar_count, gridDim.x, 0, bar_ok, abort_flag)) {
             if (threadIdx.x == 0) atomicExch(a.status, 1);
             return;
@@ -947,22 +948,23 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             // Nothing follows the selection in this launch: CTAs check out of the barrier now
             // (no CTA waits on it again) and those without a head leave at once.
             grid_barrier_finish(la.bar_count, la.bar_count + 8, gridDim.x);
-            if (static_cast<int>(blockIdx.x) >= a.Hkv) return;
+            if (static_cast<int>(blockIdx.x) >= la.Hkv_out) return;
         }
-        for (int h = blockIdx.x; h < a.Hkv; h += gridDim.x) {
-            const float* sc = la.chunk_scores + static_cast<size_t>(h) * la.C;
+        for (int h = blockIdx.x; h < la.Hkv_out; h += gridDim.x) {
+            const float* sc = la.chunk_scores + (static_cast<size_t>(h) << a.kv_shift) * la.C;
+            const float* sc2 = a.kv_shift ? sc + la.C : nullptr;        // the head's second scoring head
             int32_t* out = la.out_idx + static_cast<size_t>(h) * la.n_max;
             if (la.C <= kThreads * 6)
-                select_head<6>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+                select_head<6>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
             else if (la.C <= kThreads * kSelPerThread)
-                select_head<kSelPerThread>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+                select_head<kSelPerThread>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
             else if (C_STATIC == 1 && la.C <= kThreads * kSelPerThreadMax) {
                 // token-level selection: tens of thousands of keys per head (compiled only into the
                 // c = 1 variant; its register spills stay out of the chunk-level kernels)
                 if constexpr (C_STATIC == 1)
-                    select_head<kSelPerThreadMax>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+                    select_head<kSelPerThreadMax>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
             } else
-                select_head<0>(sc, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+                select_head<0>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
         }
         if (rows_elsewhere) return;
         if (!solo) {
@@ -976,7 +978,7 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const int vpr = a.d >> 3;
         const int rows_per_pass = (kThreads / vpr) * kGatherRowsPerThread;
         // (32-bit arithmetic: the host checks that Hkv * n_max * (grid + 1) fits)
-        const unsigned rows_total = static_cast<unsigned>(a.Hkv) * la.n_max;
+        const unsigned rows_total = static_cast<unsigned>(la.Hkv_out) * la.n_max;
         const int r_begin = static_cast<int>(rows_total * blockIdx.x / gridDim.x);
         const int r_end = static_cast<int>(rows_total * (blockIdx.x + 1) / gridDim.x);
         // The indices of this CTA's rows (contiguous in [Hkv, n_max] order) go to shared memory
@@ -1190,8 +1192,16 @@ cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, c
     la.C = io.C;
     la.k = io.k;
     la.n_max = io.n_max;
+    la.Hkv_out = io.Hkv_out;
     la.bar_count = io.bar_count;
     return dispatch_variant<true>(plan, tm_q, tm_k, args, la, stream);
+}
+
+__global__ void pair_sum_kernel(const float* __restrict__ in, float* __restrict__ out, int C, size_t n) {
+    const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const size_t h = i / C, ch = i - h * C;
+    out[i] = in[(2 * h) * C + ch] + in[(2 * h + 1) * C + ch];
 }
 
 // Chunk scores for compile-time chunk sizes (chunks never straddle panels) and R % 4 == 0, in CTAs
@@ -1209,6 +1219,13 @@ finalize_panels_kernel(const ScoreArgs a, const FinGeom g, float* __restrict__ o
     if (p_lo >= p_hi) return;
     const float* rs = a.row_stat + static_cast<size_t>(h) * 512;
     contract_panels_aligned<RV, PP, SB>(a, g, h, p_lo, p_hi, rs, rs + 256, out);
+}
+
+cudaError_t launch_pair_sum(const float* in, float* out, int Hkv, int C, cudaStream_t stream) {
+    const size_t n = static_cast<size_t>(Hkv) * C;
+    if (n == 0) return cudaSuccess;
+    pair_sum_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, stream>>>(in, out, C, n);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,

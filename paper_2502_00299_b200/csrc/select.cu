@@ -14,7 +14,7 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
               int32_t* __restrict__ out_idx) {
     __shared__ SelectSmem sm;
     const int h = blockIdx.x;
-    select_head<KPT>(scores + static_cast<size_t>(h) * C, L, w, c, C, k, n_max,
+    select_head<KPT>(scores + static_cast<size_t>(h) * C, nullptr, L, w, c, C, k, n_max,
                      out_idx + static_cast<size_t>(h) * n_max, sm);
 }
 

@@ -38,9 +38,11 @@ __device__ __forceinline__ uint32_t select_order_key(float x) {
 // All threads of the CTA must call this (it uses __syncthreads); blockDim.x must be a multiple
 // of 32 and at most 1024. KPT > 0: every thread keeps up to KPT keys in registers, which needs
 // C <= blockDim.x * KPT; KPT = 0: keys are re-read from memory on every use.
+// sc2 != NULL: the head's scores are sc[ch] + sc2[ch] (a KV head scored as two heads of half the rows).
 template <int KPT>
-__device__ __forceinline__ void select_head(const float* __restrict__ sc, int L, int w, int c, int C, int k,
-                                            int n_max, int32_t* __restrict__ out, SelectSmem& sm) {
+__device__ __forceinline__ void select_head(const float* __restrict__ sc, const float* __restrict__ sc2, int L, int w, int c,
+                                            int C, int k, int n_max, int32_t* __restrict__ out, SelectSmem& sm) {
+    auto score_at = [&](int ch) { return sc2 != nullptr ? sc[ch] + sc2[ch] : sc[ch]; };
     const int P = L - w;
     const int nt = blockDim.x, nwarps = nt >> 5;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -55,7 +57,7 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
     uint32_t keys[KR];
     if (IN_REGS && kk > 0 && !keep_all) {
 #pragma unroll
-        for (int u = 0; u < KR; ++u) keys[u] = (c0 + u < c1) ? select_order_key(sc[c0 + u]) : 0u;
+        for (int u = 0; u < KR; ++u) keys[u] = (c0 + u < c1) ? select_order_key(score_at(c0 + u)) : 0u;
     }
     if (tid == 0) sm.last_kept = 0;
 
@@ -99,7 +101,7 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
                     if (u < per) count_one(c0 + u < c1, keys[u]);      // `per` is uniform: no divergence
             } else {
                 for (int u = 0; u < per; ++u)
-                    count_one(c0 + u < c1, (c0 + u < c1) ? select_order_key(sc[c0 + u]) : 0u);
+                    count_one(c0 + u < c1, (c0 + u < c1) ? select_order_key(score_at(c0 + u)) : 0u);
             }
             __syncthreads();
             if (grouped) {
@@ -149,7 +151,7 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
                 if (c0 + u < c1) { gt_n += keys[u] > thresh; eq_n += keys[u] == thresh; }
         } else {
             for (int ch = c0; ch < c1; ++ch) {
-                const uint32_t key = select_order_key(sc[ch]);
+                const uint32_t key = select_order_key(score_at(ch));
                 gt_n += key > thresh;
                 eq_n += key == thresh;
             }
@@ -198,7 +200,7 @@ __device__ __forceinline__ void select_head(const float* __restrict__ sc, int L,
             for (int u = 0; u < KR; ++u)
                 if (c0 + u < c1) visit(c0 + u, keys[u]);
         } else {
-            for (int ch = c0; ch < c1; ++ch) visit(ch, keep_all ? 0u : select_order_key(sc[ch]));
+            for (int ch = c0; ch < c1; ++ch) visit(ch, keep_all ? 0u : select_order_key(score_at(ch)));
         }
     }
     __syncthreads();
