@@ -954,17 +954,17 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
             const float* sc = la.chunk_scores + (static_cast<size_t>(h) << a.kv_shift) * la.C;
             const float* sc2 = a.kv_shift ? sc + la.C : nullptr;        // the head's second scoring head
             int32_t* out = la.out_idx + static_cast<size_t>(h) * la.n_max;
-            if (la.C <= kThreads * 6)
-                select_head<6>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
-            else if (la.C <= kThreads * kSelPerThread)
-                select_head<kSelPerThread>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
-            else if (C_STATIC == 1 && la.C <= kThreads * kSelPerThreadMax) {
-                // token-level selection: tens of thousands of keys per head (compiled only into the
-                // c = 1 variant; its register spills stay out of the chunk-level kernels)
-                if constexpr (C_STATIC == 1)
-                    select_head<kSelPerThreadMax>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
-            } else
-                select_head<0>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+            if (la.C <= kThreads * 6) {
+                select_head_regs<6>(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss);
+            } else {
+                // keys go to the idle dynamic shared memory behind the selection scratch; if they do
+                // not fit there (token-level selection of very long sequences) they replace the
+                // chunk scores, which nothing reads after the selection
+                uint32_t* kbuf = reinterpret_cast<uint32_t*>(dyn + ((sizeof(SelectSmem) + 127) & ~size_t(127)));
+                const bool fits = static_cast<size_t>(la.C) * 4 + sizeof(SelectSmem) + 256 <= static_cast<size_t>(g.dyn_bytes);
+                select_head_rows(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss,
+                                 fits ? kbuf : reinterpret_cast<uint32_t*>(const_cast<float*>(sc)));
+            }
         }
         if (rows_elsewhere) return;
         if (!solo) {
