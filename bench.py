@@ -40,6 +40,7 @@ NSETS = 4
 LAYERS_PER_STEP = 32
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
+FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one cfg2 layer through a lane, from ncu captures
 # of both launches (layer kernel + row gather): 8 CTAs 69.3 + 13.5 MB, 18 CTAs 69.4 + 13.5 MB
 TRAFFIC_BYTES_PER_LAYER = {8: 82.8e6, 18: 82.9e6}
@@ -54,12 +55,21 @@ def parse_args():
     ap.add_argument("--config", type=int, default=2, help="workload table entry (2 = headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-long", action="store_true", help="skip the 128K / 64K long-context layer timings")
     ap.add_argument("--lanes", type=int, default=18, help="layers in flight (each on 1/lanes of the SMs)")
     ap.add_argument("--lane-ctas", type=int, default=0, help="CTA budget of a lane (0: SMs // lanes)")
     ap.add_argument("--mode", choices=("pipe", "lane"), default="pipe",
                     help="pipe: chunkkv_pipe_layer (layer kernels back to back, row gathers on side streams); "
                          "lane: chunkkv_compress_layer_lane (one layer at a time per lane)")
     return ap.parse_args()
+
+
+def measured_bf16_sustained_tflops():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return FALLBACK_BF16_SUSTAINED_TFLOPS, "fallback"
 
 
 def measured_hbm_peak():
@@ -202,7 +212,7 @@ def run_ours(args, wl):
     _build.build()
     import paper_2502_00299_b200 as ck
     from paper_2502_00299_b200.sharding import job_throughput, max_over_ranks
-    from workloads import make_layer
+    from workloads import CONFIGS, make_layer, scaled
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -447,6 +457,54 @@ def run_ours(args, wl):
                                        "note": "chunkkv_compress_layer with c = 1, one layer at a time on all SMs"}
     extra_roof["jaccard"] = {"us": us_jac, "note": "chunkkv_jaccard on the kept indices of two layers "
                                                    f"([{wl.Hkv}, {n_max}] int32 each; latency-bound, includes the binding's two small allocations)"}
+
+    # ---- the long-context shapes (256 score rows per KV head: bound by exponentials and the tensor
+    #      pipe rather than by HBM), one layer at a time on the whole GPU
+    if not args.no_long and rank == 0:
+        tf_peak, tf_src = measured_bf16_sustained_tflops()
+        sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+        long_rows = {}
+        for name, lw in (("cfg4_128k", CONFIGS[4]), ("cfg5_longest_64k", scaled(CONFIGS[5], L=65536))):
+            lsets = []
+            for i in range(2):
+                lx = make_layer(lw, layer=i)
+                lsets.append(tuple(torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16)
+                                   for b in (lx.q_obs, lx.K, lx.V)))
+            ln = ck.out_len(lw.L, lw.w, lw.c, lw.budget)
+            lo = [torch.empty((lw.Hkv, ln, lw.d), dtype=torch.bfloat16, device=dev) for _ in range(2)]
+            lo.append(torch.empty((lw.Hkv, ln), dtype=torch.int32, device=dev))
+            cnt = [0]
+
+            def long_layer():
+                q, K, V = lsets[cnt[0] % 2]
+                cnt[0] += 1
+                st = lib.chunkkv_compress_layer(q.data_ptr(), K.data_ptr(), V.data_ptr(), lw.L, lw.Hq, lw.Hkv, lw.d, lw.w,
+                                                lw.c, lw.budget, None, lo[0].data_ptr(), lo[1].data_ptr(),
+                                                lo[2].data_ptr(), stream.cuda_stream)
+                if st != 0:
+                    raise ck.ChunkKVError(st, "chunkkv_compress_layer (long context)")
+
+            with torch.cuda.stream(stream):
+                us = time_calls(long_layer, n=20)
+            if ck.device_status() != 0:
+                raise RuntimeError("a kernel reported an abandoned wait")
+            lb = layer_bytes(lw, ln)["layer"]
+            R = lw.w * lw.Hq // lw.Hkv
+            flops = 2.0 * R * lw.L * lw.d * lw.Hkv
+            exps = float(R) * lw.L * lw.Hkv
+            clock_max_mhz = clocks.get("sm_max_mhz")
+            sfu_floor_us = exps / (16.0 * sm_count * clock_max_mhz * 1e6) * 1e6 if clock_max_mhz else None
+            long_rows[name] = {
+                "Hq": lw.Hq, "Hkv": lw.Hkv, "L": lw.L, "w": lw.w, "c": lw.c, "budget": lw.budget, "score_rows_per_kv_head": R,
+                "us": us, "tokens_per_s": lw.L / (us * 1e-6), "algorithmic_bytes": lb,
+                "GB/s": lb / (us * 1e-6) / 1e9, "frac_of_measured_hbm_peak": lb / (us * 1e-6) / 1e9 / peak,
+                "bf16_TFLOP/s": flops / (us * 1e-6) / 1e12,
+                "frac_of_sustained_bf16_peak": flops / (us * 1e-6) / 1e12 / tf_peak, "bf16_peak_source": tf_src,
+                "exponentials": exps, "special_function_floor_us": sfu_floor_us,
+                "note": "chunkkv_compress_layer, one layer at a time on all SMs, two K/V sets alternating (each > L2); "
+                        "floor = exponentials / (16 per clock per SM at the maximum SM clock)"}
+            del lsets, lo
+        extra_roof["long_context_layers"] = long_rows
 
     # ---- end to end: pinned host buffers in, host buffers out, copies inside the timed region
     e2e = None
