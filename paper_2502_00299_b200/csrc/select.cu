@@ -39,23 +39,18 @@ cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int
         return cudaGetLastError();
     }
     // more: the keys of a head live in dynamic shared memory if they fit beside the static scratch
-    constexpr size_t kPlain = 48 * 1024 - sizeof(SelectSmem) - 512;     // available without opting in
+    // (beyond the 48 KB every kernel may use, so the kernel opts in), else they are recomputed
     const size_t want = static_cast<size_t>(C) * 4;
-    int key_bytes = 0;
-    if (want <= kPlain) {
-        key_bytes = static_cast<int>(want);
-    } else {
-        int dev = 0, optin = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-        const long room = static_cast<long>(optin) - static_cast<long>(sizeof(SelectSmem)) - 1024;
-        if (room > 0 && want <= static_cast<size_t>(room)) {
-            if (cudaFuncSetAttribute(select_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     static_cast<int>(room)) == cudaSuccess)
-                key_bytes = static_cast<int>(want);
-            else
-                cudaGetLastError();
-        }
+    int key_bytes = 0, dev = 0, optin = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    const long room = static_cast<long>(optin) - static_cast<long>(sizeof(SelectSmem)) - 1024;
+    if (room > 0 && want <= static_cast<size_t>(room)) {
+        if (cudaFuncSetAttribute(select_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(room)) == cudaSuccess)
+            key_bytes = static_cast<int>(want);
+        else
+            cudaGetLastError();
     }
     select_kernel<0><<<Hkv, kSelThreads, key_bytes, stream>>>(scores, L, w, c, C, k, n_max, out_idx, key_bytes);
     return cudaGetLastError();

@@ -46,6 +46,9 @@ def test_gather_bit_exact(ck, Hkv, L, d, n_max):
 @pytest.mark.parametrize("L,w,c,budget,Hkv", [
     (2048, 16, 10, 256, 2), (1003, 8, 10, 203, 3), (500, 4, 7, 4 + 7 * 20, 2), (26, 4, 5, 1000, 1),
     (26, 4, 5, 8, 1), (4, 4, 5, 4, 2), (9000, 32, 1, 32 + 777, 2), (20000, 32, 3, 32 + 3 * 2500, 1),
+    (3000, 8, 1, 8 + 300, 2),          # 2992 chunks: eight keys per thread in registers
+    (40000, 32, 1, 32 + 4000, 2),      # 39968 chunks: keys in opted-in shared memory
+    (70000, 16, 1, 16 + 5000, 2),      # 69984 chunks: more keys than shared memory holds
 ])
 def test_select_bit_exact_on_given_scores(ck, L, w, c, budget, Hkv):
     rng = np.random.default_rng(L * 7 + c)
@@ -67,6 +70,22 @@ def test_select_ties_go_to_lower_chunk_ids(ck):
     s[2, ::2] = -0.0                                                # -0 ties with +0
     s[2, 1::2] = 0.0
     for budget in (w + c * 1, w + c * 37, w + c * (C // 2), w + c * (C - 1)):
+        idx = ck.select(torch.from_numpy(s).cuda(), L, w, c, budget).cpu().numpy()
+        assert np.array_equal(idx, ora.select(s.astype(np.float64), L, w, c, budget))
+
+
+@pytest.mark.parametrize("L", [9000, 70000])      # keys in shared memory / recomputed from the scores
+def test_select_ties_with_many_chunks_per_thread(ck, L):
+    w, c, Hkv = 8, 1, 4
+    C = ora.num_chunks(L, w, c)
+    rng = np.random.default_rng(L)
+    s = rng.integers(0, 6, size=(Hkv, C)).astype(np.float32)       # massive ties
+    s[1] = 1.0                                                      # all equal
+    s[2, ::2] = -0.0                                                # -0 ties with +0
+    s[2, 1::2] = 0.0
+    s[3] = (rng.standard_normal(C) * 1e3).astype(np.float32)        # both signs, many exponents
+    s[3, ::7] = s[3, 3]
+    for budget in (w + 1, w + 37, w + C // 2, w + C - 1):
         idx = ck.select(torch.from_numpy(s).cuda(), L, w, c, budget).cpu().numpy()
         assert np.array_equal(idx, ora.select(s.astype(np.float64), L, w, c, budget))
 
