@@ -29,7 +29,9 @@ prints; parity on these choices is UNPINNED by the paper itself):
 What pins it (tests/test_oracle_*.py): brute-force enumeration of chunk subsets, softmax
 row sums, mass conservation, the uniform-attention closed form (q = 0), a dominant-key
 limit, an e-ratio logit case that fixes the 1/sqrt(d) scale, an independent library
-softmax, library top-k for c = 1, the budget/ordering/window invariants, reuse identity.
+softmax, library top-k for c = 1, the budget/ordering/window invariants, reuse identity;
+for Algorithm 1's budget rule (select_alg1): hand-worked cases, brute-force enumeration of
+chunk subsets followed by the cut, and the exact output length.
 
 Layouts (numpy arrays; bf16 tensors arrive as uint16 bit patterns):
   q_obs [Hq, w, d]   K, V [Hkv, L, d]   token scores [Hkv, P]   chunk scores [Hkv, C]
@@ -168,6 +170,58 @@ def select(scores: np.ndarray, L: int, w: int, c: int, budget: int) -> np.ndarra
     return out
 
 
+# --------------------------------------------------------------------------- Algorithm 1's budget rule
+# The alternative selection policy printed in Algorithm 1 (section "Chunk Based KV Compression")
+# and the paragraph after it: k = floor(L_max / c) chunks are selected, their tokens are taken in
+# the original order, only the first L_max - w of them are kept, and the observe window takes the
+# last w places. Compression-ratio budgets (the 10 % / 20 % / 30 % settings of the experiments)
+# are L_max = floor(ratio * L). Same readings as above for everything the algorithm leaves open
+# (chunk grid over the prefix, ties to the lower chunk id).
+def budget_from_ratio(L: int, ratio: float) -> int:
+    """L_max for a compression ratio (fraction of the L tokens that is kept)."""
+    if not (0.0 <= ratio <= 1.0):
+        raise ValueError("ratio must lie in [0, 1]")
+    return int(math.floor(ratio * L))
+
+
+def num_kept_chunks_alg1(L: int, w: int, c: int, budget: int) -> int:
+    """k = floor(L_max / c), limited to the chunks that exist. (Algorithm 1, "Top-K Chunk Selection".)"""
+    _check(L, w, c, budget)
+    return min(budget // c, num_chunks(L, w, c))
+
+
+def out_len_alg1(L: int, w: int, c: int, budget: int) -> int:
+    """Row count of the outputs: at most L_max - w selected tokens, then the window."""
+    return min(num_kept_chunks_alg1(L, w, c, budget) * c, budget - w) + w
+
+
+def kept_indices_alg1(kept: Sequence[int], L: int, w: int, c: int, budget: int, n_max: int) -> np.ndarray:
+    """Tokens of the kept chunks in ascending order, cut to the first L_max - w, then the window.
+
+    (Algorithm 1, "Compression" and "Concatenation": K' <- concat(K'[0 : L_max - w], K[T_k - w : T_k]).)
+    """
+    P = L - w
+    sel: List[int] = []
+    for ch in sorted(int(v) for v in kept):
+        sel.extend(range(ch * c, min((ch + 1) * c, P)))
+    sel = sel[:budget - w]
+    idx = np.asarray(sel + list(range(P, L)), dtype=np.int32)
+    out = np.full(n_max, -1, dtype=np.int32)
+    out[:idx.size] = idx
+    return out
+
+
+def select_alg1(scores: np.ndarray, L: int, w: int, c: int, budget: int) -> np.ndarray:
+    """idx [Hkv, n_max] from chunk scores [Hkv, C] under Algorithm 1's budget rule."""
+    k = num_kept_chunks_alg1(L, w, c, budget)
+    n_max = out_len_alg1(L, w, c, budget)
+    Hkv = scores.shape[0]
+    out = np.empty((Hkv, n_max), dtype=np.int32)
+    for h in range(Hkv):
+        out[h] = kept_indices_alg1(select_chunks(scores[h], k), L, w, c, budget, n_max)
+    return out
+
+
 # --------------------------------------------------------------------------- step 4: gather
 def gather(K: np.ndarray, V: np.ndarray, idx: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     """out_K[h, n] = K[h, idx[h, n]] (bit copies), zero rows where idx is -1.
@@ -210,6 +264,17 @@ def compress_layer(q_obs: np.ndarray, K: np.ndarray, V: np.ndarray, Hq: int, Hkv
     out_K, out_V = gather(K, V, idx)
     res.update(out_K=out_K, out_V=out_V, idx=idx)
     return res
+
+
+def compress_layer_alg1(q_obs: np.ndarray, K: np.ndarray, V: np.ndarray, Hq: int, Hkv: int,
+                        w: int, c: int, budget: int) -> Dict[str, np.ndarray]:
+    """One layer under Algorithm 1's budget rule: same scores, select_alg1, same gather."""
+    L = K.shape[1]
+    t = token_scores(q_obs, K, Hq, Hkv, w)
+    s = chunk_scores(t, c)
+    idx = select_alg1(s, L, w, c, budget)
+    out_K, out_V = gather(K, V, idx)
+    return dict(token_scores=t, chunk_scores=s, idx=idx, out_K=out_K, out_V=out_V)
 
 
 # --------------------------------------------------------------------------- many layers
