@@ -160,6 +160,27 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
                            void* out_K, void* out_V, int32_t* out_idx, void* stream);
 
 /*
+ * Algorithm 1's budget rule, as an alternative to Algorithm 3's (which the calls above follow):
+ * k = floor(L_max / c) chunks are selected (at most the C that exist), their tokens are taken in
+ * ascending order and cut to the first L_max - w ("K'[0 : L_max - w]"), and the observe window
+ * takes the last w places. `budget` is L_max. chunkkv_budget_from_ratio gives L_max for the
+ * compression ratios of the paper's experiments: floor(ratio * L), ratio in [0, 1].
+ * chunkkv_out_len_alg1 = min(k * c, L_max - w) + w is the row count n_max of out_idx / out_K /
+ * out_V for these two calls; a kept clipped last chunk leaves -1 / zero-row padding at the end.
+ * Chunk grid, tie-break, layouts, ownership and error codes are those of chunkkv_select and
+ * chunkkv_compress_layer (no index reuse argument: reuse layers call chunkkv_compress_layer or
+ * chunkkv_gather with these indices). Scoring, selection and gathering run as three launches.
+ */
+CHUNKKV_API int chunkkv_budget_from_ratio(int L, double ratio);
+CHUNKKV_API int chunkkv_num_kept_chunks_alg1(int L, int w, int c, int budget);
+CHUNKKV_API int chunkkv_out_len_alg1(int L, int w, int c, int budget);
+CHUNKKV_API int chunkkv_select_alg1(const float* chunk_scores, int L, int Hkv, int w, int c, int budget,
+                        int32_t* out_idx, void* stream);
+CHUNKKV_API int chunkkv_compress_layer_alg1(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                                int d, int w, int c, int budget, void* out_K, void* out_V, int32_t* out_idx,
+                                void* stream);
+
+/*
  * Index similarity between two layers (the paper's section on layer-wise index reuse reports the
  * Jaccard similarity of the preserved indices of adjacent layers; Algorithm 2 shares indices
  * because it is high). Per KV head h: out_ratio[h] = |A n B| / |A u B| (1 when both are empty),

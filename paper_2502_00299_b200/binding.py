@@ -72,6 +72,16 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_jaccard.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     L.chunkkv_score_noalloc.restype = i32
     L.chunkkv_score_noalloc.argtypes = [vp, vp] + [i32] * 6 + [vp, vp]
+    L.chunkkv_budget_from_ratio.restype = i32
+    L.chunkkv_budget_from_ratio.argtypes = [i32, ctypes.c_double]
+    L.chunkkv_num_kept_chunks_alg1.restype = i32
+    L.chunkkv_num_kept_chunks_alg1.argtypes = [i32] * 4
+    L.chunkkv_out_len_alg1.restype = i32
+    L.chunkkv_out_len_alg1.argtypes = [i32] * 4
+    L.chunkkv_select_alg1.restype = i32
+    L.chunkkv_select_alg1.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp]
+    L.chunkkv_compress_layer_alg1.restype = i32
+    L.chunkkv_compress_layer_alg1.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, vp, vp]
     L.chunkkv_profile_enable.restype = i32
     L.chunkkv_profile_enable.argtypes = [i32]
     L.chunkkv_profile_read.restype = i32
@@ -166,6 +176,44 @@ def select(chunk_scores: torch.Tensor, L: int, w: int, c: int, budget: int,
     _check(lib.chunkkv_select(chunk_scores.data_ptr(), L, Hkv, w, c, budget, idx.data_ptr(),
                               _stream(stream)), "chunkkv_select")
     return idx
+
+
+def budget_from_ratio(L: int, ratio: float) -> int:
+    v = lib.chunkkv_budget_from_ratio(L, float(ratio))
+    _check(min(v, 0), "chunkkv_budget_from_ratio")
+    return v
+
+
+def out_len_alg1(L: int, w: int, c: int, budget: int) -> int:
+    v = lib.chunkkv_out_len_alg1(L, w, c, budget)
+    _check(min(v, 0), "chunkkv_out_len_alg1")
+    return v
+
+
+def select_alg1(chunk_scores: torch.Tensor, L: int, w: int, c: int, budget: int,
+                stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """idx [Hkv, n_max] int32 from chunk scores [Hkv, C] f32 under Algorithm 1's budget rule."""
+    _dev(chunk_scores, torch.float32, "chunk_scores")
+    Hkv = chunk_scores.shape[0]
+    idx = torch.empty((Hkv, out_len_alg1(L, w, c, budget)), dtype=torch.int32, device=chunk_scores.device)
+    _check(lib.chunkkv_select_alg1(chunk_scores.data_ptr(), L, Hkv, w, c, budget, idx.data_ptr(),
+                                   _stream(stream)), "chunkkv_select_alg1")
+    return idx
+
+
+def compress_layer_alg1(q_obs: torch.Tensor, K: torch.Tensor, V: torch.Tensor, Hq: int, w: int, c: int, budget: int,
+                        stream: Optional[torch.cuda.Stream] = None) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """out_K, out_V [Hkv, n_max, d], idx [Hkv, n_max] for one layer under Algorithm 1's budget rule."""
+    _dev(q_obs, torch.bfloat16, "q_obs"); _dev(K, torch.bfloat16, "K"); _dev(V, torch.bfloat16, "V")
+    Hkv, L, d = K.shape
+    n_max = out_len_alg1(L, w, c, budget)
+    out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=K.device)
+    out_V = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=K.device)
+    idx = torch.empty((Hkv, n_max), dtype=torch.int32, device=K.device)
+    _check(lib.chunkkv_compress_layer_alg1(q_obs.data_ptr(), K.data_ptr(), V.data_ptr(), L, Hq, Hkv, d, w, c, budget,
+                                           out_K.data_ptr(), out_V.data_ptr(), idx.data_ptr(), _stream(stream)),
+           "chunkkv_compress_layer_alg1")
+    return out_K, out_V, idx
 
 
 def gather(K: torch.Tensor, V: torch.Tensor, idx: torch.Tensor,

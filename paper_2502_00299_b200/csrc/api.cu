@@ -585,6 +585,81 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
                          stream);
 }
 
+// ---- Algorithm 1's budget rule: k = floor(L_max / c) chunks, their tokens cut to the first
+//      L_max - w, the window last. Scoring and gathering are the calls above; only the number of
+//      kept chunks, the output length and the cut differ.
+int chunkkv_budget_from_ratio(int L, double ratio) {
+    if (L < 0 || !(ratio >= 0.0 && ratio <= 1.0)) return CHUNKKV_EINVAL_SHAPE;
+    return static_cast<int>(floor(ratio * static_cast<double>(L)));
+}
+
+int chunkkv_num_kept_chunks_alg1(int L, int w, int c, int budget) {
+    int st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    const int C = (L - w + c - 1) / c;
+    const int k = budget / c;
+    return k < C ? k : C;
+}
+
+int chunkkv_out_len_alg1(int L, int w, int c, int budget) {
+    const int k = chunkkv_num_kept_chunks_alg1(L, w, c, budget);
+    if (k < 0) return k;
+    const long long full = static_cast<long long>(k) * c, cap = budget - w;
+    return static_cast<int>((full < cap ? full : cap) + w);
+}
+
+int chunkkv_select_alg1(const float* chunk_scores, int L, int Hkv, int w, int c, int budget,
+                        int32_t* out_idx, void* stream) {
+    int st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    if (Hkv < 1 || Hkv > 65535) return CHUNKKV_EINVAL_SHAPE;
+    const int C = chunkkv_num_chunks(L, w, c);
+    const int k = chunkkv_num_kept_chunks_alg1(L, w, c, budget);
+    const int n_max = chunkkv_out_len_alg1(L, w, c, budget);
+    if (out_idx == nullptr || (C > 0 && k > 0 && chunk_scores == nullptr)) return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(out_idx) || !aligned16(chunk_scores)) return CHUNKKV_EINVAL_ALIGN;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaError_t e = launch_select(chunk_scores, L, Hkv, w, c, C, k, n_max, out_idx,
+                                  static_cast<cudaStream_t>(stream), budget - w);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+int chunkkv_compress_layer_alg1(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                                int d, int w, int c, int budget, void* out_K, void* out_V, int32_t* out_idx,
+                                void* stream) {
+    int st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    st = check_heads(L, Hq, Hkv, d, w);
+    if (st != CHUNKKV_OK) return st;
+    if (q_obs == nullptr || K == nullptr || V == nullptr || out_K == nullptr || out_V == nullptr || out_idx == nullptr)
+        return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(q_obs) || !aligned16(K) || !aligned16(V) || !aligned16(out_K) || !aligned16(out_V) ||
+        !aligned16(out_idx))
+        return CHUNKKV_EINVAL_ALIGN;
+    const int C = chunkkv_num_chunks(L, w, c);
+    const int k = chunkkv_num_kept_chunks_alg1(L, w, c, budget);
+    const int n_max = chunkkv_out_len_alg1(L, w, c, budget);
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float* chunk_scores = nullptr;
+    if (C > 0 && k > 0) {
+        st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, round64(static_cast<size_t>(Hkv) * C), &chunk_scores, s);
+        if (st != CHUNKKV_OK) return st;
+    }
+    cudaError_t e = launch_select(chunk_scores, L, Hkv, w, c, C, k, n_max, out_idx, s, budget - w);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_gather(K, V, out_idx, L, Hkv, d, n_max, out_K, out_V, nullptr, ctx->num_sms, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
 size_t chunkkv_lane_bytes(int L, int Hq, int Hkv, int d, int w, int c, int max_ctas) {
     if (w < 1 || c < 1 || L < w || max_ctas < 0) return 0;
     if (check_heads(L, Hq, Hkv, d, w) != CHUNKKV_OK) return 0;

@@ -69,8 +69,9 @@ cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, c
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
                             int num_sms, cudaStream_t stream);
 
+// tok_cap: at most this many tokens of the kept chunks are emitted (lowest positions first)
 cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int C, int k, int n_max,
-                          int32_t* out_idx, cudaStream_t stream);
+                          int32_t* out_idx, cudaStream_t stream, int tok_cap = 0x7fffffff);
 
 cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
                           int n_max, void* out_K, void* out_V, int32_t* idx_copy_or_null,

@@ -13,29 +13,29 @@ constexpr int kSelThreads = 512;
 template <int KPT>
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int k, int n_max,
-              int32_t* __restrict__ out_idx, int key_bytes) {
+              int32_t* __restrict__ out_idx, int key_bytes, int tok_cap) {
     __shared__ SelectSmem sm;
     extern __shared__ uint32_t key_buf[];
     const int h = blockIdx.x;
     const float* sc = scores + static_cast<size_t>(h) * C;
     int32_t* out = out_idx + static_cast<size_t>(h) * n_max;
     if constexpr (KPT > 0)
-        select_head_regs<KPT>(sc, nullptr, L, w, c, C, k, n_max, out, sm);
+        select_head_regs<KPT>(sc, nullptr, L, w, c, C, k, n_max, out, sm, tok_cap);
     else
-        select_head_rows(sc, nullptr, L, w, c, C, k, n_max, out, sm, key_bytes > 0 ? key_buf : nullptr);
+        select_head_rows(sc, nullptr, L, w, c, C, k, n_max, out, sm, key_bytes > 0 ? key_buf : nullptr, tok_cap);
 }
 
 }  // namespace
 
 cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int C, int k, int n_max,
-                          int32_t* out_idx, cudaStream_t stream) {
+                          int32_t* out_idx, cudaStream_t stream, int tok_cap) {
     // a few keys per thread: registers (the fewest that hold every key)
     if (C <= kSelThreads * 4) {
-        select_kernel<4><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx, 0);
+        select_kernel<4><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx, 0, tok_cap);
         return cudaGetLastError();
     }
     if (C <= kSelThreads * 8) {
-        select_kernel<8><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx, 0);
+        select_kernel<8><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx, 0, tok_cap);
         return cudaGetLastError();
     }
     // more: the keys of a head live in dynamic shared memory if they fit beside the static scratch
@@ -52,7 +52,7 @@ cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int
         else
             cudaGetLastError();
     }
-    select_kernel<0><<<Hkv, kSelThreads, key_bytes, stream>>>(scores, L, w, c, C, k, n_max, out_idx, key_bytes);
+    select_kernel<0><<<Hkv, kSelThreads, key_bytes, stream>>>(scores, L, w, c, C, k, n_max, out_idx, key_bytes, tok_cap);
     return cudaGetLastError();
 }
 

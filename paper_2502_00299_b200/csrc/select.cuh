@@ -53,7 +53,8 @@ __device__ __forceinline__ uint32_t select_order_key(float x) {
 // sc2 != NULL: the head's scores are sc[ch] + sc2[ch] (a KV head scored as two heads of half the rows).
 template <int KPT>
 __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, const float* __restrict__ sc2, int L, int w, int c,
-                                            int C, int k, int n_max, int32_t* __restrict__ out, SelectSmem& sm) {
+                                            int C, int k, int n_max, int32_t* __restrict__ out, SelectSmem& sm,
+                                            int tok_cap = 0x7fffffff) {
     auto score_at = [&](int ch) { return sc2 != nullptr ? sc[ch] + sc2[ch] : sc[ch]; };
     const int P = L - w;
     const int nt = blockDim.x, nwarps = nt >> 5;
@@ -200,7 +201,8 @@ __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, c
                 else {
                     const int j0 = ch * c, len = min(c, P - j0);
                     int32_t* dst = out + static_cast<size_t>(rank) * c;
-                    for (int t = 0; t < len; ++t) dst[t] = j0 + t;
+                    for (int t = 0; t < len; ++t)
+                        if (rank * c + t < tok_cap) dst[t] = j0 + t;
                 }
                 if (ch == C - 1) sm.last_kept = 1;
             }
@@ -218,7 +220,9 @@ __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, c
     __syncthreads();
     // Every kept chunk is full except possibly chunk C-1, which can only be the last kept one.
     const int tail = (C > 0) ? (P - (C - 1) * c) : 0;
-    const int n_tok = kk * c - ((sm.last_kept && kk > 0) ? (c - tail) : 0);
+    // tok_cap: at most this many tokens of the kept chunks are emitted, lowest positions first
+    // (Algorithm 1 keeps the first L_max - w selected tokens); no cap by default
+    const int n_tok = min(kk * c - ((sm.last_kept && kk > 0) ? (c - tail) : 0), tok_cap);
     if (stage_sel)
         for (int n = tid; n < n_tok; n += nt) {
             const int rank = n / c;
@@ -235,7 +239,8 @@ __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, c
 // NULL: keys are then recomputed from the scores on every use. sc2 != NULL: the head's scores are sc[ch] + sc2[ch] (a KV head scored as two
 // heads of half the rows).
 __device__ __forceinline__ void select_head_rows(const float* sc, const float* sc2, int L, int w, int c, int C, int k,
-                                            int n_max, int32_t* __restrict__ out, SelectSmem& sm, uint32_t* kbuf) {
+                                            int n_max, int32_t* __restrict__ out, SelectSmem& sm, uint32_t* kbuf,
+                                            int tok_cap = 0x7fffffff) {
     auto score_at = [&](int ch) { return sc2 != nullptr ? __ldcg(sc + ch) + __ldcg(sc2 + ch) : __ldcg(sc + ch); };
     constexpr unsigned kFull = 0xffffffffu;
     const int P = L - w;
@@ -401,7 +406,8 @@ __device__ __forceinline__ void select_head_rows(const float* sc, const float* s
                 else {
                     const int j0 = ch * c, len = min(c, P - j0);
                     int32_t* dst = out + static_cast<size_t>(rank) * c;
-                    for (int t = 0; t < len; ++t) dst[t] = j0 + t;
+                    for (int t = 0; t < len; ++t)
+                        if (rank * c + t < tok_cap) dst[t] = j0 + t;
                 }
                 if (ch == C - 1) sm.last_kept = 1;
             }
@@ -412,7 +418,9 @@ __device__ __forceinline__ void select_head_rows(const float* sc, const float* s
     __syncthreads();
     // Every kept chunk is full except possibly chunk C-1, which can only be the last kept one.
     const int tail = (C > 0) ? (P - (C - 1) * c) : 0;
-    const int n_tok = kk * c - ((sm.last_kept && kk > 0) ? (c - tail) : 0);
+    // tok_cap: at most this many tokens of the kept chunks are emitted, lowest positions first
+    // (Algorithm 1 keeps the first L_max - w selected tokens); no cap by default
+    const int n_tok = min(kk * c - ((sm.last_kept && kk > 0) ? (c - tail) : 0), tok_cap);
     if (stage_sel)
         for (int n = tid; n < n_tok; n += nt) {
             const int rank = n / c;

@@ -484,3 +484,51 @@ def test_compress_layer_at_the_largest_supported_length(ck):
     oK, oV, idx = _run_layer(ck, x, wl)
     _check_layer(x, wl, oK, oV, idx)
 
+
+
+# ------------------------------------------------------------------------------ Algorithm 1's budget rule
+@pytest.mark.parametrize("L,w,c,budget,Hkv", [
+    (26, 4, 5, 12, 1), (26, 4, 5, 14, 1), (2048, 16, 10, 256, 2), (1003, 8, 10, 203, 3), (500, 4, 7, 150, 2),
+    (26, 4, 5, 1000, 1), (26, 4, 5, 4, 1), (9000, 32, 1, 32 + 777, 2), (40000, 32, 3, 5000, 2),
+    (60000, 16, 1, 50000, 1),          # more than 4096 kept chunks: positions written without staging
+])
+def test_select_alg1_bit_exact_on_given_scores(ck, L, w, c, budget, Hkv):
+    rng = np.random.default_rng(L * 5 + budget)
+    C = ora.num_chunks(L, w, c)
+    s = rng.random((Hkv, max(C, 1))).astype(np.float32)[:, :C]
+    s[0, C - 1] = 2.0                              # the clipped last chunk is selected in head 0
+    idx = ck.select_alg1(torch.from_numpy(np.ascontiguousarray(s)).cuda(), L, w, c, budget).cpu().numpy()
+    assert ck.out_len_alg1(L, w, c, budget) == ora.out_len_alg1(L, w, c, budget) == idx.shape[1]
+    assert np.array_equal(idx, ora.select_alg1(s.astype(np.float64), L, w, c, budget))
+
+
+def test_budget_from_ratio_matches_oracle(ck):
+    for L, r in ((32768, 0.10), (32768, 0.2), (131072, 0.3), (1000, 0.0), (1000, 1.0), (777, 0.333)):
+        assert ck.budget_from_ratio(L, r) == ora.budget_from_ratio(L, r)
+    with pytest.raises(ck.ChunkKVError):
+        ck.budget_from_ratio(100, 1.5)
+
+
+@pytest.mark.parametrize("cfg,L,ratio", [(1, 2048, 0.125), (2, 6000, 0.10), (4, 9000, 0.2)])
+def test_compress_layer_alg1_matches_oracle(ck, cfg, L, ratio):
+    budget = ora.budget_from_ratio(L, ratio)
+    wl = scaled(CONFIGS[cfg], L=L, budget=budget)
+    x = make_layer(wl)
+    oK, oV, idx = ck.compress_layer_alg1(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V), wl.Hq, wl.w, wl.c, budget)
+    assert ck.device_status() == 0
+    ref = ora.compress_layer_alg1(x.q_obs, x.K, x.V, wl.Hq, wl.Hkv, wl.w, wl.c, budget)
+    idx_np = idx.cpu().numpy()
+    assert idx_np.shape == ref["idx"].shape
+    s = ref["chunk_scores"]
+    k = ora.num_kept_chunks_alg1(L, wl.w, wl.c, budget)
+    for h in range(wl.Hkv):
+        if not np.array_equal(idx_np[h], ref["idx"][h]):
+            # swaps only among chunks within 1e-4 (relative) of the k-th oracle score
+            got = set((idx_np[h][idx_np[h] >= 0][:-wl.w] // wl.c).tolist())
+            want = set(ora.select_chunks(s[h], k).tolist())
+            kth = np.sort(s[h])[::-1][k - 1]
+            assert all(abs(s[h][ch] - kth) <= 1e-4 * kth for ch in got ^ want)
+    gK, gV = ora.gather(x.K, x.V, idx_np)
+    assert np.array_equal(bits_of(oK), gK) and np.array_equal(bits_of(oV), gV)
+    n_kept = (idx_np >= 0).sum(axis=1)
+    assert np.all(n_kept <= max(budget, wl.w)) and np.all(idx_np[np.arange(wl.Hkv), n_kept - 1] == L - 1)
