@@ -42,8 +42,8 @@ FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one cfg2 layer through a lane, from ncu captures
-# of both launches (layer kernel + row gather): 8 CTAs 69.6 + 13.5 MB, 18 CTAs 69.4 + 13.5 MB
-TRAFFIC_BYTES_PER_LAYER = {8: 83.1e6, 18: 82.9e6}
+# of both launches (layer kernel + row gather): 8 CTAs 69.6 + 13.5 MB, 18 CTAs 69.5 + 13.5 MB
+TRAFFIC_BYTES_PER_LAYER = {8: 83.1e6, 18: 83.0e6}
 
 
 def parse_args():
