@@ -32,11 +32,12 @@
  *     c >= 1; budget >= w; Hkv * L < 2^23 (8 M keys per layer).
  *   - Return value: CHUNKKV_OK (0) or a negative CHUNKKV_E* code. Arguments are checked on
  *     the host before anything is launched; nothing is thrown and nothing aborts.
- *   - Scratch memory: scoring needs device scratch (chunkkv_workspace_bytes). Either hand the
- *     library a buffer with chunkkv_set_workspace, or let it allocate one on first use (one
- *     cudaMalloc per device, grown when a larger problem arrives; growing synchronises the
- *     device). Calls that use the scratch of one device must be ordered on the GPU (same
- *     stream, or otherwise serialised): concurrent calls would share it.
+ *   - Scratch memory: scoring needs device scratch of chunkkv_workspace_bytes(...) bytes. The
+ *     library never allocates and never frees: the caller hands it a buffer once with
+ *     chunkkv_set_workspace (a set-up call), and every entry point that scores returns
+ *     CHUNKKV_ENOWORKSPACE while no buffer, or too small a buffer, is set. Calls that use the
+ *     scratch of one device must be ordered on the GPU (same stream, or otherwise serialised):
+ *     concurrent calls would share it. Lanes and pipes (below) take their scratch per object.
  */
 #ifndef CHUNKKV_H_
 #define CHUNKKV_H_
@@ -58,7 +59,7 @@ extern "C" {
 #define CHUNKKV_EINVAL_NULL    -1  /* a required pointer is NULL */
 #define CHUNKKV_EINVAL_SHAPE   -2  /* a size violates the limits above */
 #define CHUNKKV_EINVAL_ALIGN   -3  /* a tensor pointer is not 16-byte aligned */
-#define CHUNKKV_ENOWORKSPACE   -4  /* caller-provided workspace too small / allocation failed */
+#define CHUNKKV_ENOWORKSPACE   -4  /* no workspace set (chunkkv_set_workspace), or too small for the shape */
 #define CHUNKKV_ECUDA          -5  /* a CUDA runtime or driver call failed (see chunkkv_last_cuda_error) */
 #define CHUNKKV_EDEVICE        -6  /* a kernel gave up on a bounded wait (see chunkkv_device_status) */
 #define CHUNKKV_ETOOLARGE      -7  /* the problem needs more scratch than a fixed-size variant provides */
@@ -82,10 +83,11 @@ CHUNKKV_API int chunkkv_out_len(int L, int w, int c, int budget);
 CHUNKKV_API size_t chunkkv_workspace_bytes(int L, int Hq, int Hkv, int d, int w, int c);
 
 /*
- * Use caller-owned device memory (256-byte aligned, on the current device) as scratch for all
- * later calls on this device. Its first 256 bytes hold the library's device status word and are
- * cleared by this call (which synchronises the device). Passing (NULL, 0) returns to
- * library-managed scratch. The caller keeps ownership.
+ * Set-up: use caller-owned device memory (256-byte aligned, on the current device) as scratch for
+ * all later calls on this device. Its first 256 bytes hold the library's device status word and
+ * hand-over counters and are cleared by this call. This is the one call that synchronises the
+ * device (work queued earlier may still be using the previous buffer). Passing (NULL, 0) detaches
+ * the buffer. The caller keeps ownership and must keep the buffer alive while calls may use it.
  */
 CHUNKKV_API int chunkkv_set_workspace(void* dev_ptr, size_t bytes);
 
@@ -113,25 +115,34 @@ CHUNKKV_API int chunkkv_score(const void* q_obs, const void* K, int L, int Hq, i
  * deployment convenience, not a step of the method.)
  *
  * Who needs it: serving processes that hand every free byte of HBM to their own cache pool at
- * start-up, so that a later cudaMalloc either fails or eats into memory they have promised
- * elsewhere; and callers inside latency-critical loops that cannot accept the device-wide
- * synchronisation cudaMalloc / cudaFree imply. This entry point calls no cudaMalloc, cudaFree or
- * any other allocating routine, and ignores chunkkv_set_workspace: its scratch is a fixed
- * 8 MiB array that lives in the library's device image (every GPU that loads the library holds
- * those 8 MiB until the process exits).
+ * start-up and therefore have no buffer left to pass to chunkkv_set_workspace later, and callers
+ * that cannot reach an allocator at all (a plug-in that only sees raw pointers). This entry point
+ * calls no cudaMalloc, cudaFree or any other allocating routine, and ignores
+ * chunkkv_set_workspace: its scratch is a fixed 8 MiB array that lives in the library's device
+ * image (every GPU on which this entry point has been called holds those 8 MiB until the process
+ * exits).
  *
  * Same arguments, layouts and result as chunkkv_score without the token-score output:
  * out_chunk_scores [Hkv, C] f32. Shapes whose chunkkv_workspace_bytes(L, Hq, Hkv, d, w, c)
- * exceeds 8 MiB are rejected with CHUNKKV_ETOOLARGE and nothing is launched.
+ * exceeds 8 MiB are rejected with CHUNKKV_ETOOLARGE, shapes outside the library's limits with
+ * CHUNKKV_EINVAL_SHAPE, and nothing is launched.
  *
  * The first call on each device looks up the device address of the array (with that device
- * current); make that first call outside any stream capture. All calls on a device share the one
- * array, which keeps whatever the previous call left in it: the library clears the status word it
- * needs zeroed on every call, and calls that overlap on the GPU (different streams, no ordering)
- * race on the scratch - order them.
+ * current). The CUDA runtime loads device code lazily, so that first call is also the moment the
+ * array takes its 8 MiB: make one warm-up call per device at start-up, before the process gives
+ * its free memory away and outside any stream capture. Later calls leave the amount of free
+ * device memory unchanged. All calls on a device share the one array, which keeps whatever the
+ * previous call left in it; nothing in it needs clearing between calls, and calls that overlap on
+ * the GPU (different streams, no ordering) race on it - order them.
+ *
+ * chunkkv_score_noalloc_status synchronises `stream`, then reports whether a kernel launched by
+ * chunkkv_score_noalloc on the current device abandoned a bounded wait since the last status call
+ * (CHUNKKV_EDEVICE; out_chunk_scores of that call are then incomplete) and clears the mark.
+ * chunkkv_device_status does not cover this entry point.
  */
 CHUNKKV_API int chunkkv_score_noalloc(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d,
                                       int w, int c, float* out_chunk_scores, void* stream);
+CHUNKKV_API int chunkkv_score_noalloc_status(void* stream);
 
 /*
  * Step "top-k chunk selection" and the kept-index list (Algorithm 3: Top-K, selection mask,

@@ -9,7 +9,7 @@ so that the build module itself can be imported before the library exists.
 _EXPORTS = (
     "ChunkKVError", "LIB_PATH", "Lane", "Pipe", "budget_from_ratio", "compress_layer", "compress_layer_alg1",
     "compress_layer_host", "compress_model", "out_len_alg1", "select_alg1",
-    "device_status", "gather", "jaccard", "lib", "num_chunks", "num_kept_chunks", "out_len", "profile_enable",
+    "device_status", "ensure_workspace", "gather", "jaccard", "lib", "num_chunks", "num_kept_chunks", "out_len", "profile_enable",
     "profile_read", "score", "select", "set_workspace", "strerror", "workspace_bytes",
 )
 __all__ = list(_EXPORTS)

@@ -72,6 +72,8 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_jaccard.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
     L.chunkkv_score_noalloc.restype = i32
     L.chunkkv_score_noalloc.argtypes = [vp, vp] + [i32] * 6 + [vp, vp]
+    L.chunkkv_score_noalloc_status.restype = i32
+    L.chunkkv_score_noalloc_status.argtypes = [vp]
     L.chunkkv_budget_from_ratio.restype = i32
     L.chunkkv_budget_from_ratio.argtypes = [i32, ctypes.c_double]
     L.chunkkv_num_kept_chunks_alg1.restype = i32
@@ -138,13 +140,34 @@ def workspace_bytes(L: int, Hq: int, Hkv: int, d: int, w: int, c: int) -> int:
     return int(lib.chunkkv_workspace_bytes(L, Hq, Hkv, d, w, c))
 
 
+_workspaces = {}      # device index -> uint8 tensor currently handed to the library
+
+
 def set_workspace(buf: Optional[torch.Tensor]) -> None:
-    """Hand the library a caller-owned scratch buffer (uint8 CUDA tensor), or None to undo."""
+    """Hand the library a caller-owned scratch buffer (uint8 CUDA tensor on the current device), or
+    None to detach it. The library itself never allocates; see ensure_workspace."""
+    dev = torch.cuda.current_device()
     if buf is None:
         _check(lib.chunkkv_set_workspace(None, 0), "chunkkv_set_workspace")
+        _workspaces.pop(dev, None)
     else:
         _check(lib.chunkkv_set_workspace(buf.data_ptr(), buf.numel() * buf.element_size()),
                "chunkkv_set_workspace")
+        _workspaces[dev] = buf
+
+
+def ensure_workspace(L: int, Hq: int, Hkv: int, d: int, w: int, c: int) -> None:
+    """Make sure the current device's scratch covers this shape: the device memory is a torch
+    tensor allocated here (grown when a larger shape arrives) and handed over with
+    chunkkv_set_workspace. A buffer given through set_workspace is kept if it is large enough."""
+    need = workspace_bytes(L, Hq, Hkv, d, w, c)
+    if need == 0:
+        raise ChunkKVError(-2, "chunkkv_workspace_bytes")
+    dev = torch.cuda.current_device()
+    cur = _workspaces.get(dev)
+    if cur is not None and cur.numel() >= need:
+        return
+    set_workspace(torch.empty(need + (need >> 2), dtype=torch.uint8, device=torch.device("cuda", dev)))
 
 
 def device_status(stream: Optional[torch.cuda.Stream] = None) -> int:
@@ -159,6 +182,9 @@ def score(q_obs: torch.Tensor, K: torch.Tensor, w: int, c: int, want_token_score
     Hq, d = q_obs.shape[0], q_obs.shape[2]
     Hkv, L = K.shape[0], K.shape[1]
     C = num_chunks(L, w, c)
+    ensure_workspace(L, Hq, Hkv, d, w, c)
+    if want_token_scores:
+        ensure_workspace(L, Hq, Hkv, d, w, 1)
     cs = torch.empty((Hkv, C), dtype=torch.float32, device=K.device)
     ts = torch.empty((Hkv, L - w), dtype=torch.float32, device=K.device) if want_token_scores else None
     _check(lib.chunkkv_score(q_obs.data_ptr(), K.data_ptr(), L, Hq, Hkv, d, w, c, _ptr(ts),
@@ -202,14 +228,19 @@ def select_alg1(chunk_scores: torch.Tensor, L: int, w: int, c: int, budget: int,
 
 
 def compress_layer_alg1(q_obs: torch.Tensor, K: torch.Tensor, V: torch.Tensor, Hq: int, w: int, c: int, budget: int,
+                        out_K: Optional[torch.Tensor] = None, out_V: Optional[torch.Tensor] = None,
+                        out_idx: Optional[torch.Tensor] = None,
                         stream: Optional[torch.cuda.Stream] = None) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
     """out_K, out_V [Hkv, n_max, d], idx [Hkv, n_max] for one layer under Algorithm 1's budget rule."""
     _dev(q_obs, torch.bfloat16, "q_obs"); _dev(K, torch.bfloat16, "K"); _dev(V, torch.bfloat16, "V")
     Hkv, L, d = K.shape
     n_max = out_len_alg1(L, w, c, budget)
-    out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=K.device)
-    out_V = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=K.device)
-    idx = torch.empty((Hkv, n_max), dtype=torch.int32, device=K.device)
+    ensure_workspace(L, Hq, Hkv, d, w, c)
+    if out_K is None:
+        out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=K.device)
+    if out_V is None:
+        out_V = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=K.device)
+    idx = out_idx if out_idx is not None else torch.empty((Hkv, n_max), dtype=torch.int32, device=K.device)
     _check(lib.chunkkv_compress_layer_alg1(q_obs.data_ptr(), K.data_ptr(), V.data_ptr(), L, Hq, Hkv, d, w, c, budget,
                                            out_K.data_ptr(), out_V.data_ptr(), idx.data_ptr(), _stream(stream)),
            "chunkkv_compress_layer_alg1")
@@ -247,6 +278,8 @@ def compress_layer(q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tens
     Hkv, L, d = K.shape
     n_max = out_len(L, w, c, budget)
     dev = K.device
+    if reuse_idx is None:
+        ensure_workspace(L, Hq, Hkv, d, w, c)
     if out_K is None:
         out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
     if out_V is None:
@@ -280,12 +313,15 @@ class Lane:
     up to at most the number of SMs."""
 
     def __init__(self, L: int, Hq: int, Hkv: int, d: int, w: int, c: int, max_ctas: int = 0,
-                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None,
+                 buf: Optional[torch.Tensor] = None):
         self.max_ctas = int(max_ctas)
         self.bytes = int(lib.chunkkv_lane_bytes(L, Hq, Hkv, d, w, c, self.max_ctas))
         if self.bytes == 0:
             raise ChunkKVError(-2, "chunkkv_lane_bytes")
-        self.buf = torch.empty(self.bytes, dtype=torch.uint8, device=device or "cuda")
+        if buf is not None and buf.numel() * buf.element_size() < self.bytes:
+            raise ValueError("the given scratch tensor is smaller than chunkkv_lane_bytes")
+        self.buf = buf if buf is not None else torch.empty(self.bytes, dtype=torch.uint8, device=device or "cuda")
         self.stream = stream if stream is not None else torch.cuda.Stream(device=self.buf.device)
         _check(lib.chunkkv_lane_init(self.buf.data_ptr(), self.bytes, self.stream.cuda_stream or None),
                "chunkkv_lane_init")
@@ -321,12 +357,15 @@ class Pipe:
     `stream`, everything after scoring on the pipe's own stream. Call join() before using outputs."""
 
     def __init__(self, L: int, Hq: int, Hkv: int, d: int, w: int, c: int, max_ctas: int = 0,
-                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None,
+                 buf: Optional[torch.Tensor] = None):
         self.max_ctas = int(max_ctas)
         self.bytes = int(lib.chunkkv_pipe_bytes(L, Hq, Hkv, d, w, c, self.max_ctas))
         if self.bytes == 0:
             raise ChunkKVError(-2, "chunkkv_pipe_bytes")
-        self.buf = torch.empty(self.bytes, dtype=torch.uint8, device=device or "cuda")
+        if buf is not None and buf.numel() * buf.element_size() < self.bytes:
+            raise ValueError("the given scratch tensor is smaller than chunkkv_pipe_bytes")
+        self.buf = buf if buf is not None else torch.empty(self.bytes, dtype=torch.uint8, device=device or "cuda")
         self.stream = stream if stream is not None else torch.cuda.Stream(device=self.buf.device)
         handle = ctypes.c_void_p()
         _check(lib.chunkkv_pipe_open(self.buf.data_ptr(), self.bytes, self.max_ctas, ctypes.byref(handle)),
@@ -379,6 +418,7 @@ def compress_layer_host(host_q: torch.Tensor, host_K: torch.Tensor, host_V: torc
     Hkv, L, d = host_K.shape
     dq, dK, dV, doK, doV, dI = dev_bufs
     hK, hV, hI = host_outs
+    ensure_workspace(L, Hq, Hkv, d, w, c)
     _check(lib.chunkkv_compress_layer_host(
         host_q.data_ptr(), host_K.data_ptr(), host_V.data_ptr(), L, Hq, Hkv, d, w, c, budget,
         dq.data_ptr(), dK.data_ptr(), dV.data_ptr(), doK.data_ptr(), doV.data_ptr(), dI.data_ptr(),

@@ -5,7 +5,6 @@
 #include "internal.h"
 
 #include <math.h>
-#include <stdlib.h>
 #include <mutex>
 #include <vector>
 
@@ -32,10 +31,8 @@ struct DeviceCtx {
     bool init = false;
     int num_sms = 0;
     int smem_optin = 0;
-    void* ws = nullptr;        // current scratch (header + payload)
+    void* ws = nullptr;        // scratch handed over with chunkkv_set_workspace (header + payload)
     size_t ws_bytes = 0;
-    bool ws_owned = false;     // allocated by the library
-    bool ws_user = false;      // provided by chunkkv_set_workspace
     std::vector<ProfileRec> recs;
     float prof_ms[CHUNKKV_PROFILE_SLOTS] = {0, 0, 0, 0};
     int prof_n[CHUNKKV_PROFILE_SLOTS] = {0, 0, 0, 0};
@@ -58,9 +55,6 @@ struct Pipe {
 DeviceCtx g_ctx[kMaxDevices];
 EncodeTiledFn g_encode = nullptr;
 bool g_profile = false;
-// CHUNKKV_UNFUSED=1 makes chunkkv_compress_layer use the separate score / finalize / select /
-// gather kernels instead of the single fused launch (for comparison and debugging).
-const bool g_unfused = [] { const char* v = getenv("CHUNKKV_UNFUSED"); return v != nullptr && v[0] == '1'; }();
 
 int cuda_fail(cudaError_t e) {
     g_last_cuda_error = static_cast<int>(e);
@@ -96,29 +90,11 @@ int get_ctx(DeviceCtx** out) {
 // Shared-memory budget for the dynamic part of the score kernel (static control block excluded).
 int smem_budget(const DeviceCtx& c) { return c.smem_optin - 1024; }
 
+// The library never allocates: the scratch is whatever chunkkv_set_workspace was given.
 int ensure_workspace(DeviceCtx& c, size_t payload_bytes) {
     const size_t need = kHeaderBytes + payload_bytes;
     if (c.ws != nullptr && c.ws_bytes >= need) return CHUNKKV_OK;
-    if (c.ws_user) return CHUNKKV_ENOWORKSPACE;
-    cudaError_t e = cudaDeviceSynchronize();
-    if (e != cudaSuccess) return cuda_fail(e);
-    if (c.ws_owned && c.ws != nullptr) cudaFree(c.ws);
-    c.ws = nullptr;
-    c.ws_bytes = 0;
-    size_t bytes = need + (need >> 2);
-    bytes = (bytes + 255) & ~static_cast<size_t>(255);
-    e = cudaMalloc(&c.ws, bytes);
-    if (e != cudaSuccess) {
-        c.ws = nullptr;
-        g_last_cuda_error = static_cast<int>(e);
-        cudaGetLastError();
-        return CHUNKKV_ENOWORKSPACE;
-    }
-    e = cudaMemset(c.ws, 0, kHeaderBytes);
-    if (e != cudaSuccess) return cuda_fail(e);
-    c.ws_bytes = bytes;
-    c.ws_owned = true;
-    return CHUNKKV_OK;
+    return CHUNKKV_ENOWORKSPACE;
 }
 
 // How the R = w * Hq / Hkv window rows of a KV head are scored. Rows are independent (each has its
@@ -142,17 +118,6 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 int check_sizes(int L, int w, int c, int budget) {
     if (w < 1 || c < 1 || L < w || budget < w) return CHUNKKV_EINVAL_SHAPE;
-    return CHUNKKV_OK;
-}
-
-int check_heads(int L, int Hq, int Hkv, int d, int w) {
-    if (Hkv < 1 || Hq < Hkv || Hq % Hkv != 0) return CHUNKKV_EINVAL_SHAPE;
-    if (d != 64 && d != 128) return CHUNKKV_EINVAL_SHAPE;
-    const long long R = static_cast<long long>(w) * (Hq / Hkv);
-    if (R > 256) return CHUNKKV_EINVAL_SHAPE;
-    if (static_cast<long long>(Hkv) * L * d >= (1LL << 40)) return CHUNKKV_EINVAL_SHAPE;
-    if (Hkv > 65535) return CHUNKKV_EINVAL_SHAPE;
-    if (static_cast<long long>(Hkv) * L >= (1LL << 23)) return CHUNKKV_EINVAL_SHAPE;   // 32-bit row arithmetic in the kernels
     return CHUNKKV_OK;
 }
 
@@ -259,6 +224,17 @@ size_t scratch_floats_for(const DeviceCtx& ctx, int L, int R, int Hkv, int d, in
 
 namespace chunkkv {
 
+int check_heads(int L, int Hq, int Hkv, int d, int w) {
+    if (Hkv < 1 || Hq < Hkv || Hq % Hkv != 0) return CHUNKKV_EINVAL_SHAPE;
+    if (d != 64 && d != 128) return CHUNKKV_EINVAL_SHAPE;
+    const long long R = static_cast<long long>(w) * (Hq / Hkv);
+    if (R > 256) return CHUNKKV_EINVAL_SHAPE;
+    if (static_cast<long long>(Hkv) * L * d >= (1LL << 40)) return CHUNKKV_EINVAL_SHAPE;
+    if (Hkv > 65535) return CHUNKKV_EINVAL_SHAPE;
+    if (static_cast<long long>(Hkv) * L >= (1LL << 23)) return CHUNKKV_EINVAL_SHAPE;   // 32-bit row arithmetic in the kernels
+    return CHUNKKV_OK;
+}
+
 // Scoring into caller-supplied scratch (256-byte header + payload). Used by the fixed-scratch
 // entry point; allocates nothing and records no profiling events.
 int score_with_scratch(const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w, int c,
@@ -307,7 +283,7 @@ const char* chunkkv_strerror(int status) {
         case CHUNKKV_EINVAL_NULL: return "a required pointer is NULL";
         case CHUNKKV_EINVAL_SHAPE: return "a size is outside the supported range";
         case CHUNKKV_EINVAL_ALIGN: return "a tensor pointer is not 16-byte aligned";
-        case CHUNKKV_ENOWORKSPACE: return "scratch workspace too small or could not be allocated";
+        case CHUNKKV_ENOWORKSPACE: return "no scratch workspace was set, or it is too small for this shape";
         case CHUNKKV_ECUDA: return "a CUDA call failed";
         case CHUNKKV_EDEVICE: return "a kernel abandoned a bounded wait";
         case CHUNKKV_ETOOLARGE: return "the problem needs more scratch than the fixed-size variant provides";
@@ -357,23 +333,22 @@ int chunkkv_set_workspace(void* dev_ptr, size_t bytes) {
     DeviceCtx* ctx;
     int st = get_ctx(&ctx);
     if (st != CHUNKKV_OK) return st;
+    // set-up call: work queued earlier may still use the previous scratch
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return cuda_fail(e);
     if (dev_ptr == nullptr) {
-        if (ctx->ws_user) { ctx->ws = nullptr; ctx->ws_bytes = 0; ctx->ws_user = false; }
+        ctx->ws = nullptr;
+        ctx->ws_bytes = 0;
         return CHUNKKV_OK;
     }
     if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return CHUNKKV_EINVAL_ALIGN;
     if (bytes < kHeaderBytes) return CHUNKKV_ENOWORKSPACE;
-    if (ctx->ws_owned && ctx->ws != nullptr) cudaFree(ctx->ws);
-    ctx->ws_owned = false;
     e = cudaMemset(dev_ptr, 0, kHeaderBytes);
     if (e != cudaSuccess) return cuda_fail(e);
     e = cudaDeviceSynchronize();
     if (e != cudaSuccess) return cuda_fail(e);
     ctx->ws = dev_ptr;
     ctx->ws_bytes = bytes;
-    ctx->ws_user = true;
     return CHUNKKV_OK;
 }
 
@@ -508,7 +483,7 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
         // kernels' scratch after them
         const size_t cs_floats = round64(static_cast<size_t>(sh.Hs) * C);
         ScorePlan plan;
-        if ((lane != nullptr || !g_unfused) && make_score_plan(L, R, sh.Hs, d, c, ctas, smem_budget(*ctx), true, &plan)) {
+        if (make_score_plan(L, R, sh.Hs, d, c, ctas, smem_budget(*ctx), true, &plan)) {
             // One cooperative launch for the whole layer.
             const size_t need = (cs_floats + score_scratch_floats(plan, sh.Hs, R)) * sizeof(float);
             char* base;

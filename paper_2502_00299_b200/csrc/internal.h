@@ -34,6 +34,9 @@ struct ScoreArgs {
     int* status;          // device status word
 };
 
+// Head-count and size limits shared by every entry point that scores (CHUNKKV_OK or CHUNKKV_EINVAL_SHAPE).
+int check_heads(int L, int Hq, int Hkv, int d, int w);
+
 // Chooses kernel variant and tile geometry for a shape. Returns false if unsupported.
 // full_grid: launch one CTA per SM even if there are fewer tiles (the fused layer kernel wants
 // every SM for its later phases).

@@ -81,3 +81,30 @@ def assert_gather_exact(out_K: np.ndarray, out_V: np.ndarray, idx: np.ndarray, K
     ref_K, ref_V = ora.gather(K, V, idx)
     assert np.array_equal(out_K, ref_K), "out_K differs from K[idx]"
     assert np.array_equal(out_V, ref_V), "out_V differs from V[idx]"
+
+
+class Guarded:
+    """A CUDA tensor carved out of a larger allocation whose margins hold a known byte pattern:
+    `check()` fails if anything wrote before the first or after the last element. Stands in for a
+    memory checker on the buffers the library writes (outputs, indices, scores, scratch)."""
+    PATTERN = 0xA5
+
+    def __init__(self, shape, dtype, margin: int = 4096):
+        assert margin % 256 == 0
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.n, self.margin = n, margin
+        body = (n + 255) // 256 * 256
+        self.raw = torch.full((margin + body + margin,), self.PATTERN, dtype=torch.uint8, device="cuda")
+        self.t = self.raw[margin:margin + n].view(dtype).view(shape)
+
+    def check(self, what: str = "buffer") -> None:
+        lo = self.raw[:self.margin]
+        hi = self.raw[self.margin + self.n:]
+        assert bool((lo == self.PATTERN).all()), f"{what}: bytes before the buffer were overwritten"
+        assert bool((hi == self.PATTERN).all()), f"{what}: bytes after the buffer were overwritten"
+
+
+def guarded_outputs(Hkv: int, n_max: int, d: int):
+    """out_K, out_V, out_idx with guard margins (Guarded objects)."""
+    return (Guarded((Hkv, n_max, d), torch.bfloat16), Guarded((Hkv, n_max, d), torch.bfloat16),
+            Guarded((Hkv, n_max), torch.int32))

@@ -63,6 +63,10 @@ def test_invalid_sizes_are_rejected_on_the_host(ck):
                                       None, None) == -1        # sizes accepted, then the NULL pointers are seen
     assert lib.chunkkv_compress_layer(None, None, None, 1 << 20, 8, 8, 128, 16, 10, 256, None, None, None,
                                       None, None) == -2
+    # the fixed-scratch scoring call applies the same limits (8 heads of 2^20 keys is one key too many)
+    assert lib.chunkkv_score_noalloc(16, 16, 1 << 20, 8, 8, 128, 1, 64, 16, None) == -2
+    assert lib.chunkkv_score_noalloc(16, 16, 1024, 8, 3, 128, 16, 10, 16, None) == -2
+    assert lib.chunkkv_score_noalloc(None, None, 1024, 8, 2, 128, 16, 10, None, None) == -1
     # the new entry points check their arguments the same way
     assert lib.chunkkv_jaccard(None, None, 2, 10, 10, None, None, None) == -1
     assert lib.chunkkv_jaccard(None, None, 0, 10, 10, None, None, None) == -2

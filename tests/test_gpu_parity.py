@@ -9,8 +9,8 @@ import pytest
 import torch
 
 from oracle import chunkkv_oracle as ora
-from tests.helpers import (assert_gather_exact, assert_scores_close, assert_selection_matches,
-                           bits_of, chunks_of_idx, rand_bits, to_dev)
+from tests.helpers import (Guarded, assert_gather_exact, assert_scores_close, assert_selection_matches,
+                           bits_of, chunks_of_idx, guarded_outputs, rand_bits, to_dev)
 from workloads import CONFIGS, iter_layers, make_layer, ragged_lengths, scaled
 
 pytestmark = pytest.mark.gpu
@@ -145,10 +145,14 @@ def test_score_is_deterministic(ck):
 
 # ------------------------------------------------------------------------------ whole layer
 def _run_layer(ck, x, wl, budget=None, L=None):
+    # outputs sit between guard margins: nothing may be written outside them
     budget = wl.budget if budget is None else budget
     q, K, V = to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)
-    oK, oV, idx = ck.compress_layer(q, K, V, wl.Hq, wl.w, wl.c, budget)
+    gK, gV, gI = guarded_outputs(K.shape[0], ck.out_len(K.shape[1], wl.w, wl.c, budget), K.shape[2])
+    oK, oV, idx = ck.compress_layer(q, K, V, wl.Hq, wl.w, wl.c, budget, out_K=gK.t, out_V=gV.t, out_idx=gI.t)
     _status_ok(ck)
+    for g, name in ((gK, "out_K"), (gV, "out_V"), (gI, "out_idx")):
+        g.check(name)
     return bits_of(oK), bits_of(oV), idx.cpu().numpy()
 
 
@@ -244,6 +248,47 @@ def test_ragged_batch_config5_scaled(ck):
         _check_layer(x, wl, oK, oV, idx)
 
 
+def test_config3_full_size_reuse_depth_2(ck):
+    # the 32K-token, 32-layer workload with reuse depth 2 at its real layer size, correlated layers
+    # (the first eight layers = four reuse groups: generating and checking all 32 would take minutes)
+    wl = CONFIGS[3]
+    layers = list(iter_layers(wl, 8))
+    dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in layers]
+    outs = ck.compress_model(dev, wl.Hq, wl.w, wl.c, wl.budget, n_reuse=wl.reuse_depth)
+    _status_ok(ck)
+    for l, (x, (oK, oV, idx)) in enumerate(zip(layers, outs)):
+        src = (l // wl.reuse_depth) * wl.reuse_depth
+        idx_np = idx.cpu().numpy()
+        if l == src:
+            _check_layer(x, wl, bits_of(oK), bits_of(oV), idx_np)          # selection vs the oracle, rows bit-exact
+        else:
+            assert np.array_equal(idx_np, outs[src][2].cpu().numpy())      # Algorithm 2: the source layer's indices
+            assert_gather_exact(bits_of(oK), bits_of(oV), idx_np, x.K, x.V)
+    # adjacent compute layers of the correlated inputs keep overlapping sets (a diagnostic, cf. the
+    # paper's index-similarity table; no threshold is part of the method)
+    ratio, _ = ck.jaccard(outs[0][2], outs[2][2])
+    assert 0.0 < float(ratio.min()) <= 1.0
+
+
+def test_config5_all_ragged_lengths_one_reuse_group(ck):
+    # the batched workload: all eight sequences at their real lengths (8192..65536 tokens, 64 query
+    # heads), one reuse group each (depth 3: one computed layer, two gather-only layers)
+    wl = CONFIGS[5]
+    lens = ragged_lengths(wl)
+    assert len(lens) == 8 and min(lens) >= 8192 and max(lens) <= 65536 and len(set(lens)) == 8
+    for seq, L in enumerate(lens):
+        layers = [make_layer(wl, layer=l, seq=seq, L=L) for l in range(wl.reuse_depth)]
+        dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in layers]
+        outs = ck.compress_model(dev, wl.Hq, wl.w, wl.c, wl.budget, n_reuse=wl.reuse_depth)
+        _status_ok(ck)
+        idx0 = outs[0][2].cpu().numpy()
+        _check_layer(layers[0], wl, bits_of(outs[0][0]), bits_of(outs[0][1]), idx0)
+        for x, (oK, oV, idx) in zip(layers[1:], outs[1:]):
+            assert np.array_equal(idx.cpu().numpy(), idx0)
+            assert_gather_exact(bits_of(oK), bits_of(oV), idx0, x.K, x.V)
+        del dev, outs
+
+
 def test_compress_layer_host_round_trip(ck):
     wl = scaled(CONFIGS[2], L=3000, budget=300)
     x = make_layer(wl)
@@ -261,21 +306,39 @@ def test_compress_layer_host_round_trip(ck):
     _check_layer(x, wl, bits_of(outs[0]), bits_of(outs[1]), outs[2].numpy())
 
 
-def test_caller_provided_workspace(ck):
+def test_scratch_is_caller_owned_and_never_overrun(ck):
+    # the library allocates nothing: without a workspace the scoring calls refuse; with one placed
+    # between guard margins they work and write nothing outside it
     wl = scaled(CONFIGS[2], L=2500, budget=250)
     x = make_layer(wl)
+    q, K, V = to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)
     need = ck.workspace_bytes(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c)
     assert need > 0
-    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
-    ck.set_workspace(small)
+    n_max = ck.out_len(wl.L, wl.w, wl.c, wl.budget)
+    gK, gV, gI = guarded_outputs(wl.Hkv, n_max, wl.d)
+    gS = Guarded((wl.Hkv, ck.num_chunks(wl.L, wl.w, wl.c)), torch.float32)
+    args = (q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, wl.budget, None,
+            gK.t.data_ptr(), gV.t.data_ptr(), gI.t.data_ptr(), None)
+    ck.set_workspace(None)
     try:
-        with pytest.raises(ck.ChunkKVError) as e:
-            _run_layer(ck, x, wl)
-        assert e.value.status == -4
-        buf = torch.empty(need, dtype=torch.uint8, device="cuda")
-        ck.set_workspace(buf)
-        oK, oV, idx = _run_layer(ck, x, wl)
-        _check_layer(x, wl, oK, oV, idx)
+        assert ck.lib.chunkkv_compress_layer(*args) == -4
+        assert ck.lib.chunkkv_score(q.data_ptr(), K.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, None,
+                                    gS.t.data_ptr(), None) == -4
+        small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+        ck.set_workspace(small)
+        assert ck.lib.chunkkv_compress_layer(*args) == -4
+        ws = Guarded((need,), torch.uint8)
+        ck.set_workspace(ws.t)
+        for _ in range(2):
+            assert ck.lib.chunkkv_compress_layer(*args) == 0
+            assert ck.lib.chunkkv_score(q.data_ptr(), K.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, None,
+                                        gS.t.data_ptr(), None) == 0
+        _status_ok(ck)
+        for g, name in ((ws, "workspace"), (gK, "out_K"), (gV, "out_V"), (gI, "out_idx"), (gS, "chunk scores")):
+            g.check(name)
+        _check_layer(x, wl, bits_of(gK.t), bits_of(gV.t), gI.t.cpu().numpy())
+        t = ora.token_scores(x.q_obs, x.K, wl.Hq, wl.Hkv, wl.w)
+        assert_scores_close(gS.t.cpu().numpy(), ora.chunk_scores(t, wl.c), wl.w * wl.Hq // wl.Hkv, wl.L, "chunk scores")
     finally:
         ck.set_workspace(None)
 
@@ -312,12 +375,16 @@ def test_lane_with_few_ctas_matches_oracle(ck, cfg, L, budget, ctas):
     # a lane with a small share of the SMs (rows gathered by the second launch), shapes with
     # d = 64, R = 256, c = 20, a ragged last chunk and a budget just above the window
     wl = scaled(CONFIGS[cfg], L=L, budget=budget)
-    lane = ck.Lane(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=ctas)
+    scratch = Guarded((ck.lib.chunkkv_lane_bytes(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, ctas),), torch.uint8)
+    lane = ck.Lane(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=ctas, buf=scratch.t)
     x = make_layer(wl)
     dev = (to_dev(x.q_obs), to_dev(x.K), to_dev(x.V))
+    gK, gV, gI = guarded_outputs(wl.Hkv, ck.out_len(wl.L, wl.w, wl.c, wl.budget), wl.d)
     for rep in range(2):
-        oK, oV, idx = lane.compress_layer(*dev, wl.Hq, wl.w, wl.c, wl.budget)
+        oK, oV, idx = lane.compress_layer(*dev, wl.Hq, wl.w, wl.c, wl.budget, out_K=gK.t, out_V=gV.t, out_idx=gI.t)
     assert lane.status() == 0
+    for g, name in ((scratch, "lane scratch"), (gK, "out_K"), (gV, "out_V"), (gI, "out_idx")):
+        g.check(name)
     _check_layer(x, wl, bits_of(oK), bits_of(oV), idx.cpu().numpy())
 
 
@@ -327,14 +394,21 @@ def test_pipe_overlapped_layers_match_oracle(ck, cfg, L, budget, ctas):
     # five layers through one pipe (scoring back to back, the rest on the pipe's own stream, two
     # scratch halves taking turns), then the same pipe again after a join
     wl = scaled(CONFIGS[cfg], L=L, budget=budget)
-    pipe = ck.Pipe(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=ctas)
+    scratch = Guarded((ck.lib.chunkkv_pipe_bytes(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, ctas),), torch.uint8)
+    pipe = ck.Pipe(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=ctas, buf=scratch.t)
     layers = [make_layer(wl, layer=i) for i in range(5)]
     dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in layers]
+    guards = [guarded_outputs(wl.Hkv, ck.out_len(wl.L, wl.w, wl.c, wl.budget), wl.d) for _ in range(5)]
     torch.cuda.synchronize()
     for rep in range(2):
-        outs = [pipe.layer(*dev[i], wl.Hq, wl.w, wl.c, wl.budget) for i in range(5)]
+        outs = [pipe.layer(*dev[i], wl.Hq, wl.w, wl.c, wl.budget, out_K=guards[i][0].t, out_V=guards[i][1].t,
+                           out_idx=guards[i][2].t) for i in range(5)]
         pipe.join()
     assert pipe.status() == 0
+    scratch.check("pipe scratch")
+    for gs in guards:
+        for g, name in zip(gs, ("out_K", "out_V", "out_idx")):
+            g.check(name)
     for x, (oK, oV, idx) in zip(layers, outs):
         _check_layer(x, wl, bits_of(oK), bits_of(oV), idx.cpu().numpy())
     pipe.close()
@@ -514,8 +588,12 @@ def test_compress_layer_alg1_matches_oracle(ck, cfg, L, ratio):
     budget = ora.budget_from_ratio(L, ratio)
     wl = scaled(CONFIGS[cfg], L=L, budget=budget)
     x = make_layer(wl)
-    oK, oV, idx = ck.compress_layer_alg1(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V), wl.Hq, wl.w, wl.c, budget)
+    gK, gV, gI = guarded_outputs(wl.Hkv, ck.out_len_alg1(L, wl.w, wl.c, budget), wl.d)
+    oK, oV, idx = ck.compress_layer_alg1(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V), wl.Hq, wl.w, wl.c, budget,
+                                         out_K=gK.t, out_V=gV.t, out_idx=gI.t)
     assert ck.device_status() == 0
+    for g, name in ((gK, "out_K"), (gV, "out_V"), (gI, "out_idx")):
+        g.check(name)
     ref = ora.compress_layer_alg1(x.q_obs, x.K, x.V, wl.Hq, wl.Hkv, wl.w, wl.c, budget)
     idx_np = idx.cpu().numpy()
     assert idx_np.shape == ref["idx"].shape
