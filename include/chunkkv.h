@@ -171,6 +171,30 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
                            void* out_K, void* out_V, int32_t* out_idx, void* stream);
 
 /*
+ * A whole model with layer-wise index reuse (Algorithm 2): layer l computes its indices iff
+ * l mod reuse_depth == 0 (Algorithm 3 on q_obs[l], K[l], V[l]); every other layer gathers with the
+ * indices of layer floor(l / reuse_depth) * reuse_depth, which are also copied to its out_idx.
+ * All layers share L, Hq, Hkv, d, w, c and budget.
+ *   q_obs, K, V, out_K, out_V, out_idx   HOST arrays of n_layers DEVICE pointers (layouts as in
+ *                                        chunkkv_compress_layer); q_obs[l] may be NULL for layers
+ *                                        that reuse indices. The arrays are read during the call
+ *                                        only. Output buffers of different layers must not overlap.
+ * Same results as the corresponding sequence of chunkkv_compress_layer calls. Where the shape
+ * allows (chunk size 10 or 20, at most 128 query rows per KV head or an even number of grouped query
+ * heads, key range per SM within tensor memory) the layers run through one persistent kernel per
+ * group of up to 32 layers in which scoring layer l + 1 overlaps selecting and gathering layer l;
+ * otherwise they run layer by layer. Needs a workspace of chunkkv_model_workspace_bytes(...) bytes
+ * (chunkkv_set_workspace); returns CHUNKKV_ENOWORKSPACE otherwise. Queued on `stream`; the calls of
+ * one device that use the workspace must be ordered.
+ */
+CHUNKKV_API size_t chunkkv_model_workspace_bytes(int n_layers, int L, int Hq, int Hkv, int d, int w, int c,
+                                                 int budget, int reuse_depth);
+CHUNKKV_API int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* const* K,
+                                       const void* const* V, int L, int Hq, int Hkv, int d, int w, int c,
+                                       int budget, int reuse_depth, void* const* out_K, void* const* out_V,
+                                       int32_t* const* out_idx, void* stream);
+
+/*
  * Algorithm 1's budget rule, as an alternative to Algorithm 3's (which the calls above follow):
  * k = floor(L_max / c) chunks are selected (at most the C that exist), their tokens are taken in
  * ascending order and cut to the first L_max - w ("K'[0 : L_max - w]"), and the observe window

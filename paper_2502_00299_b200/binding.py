@@ -46,6 +46,10 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_gather.argtypes = [vp, vp, vp] + [i32] * 4 + [vp, vp, vp]
     L.chunkkv_compress_layer.restype = i32
     L.chunkkv_compress_layer.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, vp, vp, vp]
+    L.chunkkv_model_workspace_bytes.restype = sz
+    L.chunkkv_model_workspace_bytes.argtypes = [i32] * 9
+    L.chunkkv_compress_model.restype = i32
+    L.chunkkv_compress_model.argtypes = [i32, vp, vp, vp] + [i32] * 8 + [vp, vp, vp, vp]
     L.chunkkv_compress_layer_host.restype = i32
     L.chunkkv_compress_layer_host.argtypes = [vp, vp, vp] + [i32] * 7 + [vp] * 10
     L.chunkkv_lane_bytes.restype = sz
@@ -425,26 +429,63 @@ def compress_layer_host(host_q: torch.Tensor, host_K: torch.Tensor, host_V: torc
         hK.data_ptr(), hV.data_ptr(), hI.data_ptr(), _stream(stream)), "chunkkv_compress_layer_host")
 
 
-def compress_model(layers: Sequence[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]], Hq: int, w: int,
+def _ensure_bytes(need: int) -> None:
+    dev = torch.cuda.current_device()
+    cur = _workspaces.get(dev)
+    if cur is None or cur.numel() < need:
+        set_workspace(torch.empty(need + (need >> 2), dtype=torch.uint8, device=torch.device("cuda", dev)))
+
+
+def compress_model(layers: Sequence[Tuple[Optional[torch.Tensor], torch.Tensor, torch.Tensor]], Hq: int, w: int,
                    c, budget: int, n_reuse: int = 1,
                    stream: Optional[torch.cuda.Stream] = None,
+                   outs: Optional[Sequence[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]]] = None,
                    ) -> List[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]]:
     """Layer-wise index reuse: layer l computes indices iff l % n_reuse == 0, otherwise it
-    gathers with the indices of layer (l // n_reuse) * n_reuse. Only the call sequence lives
-    here; every layer is one chunkkv_compress_layer call. ``c`` is one chunk size or one per
-    layer (chunk-level layers followed by token-level ones, c = 1); a layer that reuses indices
-    takes its source layer's chunk size."""
-    cs = [int(c)] * len(layers) if isinstance(c, int) else [int(v) for v in c]
-    if len(cs) != len(layers):
-        raise ValueError("one chunk size per layer expected")
-    outs: List[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = []
-    for l, (q, K, V) in enumerate(layers):
-        if l % n_reuse == 0:
-            outs.append(compress_layer(q, K, V, Hq, w, cs[l], budget, stream=stream))
-        else:
-            s_l = (l // n_reuse) * n_reuse
-            outs.append(compress_layer(None, K, V, Hq, w, cs[s_l], budget, reuse_idx=outs[s_l][2], stream=stream))
-    return outs
+    gathers with the indices of layer (l // n_reuse) * n_reuse. ``layers`` = (q_obs, K, V) per layer
+    (q_obs may be None for layers that reuse). With one chunk size for all layers this is one
+    chunkkv_compress_model call; with one chunk size per layer (chunk-level layers followed by
+    token-level ones, c = 1) it is the same call sequence over chunkkv_compress_layer, a layer that
+    reuses indices taking its source layer's chunk size. Only marshalling lives here."""
+    n = len(layers)
+    if not isinstance(c, int):
+        cs = [int(v) for v in c]
+        if len(cs) != n:
+            raise ValueError("one chunk size per layer expected")
+        res: List[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]] = []
+        for l, (q, K, V) in enumerate(layers):
+            o = outs[l] if outs is not None else (None, None, None)
+            if l % n_reuse == 0:
+                res.append(compress_layer(q, K, V, Hq, w, cs[l], budget, out_K=o[0], out_V=o[1], out_idx=o[2], stream=stream))
+            else:
+                s_l = (l // n_reuse) * n_reuse
+                res.append(compress_layer(None, K, V, Hq, w, cs[s_l], budget, reuse_idx=res[s_l][2], out_K=o[0],
+                                          out_V=o[1], out_idx=o[2], stream=stream))
+        return res
+    Hkv, L, d = layers[0][1].shape
+    for q, K, V in layers:
+        _dev(K, torch.bfloat16, "K"); _dev(V, torch.bfloat16, "V")
+        if q is not None:
+            _dev(q, torch.bfloat16, "q_obs")
+        if tuple(K.shape) != (Hkv, L, d) or tuple(V.shape) != (Hkv, L, d):
+            raise ValueError("all layers must share one K/V shape")
+    n_max = out_len(L, w, c, budget)
+    dev = layers[0][1].device
+    if outs is None:
+        outs = [(torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev),
+                 torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev),
+                 torch.empty((Hkv, n_max), dtype=torch.int32, device=dev)) for _ in range(n)]
+    _ensure_bytes(int(lib.chunkkv_model_workspace_bytes(n, L, Hq, Hkv, d, w, c, budget, n_reuse)))
+    arr = ctypes.c_void_p * n
+    qa = arr(*[None if t[0] is None else t[0].data_ptr() for t in layers])
+    ka = arr(*[t[1].data_ptr() for t in layers])
+    va = arr(*[t[2].data_ptr() for t in layers])
+    oka = arr(*[o[0].data_ptr() for o in outs])
+    ova = arr(*[o[1].data_ptr() for o in outs])
+    oia = arr(*[o[2].data_ptr() for o in outs])
+    _check(lib.chunkkv_compress_model(n, qa, ka, va, L, Hq, Hkv, d, w, c, budget, n_reuse, oka, ova, oia,
+                                      _stream(stream)), "chunkkv_compress_model")
+    return [tuple(o) for o in outs]
 
 
 def profile_enable(on: bool) -> None:

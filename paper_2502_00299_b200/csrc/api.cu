@@ -13,7 +13,6 @@ using namespace chunkkv;
 namespace {
 
 constexpr int kMaxDevices = 64;
-constexpr size_t kHeaderBytes = 256;   // device status word lives at the start of the scratch
 
 thread_local int g_last_cuda_error = 0;
 
@@ -323,8 +322,13 @@ size_t chunkkv_workspace_bytes(int L, int Hq, int Hkv, int d, int w, int c) {
     const ScoreShape sh = score_shape(Hq, Hkv, w);
     const int C = (L - w + c - 1) / c;
     // chunk scores of the KV heads, those of the scoring heads, and the scoring kernels' scratch
-    const size_t floats = scratch_floats_for(*ctx, L, sh.Rs, sh.Hs, d, c) + round64(static_cast<size_t>(Hkv) * C) +
-                          round64(static_cast<size_t>(sh.Hs) * C);
+    size_t floats = scratch_floats_for(*ctx, L, sh.Rs, sh.Hs, d, c) + round64(static_cast<size_t>(Hkv) * C) +
+                    round64(static_cast<size_t>(sh.Hs) * C);
+    ResidentPlan rplan;
+    if (C > 0 && make_resident_plan(L, sh.Rs, sh.Hs, sh.shift, d, c, C, 0, ctx->num_sms, smem_budget(*ctx), &rplan)) {
+        const size_t rf = resident_scratch_floats(rplan, sh.Hs, C);
+        floats = rf > floats ? rf : floats;
+    }
     return kHeaderBytes + floats * sizeof(float);
 }
 
@@ -482,6 +486,44 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
         // chunk scores (of the scoring heads) sit at the start of the scratch payload, the score
         // kernels' scratch after them
         const size_t cs_floats = round64(static_cast<size_t>(sh.Hs) * C);
+        // A lane that owns at most half of the SMs leaves the row gather to a second launch of
+        // small CTAs that spread over every SM (they fit beside the other lanes' resident
+        // CTAs), instead of moving the rows through its own few SMs.
+        const bool split = rows_elsewhere != nullptr || (lane != nullptr && 2 * ctas <= ctx->num_sms);
+        ResidentPlan rplan;
+        if (!split && make_resident_plan(L, R, sh.Hs, sh.shift, d, c, C, n_max, ctas, smem_budget(*ctx), &rplan)) {
+            // One cooperative launch; the chunk partial sums never leave the SMs.
+            const size_t need = resident_scratch_floats(rplan, sh.Hs, C) * sizeof(float);
+            char* base;
+            if (lane != nullptr) {
+                if (kHeaderBytes + need > lane_bytes) return CHUNKKV_ENOWORKSPACE;
+                base = static_cast<char*>(lane);
+            } else {
+                st = ensure_workspace(*ctx, need);
+                if (st != CHUNKKV_OK) return st;
+                base = static_cast<char*>(ctx->ws);
+            }
+            CUtensorMap tm_q, tm_k;
+            st = encode_bf16_3d(&tm_q, q_obs, d, R, sh.Hs, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+            if (st != CHUNKKV_OK) return st;
+            st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+            if (st != CHUNKKV_OK) return st;
+            ResidentIO io;
+            io.L = L; io.w = w; io.Rs = R; io.Hs = sh.Hs; io.d = d; io.kv_shift = sh.shift;
+            io.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
+            io.C = C; io.k = k; io.n_max = n_max;
+            io.K = K; io.V = V; io.out_K = out_K; io.out_V = out_V; io.out_idx = out_idx;
+            io.scratch = reinterpret_cast<float*>(base + kHeaderBytes);
+            io.counters = reinterpret_cast<unsigned*>(base + kResidentCountersOffset);
+            io.status = reinterpret_cast<int*>(base);
+            io.cooperative = lane != nullptr;
+            {
+                Timer t(ctx, s, 0);
+                e = launch_layer_resident(rplan, tm_q, tm_k, io, s);
+            }
+            if (e != cudaSuccess) return cuda_fail(e);
+            return CHUNKKV_OK;
+        }
         ScorePlan plan;
         if (make_score_plan(L, R, sh.Hs, d, c, ctas, smem_budget(*ctx), true, &plan)) {
             // One cooperative launch for the whole layer.
@@ -508,10 +550,6 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
             if (st != CHUNKKV_OK) return st;
             FusedLayerIO io;
-            // A lane that owns at most half of the SMs leaves the row gather to a second launch of
-            // small CTAs that spread over every SM (they fit beside the other lanes' resident
-            // CTAs), instead of moving the rows through its own few SMs.
-            const bool split = rows_elsewhere != nullptr || (lane != nullptr && 2 * ctas <= ctx->num_sms);
             io.K = K; io.V = V; io.out_K = split ? nullptr : out_K; io.out_V = out_V; io.out_idx = out_idx;
             io.chunk_scores = payload;
             io.C = C; io.k = k; io.n_max = n_max; io.Hkv_out = Hkv;
@@ -558,6 +596,151 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
                            void* out_K, void* out_V, int32_t* out_idx, void* stream) {
     return compress_impl(q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_idx, out_K, out_V, out_idx, nullptr, 0, 0,
                          stream);
+}
+
+// ---- Algorithm 2 over a whole model: every reuse_depth-th layer computes indices, the layers
+//      between gather with them. Where the shape fits the persistent kernel the layers go through
+//      it in launches of up to kModelMaxLayers; otherwise layer by layer.
+static int model_args_ok(int n_layers, int reuse_depth) {
+    if (n_layers < 1 || reuse_depth < 1) return CHUNKKV_EINVAL_SHAPE;
+    return CHUNKKV_OK;
+}
+
+size_t chunkkv_model_workspace_bytes(int n_layers, int L, int Hq, int Hkv, int d, int w, int c, int budget,
+                                     int reuse_depth) {
+    if (model_args_ok(n_layers, reuse_depth) != CHUNKKV_OK || check_sizes(L, w, c, budget) != CHUNKKV_OK) return 0;
+    const size_t per_layer = chunkkv_workspace_bytes(L, Hq, Hkv, d, w, c);
+    if (per_layer == 0) return 0;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    if (get_ctx(&ctx) != CHUNKKV_OK) return 0;
+    const ScoreShape sh = score_shape(Hq, Hkv, w);
+    const int C = (L - w + c - 1) / c;
+    const int k = chunkkv_num_kept_chunks(L, w, c, budget);
+    ModelPlan mp;
+    size_t need = per_layer;
+    if (C > 0 && k > 0 && make_model_plan(L, sh.Rs, sh.Hs, sh.shift, d, c, C, k, ctx->num_sms, smem_budget(*ctx), &mp)) {
+        const int per_launch = n_layers < kModelMaxLayers ? n_layers : kModelMaxLayers;
+        const int n_compute = (per_launch + reuse_depth - 1) / reuse_depth + 1;
+        const size_t m = kHeaderBytes + model_scratch_floats(mp, sh.Hs, C, n_compute) * sizeof(float);
+        need = m > need ? m : need;
+    }
+    return need;
+}
+
+int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* const* K, const void* const* V,
+                           int L, int Hq, int Hkv, int d, int w, int c, int budget, int reuse_depth,
+                           void* const* out_K, void* const* out_V, int32_t* const* out_idx, void* stream) {
+    int st = model_args_ok(n_layers, reuse_depth);
+    if (st != CHUNKKV_OK) return st;
+    st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    st = check_heads(L, Hq, Hkv, d, w);
+    if (st != CHUNKKV_OK) return st;
+    if (q_obs == nullptr || K == nullptr || V == nullptr || out_K == nullptr || out_V == nullptr || out_idx == nullptr)
+        return CHUNKKV_EINVAL_NULL;
+    for (int l = 0; l < n_layers; ++l) {
+        const bool computes = (l % reuse_depth) == 0;
+        if (K[l] == nullptr || V[l] == nullptr || out_K[l] == nullptr || out_V[l] == nullptr || out_idx[l] == nullptr ||
+            (computes && q_obs[l] == nullptr))
+            return CHUNKKV_EINVAL_NULL;
+        if (!aligned16(K[l]) || !aligned16(V[l]) || !aligned16(out_K[l]) || !aligned16(out_V[l]) ||
+            !aligned16(out_idx[l]) || (computes && !aligned16(q_obs[l])))
+            return CHUNKKV_EINVAL_ALIGN;
+    }
+    const int C = chunkkv_num_chunks(L, w, c);
+    const int k = chunkkv_num_kept_chunks(L, w, c, budget);
+    const int n_max = chunkkv_out_len(L, w, c, budget);
+    if (n_max < 0) return n_max;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    ModelPlan mp;
+    bool persistent = false;
+    DeviceCtx* ctx = nullptr;
+    ScoreShape sh = score_shape(Hq, Hkv, w);
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        st = get_ctx(&ctx);
+        if (st != CHUNKKV_OK) return st;
+        persistent = C > 0 && k > 0 &&
+                     make_model_plan(L, sh.Rs, sh.Hs, sh.shift, d, c, C, k, ctx->num_sms, smem_budget(*ctx), &mp);
+    }
+    if (!persistent) {
+        // layer by layer: Algorithm 2's call sequence over chunkkv_compress_layer
+        for (int l = 0; l < n_layers; ++l) {
+            const int src = (l / reuse_depth) * reuse_depth;
+            st = chunkkv_compress_layer(l == src ? q_obs[l] : nullptr, K[l], V[l], L, Hq, Hkv, d, w, c, budget,
+                                        l == src ? nullptr : out_idx[src], out_K[l], out_V[l], out_idx[l], stream);
+            if (st != CHUNKKV_OK) return st;
+        }
+        return CHUNKKV_OK;
+    }
+    std::lock_guard<std::mutex> lk(g_mu);
+    std::vector<CUtensorMap> tm_q(kModelMaxCompute), tm_k(kModelMaxCompute);
+    std::vector<ModelLayerIO> lay(kModelMaxLayers);
+    for (int l0 = 0; l0 < n_layers;) {
+        // a launch takes whole reuse groups, at most kModelMaxLayers layers
+        int l1 = l0;
+        int n_compute = 0;
+        while (l1 < n_layers) {
+            const int group_end = (l1 + reuse_depth < n_layers) ? l1 + reuse_depth : n_layers;
+            if (group_end - l0 > kModelMaxLayers && l1 > l0) break;
+            if (group_end - l0 > kModelMaxLayers) {         // a single reuse group longer than a launch: split it
+                l1 = l0 + kModelMaxLayers;
+                if (n_compute == 0) n_compute = 1;
+                break;
+            }
+            l1 = group_end;
+            ++n_compute;
+        }
+        const int n = l1 - l0;
+        const size_t need = model_scratch_floats(mp, sh.Hs, C, n_compute) * sizeof(float);
+        st = ensure_workspace(*ctx, need);
+        if (st != CHUNKKV_OK) return st;
+        char* base = static_cast<char*>(ctx->ws);
+        int nc = 0;
+        for (int i = 0; i < n; ++i) {
+            const int l = l0 + i;
+            const bool computes = (l % reuse_depth) == 0;
+            lay[i].K = K[l]; lay[i].V = V[l]; lay[i].out_K = out_K[l]; lay[i].out_V = out_V[l]; lay[i].out_idx = out_idx[l];
+            lay[i].computes = computes;
+            if (computes) {
+                st = encode_bf16_3d(&tm_q[nc], q_obs[l], d, sh.Rs, sh.Hs, sh.Rs < 128 ? sh.Rs : 128,
+                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+                if (st != CHUNKKV_OK) return st;
+                st = encode_bf16_3d(&tm_k[nc], K[l], d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+                if (st != CHUNKKV_OK) return st;
+                ++nc;
+            }
+        }
+        if (!lay[0].computes) {
+            // the launch starts inside a reuse group (a group longer than a launch): these layers gather
+            // with indices computed by an earlier launch
+            int i = 0;
+            for (; i < n && !lay[i].computes; ++i) {
+                const int l = l0 + i, src = (l / reuse_depth) * reuse_depth;
+                cudaError_t e = launch_gather(K[l], V[l], out_idx[src], L, Hkv, d, n_max, out_K[l], out_V[l], out_idx[l],
+                                              ctx->num_sms, s);
+                if (e != cudaSuccess) return cuda_fail(e);
+            }
+            l0 += i;
+            continue;
+        }
+        ModelIO io;
+        io.L = L; io.w = w; io.Rs = sh.Rs; io.Hs = sh.Hs; io.d = d; io.kv_shift = sh.shift;
+        io.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
+        io.C = C; io.k = k; io.n_max = n_max;
+        io.scratch = reinterpret_cast<float*>(base + kHeaderBytes);
+        io.counters = reinterpret_cast<unsigned*>(base + kResidentCountersOffset);
+        io.status = reinterpret_cast<int*>(base);
+        cudaError_t e;
+        {
+            Timer t(ctx, s, 0);
+            e = launch_model(mp, io, tm_q.data(), tm_k.data(), lay.data(), n, s);
+        }
+        if (e != cudaSuccess) return cuda_fail(e);
+        l0 = l1;
+    }
+    return CHUNKKV_OK;
 }
 
 // ---- Algorithm 1's budget rule: k = floor(L_max / c) chunks, their tokens cut to the first
@@ -646,7 +829,12 @@ size_t chunkkv_lane_bytes(int L, int Hq, int Hkv, int d, int w, int c, int max_c
     const int C = (L - w + c - 1) / c;
     ScorePlan plan;
     if (!make_score_plan(L, sh.Rs, sh.Hs, d, c, ctas, smem_budget(*ctx), true, &plan)) return 0;
-    const size_t floats = score_scratch_floats(plan, sh.Hs, sh.Rs) + round64(static_cast<size_t>(sh.Hs) * C);
+    size_t floats = score_scratch_floats(plan, sh.Hs, sh.Rs) + round64(static_cast<size_t>(sh.Hs) * C);
+    ResidentPlan rplan;
+    if (C > 0 && make_resident_plan(L, sh.Rs, sh.Hs, sh.shift, d, c, C, 0, ctas, smem_budget(*ctx), &rplan)) {
+        const size_t rf = resident_scratch_floats(rplan, sh.Hs, C);
+        floats = rf > floats ? rf : floats;
+    }
     return kHeaderBytes + floats * sizeof(float);
 }
 

@@ -7,6 +7,14 @@
 
 namespace chunkkv {
 
+// Every scratch buffer (device workspace, lane, pipe) starts with a header of this many bytes that is
+// zero between launches: device status word at +0, the grid barrier's ticket and exit counters at
+// +64 / +128, and from +192 the counters of the layer kernel with on-chip partial sums (exit
+// counter, then one hand-over counter per scoring head and one per KV head).
+constexpr size_t kHeaderBytes = 2048;
+constexpr size_t kResidentCountersOffset = 192;
+constexpr int kResidentMaxHeads = 224;
+
 // Geometry of one scoring launch, fixed on the host.
 struct ScorePlan {
     int c_static;   // chunk size baked into the kernel (0 = run-time chunk size)
@@ -68,6 +76,76 @@ struct FusedLayerIO {
 // The whole layer in one cooperative launch (plan made with full_grid = true, C > 0, k > 0).
 cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                const ScoreArgs& args, const FusedLayerIO& io, cudaStream_t stream);
+
+// The layer kernel that keeps its chunk partial sums in tensor memory (layer_resident.cu): every CTA
+// belongs to one scoring head, `cph` CTAs per head.
+struct ResidentPlan {
+    int c_static;     // 10 or 20
+    int grid, cph;
+    int n_tiles;      // 120-key accumulator tiles per head
+    int t_max;        // most tiles any CTA takes
+    int n_stages;
+    int smem_bytes;
+    int off_ring, ring_bytes, off_pmax, off_misc;
+};
+
+struct ResidentIO {
+    int L, w, Rs, Hs, d, kv_shift;   // Rs rows per scoring head, Hs scoring heads, KV head = scoring head >> kv_shift
+    float sl2;
+    int C, k, n_max;
+    const void* K;
+    const void* V;
+    void* out_K;
+    void* out_V;
+    int32_t* out_idx;
+    float* scratch;       // resident_scratch_floats() floats
+    unsigned* counters;   // header + kResidentCountersOffset
+    int* status;
+    bool cooperative;     // cooperative launch (lanes: several launches share the GPU) instead of a programmatic dependent one
+};
+
+// false when the shape does not fit this kernel (chunk size other than 10 / 20, more than 128 rows
+// per scoring head, more chunks per CTA than tensor memory holds, fewer CTAs than scoring heads).
+bool make_resident_plan(int L, int Rs, int Hs, int kv_shift, int d, int c, int C, int n_max, int max_ctas,
+                        int smem_limit, ResidentPlan* plan);
+size_t resident_scratch_floats(const ResidentPlan& plan, int Hs, int C);
+cudaError_t launch_layer_resident(const ResidentPlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                                  const ResidentIO& io, cudaStream_t stream);
+
+// The persistent kernel that runs many layers per launch (model_kernel.cu). Same tiling as the
+// layer kernel above, plus two tail warps per CTA that select and copy rows behind the scoring.
+constexpr int kModelMaxLayers = 32;     // layers per launch (computed + reusing)
+constexpr int kModelMaxCompute = 32;    // computed layers per launch
+
+struct ModelPlan {
+    int c_static, grid, cph, n_tiles, t_max, n_stages, smem_bytes;
+    int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes;
+};
+
+struct ModelIO {
+    int L, w, Rs, Hs, d, kv_shift;
+    float sl2;
+    int C, k, n_max;
+    float* scratch;       // model_scratch_floats() floats
+    unsigned* counters;   // header + kResidentCountersOffset
+    int* status;
+};
+
+struct ModelLayerIO {
+    const void* K;
+    const void* V;
+    void* out_K;
+    void* out_V;
+    int32_t* out_idx;
+    bool computes;        // false: gather with the indices of the nearest computed layer before it
+};
+
+bool make_model_plan(int L, int Rs, int Hs, int kv_shift, int d, int c, int C, int k, int max_ctas, int smem_limit,
+                     ModelPlan* plan);
+size_t model_scratch_floats(const ModelPlan& plan, int Hs, int C, int n_compute);
+// layers[0] must compute; tm_q / tm_k hold one tensor map per computed layer, in order.
+cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
+                         const ModelLayerIO* layers, int n_layers, cudaStream_t stream);
 
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
                             int num_sms, cudaStream_t stream);

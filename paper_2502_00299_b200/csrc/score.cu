@@ -19,6 +19,7 @@
 #include "gather.cuh"
 #include "internal.h"
 #include "ptx.cuh"
+#include "panels.cuh"
 #include "select.cuh"
 
 #include <math_constants.h>
@@ -43,113 +44,6 @@ struct SharedCtl {
     uint32_t tmem_base;
     int abort_flag;
 };
-
-// Pull WP consecutive accumulator columns of this thread's row into registers.
-template <int WP>
-__device__ __forceinline__ void load_panel(uint32_t taddr, float (&v)[WP]) {
-    static_assert(WP % 4 == 0, "panel width must be a multiple of 4 columns");
-    int o = 0;
-#pragma unroll
-    for (int b = 0; b < WP / 32; ++b, o += 32) tmem_ld_x32(taddr + o, &v[o]);
-    if constexpr ((WP & 16) != 0) { tmem_ld_x16(taddr + o, &v[o]); o += 16; }
-    if constexpr ((WP & 8) != 0) { tmem_ld_x8(taddr + o, &v[o]); o += 8; }
-    if constexpr ((WP & 4) != 0) { tmem_ld_x4(taddr + o, &v[o]); o += 4; }
-    tmem_ld_wait();
-}
-
-// Panel that lies wholly inside the prefix and starts on a chunk boundary, chunk size known at
-// compile time: all control flow below folds away after unrolling.
-template <int C, int WP>
-__device__ __forceinline__ void panel_fast(float (&v)[WP], float sl2, bool active, float* part,
-                                           int row_stride, uint64_t keep, float* out_m, float* out_l) {
-    static_assert(WP % 4 == 0 && WP >= 8, "panel width");
-    // row max with three-input max instructions, two independent chains
-    float m0 = fmaxf(v[0], v[1]), m1 = fmaxf(v[2], v[3]);
-#pragma unroll
-    for (int u = 4; u + 3 < WP; u += 4) {
-        m0 = fmax3(m0, v[u], v[u + 1]);
-        m1 = fmax3(m1, v[u + 2], v[u + 3]);
-    }
-    const float mx = fmaxf(m0, m1);
-    const float neg_m2 = -mx * sl2;
-    float l = 0.f;
-    if constexpr (C % 2 == 0) {
-        // Two columns per instruction: scale-and-shift and the chunk sums run on packed pairs
-        // (same arithmetic, fewer instructions issued).
-        const unsigned long long s2 = pack2(sl2, sl2), n2 = pack2(neg_m2, neg_m2);
-        unsigned long long e[WP / 2];
-#pragma unroll
-        for (int u = 0; u < WP / 2; ++u) {
-            float x0, x1;
-            unpack2(fma2(pack2(v[2 * u], v[2 * u + 1]), s2, n2), x0, x1);
-            e[u] = pack2(ex2_approx(x0), ex2_approx(x1));
-        }
-        constexpr int H = C / 2;     // pairs per chunk
-#pragma unroll
-        for (int ch = 0; ch < WP / C; ++ch) {
-            unsigned long long s0 = e[ch * H];
-            unsigned long long s1 = (H > 1) ? e[ch * H + 1] : 0ull;
-#pragma unroll
-            for (int t = 2; t < H; t += 2) {
-                s0 = add2(s0, e[ch * H + t]);
-                if (t + 1 < H) s1 = add2(s1, e[ch * H + t + 1]);
-            }
-            if (H > 1) s0 = add2(s0, s1);
-            float lo, hi;
-            unpack2(s0, lo, hi);
-            const float acc = lo + hi;
-            if (active) st_keep(part + static_cast<size_t>(ch) * row_stride, acc, keep);
-            l += acc;
-        }
-    } else {
-        // exponentials first, in place: WP independent operations the scheduler can overlap freely
-#pragma unroll
-        for (int u = 0; u < WP; ++u) v[u] = ex2_approx(fmaf(v[u], sl2, neg_m2));
-        // chunk sums as balanced trees (short dependency chains), one store per chunk
-#pragma unroll
-        for (int ch = 0; ch < WP / C; ++ch) {
-            float s0 = 0.f, s1 = 0.f;
-#pragma unroll
-            for (int t = 0; t < C; t += 2) {
-                s0 += v[ch * C + t];
-                if (t + 1 < C) s1 += v[ch * C + t + 1];
-            }
-            const float acc = s0 + s1;
-            if (active) st_keep(part + static_cast<size_t>(ch) * row_stride, acc, keep);
-            l += acc;
-        }
-    }
-    *out_m = mx * sl2;
-    *out_l = l;
-}
-
-// Panel of a compile-time chunk size that starts on a chunk boundary but reaches past the
-// prefix: chunk positions are still static; columns at or past P only feed the row sum, and
-// columns the row cannot see (causal mask in the window, or past L) contribute nothing.
-template <int C, int WP>
-__device__ __forceinline__ void panel_static_tail(const float (&v)[WP], float sl2, bool active, float* part,
-                                                  int row_stride, uint64_t keep, int j0, int P, int last_visible,
-                                                  float* out_m, float* out_l) {
-    const int n_vis = last_visible - j0 + 1;     // columns u < n_vis are visible
-    const int n_pre = P - j0;                    // columns u < n_pre belong to the prefix
-    float mx = -CUDART_INF_F;
-#pragma unroll
-    for (int u = 0; u < WP; ++u) mx = (u < n_vis) ? fmaxf(mx, v[u]) : mx;
-    const float neg_m2 = (mx == -CUDART_INF_F) ? 0.f : -mx * sl2;
-    float l = 0.f, acc = 0.f;
-#pragma unroll
-    for (int u = 0; u < WP; ++u) {
-        const float e = (u < n_vis) ? ex2_approx(fmaf(v[u], sl2, neg_m2)) : 0.f;
-        l += e;
-        const float pe = (u < n_pre) ? e : 0.f;
-        acc = (u % C == 0) ? pe : acc + pe;
-        if ((u + 1) % C == 0) {
-            if (active && (u + 1 - C) < n_pre) st_keep(part + static_cast<size_t>((u + 1) / C - 1) * row_stride, acc, keep);
-        }
-    }
-    *out_m = (mx == -CUDART_INF_F) ? -CUDART_INF_F : mx * sl2;
-    *out_l = l;
-}
 
 // Any panel: run-time chunk size, chunk grid clipped at P, causal mask inside the window
 // columns [P, L), nothing visible at or beyond L. Window columns add to the row sum only.
@@ -794,10 +688,14 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 const int j0 = panel * WPP;
                 float m2, l;
                 if constexpr (C_STATIC > 0) {
+                    const int n_pre = a.P - j0;      // chunk slots that start before P hold a chunk
+                    auto emit = [&](int ch, float acc) {
+                        if (active && ch * C_STATIC < n_pre) st_keep(part + static_cast<size_t>(ch) * a.R, acc, keep);
+                    };
                     if (j0 + WPP <= a.P)
-                        panel_fast<C_STATIC, WPP>(v, a.sl2, active, part, a.R, keep, &m2, &l);
+                        panel_fast<C_STATIC, WPP>(v, a.sl2, emit, &m2, &l);
                     else
-                        panel_static_tail<C_STATIC, WPP>(v, a.sl2, active, part, a.R, keep, j0, a.P, last_visible, &m2, &l);
+                        panel_static_tail<C_STATIC, WPP>(v, a.sl2, emit, j0, a.P, last_visible, &m2, &l);
                 } else {
                     panel_general<WPP>(v, a.sl2, active, part, a.R, j0, a.P, a.c, last_visible, &m2, &l);
                 }

@@ -2,16 +2,16 @@
 // the selection mask, "always keep most recent tokens", "nonzero(mask)"), shared by the
 // stand-alone select kernel and the fused layer kernel. One CTA works on one KV head.
 //
-// Both bodies find the k-th largest of the order-preserving 32-bit keys by an exact 4-pass radix
-// select and then rank every chunk among the kept ones: rank = #above before it + min(#equal
-// before it, ties to keep) - ties go to the lower chunk id. Token positions are written directly
-// in ascending order: no mask, no sort.
+// Both bodies find the k-th largest of the order-preserving 32-bit keys exactly and then rank
+// every chunk among the kept ones: rank = #above before it + min(#equal before it, ties to keep) -
+// ties go to the lower chunk id. Token positions are written directly in ascending order: no
+// mask, no sort.
 //
 // select_head_regs (a few chunks per thread): each thread owns a contiguous run of chunk ids and
-// keeps their keys in registers. In the first radix pass, whose digit (sign and high exponent
-// bits) is nearly constant, every warp counts into its own 16-bit histogram row (lanes that hit
-// the same bin add once); later passes add one shared-memory atomic per surviving key. One
-// block-wide prefix sum over the threads' (#above, #equal) gives the ranks. Fully unrolled.
+// keeps their keys in registers; the threshold comes from an adaptive radix select (2048 equal
+// sub-intervals of [min key, max key], repeated on the sub-interval that holds the k-th largest
+// until few enough keys remain to rank directly). One block-wide prefix sum over the threads'
+// (#above, #equal) gives the ranks.
 //
 // select_head_rows (many chunks per thread, e.g. token-level selection of tens of thousands of
 // keys): unrolled code over registers would spill and spend its time fetching instructions that
@@ -36,8 +36,11 @@ struct SelectSmem {
     int sel[kSelCap];
     int hist[256];
     unsigned long long warp_sums[kSelMaxWarps + 1];
+    int warp_tot[kSelMaxWarps];
     uint32_t prefix;
     int need;
+    int bin_count;
+    int n_cand;
     int last_kept;
 };
 
@@ -47,15 +50,27 @@ __device__ __forceinline__ uint32_t select_order_key(float x) {
 }
 
 // Selection for a few chunks per thread. All threads of the CTA must call this (it uses
-// __syncthreads); blockDim.x must be a multiple of 32 and at most 1024. Every thread keeps up to
-// KPT keys in registers, which needs C <= blockDim.x * KPT (KPT = 0 re-reads keys from memory
-// on every use instead).
+// __syncthreads); blockDim.x must be a multiple of 32, at least 512 and at most 1024. Every thread
+// keeps up to KPT keys in registers, which needs C <= blockDim.x * KPT.
 // sc2 != NULL: the head's scores are sc[ch] + sc2[ch] (a KV head scored as two heads of half the rows).
+//
+// The k-th largest key is found by an adaptive radix select: the keys of interest always lie in a
+// known interval [base, base + span]; one round histograms them into 2048 equal sub-intervals,
+// finds the sub-interval that holds the k-th largest and makes it the new interval. Chunk scores
+// of one head sit in a narrow band of the float range, so the first round (over [min, max] of the
+// keys) already leaves a handful of candidates; as soon as at most kSelCandCap keys remain they are
+// ranked against each other directly. Ties and degenerate inputs (all keys equal) end with
+// span = 0, i.e. a single key value. Exact for any input.
+constexpr int kSelBins = 2048;
+constexpr int kSelCandCap = 1024;
+
 template <int KPT>
-__device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, const float* __restrict__ sc2, int L, int w, int c,
-                                            int C, int k, int n_max, int32_t* __restrict__ out, SelectSmem& sm,
+__device__ __forceinline__ void select_head_regs(const float* sc, const float* sc2, int L, int w, int c,
+                                            int C, int k, int n_max, int32_t* out, SelectSmem& sm,
                                             int tok_cap = 0x7fffffff) {
-    auto score_at = [&](int ch) { return sc2 != nullptr ? sc[ch] + sc2[ch] : sc[ch]; };
+    static_assert(KPT > 0, "keys live in registers");
+    constexpr unsigned kFull = 0xffffffffu;
+    auto score_at = [&](int ch) { return sc2 != nullptr ? __ldcg(sc + ch) + __ldcg(sc2 + ch) : __ldcg(sc + ch); };
     const int P = L - w;
     const int nt = blockDim.x, nwarps = nt >> 5;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -65,92 +80,105 @@ __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, c
     // thread t owns chunk ids [c0, c1)
     const int per = (C + nt - 1) / nt;
     const int c0 = min(tid * per, C), c1 = min(c0 + per, C);
-    constexpr bool IN_REGS = KPT > 0;
-    constexpr int KR = IN_REGS ? KPT : 1;
-    uint32_t keys[KR];
-    if (IN_REGS && kk > 0 && !keep_all) {
+    uint32_t keys[KPT];
+    if (kk > 0 && !keep_all) {
 #pragma unroll
-        for (int u = 0; u < KR; ++u) keys[u] = (c0 + u < c1) ? select_order_key(score_at(c0 + u)) : 0u;
+        for (int u = 0; u < KPT; ++u) keys[u] = (c0 + u < c1) ? select_order_key(score_at(c0 + u)) : 0u;
     }
     if (tid == 0) sm.last_kept = 0;
 
     uint32_t thresh = 0;   // key of the k-th largest score
     int need_eq = 0;       // how many chunks equal to the threshold are kept
     if (!keep_all && kk > 0) {
-        uint32_t prefix = 0;
-        int need = k;
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
-            // Pass 0 sees the sign and exponent bits, which are nearly the same for all scores:
-            // lanes that hit the same bin are grouped with a match and add once to the warp's own
-            // histogram row. Later passes see spread-out digits of the few keys that still carry
-            // the prefix: there one atomic add per key into the shared histogram is cheaper.
-            const bool grouped = (pass == 0);
-            if (grouped) {   // clear this warp's histogram row (256 x 16 bit = 128 words)
-                uint32_t* row = reinterpret_cast<uint32_t*>(sm.whist[warp]);
+        int* hist = reinterpret_cast<int*>(&sm.whist[0][0]);            // kSelBins counters
+        uint32_t* cand = reinterpret_cast<uint32_t*>(&sm.sel[0]);       // kSelCandCap keys (sel is written later)
+        // smallest and largest key of the head
+        uint32_t lo = 0xffffffffu, hi = 0u;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) row[lane + 32 * q] = 0u;
-                __syncwarp();
-            } else {
-                if (tid < 256) sm.hist[tid] = 0;
-                __syncthreads();
-            }
-            const uint32_t himask = (pass == 0) ? 0u : (0xFFFFFFFFu << (shift + 8));
-            auto count_one = [&](bool have, uint32_t key) {
-                const bool in = have && (key & himask) == prefix;
-                const int bin = in ? static_cast<int>((key >> shift) & 0xFF) : -1;
-                if (grouped) {
-                    const unsigned peers = __match_any_sync(0xffffffffu, bin);
-                    if (in && lane == __ffs(peers) - 1)
-                        sm.whist[warp][bin] += static_cast<unsigned short>(__popc(peers));
-                    __syncwarp();
-                } else if (in) {
-                    atomicAdd(&sm.hist[bin], 1);
-                }
-            };
-            if (IN_REGS) {
-#pragma unroll
-                for (int u = 0; u < KR; ++u)
-                    if (u < per) count_one(c0 + u < c1, keys[u]);      // `per` is uniform: no divergence
-            } else {
-                for (int u = 0; u < per; ++u)
-                    count_one(c0 + u < c1, (c0 + u < c1) ? select_order_key(score_at(c0 + u)) : 0u);
-            }
-            __syncthreads();
-            if (grouped) {
-                if (tid < 256) {
-                    int sum = 0;
-                    for (int wv = 0; wv < nwarps; ++wv) sum += sm.whist[wv][tid];
-                    sm.hist[tid] = sum;
-                }
-                __syncthreads();
-            }
-            if (warp == 0) {
-                // lane t owns bins 255-8t .. 248-8t (descending), so a prefix over lanes counts from the top
-                int cnt[8], sum = 0;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) { cnt[q] = sm.hist[255 - 8 * lane - q]; sum += cnt[q]; }
-                int inc = sum;
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const int n = __shfl_up_sync(0xffffffffu, inc, off);
-                    if (lane >= off) inc += n;
-                }
-                const unsigned reach = __ballot_sync(0xffffffffu, inc >= need);
-                const int owner = reach ? (__ffs(reach) - 1) : 31;
-                if (lane == owner) {
-                    int above = inc - sum, q = 0;
-                    while (q < 7 && above + cnt[q] < need) { above += cnt[q]; ++q; }
-                    sm.prefix = prefix | (static_cast<uint32_t>(255 - 8 * lane - q) << shift);
-                    sm.need = need - above;
-                }
-            }
-            __syncthreads();
-            prefix = sm.prefix;
-            need = sm.need;
+        for (int u = 0; u < KPT; ++u)
+            if (c0 + u < c1) { lo = min(lo, keys[u]); hi = max(hi, keys[u]); }
+        lo = __reduce_min_sync(kFull, lo);
+        hi = __reduce_max_sync(kFull, hi);
+        if (lane == 0) sm.warp_sums[warp] = (static_cast<unsigned long long>(hi) << 32) | lo;
+        for (int i = tid; i < kSelBins; i += nt) hist[i] = 0;
+        if (tid == 0) sm.n_cand = 0;
+        __syncthreads();
+        uint32_t base = 0xffffffffu, top = 0u;
+        for (int wv = 0; wv < nwarps; ++wv) {
+            const unsigned long long v = sm.warp_sums[wv];
+            base = min(base, static_cast<uint32_t>(v));
+            top = max(top, static_cast<uint32_t>(v >> 32));
         }
-        thresh = prefix;
-        need_eq = need;
+        uint32_t span = top - base;          // the keys of interest lie in [base, base + span]
+        int need = k;                        // the need-th largest of them is the threshold
+        for (int round = 0;; ++round) {
+            if (span == 0u) { thresh = base; need_eq = need; break; }
+            const int shift = max(0, 21 - __clz(span));      // (span >> shift) < kSelBins
+            if (round > 0) {
+                for (int i = tid; i < kSelBins; i += nt) hist[i] = 0;
+                __syncthreads();
+            }
+#pragma unroll
+            for (int u = 0; u < KPT; ++u) {
+                const uint32_t dlt = keys[u] - base;
+                if (c0 + u < c1 && keys[u] >= base && dlt <= span) atomicAdd(&hist[dlt >> shift], 1);
+            }
+            __syncthreads();
+            // thread t < 512 owns bins 2047 - 4t .. 2044 - 4t, so a prefix over threads counts from the top
+            int cnt[4] = {0, 0, 0, 0}, sum = 0;
+            if (tid < kSelBins / 4) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) { cnt[q] = hist[kSelBins - 1 - 4 * tid - q]; sum += cnt[q]; }
+            }
+            int inc = sum;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int n = __shfl_up_sync(kFull, inc, off);
+                if (lane >= off) inc += n;
+            }
+            if (lane == 31) sm.warp_tot[warp] = inc;
+            __syncthreads();
+            int before = 0;
+            for (int wv = 0; wv < warp; ++wv) before += sm.warp_tot[wv];
+            inc += before;
+            if (tid < kSelBins / 4 && inc - sum < need && need <= inc) {     // exactly one thread
+                int above = inc - sum, q = 0, cq = cnt[0];
+#pragma unroll
+                for (int t = 0; t < 3; ++t)          // (unrolled: cnt stays in registers)
+                    if (q == t && above + cnt[t] < need) { above += cnt[t]; q = t + 1; cq = cnt[t + 1]; }
+                sm.prefix = static_cast<uint32_t>(kSelBins - 1 - 4 * tid - q);
+                sm.need = need - above;
+                sm.bin_count = cq;
+            }
+            __syncthreads();
+            const uint32_t bin = sm.prefix;
+            const int n_bin = sm.bin_count;
+            need = sm.need;
+            const uint32_t sub = bin << shift;
+            const uint32_t width = (shift >= 32) ? 0xffffffffu : ((1u << shift) - 1u);
+            base += sub;
+            span = min(width, span - sub);
+            if (n_bin <= kSelCandCap) {
+                // few keys left: rank them against each other
+#pragma unroll
+                for (int u = 0; u < KPT; ++u) {
+                    const uint32_t dlt = keys[u] - base;
+                    if (c0 + u < c1 && keys[u] >= base && dlt <= span) cand[atomicAdd(&sm.n_cand, 1)] = keys[u];
+                }
+                __syncthreads();
+                for (int j = tid; j < n_bin; j += nt) {
+                    const uint32_t v = cand[j];
+                    int gt = 0, ge = 0;
+                    for (int i = 0; i < n_bin; ++i) { gt += cand[i] > v; ge += cand[i] >= v; }
+                    if (gt < need && need <= ge) { sm.prefix = v; sm.need = need - gt; }   // same values from every writer
+                }
+                __syncthreads();
+                thresh = sm.prefix;
+                need_eq = sm.need;
+                break;
+            }
+        }
+        __syncthreads();       // cand (= sel) and the shared words are reused below
     }
 
     // Ordered sweep over the chunk ids.
@@ -158,23 +186,17 @@ __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, c
     if (kk > 0) {
         unsigned gt_n = 0, eq_n = 0;
         if (keep_all) gt_n = c1 - c0;
-        else if (IN_REGS) {
+        else {
 #pragma unroll
-            for (int u = 0; u < KR; ++u)
+            for (int u = 0; u < KPT; ++u)
                 if (c0 + u < c1) { gt_n += keys[u] > thresh; eq_n += keys[u] == thresh; }
-        } else {
-            for (int ch = c0; ch < c1; ++ch) {
-                const uint32_t key = select_order_key(score_at(ch));
-                gt_n += key > thresh;
-                eq_n += key == thresh;
-            }
         }
         // block-wide exclusive prefix of the packed pair (eq in the high half, gt in the low half)
         const unsigned long long mine = (static_cast<unsigned long long>(eq_n) << 32) | gt_n;
         unsigned long long inc = mine;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
-            const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, off);
+            const unsigned long long n = __shfl_up_sync(kFull, inc, off);
             if (lane >= off) inc += n;
         }
         if (lane == 31) sm.warp_sums[warp] = inc;
@@ -184,7 +206,7 @@ __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, c
             unsigned long long sinc = s;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                const unsigned long long n = __shfl_up_sync(0xffffffffu, sinc, off);
+                const unsigned long long n = __shfl_up_sync(kFull, sinc, off);
                 if (lane >= off) sinc += n;
             }
             sm.warp_sums[lane] = sinc - s;
@@ -209,12 +231,12 @@ __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, c
             gt_before += gt;
             eq_before += eq;
         };
-        if (IN_REGS && !keep_all) {
+        if (!keep_all) {
 #pragma unroll
-            for (int u = 0; u < KR; ++u)
+            for (int u = 0; u < KPT; ++u)
                 if (c0 + u < c1) visit(c0 + u, keys[u]);
         } else {
-            for (int ch = c0; ch < c1; ++ch) visit(ch, keep_all ? 0u : select_order_key(score_at(ch)));
+            for (int ch = c0; ch < c1; ++ch) visit(ch, 0u);
         }
     }
     __syncthreads();
@@ -224,9 +246,10 @@ __device__ __forceinline__ void select_head_regs(const float* __restrict__ sc, c
     // (Algorithm 1 keeps the first L_max - w selected tokens); no cap by default
     const int n_tok = min(kk * c - ((sm.last_kept && kk > 0) ? (c - tail) : 0), tok_cap);
     if (stage_sel)
-        for (int n = tid; n < n_tok; n += nt) {
-            const int rank = n / c;
-            out[n] = sm.sel[rank] * c + (n - rank * c);
+        for (int r = tid; r < kk; r += nt) {            // one kept chunk per thread: its c positions
+            const int j0 = sm.sel[r] * c, n0 = r * c;
+            for (int t = 0; t < c; ++t)
+                if (n0 + t < n_tok) out[n0 + t] = j0 + t;
         }
     for (int i = tid; i < w; i += nt) out[n_tok + i] = P + i;
     for (int i = n_tok + w + tid; i < n_max; i += nt) out[i] = -1;

@@ -289,6 +289,45 @@ def test_config5_all_ragged_lengths_one_reuse_group(ck):
         del dev, outs
 
 
+@pytest.mark.parametrize("cfg,L,budget,n_layers,n_reuse", [
+    (2, 6000, 600, 5, 2),        # several tiles per CTA, odd layer count, last group incomplete
+    (1, 2048, 256, 4, 1),        # d = 64, 64 rows, every layer computes
+    (5, 5000, 500, 7, 3),        # 256 rows per KV head: two scoring heads per KV head
+    (4, 9000, 900, 3, 3),        # c = 20, w = 64: one computed layer, two that reuse
+    (2, 3001, 47, 3, 2),         # budget just above the window (k = 1), ragged last chunk
+    (2, 150, 140, 2, 2),         # fewer tiles than CTAs per head; almost everything kept
+    (2, 2592 + 32, 2592 + 32, 2, 1),   # k = C: identity, the clipped-chunk padding path is not taken
+    (2, 2595 + 32, 5000, 2, 1),  # k = C with a clipped last chunk: -1 padding and zero rows
+])
+def test_compress_model_persistent_kernel_matches_oracle(ck, cfg, L, budget, n_layers, n_reuse):
+    # chunkkv_compress_model: all layers in one launch, scoring of a layer overlapping the selection
+    # and row copies of the one before; every computed layer against the oracle, every reusing layer
+    # against Algorithm 2 (same indices, rows bit-exact); outputs between guard margins
+    wl = scaled(CONFIGS[cfg], L=L, budget=budget, n_layers=n_layers, rho=0.0)
+    layers = [make_layer(wl, layer=i) for i in range(n_layers)]
+    dev = [(to_dev(x.q_obs) if i % n_reuse == 0 else None, to_dev(x.K), to_dev(x.V)) for i, x in enumerate(layers)]
+    n_max = ck.out_len(wl.L, wl.w, wl.c, wl.budget)
+    guards = [guarded_outputs(wl.Hkv, n_max, wl.d) for _ in range(n_layers)]
+    for rep in range(2):                       # the second call reuses scratch and counters
+        for gs in guards:
+            for g in gs:
+                g.t.view(torch.uint8).fill_(0x5A)
+        outs = ck.compress_model(dev, wl.Hq, wl.w, wl.c, wl.budget, n_reuse=n_reuse,
+                                 outs=[(g[0].t, g[1].t, g[2].t) for g in guards])
+        _status_ok(ck)
+    for gs in guards:
+        for g, name in zip(gs, ("out_K", "out_V", "out_idx")):
+            g.check(name)
+    for l, (x, (oK, oV, idx)) in enumerate(zip(layers, outs)):
+        src = (l // n_reuse) * n_reuse
+        idx_np = idx.cpu().numpy()
+        if l == src:
+            _check_layer(x, wl, bits_of(oK), bits_of(oV), idx_np)
+        else:
+            assert np.array_equal(idx_np, outs[src][2].cpu().numpy())
+            assert_gather_exact(bits_of(oK), bits_of(oV), idx_np, x.K, x.V)
+
+
 def test_compress_layer_host_round_trip(ck):
     wl = scaled(CONFIGS[2], L=3000, budget=300)
     x = make_layer(wl)
@@ -324,7 +363,7 @@ def test_scratch_is_caller_owned_and_never_overrun(ck):
         assert ck.lib.chunkkv_compress_layer(*args) == -4
         assert ck.lib.chunkkv_score(q.data_ptr(), K.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, None,
                                     gS.t.data_ptr(), None) == -4
-        small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+        small = torch.empty(4096, dtype=torch.uint8, device="cuda")      # room for the header only
         ck.set_workspace(small)
         assert ck.lib.chunkkv_compress_layer(*args) == -4
         ws = Guarded((need,), torch.uint8)
