@@ -37,7 +37,7 @@ constexpr int kMThreads = 640;
 constexpr int kMEpiThreads = 512;
 constexpr int kMTailThreads = 64;
 constexpr int kMMiscBytes = 14336;      // epilogue: group records, slices, m_i, 1 / l_i, row sums per lane quarter
-constexpr int kMSlots = 6;              // staging slots of the row copies
+constexpr int kMSlots = 8;              // staging slots of the row copies
 constexpr int kMSelBins = 2048;
 constexpr int kMCandCap = 1024;
 constexpr int kBarEpi = 1, kBarTail = 2;
@@ -128,32 +128,47 @@ __device__ __forceinline__ bool wait_counter(const unsigned* counter, unsigned t
 // Exact top-k of one head's chunk scores by the 64 tail threads (same adaptive radix select as
 // select_head_regs in select.cuh, with the keys in shared memory): fills sel[0 .. kk) with the kept
 // chunk ids in ascending order and returns whether the clipped last chunk is among them.
-__device__ __forceinline__ int tail_select(const float* row2, int C, int k, uint32_t* keys, int* hist,
+// Two warps have little latency hiding of their own, so every pass walks the keys four at a time
+// (16-byte shared-memory accesses) with several independent accesses in flight per thread.
+// keys: Cpad = C rounded up to a multiple of 4 entries; entries at or past C are ignored.
+__device__ __forceinline__ int tail_select(const float* row2, int C, int Cpad, int k, uint32_t* keys, int* hist,
                                            int* sel, ModelCtl& ctl, int tt) {
     // keys[0 .. C) holds the head's chunk scores as floats on entry (row2 != NULL: to be added to a
     // second row, the other half of the head's query rows) and their order-preserving keys afterwards
     constexpr unsigned kFull = 0xffffffffu;
     const int lane = tt & 31, tw = tt >> 5;
-    const int kk = min(k, C);
     if (tt == 0) { ctl.t_last_kept = 0; ctl.t_ncand = 0; }
     if (k >= C) {                      // everything is kept
         for (int ch = tt; ch < C; ch += kMTailThreads) sel[ch] = ch;
         named_barrier(kBarTail, kMTailThreads);
         return C > 0 ? 1 : 0;
     }
+    const int nv = Cpad >> 2;          // 16-byte groups of keys
+    uint4* kv = reinterpret_cast<uint4*>(keys);
+    const float4* r2 = reinterpret_cast<const float4*>(row2);
     uint32_t lo = 0xffffffffu, hi = 0u;
-    for (int ch = tt; ch < C; ch += kMTailThreads) {
-        float s = __uint_as_float(keys[ch]);
-        if (row2 != nullptr) s += row2[ch];
-        const uint32_t key = select_order_key(s);
-        keys[ch] = key;
-        lo = min(lo, key);
-        hi = max(hi, key);
+#pragma unroll 4
+    for (int v = tt; v < nv; v += kMTailThreads) {
+        const uint4 raw = kv[v];
+        float4 f = make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), __uint_as_float(raw.z), __uint_as_float(raw.w));
+        if (row2 != nullptr) { const float4 g = r2[v]; f.x += g.x; f.y += g.y; f.z += g.z; f.w += g.w; }
+        uint4 key = make_uint4(select_order_key(f.x), select_order_key(f.y), select_order_key(f.z), select_order_key(f.w));
+        const int ch = 4 * v;
+        if (ch + 1 >= C) key.y = key.x;      // entries past C copy a valid key: they never widen [min, max]
+        if (ch + 2 >= C) key.z = key.x;
+        if (ch + 3 >= C) key.w = key.x;
+        kv[v] = key;
+        lo = min(min(lo, key.x), min(min(key.y, key.z), key.w));
+        hi = max(max(hi, key.x), max(max(key.y, key.z), key.w));
     }
     lo = __reduce_min_sync(kFull, lo);
     hi = __reduce_max_sync(kFull, hi);
     if (lane == 0) ctl.t_pair[tw] = (static_cast<unsigned long long>(hi) << 32) | lo;
-    for (int i = tt; i < kMSelBins; i += kMTailThreads) hist[i] = 0;
+    {
+        int4* hv = reinterpret_cast<int4*>(hist);
+#pragma unroll
+        for (int i = 0; i < kMSelBins / 4 / kMTailThreads; ++i) hv[tt + i * kMTailThreads] = make_int4(0, 0, 0, 0);
+    }
     named_barrier(kBarTail, kMTailThreads);
     uint32_t base = min(static_cast<uint32_t>(ctl.t_pair[0]), static_cast<uint32_t>(ctl.t_pair[1]));
     const uint32_t top = max(static_cast<uint32_t>(ctl.t_pair[0] >> 32), static_cast<uint32_t>(ctl.t_pair[1] >> 32));
@@ -165,18 +180,31 @@ __device__ __forceinline__ int tail_select(const float* row2, int C, int k, uint
         if (span == 0u) { thresh = base; need_eq = need; break; }
         const int shift = max(0, 21 - __clz(span));
         if (round > 0) {
-            for (int i = tt; i < kMSelBins; i += kMTailThreads) hist[i] = 0;
+            int4* hv = reinterpret_cast<int4*>(hist);
+#pragma unroll
+            for (int i = 0; i < kMSelBins / 4 / kMTailThreads; ++i) hv[tt + i * kMTailThreads] = make_int4(0, 0, 0, 0);
             named_barrier(kBarTail, kMTailThreads);
         }
-        for (int ch = tt; ch < C; ch += kMTailThreads) {
-            const uint32_t key = keys[ch], dlt = key - base;
-            if (key >= base && dlt <= span) atomicAdd(&hist[dlt >> shift], 1);
+#pragma unroll 4
+        for (int v = tt; v < nv; v += kMTailThreads) {
+            const uint4 key = kv[v];
+            const int ch = 4 * v;
+            const uint32_t d0 = key.x - base, d1 = key.y - base, d2 = key.z - base, d3 = key.w - base;
+            if (key.x >= base && d0 <= span) atomicAdd(&hist[d0 >> shift], 1);
+            if (ch + 1 < C && key.y >= base && d1 <= span) atomicAdd(&hist[d1 >> shift], 1);
+            if (ch + 2 < C && key.z >= base && d2 <= span) atomicAdd(&hist[d2 >> shift], 1);
+            if (ch + 3 < C && key.w >= base && d3 <= span) atomicAdd(&hist[d3 >> shift], 1);
         }
         named_barrier(kBarTail, kMTailThreads);
-        // thread t owns bins 2047 - 32 t .. 2016 - 32 t (descending)
-        const int b_hi = kMSelBins - 1 - 32 * tt;
+        // thread t owns bins 2047 - 32 t .. 2016 - 32 t (descending): eight 16-byte loads
+        const int b_lo = kMSelBins - 32 - 32 * tt;
+        const int4* hb = reinterpret_cast<const int4*>(hist + b_lo);
+        int4 hq[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) hq[i] = hb[i];
         int sum = 0;
-        for (int q = 0; q < 32; ++q) sum += hist[b_hi - q];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sum += (hq[i].x + hq[i].y) + (hq[i].z + hq[i].w);
         int inc = sum;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -188,6 +216,7 @@ __device__ __forceinline__ int tail_select(const float* row2, int C, int k, uint
         if (tw == 1) inc += ctl.t_tot[0];
         if (inc - sum < need && need <= inc) {          // exactly one thread
             int above = inc - sum, q = 0;
+            const int b_hi = b_lo + 31;
             while (q < 31 && above + hist[b_hi - q] < need) { above += hist[b_hi - q]; ++q; }
             ctl.t_prefix = static_cast<uint32_t>(b_hi - q);
             ctl.t_need = need - above;
@@ -203,9 +232,14 @@ __device__ __forceinline__ int tail_select(const float* row2, int C, int k, uint
         if (n_bin <= kMCandCap) {
             uint32_t* cand = reinterpret_cast<uint32_t*>(hist);      // the histogram is no longer needed
             named_barrier(kBarTail, kMTailThreads);                   // ... once every thread has read it
-            for (int ch = tt; ch < C; ch += kMTailThreads) {
-                const uint32_t key = keys[ch], dlt = key - base;
-                if (key >= base && dlt <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key;
+#pragma unroll 4
+            for (int v = tt; v < nv; v += kMTailThreads) {
+                const uint4 key = kv[v];
+                const int ch = 4 * v;
+                if (key.x >= base && key.x - base <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key.x;
+                if (ch + 1 < C && key.y >= base && key.y - base <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key.y;
+                if (ch + 2 < C && key.z >= base && key.z - base <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key.z;
+                if (ch + 3 < C && key.w >= base && key.w - base <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key.w;
             }
             named_barrier(kBarTail, kMTailThreads);
             for (int j = tt; j < n_bin; j += kMTailThreads) {
@@ -220,11 +254,17 @@ __device__ __forceinline__ int tail_select(const float* row2, int C, int k, uint
             break;
         }
     }
-    // ordered sweep: thread t owns the contiguous ids [c0, c1)
-    const int per = (C + kMTailThreads - 1) / kMTailThreads;
-    const int c0 = min(tt * per, C), c1 = min(c0 + per, C);
+    // ordered sweep: thread t owns the contiguous 16-byte groups [v0, v1)
+    const int pv = (nv + kMTailThreads - 1) / kMTailThreads;
+    const int v0 = min(tt * pv, nv), v1 = min(v0 + pv, nv);
     unsigned gt_n = 0, eq_n = 0;
-    for (int ch = c0; ch < c1; ++ch) { const uint32_t key = keys[ch]; gt_n += key > thresh; eq_n += key == thresh; }
+#pragma unroll 4
+    for (int v = v0; v < v1; ++v) {
+        const uint4 key = kv[v];
+        const int ch = 4 * v;
+        gt_n += (key.x > thresh) + (ch + 1 < C && key.y > thresh) + (ch + 2 < C && key.z > thresh) + (ch + 3 < C && key.w > thresh);
+        eq_n += (key.x == thresh) + (ch + 1 < C && key.y == thresh) + (ch + 2 < C && key.z == thresh) + (ch + 3 < C && key.w == thresh);
+    }
     const unsigned long long mine = (static_cast<unsigned long long>(eq_n) << 32) | gt_n;
     unsigned long long inc = mine;
 #pragma unroll
@@ -237,8 +277,7 @@ __device__ __forceinline__ int tail_select(const float* row2, int C, int k, uint
     named_barrier(kBarTail, kMTailThreads);
     const unsigned long long excl = (tw == 1 ? ctl.t_pair[0] : 0ull) + inc - mine;
     int gt_before = static_cast<int>(excl & 0xffffffffu), eq_before = static_cast<int>(excl >> 32);
-    for (int ch = c0; ch < c1; ++ch) {
-        const uint32_t key = keys[ch];
+    auto visit = [&](int ch, uint32_t key) {
         const bool gt = key > thresh, eq = key == thresh;
         if (gt || (eq && eq_before < need_eq)) {
             sel[gt_before + min(eq_before, need_eq)] = ch;
@@ -246,9 +285,17 @@ __device__ __forceinline__ int tail_select(const float* row2, int C, int k, uint
         }
         gt_before += gt;
         eq_before += eq;
+    };
+#pragma unroll 2
+    for (int v = v0; v < v1; ++v) {
+        const uint4 key = kv[v];
+        const int ch = 4 * v;
+        visit(ch, key.x);
+        if (ch + 1 < C) visit(ch + 1, key.y);
+        if (ch + 2 < C) visit(ch + 2, key.z);
+        if (ch + 3 < C) visit(ch + 3, key.w);
     }
     named_barrier(kBarTail, kMTailThreads);
-    (void)kk;
     return ctl.t_last_kept;
 }
 
@@ -573,7 +620,7 @@ model_kernel(const __grid_constant__ ModelParams p) {
             named_barrier(kBarTail, kMTailThreads);
             if (ctl.abort_flag) { ok = false; break; }
             const float* row2 = p.kv_shift ? reinterpret_cast<const float*>(keys) + p.Cpad : nullptr;
-            const int last_kept = tail_select(row2, p.C, p.k, keys, hist, sel, ctl, tt);
+            const int last_kept = tail_select(row2, p.C, p.Cpad, p.k, keys, hist, sel, ctl, tt);
             const int n_tok = kk * C_STATIC - ((last_kept && kk > 0) ? (C_STATIC - tail_rows) : 0);
             // ---- this layer and the layers after it that reuse its indices
             int lj = li;
