@@ -622,7 +622,7 @@ size_t chunkkv_model_workspace_bytes(int n_layers, int L, int Hq, int Hkv, int d
     if (C > 0 && k > 0 && make_model_plan(L, sh.Rs, sh.Hs, sh.shift, d, c, C, k, ctx->num_sms, smem_budget(*ctx), &mp)) {
         const int per_launch = n_layers < kModelMaxLayers ? n_layers : kModelMaxLayers;
         const int n_compute = (per_launch + reuse_depth - 1) / reuse_depth + 1;
-        const size_t m = kHeaderBytes + model_scratch_floats(mp, sh.Hs, C, n_compute) * sizeof(float);
+        const size_t m = kHeaderBytes + model_scratch_floats(mp, sh.Hs, sh.shift, C, n_compute) * sizeof(float);
         need = m > need ? m : need;
     }
     return need;
@@ -693,7 +693,7 @@ int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* c
             ++n_compute;
         }
         const int n = l1 - l0;
-        const size_t need = model_scratch_floats(mp, sh.Hs, C, n_compute) * sizeof(float);
+        const size_t need = model_scratch_floats(mp, sh.Hs, sh.shift, C, n_compute) * sizeof(float);
         st = ensure_workspace(*ctx, need);
         if (st != CHUNKKV_OK) return st;
         char* base = static_cast<char*>(ctx->ws);

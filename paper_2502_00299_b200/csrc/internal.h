@@ -13,7 +13,7 @@ namespace chunkkv {
 // counter, then one hand-over counter per scoring head and one per KV head).
 constexpr size_t kHeaderBytes = 2048;
 constexpr size_t kResidentCountersOffset = 192;
-constexpr int kResidentMaxHeads = 224;
+constexpr int kResidentMaxHeads = 148;   // three counter arrays of this length follow the exit counter
 
 // Geometry of one scoring launch, fixed on the host.
 struct ScorePlan {
@@ -119,6 +119,8 @@ constexpr int kModelMaxCompute = 32;    // computed layers per launch
 
 struct ModelPlan {
     int c_static, grid, cph, n_tiles, t_max, n_stages, smem_bytes;
+    int n_score, n_sel;          // scoring CTAs, selector CTAs (grid = n_score + n_sel)
+    int sel_row_bytes, sel_keys_fit;
     int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes;
 };
 
@@ -142,7 +144,7 @@ struct ModelLayerIO {
 
 bool make_model_plan(int L, int Rs, int Hs, int kv_shift, int d, int c, int C, int k, int max_ctas, int smem_limit,
                      ModelPlan* plan);
-size_t model_scratch_floats(const ModelPlan& plan, int Hs, int C, int n_compute);
+size_t model_scratch_floats(const ModelPlan& plan, int Hs, int kv_shift, int C, int n_compute);
 // layers[0] must compute; tm_q / tm_k hold one tensor map per computed layer, in order.
 cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
                          const ModelLayerIO* layers, int n_layers, cudaStream_t stream);

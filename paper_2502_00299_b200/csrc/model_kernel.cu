@@ -33,14 +33,11 @@ namespace chunkkv {
 
 namespace {
 
-constexpr int kMThreads = 640;
+constexpr int kMThreads = 608;          // warp 0: TMA, warp 1: UMMA issue, warps 2..17: epilogue, warp 18: row copies
 constexpr int kMEpiThreads = 512;
-constexpr int kMTailThreads = 64;
 constexpr int kMMiscBytes = 14336;      // epilogue: group records, slices, m_i, 1 / l_i, row sums per lane quarter
 constexpr int kMSlots = 8;              // staging slots of the row copies
-constexpr int kMSelBins = 2048;
-constexpr int kMCandCap = 1024;
-constexpr int kBarEpi = 1, kBarTail = 2;
+constexpr int kBarEpi = 1;
 
 struct ModelCtl {
     unsigned long long full[kRMaxStages];
@@ -50,16 +47,11 @@ struct ModelCtl {
     unsigned long long qfull;
     unsigned long long qempty;
     unsigned long long gfull[kMSlots];
-    unsigned long long sfull;          // the head's chunk scores have landed in shared memory (tail warps)
+    unsigned long long sfull;          // a kept-chunk list has landed in shared memory (copy thread)
     uint32_t tmem_base;
     int abort_flag;
     int epi_ok;
-    // tail warps
-    int tail_ok;
-    unsigned long long t_pair[2];
-    int t_tot[2];
-    uint32_t t_prefix;
-    int t_need, t_bin_count, t_ncand, t_last_kept;
+    int sel_flag[2];                   // selector CTAs: wait result, abort flag
 };
 
 struct ModelLayer {
@@ -82,11 +74,16 @@ struct ModelParams {
     int cph, n_tiles, n_stages, q_box_rows, k_box_rows;
     int C, k, n_max, Hkv;
     int Cpad;              // row stride of the chunk scores (C rounded up to a multiple of 4: rows stay 16-byte aligned)
+    int n_score, n_sel;    // scoring CTAs (Hs * cph) and selector CTAs (the rest of the grid)
+    int sel_row_bytes;     // bytes of one kept-chunk list: 4 header ints + the kept chunk ids, padded to 16 bytes
+    int sel_keys_fit;      // selector: the keys of a head fit its shared memory (many chunks per thread)
     int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes;
     float* cta_stat;       // [2 (slot parity)][grid][{max, sum}][128]
     float* scores;         // [n_compute][Hs][Cpad]
     unsigned* cnt_a;       // [Hs]
-    unsigned* cnt_b;       // [Hs]
+    unsigned* cnt_b;       // [Hs]   chunk scores of a slot announced by the scoring CTAs
+    unsigned* cnt_c;       // [Hkv]  kept-chunk lists announced by the selector CTAs
+    int* sel_rows;         // [n_compute][Hkv][sel_row_bytes / 4]
     unsigned* exits;
     int* status;
 };
@@ -125,178 +122,69 @@ __device__ __forceinline__ bool wait_counter(const unsigned* counter, unsigned t
     }
 }
 
-// Exact top-k of one head's chunk scores by the 64 tail threads (same adaptive radix select as
-// select_head_regs in select.cuh, with the keys in shared memory): fills sel[0 .. kk) with the kept
-// chunk ids in ascending order and returns whether the clipped last chunk is among them.
-// Two warps have little latency hiding of their own, so every pass walks the keys four at a time
-// (16-byte shared-memory accesses) with several independent accesses in flight per thread.
-// keys: Cpad = C rounded up to a multiple of 4 entries; entries at or past C are ignored.
-__device__ __forceinline__ int tail_select(const float* row2, int C, int Cpad, int k, uint32_t* keys, int* hist,
-                                           int* sel, ModelCtl& ctl, int tt) {
-    // keys[0 .. C) holds the head's chunk scores as floats on entry (row2 != NULL: to be added to a
-    // second row, the other half of the head's query rows) and their order-preserving keys afterwards
-    constexpr unsigned kFull = 0xffffffffu;
-    const int lane = tt & 31, tw = tt >> 5;
-    if (tt == 0) { ctl.t_last_kept = 0; ctl.t_ncand = 0; }
-    if (k >= C) {                      // everything is kept
-        for (int ch = tt; ch < C; ch += kMTailThreads) sel[ch] = ch;
-        named_barrier(kBarTail, kMTailThreads);
-        return C > 0 ? 1 : 0;
-    }
-    const int nv = Cpad >> 2;          // 16-byte groups of keys
-    uint4* kv = reinterpret_cast<uint4*>(keys);
-    const float4* r2 = reinterpret_cast<const float4*>(row2);
-    uint32_t lo = 0xffffffffu, hi = 0u;
-#pragma unroll 4
-    for (int v = tt; v < nv; v += kMTailThreads) {
-        const uint4 raw = kv[v];
-        float4 f = make_float4(__uint_as_float(raw.x), __uint_as_float(raw.y), __uint_as_float(raw.z), __uint_as_float(raw.w));
-        if (row2 != nullptr) { const float4 g = r2[v]; f.x += g.x; f.y += g.y; f.z += g.z; f.w += g.w; }
-        uint4 key = make_uint4(select_order_key(f.x), select_order_key(f.y), select_order_key(f.z), select_order_key(f.w));
-        const int ch = 4 * v;
-        if (ch + 1 >= C) key.y = key.x;      // entries past C copy a valid key: they never widen [min, max]
-        if (ch + 2 >= C) key.z = key.x;
-        if (ch + 3 >= C) key.w = key.x;
-        kv[v] = key;
-        lo = min(min(lo, key.x), min(min(key.y, key.z), key.w));
-        hi = max(max(hi, key.x), max(max(key.y, key.z), key.w));
-    }
-    lo = __reduce_min_sync(kFull, lo);
-    hi = __reduce_max_sync(kFull, hi);
-    if (lane == 0) ctl.t_pair[tw] = (static_cast<unsigned long long>(hi) << 32) | lo;
-    {
-        int4* hv = reinterpret_cast<int4*>(hist);
-#pragma unroll
-        for (int i = 0; i < kMSelBins / 4 / kMTailThreads; ++i) hv[tt + i * kMTailThreads] = make_int4(0, 0, 0, 0);
-    }
-    named_barrier(kBarTail, kMTailThreads);
-    uint32_t base = min(static_cast<uint32_t>(ctl.t_pair[0]), static_cast<uint32_t>(ctl.t_pair[1]));
-    const uint32_t top = max(static_cast<uint32_t>(ctl.t_pair[0] >> 32), static_cast<uint32_t>(ctl.t_pair[1] >> 32));
-    uint32_t span = top - base;
-    int need = k;
-    uint32_t thresh = 0;
-    int need_eq = 0;
-    for (int round = 0;; ++round) {
-        if (span == 0u) { thresh = base; need_eq = need; break; }
-        const int shift = max(0, 21 - __clz(span));
-        if (round > 0) {
-            int4* hv = reinterpret_cast<int4*>(hist);
-#pragma unroll
-            for (int i = 0; i < kMSelBins / 4 / kMTailThreads; ++i) hv[tt + i * kMTailThreads] = make_int4(0, 0, 0, 0);
-            named_barrier(kBarTail, kMTailThreads);
-        }
-#pragma unroll 4
-        for (int v = tt; v < nv; v += kMTailThreads) {
-            const uint4 key = kv[v];
-            const int ch = 4 * v;
-            const uint32_t d0 = key.x - base, d1 = key.y - base, d2 = key.z - base, d3 = key.w - base;
-            if (key.x >= base && d0 <= span) atomicAdd(&hist[d0 >> shift], 1);
-            if (ch + 1 < C && key.y >= base && d1 <= span) atomicAdd(&hist[d1 >> shift], 1);
-            if (ch + 2 < C && key.z >= base && d2 <= span) atomicAdd(&hist[d2 >> shift], 1);
-            if (ch + 3 < C && key.w >= base && d3 <= span) atomicAdd(&hist[d3 >> shift], 1);
-        }
-        named_barrier(kBarTail, kMTailThreads);
-        // thread t owns bins 2047 - 32 t .. 2016 - 32 t (descending): eight 16-byte loads
-        const int b_lo = kMSelBins - 32 - 32 * tt;
-        const int4* hb = reinterpret_cast<const int4*>(hist + b_lo);
-        int4 hq[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) hq[i] = hb[i];
-        int sum = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) sum += (hq[i].x + hq[i].y) + (hq[i].z + hq[i].w);
-        int inc = sum;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int n = __shfl_up_sync(kFull, inc, off);
-            if (lane >= off) inc += n;
-        }
-        if (lane == 31) ctl.t_tot[tw] = inc;
-        named_barrier(kBarTail, kMTailThreads);
-        if (tw == 1) inc += ctl.t_tot[0];
-        if (inc - sum < need && need <= inc) {          // exactly one thread
-            int above = inc - sum, q = 0;
-            const int b_hi = b_lo + 31;
-            while (q < 31 && above + hist[b_hi - q] < need) { above += hist[b_hi - q]; ++q; }
-            ctl.t_prefix = static_cast<uint32_t>(b_hi - q);
-            ctl.t_need = need - above;
-            ctl.t_bin_count = hist[b_hi - q];
-        }
-        named_barrier(kBarTail, kMTailThreads);
-        const uint32_t bin = ctl.t_prefix;
-        const int n_bin = ctl.t_bin_count;
-        need = ctl.t_need;
-        const uint32_t sub = bin << shift;
-        base += sub;
-        span = min((1u << shift) - 1u, span - sub);
-        if (n_bin <= kMCandCap) {
-            uint32_t* cand = reinterpret_cast<uint32_t*>(hist);      // the histogram is no longer needed
-            named_barrier(kBarTail, kMTailThreads);                   // ... once every thread has read it
-#pragma unroll 4
-            for (int v = tt; v < nv; v += kMTailThreads) {
-                const uint4 key = kv[v];
-                const int ch = 4 * v;
-                if (key.x >= base && key.x - base <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key.x;
-                if (ch + 1 < C && key.y >= base && key.y - base <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key.y;
-                if (ch + 2 < C && key.z >= base && key.z - base <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key.z;
-                if (ch + 3 < C && key.w >= base && key.w - base <= span) cand[atomicAdd(&ctl.t_ncand, 1)] = key.w;
+// Selector CTA (the CTAs after the scoring CTAs; they run on SMs the scoring grid leaves free): for
+// every slot and each of its KV heads, once the head's chunk scores are complete, the whole CTA
+// runs the exact top-k (select.cuh), writes the kept positions to out_idx of the computed layer
+// and of every layer that reuses its indices (and zero rows behind the kept rows, which exist
+// only when the clipped last chunk is kept), publishes the kept-chunk list for the scoring CTAs'
+// copy threads and announces it on the head's third counter.
+template <int C_STATIC>
+__device__ __forceinline__ bool selector_loop(const ModelParams& p, uint8_t* dyn, int* flag_smem) {
+    SelectSmem& ss = *reinterpret_cast<SelectSmem*>(dyn);
+    constexpr size_t kSelBytes = (sizeof(SelectSmem) + 127) & ~size_t(127);
+    int32_t* sidx = reinterpret_cast<int32_t*>(dyn + kSelBytes);                  // [n_max] kept positions
+    const size_t idx_bytes = (static_cast<size_t>(p.n_max) * 4 + 127) & ~size_t(127);
+    uint32_t* kbuf = reinterpret_cast<uint32_t*>(dyn + kSelBytes + idx_bytes);    // keys, when there are many chunks per thread
+    const int sid = static_cast<int>(blockIdx.x) - p.n_score;
+    const int kk = min(p.k, p.C);
+    const int tail_rows = (p.C > 0) ? (p.P - (p.C - 1) * C_STATIC) : 0;
+    const int row_ints = p.sel_row_bytes / 4;
+    volatile int* flag = flag_smem;
+    for (int li = 0; li < p.n_layers;) {
+        const int s = p.layer[li].slot;
+        int lj_end = li + 1;
+        while (lj_end < p.n_layers && !p.layer[lj_end].computes) ++lj_end;
+        for (int hkv = sid; hkv < p.Hkv; hkv += p.n_sel) {
+            if (threadIdx.x == 0) {
+                const unsigned target = static_cast<unsigned>(s + 1) * p.cph;
+                bool w_ok = wait_counter(p.cnt_b + (hkv << p.kv_shift), target, flag + 1, 100);
+                if (w_ok && p.kv_shift) w_ok = wait_counter(p.cnt_b + (hkv << p.kv_shift) + 1, target, flag + 1, 100);
+                asm volatile("fence.acq_rel.gpu;" ::: "memory");
+                flag[0] = w_ok ? 1 : 0;
             }
-            named_barrier(kBarTail, kMTailThreads);
-            for (int j = tt; j < n_bin; j += kMTailThreads) {
-                const uint32_t v = cand[j];
-                int gt = 0, ge = 0;
-                for (int i = 0; i < n_bin; ++i) { gt += cand[i] > v; ge += cand[i] >= v; }
-                if (gt < need && need <= ge) { ctl.t_prefix = v; ctl.t_need = need - gt; }
+            __syncthreads();
+            if (!flag[0]) return false;
+            const float* sc = p.scores + (static_cast<size_t>(s) * p.Hs + (hkv << p.kv_shift)) * p.Cpad;
+            const float* sc2 = p.kv_shift ? sc + p.Cpad : nullptr;
+            if (p.C <= kMThreads * 8)
+                select_head_regs<8>(sc, sc2, p.L, p.w, C_STATIC, p.C, p.k, p.n_max, sidx, ss);
+            else
+                select_head_rows(sc, sc2, p.L, p.w, C_STATIC, p.C, p.k, p.n_max, sidx, ss,
+                                 p.sel_keys_fit ? kbuf : nullptr);
+            const int n_tok = kk * C_STATIC - ((ss.last_kept && kk > 0) ? (C_STATIC - tail_rows) : 0);
+            // the kept-chunk list for the copy threads: [n_tok, -, -, -, chunk ids]
+            int* row = p.sel_rows + (static_cast<size_t>(s) * p.Hkv + hkv) * row_ints;
+            if (threadIdx.x == 0) row[0] = n_tok;
+            for (int r = threadIdx.x; r < kk; r += kMThreads) row[4 + r] = ss.sel[r];
+            const int vpr = p.d >> 3;
+            for (int lj = li; lj < lj_end; ++lj) {
+                const ModelLayer& ly = p.layer[lj];
+                int32_t* dst = ly.out_idx + static_cast<size_t>(hkv) * p.n_max;
+                for (int n = threadIdx.x; n < p.n_max; n += kMThreads) dst[n] = sidx[n];
+                uint4* zk = ly.out_K + (static_cast<size_t>(hkv) * p.n_max + n_tok + p.w) * vpr;
+                uint4* zv = ly.out_V + (static_cast<size_t>(hkv) * p.n_max + n_tok + p.w) * vpr;
+                const int nz = (p.n_max - n_tok - p.w) * vpr;
+                for (int i = threadIdx.x; i < nz; i += kMThreads) { zk[i] = make_uint4(0, 0, 0, 0); zv[i] = make_uint4(0, 0, 0, 0); }
             }
-            named_barrier(kBarTail, kMTailThreads);
-            thresh = ctl.t_prefix;
-            need_eq = ctl.t_need;
-            break;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                unsigned old;   // release: the list and the positions written above are visible to whoever sees the count
+                asm volatile("atom.add.release.gpu.u32 %0, [%1], 1;" : "=r"(old) : "l"(p.cnt_c + hkv) : "memory");
+            }
         }
+        li = lj_end;
     }
-    // ordered sweep: thread t owns the contiguous 16-byte groups [v0, v1)
-    const int pv = (nv + kMTailThreads - 1) / kMTailThreads;
-    const int v0 = min(tt * pv, nv), v1 = min(v0 + pv, nv);
-    unsigned gt_n = 0, eq_n = 0;
-#pragma unroll 4
-    for (int v = v0; v < v1; ++v) {
-        const uint4 key = kv[v];
-        const int ch = 4 * v;
-        gt_n += (key.x > thresh) + (ch + 1 < C && key.y > thresh) + (ch + 2 < C && key.z > thresh) + (ch + 3 < C && key.w > thresh);
-        eq_n += (key.x == thresh) + (ch + 1 < C && key.y == thresh) + (ch + 2 < C && key.z == thresh) + (ch + 3 < C && key.w == thresh);
-    }
-    const unsigned long long mine = (static_cast<unsigned long long>(eq_n) << 32) | gt_n;
-    unsigned long long inc = mine;
-#pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const unsigned long long n = __shfl_up_sync(kFull, inc, off);
-        if (lane >= off) inc += n;
-    }
-    named_barrier(kBarTail, kMTailThreads);           // t_pair was read above by every thread
-    if (lane == 31) ctl.t_pair[tw] = inc;
-    named_barrier(kBarTail, kMTailThreads);
-    const unsigned long long excl = (tw == 1 ? ctl.t_pair[0] : 0ull) + inc - mine;
-    int gt_before = static_cast<int>(excl & 0xffffffffu), eq_before = static_cast<int>(excl >> 32);
-    auto visit = [&](int ch, uint32_t key) {
-        const bool gt = key > thresh, eq = key == thresh;
-        if (gt || (eq && eq_before < need_eq)) {
-            sel[gt_before + min(eq_before, need_eq)] = ch;
-            if (ch == C - 1) ctl.t_last_kept = 1;
-        }
-        gt_before += gt;
-        eq_before += eq;
-    };
-#pragma unroll 2
-    for (int v = v0; v < v1; ++v) {
-        const uint4 key = kv[v];
-        const int ch = 4 * v;
-        visit(ch, key.x);
-        if (ch + 1 < C) visit(ch + 1, key.y);
-        if (ch + 2 < C) visit(ch + 2, key.z);
-        if (ch + 3 < C) visit(ch + 3, key.w);
-    }
-    named_barrier(kBarTail, kMTailThreads);
-    return ctl.t_last_kept;
+    return true;
 }
 
 template <int C_STATIC>
@@ -324,6 +212,26 @@ model_kernel(const __grid_constant__ ModelParams p) {
     volatile int* abort_flag = &ctl.abort_flag;
     const uint32_t n_stages = static_cast<uint32_t>(p.n_stages);
 
+    if (static_cast<int>(blockIdx.x) >= p.n_score) {
+        // ------------------------------------------------------------------ selector CTA
+        if (threadIdx.x == 0) { ctl.sel_flag[0] = 1; ctl.sel_flag[1] = 0; }
+        __syncthreads();
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        const bool s_ok = selector_loop<C_STATIC>(p, dyn, ctl.sel_flag);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            if (!s_ok) atomicExch(p.status, 1);
+            const unsigned old = atomicAdd(p.exits, 1u);
+            if (old + 1u == gridDim.x) {
+                for (int h = 0; h < p.Hs; ++h) { p.cnt_a[h] = 0u; p.cnt_b[h] = 0u; }
+                for (int h = 0; h < p.Hkv; ++h) p.cnt_c[h] = 0u;
+                *p.exits = 0u;
+                __threadfence();
+            }
+        }
+        return;
+    }
     const int hs = blockIdx.x / p.cph, part = blockIdx.x - hs * p.cph;
     const int hkv = hs >> p.kv_shift;
     const int t_begin = p.n_tiles * part / p.cph, t_end = p.n_tiles * (part + 1) / p.cph;
@@ -344,7 +252,6 @@ model_kernel(const __grid_constant__ ModelParams p) {
         mbar_init(smem_u32(&ctl.sfull), 1);
         ctl.abort_flag = 0;
         ctl.epi_ok = 1;
-        ctl.tail_ok = 1;
         fence_mbar_init();
         fence_proxy_async();
     }
@@ -572,98 +479,63 @@ model_kernel(const __grid_constant__ ModelParams p) {
         }
         if (!ok && lane == 0) ctl.abort_flag = 1;
     } else {
-        // ------------------------------------------------------------------ tail: select + row copies
-        const int tt = threadIdx.x - 576;                // 0 .. 63
-        uint8_t* tbase = dyn + p.off_tail;
-        int* hist = reinterpret_cast<int*>(tbase);                                   // 2048 bins (8 KB)
-        uint32_t* keys = reinterpret_cast<uint32_t*>(tbase + 8192);                  // [1 or 2][Cpad] scores, then C keys
-        const size_t keys_bytes = ((static_cast<size_t>(p.Cpad) * 4 << p.kv_shift) + 127) & ~size_t(127);
-        int* sel = reinterpret_cast<int*>(tbase + 8192 + keys_bytes);                // kept chunk ids
-        const size_t sel_bytes = (static_cast<size_t>(min(p.k, p.C)) * 4 + 127) & ~size_t(127);
-        const uint32_t stage0 = smem_u32(tbase + 8192 + keys_bytes + sel_bytes);     // kMSlots x stage_slot_bytes, 128-byte aligned
-        const int Q = p.cph << p.kv_shift;               // CTAs of this KV head
-        const int q = static_cast<int>(blockIdx.x) - (hkv << p.kv_shift) * p.cph;
-        const int kk = min(p.k, p.C);
-        const int wu = (p.w + C_STATIC - 1) / C_STATIC;  // the window as pseudo-chunks of up to c rows
-        const int U = kk + wu;                           // copy units of the head
-        const int u_begin = static_cast<int>(static_cast<long long>(U) * q / Q);
-        const int u_end = static_cast<int>(static_cast<long long>(U) * (q + 1) / Q);
-        const uint32_t row_bytes = static_cast<uint32_t>(p.d) * 2u;
-        const int tail_rows = (p.C > 0) ? (p.P - (p.C - 1) * C_STATIC) : 0;      // rows of the clipped last chunk
-        uint32_t g_issued = 0;                           // units loaded so far (all layers): slot = g % kMSlots
-        bool ok = true;
-        for (int li = 0; li < p.n_layers && ok;) {
-            const int s = p.layer[li].slot;
-            // ---- the head's chunk scores of slot s are complete once every CTA of its scoring heads has
-            //      announced them; one bulk copy per row brings them into shared memory
-            if (tt == 0) {
-                const unsigned target = static_cast<unsigned>(s + 1) * p.cph;
-                bool w_ok = wait_counter(p.cnt_b + (hkv << p.kv_shift), target, abort_flag, 200);
-                if (w_ok && p.kv_shift) w_ok = wait_counter(p.cnt_b + (hkv << p.kv_shift) + 1, target, abort_flag, 200);
+        // ------------------------------------------------------------------ tail: row copies
+        // One thread: waits until the selector CTA has published the head's kept-chunk list of a
+        // slot, fetches the list, and moves this CTA's share of the rows - whole chunks and window
+        // pieces - through the staging slots with bulk copies, for the computed layer and for every
+        // layer that reuses its indices.
+        if (lane == 0) {
+            uint8_t* tbase = dyn + p.off_tail;
+            int* row = reinterpret_cast<int*>(tbase);        // [4 + kkpad]: n_tok, -, -, -, kept chunk ids
+            const uint32_t stage0 = smem_u32(tbase + p.sel_row_bytes);
+            const int* sel = row + 4;
+            const int Q = p.cph << p.kv_shift;               // CTAs of this KV head
+            const int q = static_cast<int>(blockIdx.x) - (hkv << p.kv_shift) * p.cph;
+            const int kk = min(p.k, p.C);
+            const int wu = (p.w + C_STATIC - 1) / C_STATIC;  // the window as pseudo-chunks of up to c rows
+            const int U = kk + wu;                           // copy units of the head
+            const int u_begin = static_cast<int>(static_cast<long long>(U) * q / Q);
+            const int u_end = static_cast<int>(static_cast<long long>(U) * (q + 1) / Q);
+            const int n_units = u_end - u_begin;
+            const uint32_t row_bytes = static_cast<uint32_t>(p.d) * 2u;
+            const uint32_t half_slot = static_cast<uint32_t>(p.stage_slot_bytes) / 2u;
+            uint32_t g_issued = 0;                           // units loaded so far (all layers): slot = g % kMSlots
+            bool ok = true;
+            for (int li = 0; li < p.n_layers && ok;) {
+                const int s = p.layer[li].slot;
+                ok = wait_counter(p.cnt_c + hkv, static_cast<unsigned>(s + 1), abort_flag, 200);
+                if (!ok) break;
                 asm volatile("fence.acq_rel.gpu;" ::: "memory");
-                if (w_ok) {
-                    const float* sc = p.scores + (static_cast<size_t>(s) * p.Hs + (hkv << p.kv_shift)) * p.Cpad;
-                    const uint32_t bytes = static_cast<uint32_t>(p.Cpad) * 4u << p.kv_shift;     // the rows are adjacent
+                {
                     const uint32_t bar = smem_u32(&ctl.sfull);
-                    mbar_arrive_expect_tx(bar, bytes);
-                    // the scores were written with ordinary stores by other CTAs: order them before the bulk copy's reads
+                    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(p.sel_row_bytes));
+                    // the list was written with ordinary stores by the selector CTA
                     asm volatile("fence.proxy.async.global;" ::: "memory");
-                    bulk_load(smem_u32(keys), sc, bytes, bar);
+                    bulk_load(smem_u32(row), p.sel_rows + (static_cast<size_t>(s) * p.Hkv + hkv) * (p.sel_row_bytes / 4),
+                              static_cast<uint32_t>(p.sel_row_bytes), bar);
+                    ok = mbar_wait(bar, static_cast<uint32_t>(s) & 1u, abort_flag);
+                    if (!ok) break;
                 }
-                ctl.tail_ok = w_ok ? 1 : 0;
-            }
-            named_barrier(kBarTail, kMTailThreads);
-            if (!ctl.tail_ok) { ok = false; break; }
-            if (!mbar_wait(smem_u32(&ctl.sfull), static_cast<uint32_t>(s) & 1u, abort_flag)) { ok = false; }
-            // (every tail thread waits by itself; a thread that gave up has raised the abort flag, which the
-            //  others see in their own wait)
-            named_barrier(kBarTail, kMTailThreads);
-            if (ctl.abort_flag) { ok = false; break; }
-            const float* row2 = p.kv_shift ? reinterpret_cast<const float*>(keys) + p.Cpad : nullptr;
-            const int last_kept = tail_select(row2, p.C, p.Cpad, p.k, keys, hist, sel, ctl, tt);
-            const int n_tok = kk * C_STATIC - ((last_kept && kk > 0) ? (C_STATIC - tail_rows) : 0);
-            // ---- this layer and the layers after it that reuse its indices
-            int lj = li;
-            do {
-                const ModelLayer& ly = p.layer[lj];
-                if (q == 0) {        // one CTA per head writes the kept positions
-                    int32_t* dst = ly.out_idx + static_cast<size_t>(hkv) * p.n_max;
-                    for (int r = tt; r < kk; r += kMTailThreads) {
-                        const int j0 = sel[r] * C_STATIC, n0 = r * C_STATIC;
-#pragma unroll
-                        for (int t = 0; t < C_STATIC; ++t)
-                            if (n0 + t < n_tok) dst[n0 + t] = j0 + t;
+                const int n_tok = row[0];
+                auto unit = [&](int u, int& src_row, int& dst_row, int& rows) {
+                    if (u < kk) {
+                        src_row = sel[u] * C_STATIC;
+                        dst_row = u * C_STATIC;
+                        rows = min(C_STATIC, p.P - src_row);
+                    } else {
+                        const int j = u - kk;
+                        src_row = p.P + j * C_STATIC;
+                        dst_row = n_tok + j * C_STATIC;
+                        rows = min(C_STATIC, p.L - src_row);
                     }
-                    for (int i = tt; i < p.w; i += kMTailThreads) dst[n_tok + i] = p.P + i;
-                    for (int i = n_tok + p.w + tt; i < p.n_max; i += kMTailThreads) dst[i] = -1;
-                    // rows past the kept ones (only when the clipped last chunk is kept) are zero rows
-                    const int vpr = p.d >> 3;
-                    uint4* zk = ly.out_K + (static_cast<size_t>(hkv) * p.n_max + n_tok + p.w) * vpr;
-                    uint4* zv = ly.out_V + (static_cast<size_t>(hkv) * p.n_max + n_tok + p.w) * vpr;
-                    const int nz = (p.n_max - n_tok - p.w) * vpr;
-                    for (int i = tt; i < nz; i += kMTailThreads) { zk[i] = make_uint4(0, 0, 0, 0); zv[i] = make_uint4(0, 0, 0, 0); }
-                }
-                // ---- this CTA's units: whole chunks (and window pieces) through the staging slots
-                if (tt == 0) {
+                };
+                int lj = li;
+                do {
+                    const ModelLayer& ly = p.layer[lj];
                     const char* Kh = reinterpret_cast<const char*>(ly.K) + static_cast<size_t>(hkv) * p.L * row_bytes;
                     const char* Vh = reinterpret_cast<const char*>(ly.V) + static_cast<size_t>(hkv) * p.L * row_bytes;
                     char* oK = reinterpret_cast<char*>(ly.out_K) + static_cast<size_t>(hkv) * p.n_max * row_bytes;
                     char* oV = reinterpret_cast<char*>(ly.out_V) + static_cast<size_t>(hkv) * p.n_max * row_bytes;
-                    const uint32_t half_slot = static_cast<uint32_t>(p.stage_slot_bytes) / 2u;
-                    auto unit = [&](int u, int& src_row, int& dst_row, int& rows) {
-                        if (u < kk) {
-                            src_row = sel[u] * C_STATIC;
-                            dst_row = u * C_STATIC;
-                            rows = min(C_STATIC, p.P - src_row);
-                        } else {
-                            const int j = u - kk;
-                            src_row = p.P + j * C_STATIC;
-                            dst_row = n_tok + j * C_STATIC;
-                            rows = min(C_STATIC, p.L - src_row);
-                        }
-                    };
-                    const int n_units = u_end - u_begin;
-                    // loads run kMSlots - 1 units ahead of the stores
                     int loaded = 0;
                     auto issue_load = [&](int idx) {
                         int sr, dr, rows;
@@ -675,13 +547,13 @@ model_kernel(const __grid_constant__ ModelParams p) {
                         bulk_load(stage0 + slot * p.stage_slot_bytes, Kh + static_cast<size_t>(sr) * row_bytes, bytes, bar);
                         bulk_load(stage0 + slot * p.stage_slot_bytes + half_slot, Vh + static_cast<size_t>(sr) * row_bytes, bytes, bar);
                     };
+                    // loads run kMSlots - 1 units ahead of the stores
                     for (; loaded < n_units && loaded < kMSlots - 1; ++loaded) issue_load(loaded);
-                    bool c_ok = true;
-                    for (int idx = 0; idx < n_units && c_ok; ++idx) {
+                    for (int idx = 0; idx < n_units && ok; ++idx) {
                         const uint32_t gi = g_issued + idx;
                         const uint32_t slot = gi % kMSlots;
-                        c_ok = mbar_wait(smem_u32(&ctl.gfull[slot]), (gi / kMSlots) & 1u, abort_flag);
-                        if (!c_ok) break;
+                        ok = mbar_wait(smem_u32(&ctl.gfull[slot]), (gi / kMSlots) & 1u, abort_flag);
+                        if (!ok) break;
                         int sr, dr, rows;
                         unit(u_begin + idx, sr, dr, rows);
                         const uint32_t bytes = static_cast<uint32_t>(rows) * row_bytes;
@@ -697,16 +569,13 @@ model_kernel(const __grid_constant__ ModelParams p) {
                     }
                     bulk_wait_read<0>();          // the slots are reused by the next layer's first loads
                     g_issued += static_cast<uint32_t>(n_units);
-                    ctl.tail_ok = c_ok ? 1 : 0;
-                }
-                named_barrier(kBarTail, kMTailThreads);
-                if (!ctl.tail_ok) { ok = false; break; }
-                ++lj;
-            } while (lj < p.n_layers && !p.layer[lj].computes);
-            li = lj;
+                    ++lj;
+                } while (ok && lj < p.n_layers && !p.layer[lj].computes);
+                li = lj;
+            }
+            bulk_wait_all();
+            if (!ok) ctl.abort_flag = 1;
         }
-        if (tt == 0) bulk_wait_all();
-        if (!ok && tt == 0) ctl.abort_flag = 1;
     }
 
     tc_fence_before();
@@ -720,6 +589,7 @@ model_kernel(const __grid_constant__ ModelParams p) {
         const unsigned old = atomicAdd(p.exits, 1u);
         if (old + 1u == gridDim.x) {
             for (int h = 0; h < p.Hs; ++h) { p.cnt_a[h] = 0u; p.cnt_b[h] = 0u; }
+            for (int h = 0; h < p.Hkv; ++h) p.cnt_c[h] = 0u;
             *p.exits = 0u;
             __threadfence();
         }
@@ -733,22 +603,27 @@ bool make_model_plan(int L, int Rs, int Hs, int kv_shift, int d, int c, int C, i
     if (c != 10 && c != 20) return false;
     if (Rs < 1 || Rs > 128 || (d != 64 && d != 128) || L < 1 || C < 1 || k < 1 || Hs < 1 || Hs > kResidentMaxHeads)
         return false;
-    if (max_ctas < Hs) return false;
+    const int Hkv = Hs >> kv_shift;
+    const int kk = k < C ? k : C;
+    if (kk > kSelCap) return false;                          // the selector stages the kept chunk ids in shared memory
+    if (max_ctas < Hs + 1) return false;
     ModelPlan p{};
     p.c_static = c;
-    p.cph = max_ctas / Hs;
-    p.grid = p.cph * Hs;
+    // a few CTAs do nothing but select (they take the SMs the scoring grid would leave idle anyway)
+    p.n_sel = Hkv < 4 ? Hkv : 4;
+    if (max_ctas - p.n_sel < Hs) p.n_sel = max_ctas - Hs;
+    p.cph = (max_ctas - p.n_sel) / Hs;
+    p.n_score = p.cph * Hs;
+    p.grid = p.n_score + p.n_sel;
     p.n_tiles = (L + kRTile - 1) / kRTile;
     p.t_max = (p.n_tiles + p.cph - 1) / p.cph;
     if (p.t_max * (kRTile / c) > kRPartCols) return false;
     const int KB = d / 64;
     const int q_bytes = KB * kRQTileBytes;
     const int pmax_bytes = p.t_max * 2 * 128 * 4;
-    const int kk = k < C ? k : C;
     p.stage_slot_bytes = 2 * c * d * 2;                        // K rows and V rows of one chunk
-    const int cpad = (C + 3) & ~3;
-    const int tail_bytes = 8192 + (((cpad * 4 << kv_shift) + 127) & ~127) + ((kk * 4 + 127) & ~127) +
-                           kMSlots * p.stage_slot_bytes + 128;
+    p.sel_row_bytes = ((4 + kk) * 4 + 127) & ~127;
+    const int tail_bytes = p.sel_row_bytes + kMSlots * p.stage_slot_bytes + 128;
     const int fixed = 1024 + q_bytes + 1024 + pmax_bytes + kMMiscBytes + tail_bytes;
     int ns = (smem_limit - 512 - fixed) / kRStageBytes;           // (the control block is larger than the layer kernel's)
     if (ns > kRMaxStages) ns = kRMaxStages;
@@ -759,12 +634,18 @@ bool make_model_plan(int L, int Rs, int Hs, int kv_shift, int d, int c, int C, i
     p.off_misc = p.off_pmax + pmax_bytes;
     p.off_tail = p.off_misc + kMMiscBytes;
     p.smem_bytes = 1024 + p.off_tail + tail_bytes;
+    // the selector CTAs use the same allocation for their scratch, the kept positions and (many chunks) the keys
+    const size_t n_max = static_cast<size_t>(kk) * c + 4096;      // (w <= 256 rows; generous)
+    const size_t sel_need = ((sizeof(SelectSmem) + 127) & ~size_t(127)) + ((n_max * 4 + 127) & ~size_t(127));
+    if (sel_need + 1024 > static_cast<size_t>(p.smem_bytes)) return false;
+    p.sel_keys_fit = (sel_need + static_cast<size_t>(C) * 4 + 1024 <= static_cast<size_t>(p.smem_bytes)) ? 1 : 0;
     *plan = p;
     return true;
 }
 
-size_t model_scratch_floats(const ModelPlan& plan, int Hs, int C, int n_compute) {
-    return static_cast<size_t>(2) * plan.grid * 256 + static_cast<size_t>(n_compute) * Hs * ((C + 3) & ~3) + 64;
+size_t model_scratch_floats(const ModelPlan& plan, int Hs, int kv_shift, int C, int n_compute) {
+    return static_cast<size_t>(2) * plan.grid * 256 + static_cast<size_t>(n_compute) * Hs * ((C + 3) & ~3) +
+           static_cast<size_t>(n_compute) * (Hs >> kv_shift) * (plan.sel_row_bytes / 4) + 64;
 }
 
 cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
@@ -796,13 +677,17 @@ cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtenso
     p.k_box_rows = io.L < kRTile ? io.L : kRTile;
     p.C = io.C; p.k = io.k; p.n_max = io.n_max; p.Hkv = io.Hs >> io.kv_shift;
     p.Cpad = (io.C + 3) & ~3;
+    p.n_score = plan.n_score; p.n_sel = plan.n_sel;
+    p.sel_row_bytes = plan.sel_row_bytes; p.sel_keys_fit = plan.sel_keys_fit;
     p.off_ring = plan.off_ring; p.off_pmax = plan.off_pmax; p.off_misc = plan.off_misc; p.off_tail = plan.off_tail;
     p.stage_slot_bytes = plan.stage_slot_bytes;
     p.cta_stat = io.scratch;
     p.scores = io.scratch + static_cast<size_t>(2) * plan.grid * 256;
+    p.sel_rows = reinterpret_cast<int*>(p.scores + static_cast<size_t>(n_compute) * io.Hs * p.Cpad);   // 16-byte aligned: Cpad % 4 == 0
     p.exits = io.counters;
     p.cnt_a = io.counters + 16;
     p.cnt_b = io.counters + 16 + kResidentMaxHeads;
+    p.cnt_c = io.counters + 16 + 2 * kResidentMaxHeads;
     p.status = io.status;
     const void* kern = plan.c_static == 10 ? reinterpret_cast<const void*>(model_kernel<10>)
                                            : reinterpret_cast<const void*>(model_kernel<20>);
