@@ -33,11 +33,13 @@ namespace chunkkv {
 
 namespace {
 
-constexpr int kMThreads = 608;          // warp 0: TMA, warp 1: UMMA issue, warps 2..17: epilogue, warp 18: row copies
+constexpr int kMThreads = 640;          // warp 0: TMA, warp 1: UMMA issue, warps 2..17: epilogue, warp 18: row copies, warp 19: row statistics
+                                        // (five warps per scheduler: a sixth would cut every thread to 80 registers)
 constexpr int kMEpiThreads = 512;
 constexpr int kMMiscBytes = 14336;      // epilogue: group records, slices, m_i, 1 / l_i, row sums per lane quarter
 constexpr int kMSlots = 8;              // staging slots of the row copies
 constexpr int kBarEpi = 1;
+constexpr int kMRecBytes = 16 * 1024;   // staging buffer of the statistics warps: sixteen CTAs' records
 
 struct ModelCtl {
     unsigned long long full[kRMaxStages];
@@ -48,6 +50,8 @@ struct ModelCtl {
     unsigned long long qempty;
     unsigned long long gfull[kMSlots];
     unsigned long long sfull;          // a kept-chunk list has landed in shared memory (copy thread)
+    unsigned long long stat_full[2];   // m_i and 1 / l_i of a slot are in shared memory (statistics warps -> epilogue)
+    unsigned long long rfull;          // a batch of CTA records has landed in shared memory (statistics warps)
     uint32_t tmem_base;
     int abort_flag;
     int epi_ok;
@@ -78,6 +82,7 @@ struct ModelParams {
     int sel_row_bytes;     // bytes of one kept-chunk list: 4 header ints + the kept chunk ids, padded to 16 bytes
     int sel_keys_fit;      // selector: the keys of a head fit its shared memory (many chunks per thread)
     int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes;
+    int off_rec;           // record staging buffer of the statistics warps, from off_tail
     float* cta_stat;       // [2 (slot parity)][grid][{max, sum}][128]
     float* scores;         // [n_compute][Hs][Cpad]
     unsigned* cnt_a;       // [Hs]
@@ -205,9 +210,7 @@ model_kernel(const __grid_constant__ ModelParams p) {
     float* pmax = reinterpret_cast<float*>(dyn + p.off_pmax);
     float* misc = reinterpret_cast<float*>(dyn + p.off_misc);
     float* rec = misc;                 // [4 groups][{max, sum}][128]
-    float* slice = misc + 1024;        // [4 slices][{max, sum}][128]
-    float* gm = misc + 2048;
-    float* ginv = misc + 2176;
+    float* gstat = misc + 1024;        // [2 (slot parity)][{m_i, 1 / l_i}][128]
     float* red = misc + 2304;          // [4 lane quarters][256 chunk slots]
     volatile int* abort_flag = &ctl.abort_flag;
     const uint32_t n_stages = static_cast<uint32_t>(p.n_stages);
@@ -250,6 +253,9 @@ model_kernel(const __grid_constant__ ModelParams p) {
         mbar_init(smem_u32(&ctl.qempty), 1);
         for (int s = 0; s < kMSlots; ++s) mbar_init(smem_u32(&ctl.gfull[s]), 1);
         mbar_init(smem_u32(&ctl.sfull), 1);
+        mbar_init(smem_u32(&ctl.stat_full[0]), 1);
+        mbar_init(smem_u32(&ctl.stat_full[1]), 1);
+        mbar_init(smem_u32(&ctl.rfull), 1);
         ctl.abort_flag = 0;
         ctl.epi_ok = 1;
         fence_mbar_init();
@@ -342,6 +348,11 @@ model_kernel(const __grid_constant__ ModelParams p) {
         }
     } else if (warp < 18) {
         // ------------------------------------------------------------------ epilogue
+        // The chunk partial sums and panel maxima of a layer live in rings (tensor-memory columns,
+        // shared memory) that hold more than one layer's worth, so after its last tile of layer s a
+        // thread only publishes the CTA's row records and goes straight on with the first `ahead`
+        // tiles of layer s + 1; the chunk scores of layer s are formed after those, when the other
+        // CTAs' records have long arrived and the statistics warp has merged them.
         const int et = threadIdx.x - 64;                 // 0 .. 511
         const int grp = (warp - 2) >> 2, quarter = warp & 3;
         const int pair = grp >> 1, half = grp & 1;
@@ -350,14 +361,17 @@ model_kernel(const __grid_constant__ ModelParams p) {
         const int last_visible = p.P + (row % p.w);
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const int n_pl = 2 * nt;
+        constexpr int PR = kRPartCols / 6 * 6 / SPP;     // panels in the rings (252 columns)
+        const int ahead = max(0, min(nt, (PR - n_pl) / 2));   // tiles of the next layer scored before the contraction
         const int n_local = nt * (kRTile / C_STATIC);
         const int ch0 = t_begin * (kRTile / C_STATIC);
         bool ok = true;
-        int tg0 = 0;                                      // global index of the layer's first tile
-        for (int s = 0; s < p.n_compute && ok; ++s, tg0 += nt) {
-            float run_m = -CUDART_INF_F, run_l = 0.f;
-            // this pair's tiles: global tile index tg with (tg & 1) == pair
-            for (int ti = (pair - (tg0 & 1)) & 1; ti < nt; ti += 2) {
+        float run_m = -CUDART_INF_F, run_l = 0.f;
+        // tiles [ti_lo, ti_hi) of slot s that belong to this thread's pair
+        auto do_tiles = [&](int s, int ti_lo, int ti_hi) {
+            if (!ok) return;      // (a warp whose wait failed still joins the barriers below until all warps leave together)
+            const int tg0 = s * nt, pbase = (s * n_pl) % PR;
+            for (int ti = ti_lo + ((pair - ((tg0 + ti_lo) & 1)) & 1); ti < ti_hi; ti += 2) {
                 const int tg = tg0 + ti, use = tg >> 1;
                 bool ready = true;
                 if (lane == 0) ready = mbar_wait(smem_u32(&ctl.tfull[pair]), use & 1, abort_flag);
@@ -369,6 +383,8 @@ model_kernel(const __grid_constant__ ModelParams p) {
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[pair]));
                 const int pl = ti * 2 + half;
+                int slot = pbase + pl;
+                slot -= (slot >= PR) ? PR : 0;
                 const int j0 = (t_begin + ti) * kRTile + half * kRPanel;
                 float pr[SPP], m2, l;
                 auto emit = [&](int ch, float acc) { pr[ch] = acc; };
@@ -376,22 +392,24 @@ model_kernel(const __grid_constant__ ModelParams p) {
                     panel_fast<C_STATIC, kRPanel>(v, p.sl2, emit, &m2, &l);
                 else
                     panel_static_tail<C_STATIC, kRPanel>(v, p.sl2, emit, j0, p.P, last_visible, &m2, &l);
-                part_store<SPP>(lane_addr + static_cast<uint32_t>(kRPartCol0 + pl * SPP), pr);
-                pmax[pl * 128 + row] = m2;
+                part_store<SPP>(lane_addr + static_cast<uint32_t>(kRPartCol0 + slot * SPP), pr);
+                pmax[slot * 128 + row] = m2;
                 const float nm = fmaxf(run_m, m2);
                 const float s_old = (run_m == -CUDART_INF_F) ? 0.f : ex2_approx(run_m - nm);
                 const float s_new = (m2 == -CUDART_INF_F) ? 0.f : ex2_approx(m2 - nm);
                 run_l = run_l * s_old + l * s_new;
                 run_m = nm;
             }
+        };
+        // end of slot s: this CTA's (max, sum) per row -> global memory, announced on the head's first counter
+        auto publish = [&](int s) -> bool {
             tmem_st_wait();
             rec[(grp * 2 + 0) * 128 + row] = active ? run_m : -CUDART_INF_F;
             rec[(grp * 2 + 1) * 128 + row] = active ? run_l : 0.f;
-            tc_fence_before();
+            run_m = -CUDART_INF_F;
+            run_l = 0.f;
             named_barrier(kBarEpi, kMEpiThreads);
-            tc_fence_after();
-            if (ctl.abort_flag) { ok = false; break; }
-            // ---- publish this CTA's (max, sum) per row; wait for the head's other CTAs
+            if (ctl.abort_flag) return false;            // same answer in every epilogue thread
             if (et < 128) {
                 float M = -CUDART_INF_F, Ls = 0.f;
 #pragma unroll
@@ -401,69 +419,49 @@ model_kernel(const __grid_constant__ ModelParams p) {
                 dst[128 + et] = Ls;
             }
             named_barrier(kBarEpi, kMEpiThreads);
-            if (et == 0) {
-                unsigned old;
-                asm volatile("atom.add.release.gpu.u32 %0, [%1], 1;" : "=r"(old) : "l"(p.cnt_a + hs) : "memory");
-                const bool w_ok = wait_counter(p.cnt_a + hs, static_cast<unsigned>(s + 1) * p.cph, abort_flag, 0);
-                asm volatile("fence.acq_rel.gpu;" ::: "memory");
-                ctl.epi_ok = w_ok ? 1 : 0;
-            }
-            named_barrier(kBarEpi, kMEpiThreads);
-            if (!ctl.epi_ok) { ok = false; break; }
-            // ---- row statistics of the head
-            {
-                const int i = et & 127, sl = et >> 7;
-                const float* src = p.cta_stat + (static_cast<size_t>(s & 1) * gridDim.x + static_cast<size_t>(hs) * p.cph) * 256 + i;
-                float M = -CUDART_INF_F, Ls = 0.f;
-                for (int j0 = sl; j0 < p.cph; j0 += 16) {
-                    float rm[4], rl[4];
+            if (et == 0)     // (no return value: the thread does not wait for the round trip)
+                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt_a + hs) : "memory");
+            return true;
+        };
+        // chunk scores of slot s from the partial sums in the rings (see layer_resident.cu)
+        auto contract = [&](int s) -> bool {
+            const int pbase = (s * n_pl) % PR;
+            // m_i and 1 / l_i of the head, merged by the statistics warp
+            bool ready = true;
+            if (lane == 0) ready = mbar_wait(smem_u32(&ctl.stat_full[s & 1]), (s >> 1) & 1, abort_flag);
+            if (!__shfl_sync(0xffffffffu, ready, 0)) ok = false;   // (the failed wait has raised the abort flag)
+            tc_fence_before();
+            named_barrier(kBarEpi, kMEpiThreads);        // every partial sum of the slot has been stored
+            tc_fence_after();
+            if (ctl.abort_flag) return false;            // same answer in every epilogue thread
+            const float* gm = gstat + (s & 1) * 256;
+            const float mi = gm[row], li = gm[128 + row];
+            constexpr int PPB = 30 / SPP;
+            for (int b0 = 0; grp + 4 * b0 < n_pl; b0 += PPB) {
+                float v[32];
+                int slot_of[PPB];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int j = j0 + 4 * u;
-                        rm[u] = (j < p.cph) ? __ldcg(src + static_cast<size_t>(j) * 256) : -CUDART_INF_F;
-                        rl[u] = (j < p.cph) ? __ldcg(src + static_cast<size_t>(j) * 256 + 128) : 0.f;
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) merge_ml(M, Ls, rm[u], rl[u]);
+                for (int u = 0; u < PPB; ++u) {
+                    const int pl = min(grp + 4 * (b0 + u), n_pl - 1);
+                    int slot = pbase + pl;
+                    slot -= (slot >= PR) ? PR : 0;
+                    slot_of[u] = slot;
+                    part_load<SPP>(lane_addr + static_cast<uint32_t>(kRPartCol0 + slot * SPP), &v[u * SPP]);
                 }
-                slice[(sl * 2 + 0) * 128 + i] = M;
-                slice[(sl * 2 + 1) * 128 + i] = Ls;
-            }
-            named_barrier(kBarEpi, kMEpiThreads);
-            if (et < 128) {
-                float M = -CUDART_INF_F, Ls = 0.f;
+                tmem_ld_wait();
+                v[30] = 0.f;
+                v[31] = 0.f;
 #pragma unroll
-                for (int q = 0; q < 4; ++q) merge_ml(M, Ls, slice[(q * 2) * 128 + et], slice[(q * 2 + 1) * 128 + et]);
-                gm[et] = M;
-                ginv[et] = 1.0f / Ls;
-            }
-            named_barrier(kBarEpi, kMEpiThreads);
-            // ---- chunk scores of this CTA's key range (see layer_resident.cu)
-            {
-                const float mi = gm[row], li = ginv[row];
-                constexpr int PPB = 30 / SPP;
-                for (int b0 = 0; grp + 4 * b0 < n_pl; b0 += PPB) {
-                    float v[32];
+                for (int u = 0; u < PPB; ++u) {
+                    const int pl = grp + 4 * (b0 + u);
+                    const bool have = active && pl < n_pl;
+                    const float f = have ? ex2_approx(pmax[slot_of[u] * 128 + row] - mi) * li : 0.f;
 #pragma unroll
-                    for (int u = 0; u < PPB; ++u) {
-                        const int pl = min(grp + 4 * (b0 + u), n_pl - 1);
-                        part_load<SPP>(lane_addr + static_cast<uint32_t>(kRPartCol0 + pl * SPP), &v[u * SPP]);
-                    }
-                    tmem_ld_wait();
-                    v[30] = 0.f;
-                    v[31] = 0.f;
-#pragma unroll
-                    for (int u = 0; u < PPB; ++u) {
-                        const int pl = grp + 4 * (b0 + u);
-                        const bool have = active && pl < n_pl;
-                        const float f = have ? ex2_approx(pmax[min(pl, n_pl - 1) * 128 + row] - mi) * li : 0.f;
-#pragma unroll
-                        for (int q = 0; q < SPP; ++q) v[u * SPP + q] = have ? v[u * SPP + q] * f : 0.f;
-                    }
-                    const float tot = warp_transpose_reduce(v, lane);
-                    const int pl = grp + 4 * (b0 + lane / SPP);
-                    if (lane < 30 && pl < n_pl) red[quarter * 256 + pl * SPP + lane % SPP] = tot;
+                    for (int q = 0; q < SPP; ++q) v[u * SPP + q] = have ? v[u * SPP + q] * f : 0.f;
                 }
+                const float tot = warp_transpose_reduce(v, lane);
+                const int pl = grp + 4 * (b0 + lane / SPP);
+                if (lane < 30 && pl < n_pl) red[quarter * 256 + pl * SPP + lane % SPP] = tot;
             }
             tc_fence_before();
             named_barrier(kBarEpi, kMEpiThreads);
@@ -472,13 +470,67 @@ model_kernel(const __grid_constant__ ModelParams p) {
             for (int lc = et; lc < n_local; lc += kMEpiThreads)
                 if (ch0 + lc < p.C) sc_out[ch0 + lc] = (red[lc] + red[256 + lc]) + (red[512 + lc] + red[768 + lc]);
             named_barrier(kBarEpi, kMEpiThreads);
-            if (et == 0) {
-                unsigned old;     // release: the scores written above (ordered by the barrier) are visible to whoever sees the count
-                asm volatile("atom.add.release.gpu.u32 %0, [%1], 1;" : "=r"(old) : "l"(p.cnt_b + hs) : "memory");
+            if (et == 0)     // release: the scores written above (ordered by the barrier) are visible to whoever sees the count
+                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt_b + hs) : "memory");
+            return true;
+        };
+        for (int s = 0; s <= p.n_compute; ++s) {
+            if (s < p.n_compute) do_tiles(s, 0, ahead);
+            if (s > 0 && !contract(s - 1)) break;
+            if (s < p.n_compute) {
+                do_tiles(s, ahead, nt);
+                if (!publish(s)) break;
             }
         }
         if (!ok && lane == 0) ctl.abort_flag = 1;
-    } else {
+    } else if (warp == 19) {
+        // ------------------------------------------------------------------ statistics warp
+        // Per slot: wait (bounded) until every CTA of the scoring head has published its records,
+        // fetch them with bulk copies (they are contiguous in global memory; up to 16 CTAs' records
+        // per copy), merge them into m_i and 1 / l_i - four rows per lane - and hand the result to
+        // the epilogue.
+        const int r0 = 4 * lane;
+        const float* recbuf = reinterpret_cast<const float*>(dyn + p.off_tail + p.off_rec);
+        uint32_t rc = 0;                                  // record copies completed so far
+        bool ok = true;
+        for (int s = 0; s < p.n_compute && ok; ++s) {
+            bool w_ok = true;
+            if (lane == 0) {
+                w_ok = wait_counter(p.cnt_a + hs, static_cast<unsigned>(s + 1) * p.cph, abort_flag, 100);
+                asm volatile("fence.acq_rel.gpu;" ::: "memory");
+            }
+            if (!__shfl_sync(0xffffffffu, w_ok, 0)) break;
+            const float* src = p.cta_stat + (static_cast<size_t>(s & 1) * gridDim.x + static_cast<size_t>(hs) * p.cph) * 256;
+            float M[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F}, S[4] = {0.f, 0.f, 0.f, 0.f};
+            for (int j0 = 0; j0 < p.cph; j0 += 16, ++rc) {
+                const int n = min(16, p.cph - j0);
+                if (lane == 0) {
+                    const uint32_t bar = smem_u32(&ctl.rfull);
+                    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n) * 1024u);
+                    // the records were written with ordinary stores by other CTAs
+                    asm volatile("fence.proxy.async.global;" ::: "memory");
+                    bulk_load(smem_u32(recbuf), src + static_cast<size_t>(j0) * 256, static_cast<uint32_t>(n) * 1024u, bar);
+                }
+                if (!mbar_wait(smem_u32(&ctl.rfull), rc & 1u, abort_flag)) { ok = false; break; }
+#pragma unroll 2
+                for (int j = 0; j < n; ++j) {
+                    const float4 m = *reinterpret_cast<const float4*>(recbuf + j * 256 + r0);
+                    const float4 l = *reinterpret_cast<const float4*>(recbuf + j * 256 + 128 + r0);
+                    merge_ml(M[0], S[0], m.x, l.x);
+                    merge_ml(M[1], S[1], m.y, l.y);
+                    merge_ml(M[2], S[2], m.z, l.z);
+                    merge_ml(M[3], S[3], m.w, l.w);
+                }
+                __syncwarp();                             // the buffer may be overwritten by the next copy
+            }
+            if (!ok) break;
+            float* gm = gstat + (s & 1) * 256;
+            *reinterpret_cast<float4*>(gm + r0) = make_float4(M[0], M[1], M[2], M[3]);
+            *reinterpret_cast<float4*>(gm + 128 + r0) = make_float4(1.0f / S[0], 1.0f / S[1], 1.0f / S[2], 1.0f / S[3]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl.stat_full[s & 1]));
+        }
+    } else if (warp == 18) {
         // ------------------------------------------------------------------ tail: row copies
         // One thread: waits until the selector CTA has published the head's kept-chunk list of a
         // slot, fetches the list, and moves this CTA's share of the rows - whole chunks and window
@@ -617,13 +669,14 @@ bool make_model_plan(int L, int Rs, int Hs, int kv_shift, int d, int c, int C, i
     p.grid = p.n_score + p.n_sel;
     p.n_tiles = (L + kRTile - 1) / kRTile;
     p.t_max = (p.n_tiles + p.cph - 1) / p.cph;
-    if (p.t_max * (kRTile / c) > kRPartCols) return false;
+    if (p.t_max * (kRTile / c) > 252) return false;          // a layer's chunk slots must fit the 252-column ring
     const int KB = d / 64;
     const int q_bytes = KB * kRQTileBytes;
-    const int pmax_bytes = p.t_max * 2 * 128 * 4;
+    const int pmax_bytes = (252 / (kRPanel / c)) * 128 * 4;  // the panel-maxima ring: one row set per ring panel
     p.stage_slot_bytes = 2 * c * d * 2;                        // K rows and V rows of one chunk
     p.sel_row_bytes = ((4 + kk) * 4 + 127) & ~127;
-    const int tail_bytes = p.sel_row_bytes + kMSlots * p.stage_slot_bytes + 128;
+    p.off_rec = p.sel_row_bytes + kMSlots * p.stage_slot_bytes;
+    const int tail_bytes = p.off_rec + kMRecBytes + 128;
     const int fixed = 1024 + q_bytes + 1024 + pmax_bytes + kMMiscBytes + tail_bytes;
     int ns = (smem_limit - 512 - fixed) / kRStageBytes;           // (the control block is larger than the layer kernel's)
     if (ns > kRMaxStages) ns = kRMaxStages;
@@ -681,6 +734,7 @@ cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtenso
     p.sel_row_bytes = plan.sel_row_bytes; p.sel_keys_fit = plan.sel_keys_fit;
     p.off_ring = plan.off_ring; p.off_pmax = plan.off_pmax; p.off_misc = plan.off_misc; p.off_tail = plan.off_tail;
     p.stage_slot_bytes = plan.stage_slot_bytes;
+    p.off_rec = plan.off_rec;
     p.cta_stat = io.scratch;
     p.scores = io.scratch + static_cast<size_t>(2) * plan.grid * 256;
     p.sel_rows = reinterpret_cast<int*>(p.scores + static_cast<size_t>(n_compute) * io.Hs * p.Cpad);   // 16-byte aligned: Cpad % 4 == 0
