@@ -39,7 +39,8 @@ constexpr int kMEpiThreads = 512;
 constexpr int kMMiscBytes = 14336;      // epilogue: group records, slices, m_i, 1 / l_i, row sums per lane quarter
 constexpr int kMSlots = 8;              // staging slots of the row copies
 constexpr int kBarEpi = 1;
-constexpr int kMRecBytes = 16 * 1024;   // staging buffer of the statistics warps: sixteen CTAs' records
+constexpr int kMRecBatch = 24;           // CTA records fetched per bulk copy by the statistics warp
+constexpr int kMRecBytes = kMRecBatch * 1024;
 
 struct ModelCtl {
     unsigned long long full[kRMaxStages];
@@ -486,7 +487,7 @@ model_kernel(const __grid_constant__ ModelParams p) {
     } else if (warp == 19) {
         // ------------------------------------------------------------------ statistics warp
         // Per slot: wait (bounded) until every CTA of the scoring head has published its records,
-        // fetch them with bulk copies (they are contiguous in global memory; up to 16 CTAs' records
+        // fetch them with bulk copies (they are contiguous in global memory; up to 24 CTAs' records
         // per copy), merge them into m_i and 1 / l_i - four rows per lane - and hand the result to
         // the epilogue.
         const int r0 = 4 * lane;
@@ -496,14 +497,14 @@ model_kernel(const __grid_constant__ ModelParams p) {
         for (int s = 0; s < p.n_compute && ok; ++s) {
             bool w_ok = true;
             if (lane == 0) {
-                w_ok = wait_counter(p.cnt_a + hs, static_cast<unsigned>(s + 1) * p.cph, abort_flag, 100);
+                w_ok = wait_counter(p.cnt_a + hs, static_cast<unsigned>(s + 1) * p.cph, abort_flag, 0);
                 asm volatile("fence.acq_rel.gpu;" ::: "memory");
             }
             if (!__shfl_sync(0xffffffffu, w_ok, 0)) break;
             const float* src = p.cta_stat + (static_cast<size_t>(s & 1) * gridDim.x + static_cast<size_t>(hs) * p.cph) * 256;
             float M[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F}, S[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int j0 = 0; j0 < p.cph; j0 += 16, ++rc) {
-                const int n = min(16, p.cph - j0);
+            for (int j0 = 0; j0 < p.cph; j0 += kMRecBatch, ++rc) {
+                const int n = min(kMRecBatch, p.cph - j0);
                 if (lane == 0) {
                     const uint32_t bar = smem_u32(&ctl.rfull);
                     mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n) * 1024u);
