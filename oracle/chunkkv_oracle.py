@@ -31,7 +31,9 @@ row sums, mass conservation, the uniform-attention closed form (q = 0), a domina
 limit, an e-ratio logit case that fixes the 1/sqrt(d) scale, an independent library
 softmax, library top-k for c = 1, the budget/ordering/window invariants, reuse identity;
 for Algorithm 1's budget rule (select_alg1): hand-worked cases, brute-force enumeration of
-chunk subsets followed by the cut, and the exact output length.
+chunk subsets followed by the cut, and the exact output length; for the prefill-tail adapters
+(rope, window_queries, gather_paged; tests/test_oracle_adapters.py): norm preservation, identity
+at angle 0, relative-position dependence, complex multiplication, un-paging to the dense gather.
 
 Layouts (numpy arrays; bf16 tensors arrive as uint16 bit patterns):
   q_obs [Hq, w, d]   K, V [Hkv, L, d]   token scores [Hkv, P]   chunk scores [Hkv, C]
@@ -317,3 +319,61 @@ def jaccard(idx_a: np.ndarray, idx_b: np.ndarray) -> float:
     b = set(int(v) for v in np.asarray(idx_b).ravel() if v >= 0)
     u = len(a | b)
     return (len(a & b) / u) if u else 1.0
+
+
+# --------------------------------------------------------------------------- prefill-tail inputs and paged outputs
+# The paper runs the compression at the end of prefill, on the queries of the last w positions
+# ("q_observe <- Q[T_q - w : T_q]", Algorithm 3; section "Efficiency Analysis": compression happens
+# once, after prefill, and the compacted cache then serves decoding). In a model those queries sit
+# in the layer's fused QKV projection output, before the rotary position embedding, and the
+# compacted rows go to the decode cache, which serving systems keep in pages. The three functions
+# below state those two adapters; nothing in them changes what is selected.
+def f64_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """Round fp64 values to bf16 (round to nearest even, through fp32) and return the bit patterns."""
+    u = np.ascontiguousarray(x, dtype=np.float64).astype(np.float32).view(np.uint32)
+    rounded = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)
+    return rounded.astype(np.uint16)
+
+
+def rope(x: np.ndarray, cos: np.ndarray, sin: np.ndarray) -> np.ndarray:
+    """Rotary position embedding in the rotate-half convention, fp64.
+
+    x [..., d]; cos, sin [..., d/2] (broadcast against x's leading dims): the pair (x[i], x[i + d/2])
+    is rotated by the angle whose cosine / sine are cos[i] / sin[i].
+    """
+    d = x.shape[-1]
+    h = d // 2
+    x1, x2 = x[..., :h], x[..., h:]
+    return np.concatenate([x1 * cos - x2 * sin, x2 * cos + x1 * sin], axis=-1)
+
+
+def window_queries(qkv: np.ndarray, Hq: int, Hkv: int, d: int, w: int, cos: np.ndarray,
+                   sin: np.ndarray) -> np.ndarray:
+    """q_obs [Hq, w, d] (bf16 bits) from a fused QKV activation.
+
+    qkv [T, (Hq + 2 Hkv) * d] bf16 bits, token-major, query heads first, before RoPE; the window is
+    its last w rows; cos, sin [w, d/2] are the table rows of the window's positions. The rotation
+    runs in fp64 on the exactly widened inputs and the result is rounded once to bf16.
+    """
+    T = qkv.shape[0]
+    q = bf16_bits_to_f64(qkv[T - w:, :Hq * d]).reshape(w, Hq, d)
+    out = rope(q, np.asarray(cos, dtype=np.float64)[:, None, :], np.asarray(sin, dtype=np.float64)[:, None, :])
+    return f64_to_bf16_bits(np.transpose(out, (1, 0, 2)))
+
+
+def gather_paged(K: np.ndarray, V: np.ndarray, idx: np.ndarray, block_table: np.ndarray, page_size: int,
+                 cache_K: np.ndarray, cache_V: np.ndarray) -> None:
+    """Scatter the kept rows into a paged cache, in place.
+
+    cache_K, cache_V [num_pages, page_size, Hkv, d]; compacted position n of every head goes to page
+    block_table[n // page_size], slot n % page_size (zero rows where idx is -1). Pages not named
+    by the block table, and slots past n_max in the last page, are left as they are.
+    (Algorithm 3's two index_select lines, written to where a paged decode cache keeps its rows.)
+    """
+    Hkv, n_max = idx.shape
+    for h in range(Hkv):
+        for n in range(n_max):
+            page, slot = int(block_table[n // page_size]), n % page_size
+            j = int(idx[h, n])
+            cache_K[page, slot, h] = K[h, j] if j >= 0 else 0
+            cache_V[page, slot, h] = V[h, j] if j >= 0 else 0
