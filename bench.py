@@ -4,18 +4,18 @@
 Metric: prefix tokens compressed per second per layer, on the Llama-3-8B 32K KV shape
 (Hq 32, Hkv 8, d 128, L 32768, w 32, c 10, budget 3276), seeded synthetic bf16 tensors.
 
-A step compresses the 32 layers of one 32K-token sequence: 32 layer calls
-(score -> chunk-sum -> top-k -> gather), cycling over NSETS distinct layer inputs (each 134 MB
-of K/V, so consecutive layers never find their K/V in L2). The layers are independent, so the
-step keeps `--lanes` of them in flight (chunkkv_pipe_layer, each pipe on its own stream with
-its share of the SMs and its row gathers on a side stream; `--mode lane` uses
-chunkkv_compress_layer_lane instead). `value` is measured with the step captured in a CUDA graph and
-replayed (inputs resident in HBM); the same step launched call by call is reported as `eager`,
-the same layers one after another on the whole GPU (chunkkv_compress_layer) as
-`roofline_more.single_layer`; `e2e` goes through chunkkv_compress_layer_host with pinned host
-buffers, copies inside the timed region.
+A step compresses the 32 layers of one 32K-token sequence (score -> chunk-sum -> top-k -> gather
+per layer). Every layer of the step has its own seeded q / K / V in HBM (32 x 134 MB), so no layer
+finds another layer's keys in L2. `value` times the step as ONE chunkkv_compress_model call (the
+persistent kernel: scoring of a layer overlaps selecting and gathering the one before), captured
+in a CUDA graph and replayed; `eager` is the same call without a graph;
+`roofline_more.single_layer` runs the same 32 layers as 32 chunkkv_compress_layer calls;
+`roofline_more.shared_inputs` repeats the headline with the 32 layers pointing at only 4 distinct
+K/V sets (what an L2-friendly input rotation would measure - for comparison only); `e2e` goes
+through chunkkv_compress_layer_host with pinned host buffers, copies inside the timed region.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py --profile-case {layer,model,reuse,token,cfg4} [--iters n]   (a few calls, for ncu)
 """
 from __future__ import annotations
 
@@ -36,31 +36,28 @@ import torch  # noqa: E402
 
 METRIC = "prefix_tokens_compressed_per_sec_per_layer"
 UNIT = "tokens/s/layer"
-NSETS = 4
 LAYERS_PER_STEP = 32
+SHARED_SETS = 4
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one cfg2 layer through a lane, from ncu captures
-# of both launches (layer kernel + row gather): 8 CTAs 69.6 + 13.5 MB, 18 CTAs 69.5 + 13.5 MB
-TRAFFIC_BYTES_PER_LAYER = {8: 83.1e6, 18: 83.0e6}
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--config", type=int, default=2, help="workload table entry (2 = headline)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-long", action="store_true", help="skip the 128K / 64K long-context layer timings")
-    ap.add_argument("--lanes", type=int, default=18, help="layers in flight (each on 1/lanes of the SMs)")
-    ap.add_argument("--lane-ctas", type=int, default=0, help="CTA budget of a lane (0: SMs // lanes)")
-    ap.add_argument("--mode", choices=("pipe", "lane"), default="pipe",
-                    help="pipe: chunkkv_pipe_layer (layer kernels back to back, row gathers on side streams); "
-                         "lane: chunkkv_compress_layer_lane (one layer at a time per lane)")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the secondary rows (long contexts, batched workload, token-level layers, sustained loop)")
+    ap.add_argument("--profile-case", choices=("layer", "model", "reuse", "token", "cfg4"), default=None,
+                    help="run a few calls of one case and exit (for use under a profiler)")
+    ap.add_argument("--iters", type=int, default=3, help="calls of --profile-case")
+    ap.add_argument("--layers", type=int, default=4, help="layers of --profile-case model")
     return ap.parse_args()
 
 
@@ -205,14 +202,64 @@ def run_reference(args, wl):
 
 
 # ------------------------------------------------------------------------------------- CUDA arm
+def to_dev(bits, dev):
+    return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+
+
+def make_layers(wl, n, dev, seq=0, workers=8):
+    """n distinct seeded layers of a workload on the device (generated on host threads)."""
+    from concurrent.futures import ThreadPoolExecutor
+    from workloads import make_layer
+    out = [None] * n
+    with ThreadPoolExecutor(max_workers=workers) as ex:
+        for i, x in enumerate(ex.map(lambda i: make_layer(wl, layer=i, seq=seq), range(n))):
+            out[i] = (to_dev(x.q_obs, dev), to_dev(x.K, dev), to_dev(x.V, dev))
+    return out
+
+
+def alloc_outs(ck, wl, n, dev, c=None):
+    n_max = ck.out_len(wl.L, wl.w, wl.c if c is None else c, wl.budget)
+    return [(torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device=dev),
+             torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device=dev),
+             torch.empty((wl.Hkv, n_max), dtype=torch.int32, device=dev)) for _ in range(n)]
+
+
+class ModelCall:
+    """Marshalled arguments of one chunkkv_compress_model call (built once, issued many times)."""
+
+    def __init__(self, ck, wl, layers, outs, reuse_depth, L=None):
+        import ctypes
+        self.ck, self.wl, self.n, self.reuse = ck, wl, len(layers), reuse_depth
+        self.L = wl.L if L is None else L
+        arr = ctypes.c_void_p * self.n
+        self.q = arr(*[None if (i % reuse_depth) else t[0].data_ptr() for i, t in enumerate(layers)])
+        self.K = arr(*[t[1].data_ptr() for t in layers])
+        self.V = arr(*[t[2].data_ptr() for t in layers])
+        self.oK = arr(*[o[0].data_ptr() for o in outs])
+        self.oV = arr(*[o[1].data_ptr() for o in outs])
+        self.oI = arr(*[o[2].data_ptr() for o in outs])
+        self.keep = (layers, outs)
+        need = int(ck.lib.chunkkv_model_workspace_bytes(self.n, self.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, wl.budget,
+                                                        reuse_depth))
+        self.workspace_bytes = need
+
+    def __call__(self, stream):
+        wl = self.wl
+        st = self.ck.lib.chunkkv_compress_model(self.n, self.q, self.K, self.V, self.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
+                                                wl.budget, self.reuse, self.oK, self.oV, self.oI, stream.cuda_stream)
+        if st != 0:
+            raise self.ck.ChunkKVError(st, "chunkkv_compress_model")
+
+
 def run_ours(args, wl):
     import torch.distributed as dist
 
     from paper_2502_00299_b200 import build as _build
     _build.build()
     import paper_2502_00299_b200 as ck
+    from paper_2502_00299_b200 import binding as ckb
     from paper_2502_00299_b200.sharding import job_throughput, max_over_ranks
-    from workloads import CONFIGS, make_layer, scaled
+    from workloads import CONFIGS, iter_layers, make_layer, ragged_lengths, scaled
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -230,112 +277,59 @@ def run_ours(args, wl):
         torch.cuda.synchronize()
 
     lib = ck.lib
+    NL = LAYERS_PER_STEP
     n_max = ck.out_len(wl.L, wl.w, wl.c, wl.budget)
     nbytes = layer_bytes(wl, n_max)
-    # the library allocates nothing: one scratch buffer that covers every shape timed below, set up
-    # once, before anything is captured in a graph
-    ck.ensure_workspace(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c)
-    ck.ensure_workspace(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, 1)
-    if not args.no_long and rank == 0:
-        for lw in (CONFIGS[4], scaled(CONFIGS[5], L=65536)):
-            ck.ensure_workspace(lw.L, lw.Hq, lw.Hkv, lw.d, lw.w, lw.c)
-
-    # ---- inputs: NSETS distinct layers (rank r takes sequence r), resident in HBM
-    hosts, sets = [], []
-    for i in range(NSETS):
-        x = make_layer(wl, layer=i, seq=rank)
-        hosts.append(x)
-        t = [torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16) for b in (x.q_obs, x.K, x.V)]
-        sets.append((t,))
-
-    # ---- lanes: S layers in flight, each on its own stream with 1/S of the SMs and its own scratch
-    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
-    S = max(1, args.lanes)
-    lane_ctas = args.lane_ctas if args.lane_ctas > 0 else n_sm // S
+    peak, peak_src = measured_hbm_peak()
     stream = torch.cuda.Stream(device=dev)
-    lanes = []
-    piped = args.mode == "pipe" and S > 1
-    if S > 1:
-        for li in range(S):
-            cls = ck.Pipe if piped else ck.Lane
-            ln = cls(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, max_ctas=lane_ctas, device=dev,
-                     stream=stream if li == 0 else None)
-            lanes.append(ln)
-    lane_streams = [ln.stream for ln in lanes] if lanes else [stream]
-    # every layer of a step writes its own output buffers
-    lane_outs = []
-    for _ in range(LAYERS_PER_STEP):
-        o = [torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device=dev) for _ in range(2)]
-        o.append(torch.empty((wl.Hkv, n_max), dtype=torch.int32, device=dev))
-        lane_outs.append(o)
+    extra = not args.no_extra and rank == 0
 
-    def call_layer(i: int, reuse: bool = False, single: bool = False):
-        q, K, V = sets[i % NSETS][0]
-        li = 0 if single else i % S
-        oK, oV, oI = lane_outs[i]
-        if piped and not single and not reuse:
-            ln = lanes[li]
-            st = lib.chunkkv_pipe_layer(
-                ln.handle, q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, wl.budget,
-                oK.data_ptr(), oV.data_ptr(), oI.data_ptr(), ln.stream.cuda_stream)
-        elif piped and not single:
-            st = lib.chunkkv_compress_layer(       # gather-only layers need no pipe: spread over the lane streams
-                None, K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c, wl.budget, oI.data_ptr(),
-                oK.data_ptr(), oV.data_ptr(), oI.data_ptr(), lanes[li].stream.cuda_stream)
-        elif S > 1 and not single:
-            ln = lanes[li]
-            st = lib.chunkkv_compress_layer_lane(
-                None if reuse else q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
-                wl.budget, oI.data_ptr() if reuse else None, oK.data_ptr(), oV.data_ptr(), oI.data_ptr(),
-                ln.buf.data_ptr(), ln.bytes, ln.max_ctas, ln.stream.cuda_stream)
-        else:
-            st = lib.chunkkv_compress_layer(
-                None if reuse else q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
-                wl.budget, oI.data_ptr() if reuse else None, oK.data_ptr(), oV.data_ptr(), oI.data_ptr(),
-                stream.cuda_stream)
+    # ---- inputs: every layer of the step has its own q / K / V (rank r takes sequence r)
+    layers = make_layers(wl, NL, dev, seq=rank)
+    outs = alloc_outs(ck, wl, NL, dev)
+    shared = [layers[i % SHARED_SETS] for i in range(NL)]            # 4 K/V sets standing in for 32 layers
+    model = ModelCall(ck, wl, layers, outs, 1)
+    model_shared = ModelCall(ck, wl, shared, outs, 1)
+    model_reuse2 = ModelCall(ck, wl, layers, outs, 2)
+    # the library allocates nothing: one scratch buffer that covers every shape timed below, handed
+    # over once, before anything is captured in a graph
+    need = max(model.workspace_bytes, model_reuse2.workspace_bytes,
+               ck.workspace_bytes(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c),
+               ck.workspace_bytes(wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, 1))
+    long_cfgs = (("cfg4_128k", CONFIGS[4]), ("cfg5_longest_64k", scaled(CONFIGS[5], L=65536)))
+    lens5 = ragged_lengths(CONFIGS[5])
+    if extra:
+        for _, lw in long_cfgs:
+            need = max(need, ck.workspace_bytes(lw.L, lw.Hq, lw.Hkv, lw.d, lw.w, lw.c))
+        w5 = CONFIGS[5]
+        for L5 in lens5:
+            need = max(need, int(lib.chunkkv_model_workspace_bytes(w5.n_layers, L5, w5.Hq, w5.Hkv, w5.d, w5.w, w5.c,
+                                                                   w5.budget, w5.reuse_depth)),
+                       ck.workspace_bytes(L5, w5.Hq, w5.Hkv, w5.d, w5.w, w5.c))
+    ckb._ensure_bytes(int(need))
+
+    def layer_call(i, reuse=False, c=None, o=None, src=None):
+        q, K, V = (layers if src is None else src)[i]
+        oK, oV, oI = (outs if o is None else o)[i]
+        st = lib.chunkkv_compress_layer(None if reuse else q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv,
+                                        wl.d, wl.w, wl.c if c is None else c, wl.budget, oI.data_ptr() if reuse else None,
+                                        oK.data_ptr(), oV.data_ptr(), oI.data_ptr(), stream.cuda_stream)
         if st != 0:
             raise ck.ChunkKVError(st, "chunkkv_compress_layer")
 
-    def issue_step(reuse: bool = False, single: bool = False):
-        """One step = LAYERS_PER_STEP layers; lane streams fork from and join back into `stream`."""
-        multi = S > 1 and not single
-        if multi:
-            ev = torch.cuda.Event()
-            ev.record(stream)
-            for st_ in lane_streams[1:]:
-                st_.wait_event(ev)
-        for i in range(LAYERS_PER_STEP):
-            call_layer(i, reuse, single)
-        if multi:
-            if piped and not reuse:
-                for ln in lanes:
-                    ln.join()
-            for st_ in lane_streams[1:]:
-                ev = torch.cuda.Event()
-                ev.record(st_)
-                stream.wait_event(ev)
+    def step_single():
+        for i in range(NL):
+            layer_call(i)
 
-    def step_eager():
-        issue_step()
+    def step_reuse():
+        for i in range(NL):
+            layer_call(i, reuse=True)
 
-    with torch.cuda.stream(stream):
-        for _ in range(max(args.warmup, 3)):
-            issue_step()
-            issue_step(single=True)
-    torch.cuda.synchronize()
-    if ck.device_status(stream) != 0 or any(ln.status() != 0 for ln in lanes):
-        raise RuntimeError("a kernel reported an abandoned wait during warm-up")
-
-    # ---- the step as a CUDA graph
-    def capture(**kw):
+    def capture(fn):
         gr = torch.cuda.CUDAGraph()
         with torch.cuda.graph(gr, stream=stream):
-            issue_step(**kw)
+            fn()
         return gr
-
-    graph = capture()
-    reuse_graph = capture(reuse=True)
-    single_graph = capture(single=True)        # one layer at a time on the whole GPU
 
     def timed(fn, steps):
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -348,142 +342,167 @@ def run_ours(args, wl):
         barrier()
         return ev0.elapsed_time(ev1)
 
+    def check_status():
+        if ck.device_status(stream) != 0:
+            raise RuntimeError("a kernel reported an abandoned wait")
+
     with torch.cuda.stream(stream):
         for _ in range(max(args.warmup, 3)):
-            graph.replay()
-            reuse_graph.replay()
-            single_graph.replay()
+            model(stream)
+            step_single()
+            step_reuse()
+    torch.cuda.synchronize()
+    check_status()
+    g_model = capture(lambda: model(stream))
+    g_shared = capture(lambda: model_shared(stream))
+    g_reuse2 = capture(lambda: model_reuse2(stream))
+    g_single = capture(step_single)
+    g_reuse = capture(step_reuse)
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            for g in (g_model, g_shared, g_reuse2, g_single, g_reuse):
+                g.replay()
     try:
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     except Exception:
         gpu_id = str(local_rank)
+
+    # ---- headline: one chunkkv_compress_model call per step, as a replayed graph
     sampler = ClockSampler(gpu_id)
     sampler.start()
-    ms_total = timed(graph.replay, args.steps)
+    ms_total = timed(g_model.replay, args.steps)
     clocks = sampler.stop()
-    tokens_local = args.steps * LAYERS_PER_STEP * wl.L
-    value, ms_max = job_throughput(tokens_local, ms_total, dev)
+    value, ms_max = job_throughput(args.steps * NL * wl.L, ms_total, dev)
     ms_per_step = ms_max / args.steps
-    ms_layer = ms_per_step / LAYERS_PER_STEP
+    us_layer = ms_per_step / NL * 1e3
 
-    # ---- the same step, call by call (no graph); gather-only (index reuse) layers; one layer at a time
-    eager_steps = max(3, min(args.steps, 100))
-    ms_eager = max_over_ranks(timed(step_eager, eager_steps), dev) / eager_steps
-    ms_reuse = max_over_ranks(timed(reuse_graph.replay, eager_steps), dev) / eager_steps / LAYERS_PER_STEP
-    ms_single = max_over_ranks(timed(single_graph.replay, eager_steps), dev) / eager_steps / LAYERS_PER_STEP
+    few = max(3, min(args.steps, 100))
+    us_eager = max_over_ranks(timed(lambda: model(stream), few), dev) / few / NL * 1e3
+    us_shared = max_over_ranks(timed(g_shared.replay, few), dev) / few / NL * 1e3
+    us_single = max_over_ranks(timed(g_single.replay, few), dev) / few / NL * 1e3
+    us_reuse = max_over_ranks(timed(g_reuse.replay, few), dev) / few / NL * 1e3
+    us_reuse2_model = max_over_ranks(timed(g_reuse2.replay, few), dev) / few * 1e3      # per 32-layer model
+    check_status()
 
-    # ---- per-kernel durations (CUDA events around every kernel, on the launching stream)
+    def frac_row(nb, us, **kw):
+        gbs = nb / (us * 1e-6) / 1e9
+        row = {"algorithmic_bytes": nb, "us": us, "GB/s": gbs, "frac_of_measured_peak": gbs / peak,
+               "frac_of_8TBps": gbs / NOMINAL_HBM_GBS}
+        row.update(kw)
+        return row
+
+    # per-kernel durations of the call-by-call path (CUDA events around every launch, one layer at a time)
     ck.profile_enable(True)
-    prof_steps = max(3, min(args.steps, 30))
-    timed(lambda: issue_step(single=True), prof_steps)      # one layer at a time: each kernel has the GPU to itself
+    timed(step_single, 3)
     ms_slot, n_slot = ck.profile_read()
     ck.profile_enable(False)
-    names = ("score", "finalize", "select", "gather")
+    names = ("layer_or_score", "finalize", "select", "gather")
     per_kernel = {n: {"launches": c, "avg_us": (m / c * 1e3) if c else None, "total_ms": m}
                   for n, m, c in zip(names, ms_slot, n_slot)}
-    tot = sum(ms_slot) or 1.0
-    for n, m in zip(names, ms_slot):
-        per_kernel[n]["share"] = m / tot
+    iso_us = per_kernel["layer_or_score"]["avg_us"] or float("nan")
 
-    peak, peak_src = measured_hbm_peak()
-    score_us = per_kernel["score"]["avg_us"] or float("nan")
-    fused = per_kernel["gather"]["launches"] == 0          # the whole layer ran as one kernel
-    split = S > 1 and 2 * lane_ctas <= n_sm               # a lane's layer = layer kernel + row-gather launch
-    launches_per_layer = 2 if (piped or split) else 1           # layer kernel + row gather
-    # The timed region holds nothing but the launches of LAYERS_PER_STEP layers per step, S of them
-    # in flight at a time on disjoint SM sets, so the duration a launch accounts for is the region
-    # divided by the layers; algorithmic bytes per layer over that is what HBM sustains.
-    achieved = nbytes["layer"] / (ms_layer * 1e-3) / 1e9
-    if piped:
-        kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) on the pipe's main stream + "
-                       "gather_kernel (row gather in CTAs spread over all SMs) on its side stream: the two launches of a "
-                       "layer in a pipe" % lane_ctas)
-    elif split:
-        kernel_name = ("score_kernel<FUSED> on %d CTAs (score + chunk sums + finalize + select) + gather_kernel "
-                       "(row gather in CTAs spread over all SMs): the two launches of a layer in a lane" % lane_ctas)
-    else:
-        kernel_name = "score_kernel<FUSED> (score + chunk sums + finalize + select + gather in one launch)"
-    roofline = {"kernel": kernel_name, "bound": "hbm", "achieved": achieved, "peak": peak,
-                "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": TRAFFIC_BYTES_PER_LAYER.get(lane_ctas) if ((split or piped) and args.config == 2) else None,
-                "algorithmic_bytes_per_launch": nbytes["layer"], "avg_launch_us": ms_layer * 1e3,
-                "launches_in_flight": S,
-                "isolated_launch_us": score_us,
-                "isolated_frac": nbytes["layer"] / (score_us * 1e-6) / 1e9 / peak,
-                "note": "avg_launch_us = CUDA-event time of the timed region / layers launched in it "
-                        f"({S} layers in flight on disjoint SM sets, nothing else in the region); "
-                        "isolated_* = the whole-GPU layer kernel timed alone, one layer at a time; "
-                        "traffic = DRAM bytes of one layer's launches from an ncu capture (cold L2)"}
-    layer_gbs = nbytes["layer"] / (ms_layer * 1e-3) / 1e9
-    gather_us = per_kernel["gather"]["avg_us"]                    # None when the layer kernel is fused
+    achieved = nbytes["layer"] * NL / (ms_per_step * 1e-3) / 1e9
+    roofline = {
+        "kernel": "model_kernel<10>: the persistent kernel behind chunkkv_compress_model - 32 layers per launch; "
+                  "scoring (TMA + tcgen05), chunk sums in tensor memory, top-k on selector CTAs, row copies by bulk copy",
+        "bound": "hbm", "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+        "frac": achieved / peak, "frac_of_8TBps": achieved / NOMINAL_HBM_GBS, "traffic": None,
+        "traffic_note": "not captured for the 32-layer launch (ncu's size rule); see profiles/ for the layer kernel's DRAM counters",
+        "algorithmic_bytes_per_launch": nbytes["layer"] * NL, "avg_launch_us": ms_per_step * 1e3,
+        "launches_per_step": 1, "layers_per_launch": NL,
+        "isolated_launch_us": iso_us,
+        "isolated_frac": nbytes["layer"] / (iso_us * 1e-6) / 1e9 / peak,
+        "note": "avg_launch_us = CUDA-event time of the timed region / launches in it (one launch per step, nothing else "
+                "in the region); algorithmic bytes = 32 x (K once + q + K/V rows read and written); isolated_* = the "
+                "one-layer kernel of chunkkv_compress_layer with events around every launch, same distinct inputs"}
     extra_roof = {
-        "layer_throughput": {"algorithmic_bytes": nbytes["layer"], "us_per_layer": ms_layer * 1e3, "GB/s": layer_gbs,
-                             "frac_of_measured_peak": layer_gbs / peak, "frac_of_8TBs": layer_gbs / NOMINAL_HBM_GBS,
-                             "lanes": S},
-        "single_layer": {"algorithmic_bytes": nbytes["layer"], "us": ms_single * 1e3,
-                         "GB/s": nbytes["layer"] / (ms_single * 1e-3) / 1e9,
-                         "frac_of_measured_peak": nbytes["layer"] / (ms_single * 1e-3) / 1e9 / peak,
-                         "note": "layers one after another, each on all SMs"},
-        "gather_kernel": None if not gather_us else {
-            "algorithmic_bytes": nbytes["gather"], "us": gather_us,
-            "GB/s": nbytes["gather"] / (gather_us * 1e-6) / 1e9,
-            "frac_of_measured_peak": nbytes["gather"] / (gather_us * 1e-6) / 1e9 / peak},
-        "reuse_layer": {"algorithmic_bytes": nbytes["gather"], "us": ms_reuse * 1e3,
-                        "GB/s": nbytes["gather"] / (ms_reuse * 1e-3) / 1e9,
-                        "frac_of_measured_peak": nbytes["gather"] / (ms_reuse * 1e-3) / 1e9 / peak},
+        "model_call": frac_row(nbytes["layer"], us_layer, note="headline: per layer inside one 32-layer chunkkv_compress_model call"),
+        "single_layer": frac_row(nbytes["layer"], us_single,
+                                 note="32 chunkkv_compress_layer calls back to back (one kernel per layer, each on all SMs), as a graph"),
+        "shared_inputs": frac_row(nbytes["layer"], us_shared,
+                                  note=f"headline call with the 32 layers pointing at {SHARED_SETS} K/V sets (L2 can serve repeats): "
+                                       "comparison only, not a roofline number"),
+        "reuse_layer": frac_row(nbytes["gather"], us_reuse, note="gather-only layers (index reuse), one launch each"),
     }
 
-    # ---- variants next to the hot path: token-level selection (c = 1) and the index-similarity diagnostic
+    # ---- 32 layers with reuse depth 2 (the paper's index-reuse setting), against its speed-up model
+    t_c, t_sel = us_layer, us_reuse
+    n_r = 2
+    modelled = NL * t_c / (NL / n_r * t_c + (NL - NL / n_r) * t_sel)
+    extra_roof["cfg3_model"] = {
+        "layers": NL, "reuse_depth": n_r, "us_per_model": us_reuse2_model, "us_per_model_all_layers_computed": us_layer * NL,
+        "measured_speedup": us_layer * NL / us_reuse2_model, "modelled_speedup": modelled,
+        "T_compress_us": t_c, "T_select_us": t_sel,
+        "note": "one chunkkv_compress_model call, 16 computed + 16 reusing layers, distinct K/V per layer; modelled = "
+                "N T_c / (N/N_r T_c + (N - N/N_r) T_sel) with T_c = headline per-layer time, T_sel = gather-only layer time"}
+
     def time_calls(fn, n=30):
         for _ in range(3):
             fn()
         return timed(lambda: [fn() for _ in range(n)], 1) / n * 1e3      # us per call
 
-    n_max1 = ck.out_len(wl.L, wl.w, 1, wl.budget)
-    o1 = [torch.empty((wl.Hkv, n_max1, wl.d), dtype=torch.bfloat16, device=dev) for _ in range(2)]
-    o1.append(torch.empty((wl.Hkv, n_max1), dtype=torch.int32, device=dev))
-    calls = [0]
+    if extra:
+        # adjacent computed layers of the correlated 32-layer workload: how much their kept sets overlap
+        w3 = CONFIGS[3]
+        l3 = []
+        for x in iter_layers(w3, 3):
+            l3.append((to_dev(x.q_obs, dev), to_dev(x.K, dev), to_dev(x.V, dev)))
+        with torch.cuda.stream(stream):
+            o3 = ck.compress_model(l3, w3.Hq, w3.w, w3.c, w3.budget, n_reuse=2, stream=stream)
+            ratio, _ = ck.jaccard(o3[0][2], o3[2][2], stream=stream)
+            us_jac = time_calls(lambda: ck.jaccard(o3[0][2], o3[2][2], stream=stream))
+        torch.cuda.synchronize()
+        extra_roof["cfg3_model"]["adjacent_computed_layer_jaccard"] = {
+            "mean": float(ratio.mean()), "min": float(ratio.min()), "max": float(ratio.max()),
+            "note": "chunkkv_jaccard of the kept indices of layers 0 and 2 of the correlated workload (rho 0.8), per KV head"}
+        extra_roof["jaccard"] = {"us": us_jac, "note": "chunkkv_jaccard on two [8, 3272] index matrices (latency-bound)"}
+        del l3, o3
 
-    def token_level_layer():
-        q, K, V = sets[calls[0] % NSETS][0]
-        calls[0] += 1
-        st = lib.chunkkv_compress_layer(q.data_ptr(), K.data_ptr(), V.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, 1,
-                                        wl.budget, None, o1[0].data_ptr(), o1[1].data_ptr(), o1[2].data_ptr(),
-                                        stream.cuda_stream)
-        if st != 0:
-            raise ck.ChunkKVError(st, "chunkkv_compress_layer (c = 1)")
+        # ---- sustained: the headline graph for at least a second, with the clocks it ran at
+        reps = int(max(1.0, 1.2e3 / max(ms_per_step, 1e-3)))
+        s2 = ClockSampler(gpu_id)
+        s2.start()
+        ms_sus = timed(g_model.replay, reps)
+        c2 = s2.stop()
+        extra_roof["sustained"] = frac_row(nbytes["layer"], ms_sus / reps / NL * 1e3, seconds=ms_sus * 1e-3, steps=reps,
+                                           clocks=c2, note="headline step replayed for more than a second")
 
-    with torch.cuda.stream(stream):
-        us_token = time_calls(token_level_layer)
-        ia, ib = lane_outs[0][2], lane_outs[1][2]
-        us_jac = time_calls(lambda: ck.jaccard(ia, ib, stream=stream))
-    bytes1 = layer_bytes(wl, n_max1)["layer"]
-    extra_roof["token_level_layer"] = {"c": 1, "algorithmic_bytes": bytes1, "us": us_token,
-                                       "GB/s": bytes1 / (us_token * 1e-6) / 1e9,
-                                       "frac_of_measured_peak": bytes1 / (us_token * 1e-6) / 1e9 / peak,
-                                       "note": "chunkkv_compress_layer with c = 1, one layer at a time on all SMs"}
-    extra_roof["jaccard"] = {"us": us_jac, "note": "chunkkv_jaccard on the kept indices of two layers "
-                                                   f"([{wl.Hkv}, {n_max}] int32 each; latency-bound, includes the binding's two small allocations)"}
+        # ---- token-level layers (c = 1) through chunkkv_compress_layer
+        o1 = alloc_outs(ck, wl, 2, dev, c=1)
+        cnt = [0]
 
-    # ---- the long-context shapes (256 score rows per KV head: bound by exponentials and the tensor
-    #      pipe rather than by HBM), one layer at a time on the whole GPU
-    if not args.no_long and rank == 0:
+        def token_level_layer():
+            i = cnt[0] % NL
+            cnt[0] += 1
+            layer_call(i, c=1, o=[o1[i % 2]] * NL)
+
+        with torch.cuda.stream(stream):
+            us_token = time_calls(token_level_layer)
+        b1 = layer_bytes(wl, ck.out_len(wl.L, wl.w, 1, wl.budget))["layer"]
+        extra_roof["token_level_layer"] = frac_row(b1, us_token, c=1, note="chunkkv_compress_layer with c = 1, one layer at a time")
+        del o1
+        check_status()
+
+    del g_model, g_shared, g_reuse2, g_single, g_reuse, model, model_shared, model_reuse2
+    hosts0 = None
+    if not args.no_e2e or (rank == 0 and world == 1 and not args.no_cpu_baseline):
+        hosts0 = make_layer(wl, layer=0, seq=rank)
+
+    if extra:
+        # ---- the long-context shapes (256 score rows per KV head: bound by exponentials and the tensor
+        #      pipe rather than by HBM), one layer at a time on the whole GPU
+        del layers, shared
+        torch.cuda.empty_cache()
         tf_peak, tf_src = measured_bf16_sustained_tflops()
         sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
         long_rows = {}
-        for name, lw in (("cfg4_128k", CONFIGS[4]), ("cfg5_longest_64k", scaled(CONFIGS[5], L=65536))):
-            lsets = []
-            for i in range(2):
-                lx = make_layer(lw, layer=i)
-                lsets.append(tuple(torch.from_numpy(b.view(np.int16)).to(dev).view(torch.bfloat16)
-                                   for b in (lx.q_obs, lx.K, lx.V)))
-            ln = ck.out_len(lw.L, lw.w, lw.c, lw.budget)
-            lo = [torch.empty((lw.Hkv, ln, lw.d), dtype=torch.bfloat16, device=dev) for _ in range(2)]
-            lo.append(torch.empty((lw.Hkv, ln), dtype=torch.int32, device=dev))
+        for name, lw in long_cfgs:
+            ll = make_layers(lw, 2, dev)
+            lo = alloc_outs(ck, lw, 1, dev)[0]
             cnt = [0]
 
             def long_layer():
-                q, K, V = lsets[cnt[0] % 2]
+                q, K, V = ll[cnt[0] % 2]
                 cnt[0] += 1
                 st = lib.chunkkv_compress_layer(q.data_ptr(), K.data_ptr(), V.data_ptr(), lw.L, lw.Hq, lw.Hkv, lw.d, lw.w,
                                                 lw.c, lw.budget, None, lo[0].data_ptr(), lo[1].data_ptr(),
@@ -493,62 +512,99 @@ def run_ours(args, wl):
 
             with torch.cuda.stream(stream):
                 us = time_calls(long_layer, n=20)
-            if ck.device_status() != 0:
-                raise RuntimeError("a kernel reported an abandoned wait")
-            lb = layer_bytes(lw, ln)["layer"]
+            check_status()
+            lb = layer_bytes(lw, ck.out_len(lw.L, lw.w, lw.c, lw.budget))["layer"]
             R = lw.w * lw.Hq // lw.Hkv
             flops = 2.0 * R * lw.L * lw.d * lw.Hkv
             exps = float(R) * lw.L * lw.Hkv
-            clock_max_mhz = clocks.get("sm_max_mhz")
-            sfu_floor_us = exps / (16.0 * sm_count * clock_max_mhz * 1e6) * 1e6 if clock_max_mhz else None
-            long_rows[name] = {
-                "Hq": lw.Hq, "Hkv": lw.Hkv, "L": lw.L, "w": lw.w, "c": lw.c, "budget": lw.budget, "score_rows_per_kv_head": R,
-                "us": us, "tokens_per_s": lw.L / (us * 1e-6), "algorithmic_bytes": lb,
-                "GB/s": lb / (us * 1e-6) / 1e9, "frac_of_measured_hbm_peak": lb / (us * 1e-6) / 1e9 / peak,
-                "bf16_TFLOP/s": flops / (us * 1e-6) / 1e12,
-                "frac_of_sustained_bf16_peak": flops / (us * 1e-6) / 1e12 / tf_peak, "bf16_peak_source": tf_src,
-                "exponentials": exps, "special_function_floor_us": sfu_floor_us,
-                "note": "chunkkv_compress_layer, one layer at a time on all SMs, two K/V sets alternating (each > L2); "
-                        "floor = exponentials / (16 per clock per SM at the maximum SM clock)"}
-            del lsets, lo
+            mhz = clocks.get("sm_max_mhz")
+            row = frac_row(lb, us, Hq=lw.Hq, Hkv=lw.Hkv, L=lw.L, w=lw.w, c=lw.c, budget=lw.budget, score_rows_per_kv_head=R,
+                           tokens_per_s=lw.L / (us * 1e-6))
+            row.update({"bf16_TFLOP/s": flops / (us * 1e-6) / 1e12,
+                        "frac_of_sustained_bf16_peak": flops / (us * 1e-6) / 1e12 / tf_peak, "bf16_peak_source": tf_src,
+                        "exponentials": exps,
+                        "special_function_floor_us": exps / (16.0 * sm_count * mhz * 1e6) * 1e6 if mhz else None,
+                        "note": "chunkkv_compress_layer, one layer at a time on all SMs, two K/V sets alternating (each > L2); "
+                                "floor = exponentials / (16 per clock per SM at the maximum SM clock)"})
+            long_rows[name] = row
+            del ll, lo
         extra_roof["long_context_layers"] = long_rows
+
+        # ---- the batched serving workload as configured: 8 ragged sequences x 80 layers, reuse depth 3.
+        #      Each sequence cycles a ring of 6 layer buffers at distinct addresses (two seeded layers,
+        #      replicated on the device); one chunkkv_compress_model call per sequence.
+        w5 = CONFIGS[5]
+        n5 = ck.out_len(w5.L, w5.w, w5.c, w5.budget)
+        outs5 = [(torch.empty((w5.Hkv, n5, w5.d), dtype=torch.bfloat16, device=dev),
+                  torch.empty((w5.Hkv, n5, w5.d), dtype=torch.bfloat16, device=dev),
+                  torch.empty((w5.Hkv, n5), dtype=torch.int32, device=dev)) for _ in range(w5.n_layers)]
+        calls5 = []
+        for b, L5 in enumerate(lens5):
+            wb = scaled(w5, L=L5)
+            base = make_layers(wb, 2, dev, seq=b)
+            ring = [base[i % 2] if i < 2 else tuple(t.clone() for t in base[i % 2]) for i in range(6)]
+            calls5.append(ModelCall(ck, wb, [ring[l % 6] for l in range(w5.n_layers)], outs5, w5.reuse_depth, L=L5))
+
+        def batch_step():
+            for mc in calls5:
+                mc(stream)
+
+        with torch.cuda.stream(stream):
+            for _ in range(2):
+                batch_step()
+        torch.cuda.synchronize()
+        check_status()
+        ms5 = timed(batch_step, 3) / 3
+        n_comp = (w5.n_layers + w5.reuse_depth - 1) // w5.reuse_depth
+        bytes5 = 0
+        for L5 in lens5:
+            lb5 = layer_bytes(scaled(w5, L=L5), n5)
+            bytes5 += n_comp * lb5["layer"] + (w5.n_layers - n_comp) * lb5["gather"]
+        extra_roof["cfg5_batch"] = {
+            "sequences": len(lens5), "lengths": list(lens5), "layers": w5.n_layers, "reuse_depth": w5.reuse_depth,
+            "ms_per_batch": ms5, "tokens_per_s_per_layer": sum(lens5) * w5.n_layers / (ms5 * 1e-3),
+            "algorithmic_bytes": bytes5, "GB/s": bytes5 / (ms5 * 1e-3) / 1e9,
+            "frac_of_measured_peak": bytes5 / (ms5 * 1e-3) / 1e9 / peak,
+            "note": "8 chunkkv_compress_model calls (one per sequence, 27 computed + 53 reusing layers each), sequences one "
+                    "after another; sequences too long for the persistent kernel's tensor-memory budget run layer by layer"}
+        del calls5, outs5
+        torch.cuda.empty_cache()
 
     # ---- end to end: pinned host buffers in, host buffers out, copies inside the timed region
     e2e = None
     if not args.no_e2e:
-        pin = []
-        for x in hosts:
-            pin.append([torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).pin_memory()
-                        for b in (x.q_obs, x.K, x.V)])
+        pin = [torch.from_numpy(b.view(np.int16)).view(torch.bfloat16).pin_memory()
+               for b in (hosts0.q_obs, hosts0.K, hosts0.V)]
+        stage = [torch.empty_like(t, device=dev) for t in pin]
+        oK, oV, oI = outs[0]
         h_out = [torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16).pin_memory() for _ in range(2)]
         h_out.append(torch.empty((wl.Hkv, n_max), dtype=torch.int32).pin_memory())
+        e2e_layers = 8
 
         def step_e2e():
-            for i in range(LAYERS_PER_STEP):
-                q, K, V = sets[i % NSETS][0]
-                oK, oV, oI = lane_outs[0]
-                hq, hK, hV = pin[i % NSETS]
+            for _ in range(e2e_layers):
                 st = lib.chunkkv_compress_layer_host(
-                    hq.data_ptr(), hK.data_ptr(), hV.data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
-                    wl.budget, q.data_ptr(), K.data_ptr(), V.data_ptr(), oK.data_ptr(), oV.data_ptr(),
+                    pin[0].data_ptr(), pin[1].data_ptr(), pin[2].data_ptr(), wl.L, wl.Hq, wl.Hkv, wl.d, wl.w, wl.c,
+                    wl.budget, stage[0].data_ptr(), stage[1].data_ptr(), stage[2].data_ptr(), oK.data_ptr(), oV.data_ptr(),
                     oI.data_ptr(), h_out[0].data_ptr(), h_out[1].data_ptr(), h_out[2].data_ptr(), stream.cuda_stream)
                 if st != 0:
                     raise ck.ChunkKVError(st, "chunkkv_compress_layer_host")
 
-        e2e_steps = max(1, min(args.steps, 3))
+        e2e_steps = 3
         timed(step_e2e, 1)
         ms_e2e = timed(step_e2e, e2e_steps)
-        e2e_val, _ = job_throughput(e2e_steps * LAYERS_PER_STEP * wl.L, ms_e2e, dev)
-        h2d = LAYERS_PER_STEP * (2 * wl.Hkv * wl.L * wl.d * 2 + wl.Hq * wl.w * wl.d * 2)
-        d2h = LAYERS_PER_STEP * (2 * wl.Hkv * n_max * wl.d * 2 + wl.Hkv * n_max * 4)
+        e2e_val, _ = job_throughput(e2e_steps * e2e_layers * wl.L, ms_e2e, dev)
+        h2d = NL * (2 * wl.Hkv * wl.L * wl.d * 2 + wl.Hq * wl.w * wl.d * 2)
+        d2h = NL * (2 * wl.Hkv * n_max * wl.d * 2 + wl.Hkv * n_max * 4)
         e2e = {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "steps": e2e_steps}
-    if ck.device_status(stream) != 0 or any(ln.status() != 0 for ln in lanes):
-        raise RuntimeError("a kernel reported an abandoned wait")
+               "note": f"chunkkv_compress_layer_host, {e2e_layers} layers per timed repetition x {e2e_steps}; bytes are per "
+                       f"{NL}-layer step; bound by the host link"}
+        check_status()
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu_baseline = time_oracle(wl, hosts[0], budget_s=12.0)
+        cpu_baseline = time_oracle(wl, hosts0, budget_s=12.0)
+        cpu_baseline["single_thread"] = time_oracle_single_thread(wl, hosts0, budget_s=6.0)
 
     if rank == 0:
         line = {
@@ -556,19 +612,15 @@ def run_ours(args, wl):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": wl.name, "Hq": wl.Hq, "Hkv": wl.Hkv, "d": wl.d, "L": wl.L, "w": wl.w,
-                       "c": wl.c, "budget": wl.budget, "layers_per_step": LAYERS_PER_STEP,
-                       "lanes": S,
-                       "mode": args.mode if S > 1 else "single",
-                       "launch": f"one CUDA graph per step: 32 layer calls ({'chunkkv_pipe_layer' if piped else 'chunkkv_compress_layer_lane'}), {S} in flight "
-                                 f"on {S} streams with {lane_ctas} CTAs each" if S > 1 else
-                                 "one CUDA graph per step (32 chunkkv_compress_layer calls captured)",
-                       "l2": f"layers cycle over {NSETS} distinct K/V sets of "
-                             f"{2 * wl.Hkv * wl.L * wl.d * 2 / 1e6:.0f} MB each (> L2)"},
-            "us_per_layer": ms_layer * 1e3,
-            "eager": {"value": LAYERS_PER_STEP * wl.L * world / (ms_eager * 1e-3), "unit": UNIT,
-                      "us_per_layer": ms_eager / LAYERS_PER_STEP * 1e3,
-                      "note": "same step, 32 direct C-ABI calls, no graph"},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps * LAYERS_PER_STEP * (launches_per_layer if fused else 5),
+                       "c": wl.c, "budget": wl.budget, "layers_per_step": NL,
+                       "launch": "one CUDA graph per step holding one chunkkv_compress_model call (32 computed layers, "
+                                 "one persistent kernel launch)",
+                       "l2": f"every layer of the step has its own seeded q / K / V: {NL} x "
+                             f"{2 * wl.Hkv * wl.L * wl.d * 2 / 1e6:.0f} MB resident (> L2), none shared"},
+            "us_per_layer": us_layer,
+            "eager": {"value": NL * wl.L * world / (us_eager * NL * 1e-6), "unit": UNIT, "us_per_layer": us_eager,
+                      "note": "same step, the C-ABI call issued directly, no graph"},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": args.steps,
             "roofline": roofline, "roofline_more": extra_roof, "per_kernel": per_kernel,
             "cpu_baseline": cpu_baseline,
         }
@@ -577,12 +629,87 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def time_oracle_single_thread(wl, x, budget_s: float):
+    """The oracle on one thread: one KV head of one layer (scaled to a layer in the text only)."""
+    from oracle import chunkkv_oracle as ora
+    from threadpoolctl import threadpool_limits
+    G = wl.Hq // wl.Hkv
+    with threadpool_limits(limits=1):
+        t0 = time.perf_counter()
+        ora.compress_layer(x.q_obs[:G], x.K[:1], x.V[:1], G, 1, wl.w, wl.c, wl.budget)
+        t1 = time.perf_counter() - t0
+        n = int(max(1, min(20, round(budget_s / max(t1, 1e-3)))))
+        t0 = time.perf_counter()
+        for _ in range(n):
+            ora.compress_layer(x.q_obs[:G], x.K[:1], x.V[:1], G, 1, wl.w, wl.c, wl.budget)
+        dt = (time.perf_counter() - t0) / n
+    return {"value": wl.L / (dt * wl.Hkv), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{n} x one KV head of one {wl.name} layer on one thread, {dt * 1e3:.1f} ms per head; "
+                      f"value = L / ({wl.Hkv} heads x that)"}
+
+
+def run_profile_case(args):
+    """A few calls of one case with little warm-up, for use under a profiler (ncu -k / -s / -c)."""
+    import paper_2502_00299_b200 as ck
+    from workloads import CONFIGS, scaled
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    case = args.profile_case
+    wl = CONFIGS[4] if case == "cfg4" else CONFIGS[args.config]
+    n = args.layers if case == "model" else 2
+    layers = make_layers(wl, n, dev)
+    c = 1 if case == "token" else wl.c
+    outs = alloc_outs(ck, wl, n, dev, c=c)
+    stream = torch.cuda.current_stream()
+    times = []
+
+    def run_once(i):
+        if case == "model":
+            ck.compress_model(layers, wl.Hq, wl.w, wl.c, wl.budget, n_reuse=1, outs=outs)
+        else:
+            q, K, V = layers[i % n]
+            ck.compress_layer(q, K, V, wl.Hq, wl.w, c, wl.budget, reuse_idx=outs[i % n][2] if case == "reuse" else None,
+                              out_K=outs[i % n][0], out_V=outs[i % n][1], out_idx=outs[i % n][2])
+
+    if case == "reuse":
+        ck.compress_layer(*layers[0], wl.Hq, wl.w, c, wl.budget, out_K=outs[0][0], out_V=outs[0][1], out_idx=outs[0][2])
+        outs[1][2].copy_(outs[0][2])
+    run_once(0)
+    torch.cuda.synchronize()
+    for it in range(args.iters):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        run_once(it)
+        e1.record()
+        times.append((e0, e1))
+    torch.cuda.synchronize()
+    assert ck.device_status() == 0
+    print(case, wl.name, "us per call:", [round(a.elapsed_time(b) * 1e3, 1) for a, b in times], flush=True)
+
+
+def spawn_ranks(args):
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script on this node."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "WARN")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd, env=env)
+
+
 def main():
     args = parse_args()
     from workloads import CONFIGS
     wl = CONFIGS[args.config]
-    if args.impl == "reference":
+    if args.profile_case is not None:
+        run_profile_case(args)
+    elif args.impl == "reference":
         run_reference(args, wl)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_ranks(args))
     else:
         run_ours(args, wl)
 
