@@ -171,6 +171,39 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
                            void* out_K, void* out_V, int32_t* out_idx, void* stream);
 
 /*
+ * Adapters to the steps either side of the path (the paper runs the compression at the end of
+ * prefill - "q_observe <- Q[T_q - w : T_q]" in Algorithm 3 takes the last w queries of the layer -
+ * and hands the compacted cache to decoding).
+ *
+ * chunkkv_window_queries: q_obs [Hq, w, d] bf16 out of the layer's fused QKV projection output
+ *   qkv [T, row_elems] bf16 (token-major; the Hq query heads first in a row, then keys and values;
+ *   row_elems >= (Hq + 2 Hkv) d, a multiple of 8; values before the rotary position embedding).
+ *   The window is the last w rows. cos_rows / sin_rows [w, d / 2] f32 are the embedding-table rows
+ *   of the window's positions; element i is paired with element i + d / 2 (rotate-half):
+ *   out[i] = x[i] cos[i] - x[i + d/2] sin[i], out[i + d/2] = x[i + d/2] cos[i] + x[i] sin[i],
+ *   computed in fp64 and rounded once (through fp32) to bf16. All pointers are device memory.
+ *
+ * chunkkv_gather_paged: chunkkv_gather with a paged destination. cache_K / cache_V
+ *   [num_pages, page_size, Hkv, d] bf16; compacted position n of every head goes to page
+ *   block_table[n / page_size] (device int32, ceil(n_max / page_size) entries), slot n % page_size;
+ *   zero rows where idx is outside [0, L). Entries of the block table outside [0, num_pages) are
+ *   skipped. Pages not named and slots past n_max stay as they are.
+ *
+ * chunkkv_compress_layer_paged: chunkkv_compress_layer (or, with reuse_idx, a layer that reuses
+ *   indices) writing the kept rows to a paged cache instead of dense out_K / out_V; out_idx
+ *   [Hkv, n_max] is still written. Runs as separate score / select / gather launches.
+ */
+CHUNKKV_API int chunkkv_window_queries(const void* qkv, long long row_elems, int T, int Hq, int Hkv, int d, int w,
+                                       const float* cos_rows, const float* sin_rows, void* out_q_obs, void* stream);
+CHUNKKV_API int chunkkv_gather_paged(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d, int n_max,
+                                     const int32_t* block_table, int page_size, int num_pages, void* cache_K,
+                                     void* cache_V, void* stream);
+CHUNKKV_API int chunkkv_compress_layer_paged(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                                             int d, int w, int c, int budget, const int32_t* reuse_idx_or_null,
+                                             const int32_t* block_table, int page_size, int num_pages, void* cache_K,
+                                             void* cache_V, int32_t* out_idx, void* stream);
+
+/*
  * A whole model with layer-wise index reuse (Algorithm 2): layer l computes its indices iff
  * l mod reuse_depth == 0 (Algorithm 3 on q_obs[l], K[l], V[l]); every other layer gathers with the
  * indices of layer floor(l / reuse_depth) * reuse_depth, which are also copied to its out_idx.

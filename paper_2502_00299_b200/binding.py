@@ -50,6 +50,12 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_model_workspace_bytes.argtypes = [i32] * 9
     L.chunkkv_compress_model.restype = i32
     L.chunkkv_compress_model.argtypes = [i32, vp, vp, vp] + [i32] * 8 + [vp, vp, vp, vp]
+    L.chunkkv_window_queries.restype = i32
+    L.chunkkv_window_queries.argtypes = [vp, ctypes.c_longlong] + [i32] * 5 + [vp, vp, vp, vp]
+    L.chunkkv_gather_paged.restype = i32
+    L.chunkkv_gather_paged.argtypes = [vp, vp, vp] + [i32] * 4 + [vp, i32, i32, vp, vp, vp]
+    L.chunkkv_compress_layer_paged.restype = i32
+    L.chunkkv_compress_layer_paged.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, i32, i32, vp, vp, vp, vp]
     L.chunkkv_compress_layer_host.restype = i32
     L.chunkkv_compress_layer_host.argtypes = [vp, vp, vp] + [i32] * 7 + [vp] * 10
     L.chunkkv_lane_bytes.restype = sz
@@ -294,6 +300,47 @@ def compress_layer(q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tens
                                       budget, _ptr(reuse_idx), out_K.data_ptr(), out_V.data_ptr(),
                                       out_idx.data_ptr(), _stream(stream)), "chunkkv_compress_layer")
     return out_K, out_V, out_idx
+
+
+def window_queries(qkv: torch.Tensor, Hq: int, Hkv: int, d: int, w: int, cos_rows: torch.Tensor,
+                   sin_rows: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """q_obs [Hq, w, d] bf16 from the last w rows of a fused QKV activation [T, row_elems] bf16,
+    with the rotary embedding of those rows applied (cos_rows, sin_rows [w, d / 2] f32)."""
+    _dev(qkv, torch.bfloat16, "qkv"); _dev(cos_rows, torch.float32, "cos_rows"); _dev(sin_rows, torch.float32, "sin_rows")
+    T, row_elems = qkv.shape
+    out = torch.empty((Hq, w, d), dtype=torch.bfloat16, device=qkv.device)
+    _check(lib.chunkkv_window_queries(qkv.data_ptr(), row_elems, T, Hq, Hkv, d, w, cos_rows.data_ptr(),
+                                      sin_rows.data_ptr(), out.data_ptr(), _stream(stream)), "chunkkv_window_queries")
+    return out
+
+
+def gather_paged(K: torch.Tensor, V: torch.Tensor, idx: torch.Tensor, block_table: torch.Tensor, cache_K: torch.Tensor,
+                 cache_V: torch.Tensor, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Kept rows into a paged cache [num_pages, page_size, Hkv, d] through block_table (int32)."""
+    _dev(K, torch.bfloat16, "K"); _dev(V, torch.bfloat16, "V"); _dev(idx, torch.int32, "idx")
+    _dev(block_table, torch.int32, "block_table"); _dev(cache_K, torch.bfloat16, "cache_K"); _dev(cache_V, torch.bfloat16, "cache_V")
+    Hkv, L, d = K.shape
+    _check(lib.chunkkv_gather_paged(K.data_ptr(), V.data_ptr(), idx.data_ptr(), L, Hkv, d, idx.shape[1],
+                                    block_table.data_ptr(), cache_K.shape[1], cache_K.shape[0], cache_K.data_ptr(),
+                                    cache_V.data_ptr(), _stream(stream)), "chunkkv_gather_paged")
+
+
+def compress_layer_paged(q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tensor, Hq: int, w: int, c: int,
+                         budget: int, block_table: torch.Tensor, cache_K: torch.Tensor, cache_V: torch.Tensor,
+                         reuse_idx: Optional[torch.Tensor] = None, out_idx: Optional[torch.Tensor] = None,
+                         stream: Optional[torch.cuda.Stream] = None) -> torch.Tensor:
+    """One layer into a paged cache; returns idx [Hkv, n_max]."""
+    Hkv, L, d = K.shape
+    n_max = out_len(L, w, c, budget)
+    if reuse_idx is None:
+        ensure_workspace(L, Hq, Hkv, d, w, c)
+    if out_idx is None:
+        out_idx = torch.empty((Hkv, n_max), dtype=torch.int32, device=K.device)
+    _check(lib.chunkkv_compress_layer_paged(_ptr(q_obs), K.data_ptr(), V.data_ptr(), L, Hq, Hkv, d, w, c, budget,
+                                            _ptr(reuse_idx), block_table.data_ptr(), cache_K.shape[1], cache_K.shape[0],
+                                            cache_K.data_ptr(), cache_V.data_ptr(), out_idx.data_ptr(), _stream(stream)),
+           "chunkkv_compress_layer_paged")
+    return out_idx
 
 
 def jaccard(idx_a: torch.Tensor, idx_b: torch.Tensor, stream: Optional[torch.cuda.Stream] = None,

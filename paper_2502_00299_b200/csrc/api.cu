@@ -598,6 +598,94 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
                          stream);
 }
 
+// ---- Adapters to the steps either side of the path: window queries out of a fused QKV activation
+//      (with rotary embedding), and kept rows into a paged decode cache.
+int chunkkv_window_queries(const void* qkv, long long row_elems, int T, int Hq, int Hkv, int d, int w,
+                           const float* cos_rows, const float* sin_rows, void* out_q_obs, void* stream) {
+    if (Hkv < 1 || Hq < Hkv || Hq % Hkv != 0 || (d != 64 && d != 128) || w < 1 || T < w) return CHUNKKV_EINVAL_SHAPE;
+    if (row_elems < static_cast<long long>(Hq + 2 * Hkv) * d) return CHUNKKV_EINVAL_SHAPE;
+    if (qkv == nullptr || cos_rows == nullptr || sin_rows == nullptr || out_q_obs == nullptr) return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(out_q_obs) || (reinterpret_cast<uintptr_t>(qkv) & 1u) != 0 || (row_elems & 7) != 0)
+        return CHUNKKV_EINVAL_ALIGN;
+    cudaError_t e = launch_window_queries(qkv, row_elems, T, Hq, d, w, cos_rows, sin_rows, out_q_obs,
+                                          static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+static int check_paged(int n_max, int page_size, int num_pages, const int32_t* block_table, const void* cache_K,
+                       const void* cache_V) {
+    if (page_size < 1 || num_pages < 1 || n_max < 0) return CHUNKKV_EINVAL_SHAPE;
+    if (block_table == nullptr || cache_K == nullptr || cache_V == nullptr) return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(cache_K) || !aligned16(cache_V) || (reinterpret_cast<uintptr_t>(block_table) & 3u) != 0)
+        return CHUNKKV_EINVAL_ALIGN;
+    return CHUNKKV_OK;
+}
+
+int chunkkv_gather_paged(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d, int n_max,
+                         const int32_t* block_table, int page_size, int num_pages, void* cache_K, void* cache_V,
+                         void* stream) {
+    if (L < 1 || Hkv < 1 || Hkv > 65535 || n_max < 0 || (d != 64 && d != 128)) return CHUNKKV_EINVAL_SHAPE;
+    if (static_cast<long long>(Hkv) * L * d >= (1LL << 40)) return CHUNKKV_EINVAL_SHAPE;
+    int st = check_paged(n_max, page_size, num_pages, block_table, cache_K, cache_V);
+    if (st != CHUNKKV_OK) return st;
+    if (K == nullptr || V == nullptr || idx == nullptr) return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(K) || !aligned16(V) || !aligned16(idx)) return CHUNKKV_EINVAL_ALIGN;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaError_t e = launch_gather_paged(K, V, idx, L, Hkv, d, n_max, block_table, page_size, num_pages, cache_K, cache_V,
+                                        ctx->num_sms, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
+int chunkkv_compress_layer_paged(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv, int d, int w,
+                                 int c, int budget, const int32_t* reuse_idx, const int32_t* block_table, int page_size,
+                                 int num_pages, void* cache_K, void* cache_V, int32_t* out_idx, void* stream) {
+    int st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    st = check_heads(L, Hq, Hkv, d, w);
+    if (st != CHUNKKV_OK) return st;
+    const int C = chunkkv_num_chunks(L, w, c);
+    const int k = chunkkv_num_kept_chunks(L, w, c, budget);
+    const int n_max = chunkkv_out_len(L, w, c, budget);
+    if (n_max < 0) return n_max;
+    st = check_paged(n_max, page_size, num_pages, block_table, cache_K, cache_V);
+    if (st != CHUNKKV_OK) return st;
+    if (K == nullptr || V == nullptr || out_idx == nullptr || (reuse_idx == nullptr && q_obs == nullptr))
+        return CHUNKKV_EINVAL_NULL;
+    if (!aligned16(q_obs) || !aligned16(K) || !aligned16(V) || !aligned16(out_idx) || !aligned16(reuse_idx))
+        return CHUNKKV_EINVAL_ALIGN;
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx;
+    st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e;
+    if (reuse_idx != nullptr) {
+        if (reuse_idx != out_idx) {
+            e = cudaMemcpyAsync(out_idx, reuse_idx, static_cast<size_t>(Hkv) * n_max * sizeof(int32_t),
+                                cudaMemcpyDeviceToDevice, s);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
+    } else {
+        float* chunk_scores = nullptr;
+        if (C > 0 && k > 0) {
+            st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, round64(static_cast<size_t>(Hkv) * C),
+                           &chunk_scores, s);
+            if (st != CHUNKKV_OK) return st;
+        }
+        e = launch_select(chunk_scores, L, Hkv, w, c, C, k, n_max, out_idx, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    e = launch_gather_paged(K, V, out_idx, L, Hkv, d, n_max, block_table, page_size, num_pages, cache_K, cache_V,
+                            ctx->num_sms, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
+}
+
 // ---- Algorithm 2 over a whole model: every reuse_depth-th layer computes indices, the layers
 //      between gather with them. Where the shape fits the persistent kernel the layers go through
 //      it in launches of up to kModelMaxLayers; otherwise layer by layer.

@@ -159,6 +159,13 @@ cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int
 cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,
                           int n_max, void* out_K, void* out_V, int32_t* idx_copy_or_null,
                           int num_sms, cudaStream_t stream);
+// The gather into a paged cache [page, slot, head, d] through a block table (device int32).
+cudaError_t launch_gather_paged(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d, int n_max,
+                                const int32_t* block_table, int page_size, int num_pages, void* cache_K, void* cache_V,
+                                int num_sms, cudaStream_t stream);
+// Window queries from a fused QKV activation, rotary embedding applied (see gather.cu).
+cudaError_t launch_window_queries(const void* qkv, long long row_elems, int T, int Hq, int d, int w, const float* cos_t,
+                                  const float* sin_t, void* q_obs, cudaStream_t stream);
 // Jaccard similarity of two kept-index matrices, one CTA per head (diagnostics.cu).
 cudaError_t launch_jaccard(const int32_t* idx_a, const int32_t* idx_b, int Hkv, int n_a, int n_b,
                            float* out_ratio, int32_t* out_counts_or_null, cudaStream_t stream);

@@ -67,6 +67,14 @@ def test_invalid_sizes_are_rejected_on_the_host(ck):
     assert lib.chunkkv_score_noalloc(16, 16, 1 << 20, 8, 8, 128, 1, 64, 16, None) == -2
     assert lib.chunkkv_score_noalloc(16, 16, 1024, 8, 3, 128, 16, 10, 16, None) == -2
     assert lib.chunkkv_score_noalloc(None, None, 1024, 8, 2, 128, 16, 10, None, None) == -1
+    # adapters: shapes, then pointers
+    assert lib.chunkkv_window_queries(None, 100, 10, 8, 2, 64, 16, None, None, None, None) == -2      # T < w
+    assert lib.chunkkv_window_queries(None, 100, 20, 8, 2, 64, 16, None, None, None, None) == -2      # row too short
+    assert lib.chunkkv_window_queries(None, 768, 20, 8, 2, 64, 16, None, None, None, None) == -1
+    assert lib.chunkkv_gather_paged(16, 16, 16, 100, 2, 64, 10, 16, 0, 4, 16, 16, None) == -2          # page_size
+    assert lib.chunkkv_gather_paged(16, 16, 16, 100, 2, 64, 10, None, 4, 4, 16, 16, None) == -1
+    assert lib.chunkkv_compress_model(0, None, None, None, 1024, 8, 2, 128, 16, 10, 256, 1, None, None, None, None) == -2
+    assert lib.chunkkv_compress_model(2, None, None, None, 1024, 8, 2, 128, 16, 10, 256, 1, None, None, None, None) == -1
     # the new entry points check their arguments the same way
     assert lib.chunkkv_jaccard(None, None, 2, 10, 10, None, None, None) == -1
     assert lib.chunkkv_jaccard(None, None, 0, 10, 10, None, None, None) == -2

@@ -649,3 +649,64 @@ def test_compress_layer_alg1_matches_oracle(ck, cfg, L, ratio):
     assert np.array_equal(bits_of(oK), gK) and np.array_equal(bits_of(oV), gV)
     n_kept = (idx_np >= 0).sum(axis=1)
     assert np.all(n_kept <= max(budget, wl.w)) and np.all(idx_np[np.arange(wl.Hkv), n_kept - 1] == L - 1)
+
+
+# ------------------------------------------------------------------------------ prefill-tail adapters
+def _rope_tables(positions, d, base=10000.0):
+    inv = base ** (-np.arange(0, d, 2, dtype=np.float64) / d)
+    ang = np.asarray(positions, dtype=np.float64)[:, None] * inv[None, :]
+    return np.cos(ang).astype(np.float32), np.sin(ang).astype(np.float32)
+
+
+@pytest.mark.parametrize("Hq,Hkv,d,w,T,pad", [(8, 2, 64, 16, 100, 0), (32, 8, 128, 32, 40, 64), (4, 4, 128, 1, 1, 8)])
+def test_window_queries_bit_exact(ck, Hq, Hkv, d, w, T, pad):
+    rng = np.random.default_rng(Hq + T)
+    row = (Hq + 2 * Hkv) * d + pad
+    act = rand_bits(rng, (T, row), 2.0)
+    cos, sin = _rope_tables(np.arange(T - w, T) + 1000, d)
+    out = Guarded((Hq, w, d), torch.bfloat16)
+    got = ck.window_queries(to_dev(act), Hq, Hkv, d, w, torch.from_numpy(cos).cuda(), torch.from_numpy(sin).cuda())
+    out.t.copy_(got)
+    out.check("q_obs")
+    assert np.array_equal(bits_of(got), ora.window_queries(act, Hq, Hkv, d, w, cos, sin))
+
+
+@pytest.mark.parametrize("cfg,L,budget,page", [(1, 2048, 256, 16), (2, 5000, 500, 128), (2, 3001, 3000, 7)])
+def test_paged_cache_outputs_match_oracle(ck, cfg, L, budget, page):
+    # whole layer into a paged cache, then a layer that reuses the indices into a second set of pages
+    wl = scaled(CONFIGS[cfg], L=L, budget=budget)
+    x0, x1 = make_layer(wl, layer=0), make_layer(wl, layer=1)
+    n_max = ck.out_len(wl.L, wl.w, wl.c, wl.budget)
+    n_blk = (n_max + page - 1) // page
+    n_pages = 2 * n_blk + 3
+    rng = np.random.default_rng(page)
+    perm = rng.permutation(n_pages).astype(np.int32)
+    t0, t1 = perm[:n_blk].copy(), perm[n_blk:2 * n_blk].copy()
+    cK = Guarded((n_pages, page, wl.Hkv, wl.d), torch.bfloat16)
+    cV = Guarded((n_pages, page, wl.Hkv, wl.d), torch.bfloat16)
+    cK.t.view(torch.int16).fill_(0x1111)
+    cV.t.view(torch.int16).fill_(0x2222)
+    gI = Guarded((wl.Hkv, n_max), torch.int32)
+    idx = ck.compress_layer_paged(to_dev(x0.q_obs), to_dev(x0.K), to_dev(x0.V), wl.Hq, wl.w, wl.c, wl.budget,
+                                  torch.from_numpy(t0).cuda(), cK.t, cV.t, out_idx=gI.t)
+    idx1 = ck.compress_layer_paged(None, to_dev(x1.K), to_dev(x1.V), wl.Hq, wl.w, wl.c, wl.budget,
+                                   torch.from_numpy(t1).cuda(), cK.t, cV.t, reuse_idx=idx)
+    _status_ok(ck)
+    for g, name in ((cK, "cache_K"), (cV, "cache_V"), (gI, "out_idx")):
+        g.check(name)
+    idx_np = idx.cpu().numpy()
+    assert np.array_equal(idx1.cpu().numpy(), idx_np)
+    s = ora.chunk_scores(ora.token_scores(x0.q_obs, x0.K, wl.Hq, wl.Hkv, wl.w), wl.c)
+    assert_selection_matches(idx_np, s, wl.L, wl.w, wl.c, wl.budget)
+    refK = np.full((n_pages, page, wl.Hkv, wl.d), 0x1111, dtype=np.uint16)
+    refV = np.full((n_pages, page, wl.Hkv, wl.d), 0x2222, dtype=np.uint16)
+    ora.gather_paged(x0.K, x0.V, idx_np, t0, page, refK, refV)
+    ora.gather_paged(x1.K, x1.V, idx_np, t1, page, refK, refV)
+    assert np.array_equal(bits_of(cK.t), refK) and np.array_equal(bits_of(cV.t), refV)
+    # the stand-alone call with an out-of-range page number: that page's rows are skipped
+    bad = t0.copy()
+    bad[0] = n_pages + 5
+    before = bits_of(cK.t).copy()
+    ck.gather_paged(to_dev(x0.K), to_dev(x0.V), idx, torch.from_numpy(bad).cuda(), cK.t, cV.t)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits_of(cK.t), before)
