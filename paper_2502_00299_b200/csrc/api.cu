@@ -169,10 +169,41 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
     if (C <= 0) return CHUNKKV_OK;
     const ScoreShape sh = score_shape(Hq, Hkv, w);
     const int R = sh.Rs;
-    ScorePlan plan;
-    if (!make_score_plan(L, R, sh.Hs, d, c, ctx.num_sms, smem_budget(ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
     // with two scoring heads per KV head their chunk scores go to scratch first and are added into the output
     const size_t pair_floats = sh.shift ? round64(static_cast<size_t>(sh.Hs) * C) : 0;
+    TokenPlan tplan;
+    if (c == 1 && make_token_plan(L, w, R, sh.Hs, d, ctx.num_sms, smem_budget(ctx), &tplan)) {
+        // token scores: two passes over the keys in one launch, nothing but row records in scratch
+        const size_t tfloats = extra_payload_floats + pair_floats + static_cast<size_t>(tplan.grid) * 256;
+        int st2 = ensure_workspace(ctx, tfloats * sizeof(float));
+        if (st2 != CHUNKKV_OK) return st2;
+        float* payload = reinterpret_cast<float*>(static_cast<char*>(ctx.ws) + kHeaderBytes);
+        if (out_scores == nullptr) out_scores = payload;
+        if (resolved != nullptr) *resolved = out_scores;
+        float* head_scores = sh.shift ? payload + extra_payload_floats : out_scores;
+        CUtensorMap tq, tk;
+        st2 = encode_bf16_3d(&tq, q_obs, d, R, sh.Hs, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+        if (st2 != CHUNKKV_OK) return st2;
+        st2 = encode_bf16_3d(&tk, K, d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+        if (st2 != CHUNKKV_OK) return st2;
+        TokenIO io;
+        io.L = L; io.w = w; io.Rs = R; io.Hs = sh.Hs; io.d = d; io.kv_shift = sh.shift;
+        io.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
+        io.token_scores = head_scores;
+        io.scratch = payload + extra_payload_floats + pair_floats;
+        io.counters = reinterpret_cast<unsigned*>(static_cast<char*>(ctx.ws) + kResidentCountersOffset);
+        io.status = static_cast<int*>(ctx.ws);
+        cudaError_t e2;
+        {
+            Timer t(&ctx, stream, 0);
+            e2 = launch_token_scores(tplan, tq, tk, io, stream);
+            if (e2 == cudaSuccess && sh.shift) e2 = launch_pair_sum(head_scores, out_scores, Hkv, C, stream);
+        }
+        if (e2 != cudaSuccess) return cuda_fail(e2);
+        return CHUNKKV_OK;
+    }
+    ScorePlan plan;
+    if (!make_score_plan(L, R, sh.Hs, d, c, ctx.num_sms, smem_budget(ctx), false, &plan)) return CHUNKKV_EINVAL_SHAPE;
     const size_t floats = score_scratch_floats(plan, sh.Hs, R) + extra_payload_floats + pair_floats;
     int st = ensure_workspace(ctx, floats * sizeof(float));
     if (st != CHUNKKV_OK) return st;
@@ -525,7 +556,11 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
             return CHUNKKV_OK;
         }
         ScorePlan plan;
-        if (make_score_plan(L, R, sh.Hs, d, c, ctas, smem_budget(*ctx), true, &plan)) {
+        TokenPlan tplan;
+        // token-level layers on the whole GPU: the two-pass token-score kernel, then select and gather
+        const bool token_path = c == 1 && lane == nullptr && rows_elsewhere == nullptr &&
+                                make_token_plan(L, w, R, sh.Hs, d, ctx->num_sms, smem_budget(*ctx), &tplan);
+        if (!token_path && make_score_plan(L, R, sh.Hs, d, c, ctas, smem_budget(*ctx), true, &plan)) {
             // One cooperative launch for the whole layer.
             const size_t need = (cs_floats + score_scratch_floats(plan, sh.Hs, R)) * sizeof(float);
             char* base;

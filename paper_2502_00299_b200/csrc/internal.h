@@ -149,6 +149,22 @@ size_t model_scratch_floats(const ModelPlan& plan, int Hs, int kv_shift, int C, 
 cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtensorMap* tm_q, const CUtensorMap* tm_k,
                          const ModelLayerIO* layers, int n_layers, cudaStream_t stream);
 
+// Token scores in one launch, two passes over the keys (token_kernel.cu).
+struct TokenPlan {
+    int grid, cph, n_tiles, n_tiles_prefix, n_stages, smem_bytes, off_ring, off_misc;
+};
+struct TokenIO {
+    int L, w, Rs, Hs, d, kv_shift;
+    float sl2;
+    float* token_scores;  // [Hs][P]
+    float* scratch;       // grid * 256 floats
+    unsigned* counters;   // header + kResidentCountersOffset
+    int* status;
+};
+bool make_token_plan(int L, int w, int Rs, int Hs, int d, int max_ctas, int smem_limit, TokenPlan* plan);
+cudaError_t launch_token_scores(const TokenPlan& plan, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                                const TokenIO& io, cudaStream_t stream);
+
 cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C, float* out_scores,
                             int num_sms, cudaStream_t stream);
 

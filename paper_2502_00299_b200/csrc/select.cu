@@ -21,8 +21,10 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
     int32_t* out = out_idx + static_cast<size_t>(h) * n_max;
     if constexpr (KPT > 0)
         select_head_regs<KPT>(sc, nullptr, L, w, c, C, k, n_max, out, sm, tok_cap);
+    else if (key_bytes > 0)
+        select_head_smem(sc, nullptr, L, w, c, C, k, n_max, out, sm, key_buf, tok_cap);
     else
-        select_head_rows(sc, nullptr, L, w, c, C, k, n_max, out, sm, key_bytes > 0 ? key_buf : nullptr, tok_cap);
+        select_head_rows(sc, nullptr, L, w, c, C, k, n_max, out, sm, nullptr, tok_cap);
 }
 
 }  // namespace

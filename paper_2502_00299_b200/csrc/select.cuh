@@ -256,6 +256,194 @@ __device__ __forceinline__ void select_head_regs(const float* sc, const float* s
     __syncthreads();     // shared state may be reused by the caller
 }
 
+// The same selection with the keys of the head in a shared-memory buffer (kbuf, room for C keys)
+// instead of registers: for heads with many chunks per thread (token-level selection: tens of
+// thousands of keys). Same adaptive radix select and ordered sweep as select_head_regs; the passes
+// over the keys are strided loops (coalesced, conflict-free), the sweep walks thread-contiguous runs.
+// All threads of the CTA must call it; blockDim.x a multiple of 32, at least 512, at most 1024.
+__device__ __forceinline__ void select_head_smem(const float* sc, const float* sc2, int L, int w, int c, int C, int k,
+                                                 int n_max, int32_t* out, SelectSmem& sm, uint32_t* kbuf,
+                                                 int tok_cap = 0x7fffffff) {
+    constexpr unsigned kFull = 0xffffffffu;
+    const int P = L - w;
+    const int nt = blockDim.x, nwarps = nt >> 5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const bool keep_all = (k >= C);
+    const int kk = min(k, C);
+    if (tid == 0) sm.last_kept = 0;
+    uint32_t thresh = 0;
+    int need_eq = 0;
+    if (!keep_all && kk > 0) {
+        int* hist = reinterpret_cast<int*>(&sm.whist[0][0]);
+        uint32_t* cand = reinterpret_cast<uint32_t*>(&sm.sel[0]);
+        uint32_t lo = 0xffffffffu, hi = 0u;
+        constexpr int kB = 16;                             // loads in flight per thread
+#pragma unroll 1
+        for (int ch0 = tid; ch0 < C; ch0 += kB * nt) {
+            float v[kB];
+#pragma unroll
+            for (int q = 0; q < kB; ++q) v[q] = __ldcg(sc + min(ch0 + q * nt, C - 1));
+            if (sc2 != nullptr) {
+#pragma unroll
+                for (int q = 0; q < kB; ++q) v[q] += __ldcg(sc2 + min(ch0 + q * nt, C - 1));
+            }
+#pragma unroll
+            for (int q = 0; q < kB; ++q)
+                if (ch0 + q * nt < C) {
+                    const uint32_t key = select_order_key(v[q]);
+                    kbuf[ch0 + q * nt] = key;
+                    lo = min(lo, key);
+                    hi = max(hi, key);
+                }
+        }
+        lo = __reduce_min_sync(kFull, lo);
+        hi = __reduce_max_sync(kFull, hi);
+        if (lane == 0) sm.warp_sums[warp] = (static_cast<unsigned long long>(hi) << 32) | lo;
+        for (int i = tid; i < kSelBins; i += nt) hist[i] = 0;
+        if (tid == 0) sm.n_cand = 0;
+        __syncthreads();
+        uint32_t base = 0xffffffffu, top = 0u;
+        for (int wv = 0; wv < nwarps; ++wv) {
+            const unsigned long long v = sm.warp_sums[wv];
+            base = min(base, static_cast<uint32_t>(v));
+            top = max(top, static_cast<uint32_t>(v >> 32));
+        }
+        uint32_t span = top - base;
+        int need = k;
+        for (int round = 0;; ++round) {
+            if (span == 0u) { thresh = base; need_eq = need; break; }
+            const int shift = max(0, 21 - __clz(span));
+            if (round > 0) {
+                for (int i = tid; i < kSelBins; i += nt) hist[i] = 0;
+                __syncthreads();
+            }
+#pragma unroll 4
+            for (int ch = tid; ch < C; ch += nt) {
+                const uint32_t key = kbuf[ch], dlt = key - base;
+                if (key >= base && dlt <= span) atomicAdd(&hist[dlt >> shift], 1);
+            }
+            __syncthreads();
+            int cnt[4] = {0, 0, 0, 0}, sum = 0;
+            if (tid < kSelBins / 4) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) { cnt[q] = hist[kSelBins - 1 - 4 * tid - q]; sum += cnt[q]; }
+            }
+            int inc = sum;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int n = __shfl_up_sync(kFull, inc, off);
+                if (lane >= off) inc += n;
+            }
+            if (lane == 31) sm.warp_tot[warp] = inc;
+            __syncthreads();
+            int before = 0;
+            for (int wv = 0; wv < warp; ++wv) before += sm.warp_tot[wv];
+            inc += before;
+            if (tid < kSelBins / 4 && inc - sum < need && need <= inc) {
+                int above = inc - sum, q = 0, cq = cnt[0];
+#pragma unroll
+                for (int t = 0; t < 3; ++t)
+                    if (q == t && above + cnt[t] < need) { above += cnt[t]; q = t + 1; cq = cnt[t + 1]; }
+                sm.prefix = static_cast<uint32_t>(kSelBins - 1 - 4 * tid - q);
+                sm.need = need - above;
+                sm.bin_count = cq;
+            }
+            __syncthreads();
+            const uint32_t bin = sm.prefix;
+            const int n_bin = sm.bin_count;
+            need = sm.need;
+            const uint32_t sub = bin << shift;
+            base += sub;
+            span = min((1u << shift) - 1u, span - sub);
+            if (n_bin <= kSelCandCap) {
+#pragma unroll 4
+                for (int ch = tid; ch < C; ch += nt) {
+                    const uint32_t key = kbuf[ch], dlt = key - base;
+                    if (key >= base && dlt <= span) cand[atomicAdd(&sm.n_cand, 1)] = key;
+                }
+                __syncthreads();
+                for (int j = tid; j < n_bin; j += nt) {
+                    const uint32_t v = cand[j];
+                    int gt = 0, ge = 0;
+                    for (int i = 0; i < n_bin; ++i) { gt += cand[i] > v; ge += cand[i] >= v; }
+                    if (gt < need && need <= ge) { sm.prefix = v; sm.need = need - gt; }
+                }
+                __syncthreads();
+                thresh = sm.prefix;
+                need_eq = sm.need;
+                break;
+            }
+        }
+        __syncthreads();
+    }
+    // ordered sweep: warp v owns the contiguous ids [v * rows * 32, (v + 1) * rows * 32) and walks them in
+    // rows of 32 consecutive ids, one per lane; ballots give a row's (#above, #equal) in lane order
+    const bool stage_sel = kk <= kSelCap;
+    if (kk > 0) {
+        const unsigned lt_mask = (1u << lane) - 1u;
+        const int rows = (C + nt - 1) / nt;
+        const int base_id = warp * rows * 32 + lane;
+        unsigned gt_n = 0, eq_n = 0;
+#pragma unroll 4
+        for (int u = 0; u < rows; ++u) {
+            const int ch = base_id + 32 * u;
+            const uint32_t key = (ch < C && !keep_all) ? kbuf[ch] : 0u;
+            gt_n += __popc(__ballot_sync(kFull, ch < C && (keep_all || key > thresh)));
+            eq_n += __popc(__ballot_sync(kFull, ch < C && !keep_all && key == thresh));
+        }
+        if (lane == 0) sm.warp_sums[warp] = (static_cast<unsigned long long>(eq_n) << 32) | gt_n;
+        __syncthreads();
+        if (warp == 0) {
+            const unsigned long long s = (lane < nwarps) ? sm.warp_sums[lane] : 0ull;
+            unsigned long long sinc = s;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const unsigned long long n = __shfl_up_sync(kFull, sinc, off);
+                if (lane >= off) sinc += n;
+            }
+            sm.warp_sums[lane] = sinc - s;
+        }
+        __syncthreads();
+        const unsigned long long excl = sm.warp_sums[warp];
+        int gt_run = static_cast<int>(excl & 0xffffffffu), eq_run = static_cast<int>(excl >> 32);
+#pragma unroll 2
+        for (int u = 0; u < rows; ++u) {
+            const int ch = base_id + 32 * u;
+            const uint32_t key = (ch < C && !keep_all) ? kbuf[ch] : 0u;
+            const bool gt = ch < C && (keep_all || key > thresh);
+            const bool eq = ch < C && !keep_all && key == thresh;
+            const unsigned gtm = __ballot_sync(kFull, gt), eqm = __ballot_sync(kFull, eq);
+            const int gt_before = gt_run + __popc(gtm & lt_mask);
+            const int eq_before = eq_run + __popc(eqm & lt_mask);
+            if (gt || (eq && eq_before < need_eq)) {
+                const int rank = gt_before + min(eq_before, need_eq);
+                if (stage_sel) sm.sel[rank] = ch;
+                else {
+                    const int j0 = ch * c, len = min(c, P - j0);
+                    int32_t* dst = out + static_cast<size_t>(rank) * c;
+                    for (int t = 0; t < len; ++t)
+                        if (rank * c + t < tok_cap) dst[t] = j0 + t;
+                }
+                if (ch == C - 1) sm.last_kept = 1;
+            }
+            gt_run += __popc(gtm);
+            eq_run += __popc(eqm);
+        }
+    }
+    __syncthreads();
+    const int tail = (C > 0) ? (P - (C - 1) * c) : 0;
+    const int n_tok = min(kk * c - ((sm.last_kept && kk > 0) ? (c - tail) : 0), tok_cap);
+    if (stage_sel)
+        for (int r = tid; r < kk; r += nt) {
+            const int j0 = sm.sel[r] * c, n0 = r * c;
+            for (int t = 0; t < c; ++t)
+                if (n0 + t < n_tok) out[n0 + t] = j0 + t;
+        }
+    for (int i = tid; i < w; i += nt) out[n_tok + i] = P + i;
+    for (int i = n_tok + w + tid; i < n_max; i += nt) out[i] = -1;
+    __syncthreads();
+}
+
 // Selection for many chunks per thread. All threads of the CTA must call this (it uses
 // __syncthreads); blockDim.x must be a multiple of 32 and at most 1024. kbuf: room for C keys
 // (shared or global memory; it may be the score array itself, which is then overwritten), or
