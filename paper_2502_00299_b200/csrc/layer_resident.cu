@@ -391,7 +391,10 @@ layer_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
             const size_t idx_bytes = (static_cast<size_t>(a.n_max) * 4 + 127) & ~size_t(127);
             uint32_t* kbuf = reinterpret_cast<uint32_t*>(ring + kSelBytes + idx_bytes);
             const bool fits = kSelBytes + idx_bytes + static_cast<size_t>(a.C) * 4 <= static_cast<size_t>(a.ring_bytes);
-            select_head_rows(sc, sc2, a.L, a.w, C_STATIC, a.C, a.k, a.n_max, sidx, ss, fits ? kbuf : nullptr);
+            if (fits)
+                select_head_smem(sc, sc2, a.L, a.w, C_STATIC, a.C, a.k, a.n_max, sidx, ss, kbuf);
+            else
+                select_head_rows(sc, sc2, a.L, a.w, C_STATIC, a.C, a.k, a.n_max, sidx, ss, nullptr);
         }
         const int Q = a.cph << a.kv_shift;               // CTAs of this KV head
         const int q = static_cast<int>(blockIdx.x) - (hkv << a.kv_shift) * a.cph;

@@ -53,6 +53,8 @@ struct ModelCtl {
     unsigned long long sfull;          // a kept-chunk list has landed in shared memory (copy thread)
     unsigned long long stat_full[2];   // m_i and 1 / l_i of a slot are in shared memory (statistics warps -> epilogue)
     unsigned long long rfull;          // a batch of CTA records has landed in shared memory (statistics warps)
+    unsigned long long pub_done[2];    // every epilogue warp has stored its part of the slot's record (-> statistics warp)
+    unsigned long long sc_done[2];     // every epilogue warp has stored its chunk scores of the slot (-> statistics warp)
     uint32_t tmem_base;
     int abort_flag;
     int epi_ok;
@@ -165,8 +167,12 @@ __device__ __forceinline__ bool selector_loop(const ModelParams& p, uint8_t* dyn
             if (p.C <= kMThreads * 8)
                 select_head_regs<8>(sc, sc2, p.L, p.w, C_STATIC, p.C, p.k, p.n_max, sidx, ss);
             else
-                select_head_rows(sc, sc2, p.L, p.w, C_STATIC, p.C, p.k, p.n_max, sidx, ss,
-                                 p.sel_keys_fit ? kbuf : nullptr);
+{
+                if (p.sel_keys_fit)
+                    select_head_smem(sc, sc2, p.L, p.w, C_STATIC, p.C, p.k, p.n_max, sidx, ss, kbuf);
+                else
+                    select_head_rows(sc, sc2, p.L, p.w, C_STATIC, p.C, p.k, p.n_max, sidx, ss, nullptr);
+            }
             const int n_tok = kk * C_STATIC - ((ss.last_kept && kk > 0) ? (C_STATIC - tail_rows) : 0);
             // the kept-chunk list for the copy threads: [n_tok, -, -, -, chunk ids]
             int* row = p.sel_rows + (static_cast<size_t>(s) * p.Hkv + hkv) * row_ints;
@@ -257,6 +263,10 @@ model_kernel(const __grid_constant__ ModelParams p) {
         mbar_init(smem_u32(&ctl.stat_full[0]), 1);
         mbar_init(smem_u32(&ctl.stat_full[1]), 1);
         mbar_init(smem_u32(&ctl.rfull), 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&ctl.pub_done[b]), 16);
+            mbar_init(smem_u32(&ctl.sc_done[b]), 16);
+        }
         ctl.abort_flag = 0;
         ctl.epi_ok = 1;
         fence_mbar_init();
@@ -419,9 +429,10 @@ model_kernel(const __grid_constant__ ModelParams p) {
                 dst[et] = M;
                 dst[128 + et] = Ls;
             }
-            named_barrier(kBarEpi, kMEpiThreads);
-            if (et == 0)     // (no return value: the thread does not wait for the round trip)
-                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt_a + hs) : "memory");
+            // the statistics warp announces the record once every epilogue warp has got here: no block-wide
+            // barrier and no memory fence on the scoring warps' path
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl.pub_done[s & 1]));
             return true;
         };
         // chunk scores of slot s from the partial sums in the rings (see layer_resident.cu)
@@ -470,9 +481,8 @@ model_kernel(const __grid_constant__ ModelParams p) {
             float* sc_out = p.scores + (static_cast<size_t>(s) * p.Hs + hs) * p.Cpad;
             for (int lc = et; lc < n_local; lc += kMEpiThreads)
                 if (ch0 + lc < p.C) sc_out[ch0 + lc] = (red[lc] + red[256 + lc]) + (red[512 + lc] + red[768 + lc]);
-            named_barrier(kBarEpi, kMEpiThreads);
-            if (et == 0)     // release: the scores written above (ordered by the barrier) are visible to whoever sees the count
-                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt_b + hs) : "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl.sc_done[s & 1]));      // announced by the statistics warp
             return true;
         };
         for (int s = 0; s <= p.n_compute; ++s) {
@@ -497,7 +507,11 @@ model_kernel(const __grid_constant__ ModelParams p) {
         for (int s = 0; s < p.n_compute && ok; ++s) {
             bool w_ok = true;
             if (lane == 0) {
-                w_ok = wait_counter(p.cnt_a + hs, static_cast<unsigned>(s + 1) * p.cph, abort_flag, 0);
+                // this CTA's record is complete (all epilogue warps arrived): announce it. release: the
+                // record stores, ordered before by the mbarrier, are visible to whoever sees the count
+                w_ok = mbar_wait(smem_u32(&ctl.pub_done[s & 1]), static_cast<uint32_t>(s >> 1) & 1u, abort_flag);
+                if (w_ok) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt_a + hs) : "memory");
+                if (w_ok) w_ok = wait_counter(p.cnt_a + hs, static_cast<unsigned>(s + 1) * p.cph, abort_flag, 0);
                 asm volatile("fence.acq_rel.gpu;" ::: "memory");
             }
             if (!__shfl_sync(0xffffffffu, w_ok, 0)) break;
@@ -529,7 +543,15 @@ model_kernel(const __grid_constant__ ModelParams p) {
             *reinterpret_cast<float4*>(gm + r0) = make_float4(M[0], M[1], M[2], M[3]);
             *reinterpret_cast<float4*>(gm + 128 + r0) = make_float4(1.0f / S[0], 1.0f / S[1], 1.0f / S[2], 1.0f / S[3]);
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctl.stat_full[s & 1]));
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&ctl.stat_full[s & 1]));
+                // the epilogue forms the slot's chunk scores next; announce them when they are stored
+                if (mbar_wait(smem_u32(&ctl.sc_done[s & 1]), static_cast<uint32_t>(s >> 1) & 1u, abort_flag))
+                    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt_b + hs) : "memory");
+                else
+                    ok = false;
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
         }
     } else if (warp == 18) {
         // ------------------------------------------------------------------ tail: row copies

@@ -860,8 +860,11 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 // chunk scores, which nothing reads after the selection
                 uint32_t* kbuf = reinterpret_cast<uint32_t*>(dyn + ((sizeof(SelectSmem) + 127) & ~size_t(127)));
                 const bool fits = static_cast<size_t>(la.C) * 4 + sizeof(SelectSmem) + 256 <= static_cast<size_t>(g.dyn_bytes);
-                select_head_rows(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss,
-                                 fits ? kbuf : reinterpret_cast<uint32_t*>(const_cast<float*>(sc)));
+                if (fits)
+                    select_head_smem(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss, kbuf);
+                else
+                    select_head_rows(sc, sc2, a.L, a.w, a.c, la.C, la.k, la.n_max, out, ss,
+                                     reinterpret_cast<uint32_t*>(const_cast<float*>(sc)));
             }
         }
         if (rows_elsewhere) return;
