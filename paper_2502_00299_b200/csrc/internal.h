@@ -121,7 +121,7 @@ struct ModelPlan {
     int c_static, grid, cph, n_tiles, t_max, n_stages, smem_bytes;
     int n_score, n_sel;          // scoring CTAs, selector CTAs (grid = n_score + n_sel)
     int sel_row_bytes, sel_keys_fit;
-    int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes, off_rec;
+    int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes;
 };
 
 struct ModelIO {

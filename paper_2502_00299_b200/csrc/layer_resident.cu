@@ -126,7 +126,9 @@ layer_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
 
     const int hs = blockIdx.x / a.cph, part = blockIdx.x - hs * a.cph;
     const int hkv = hs >> a.kv_shift;
-    const int t_begin = a.n_tiles * part / a.cph, t_end = a.n_tiles * (part + 1) / a.cph;
+    // tiles are dealt out rounding up, so the head's last CTA - whose last panels take the slow, masked path -
+    // is never one of those that get an extra tile
+    const int t_begin = (a.n_tiles * part + a.cph - 1) / a.cph, t_end = (a.n_tiles * (part + 1) + a.cph - 1) / a.cph;
     const int nt = t_end - t_begin;
 
     if (threadIdx.x == 0) {

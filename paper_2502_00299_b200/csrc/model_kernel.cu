@@ -6,19 +6,23 @@
 //   warp 0         TMA producer: streams the Q tile and the CTA's K tiles of layer after layer
 //                  through the shared-memory ring, as far ahead as the ring allows
 //   warp 1         tcgen05.mma issuer
-//   warps 2..17    epilogue: one exponential per score element, chunk sums into tensor memory;
-//                  at the end of a layer they publish the CTA's per-row (max, sum), wait for the
-//                  head's other CTAs (bounded), merge the row statistics, contract the partial
-//                  sums over the rows into the chunk scores of the CTA's key range (global memory),
-//                  announce them on the head's second counter and go on with the next layer
-//   warps 18..19   tail: for each computed layer, once the head's chunk scores are complete, run
-//                  the exact top-k (every CTA of a head computes the same kept-chunk list), write
-//                  out_idx (one CTA per head) and move this CTA's share of the kept K/V rows with
-//                  bulk asynchronous copies (global -> shared -> global, whole chunks at a time) -
-//                  for the computed layer and for every following layer that reuses its indices
+//   warps 2..17    epilogue, four groups of four warps: one exponential per score element, chunk sums
+//                  into a ring of tensor-memory columns that holds more than one layer; at the end
+//                  of a layer a group leaves its per-row (max, sum) in shared memory and goes straight
+//                  on with the next layer; when the head's row statistics have arrived (normally long
+//                  before they are needed) it contracts the partial sums it wrote itself over the rows
+//                  into chunk scores of the CTA's key range (global memory)
+//   warp 18        one thread: for each computed layer, once a selector CTA has published the head's
+//                  kept-chunk list, moves this CTA's share of the kept K/V rows with bulk asynchronous
+//                  copies (global -> shared -> global, whole chunks at a time) - for the computed
+//                  layer and for every following layer that reuses its indices
+//   warp 19        row statistics: merges the groups' records, stores and announces the CTA's record,
+//                  waits (bounded) for the head's other CTAs, merges their records into m_i and 1 / l_i
+//                  for the contraction, and announces the CTA's chunk scores when they are stored
+// The CTAs after the scoring CTAs are selectors: exact top-k per head, out_idx, kept-chunk lists.
 //
-// So while the tail warps select and gather layer l, the other warps already score layer l + 1: the
-// latency-bound steps cost no memory bandwidth and the copies ride along with the K stream.
+// So while the selectors and copy threads work on layer l, the other warps already score layer l + 1:
+// the latency-bound steps cost no memory bandwidth and the copies ride along with the K stream.
 // Hand-over counters only grow during a launch (layer l waits for (l + 1) x CTAs arrivals); the
 // last CTA to leave clears them. Every wait is bounded and reports through the device status word.
 #include "internal.h"
@@ -36,23 +40,34 @@ namespace {
 constexpr int kMThreads = 640;          // warp 0: TMA, warp 1: UMMA issue, warps 2..17: epilogue, warp 18: row copies, warp 19: row statistics
                                         // (five warps per scheduler: a sixth would cut every thread to 80 registers)
 constexpr int kMEpiThreads = 512;
-constexpr int kMMiscBytes = 14336;      // epilogue: group records, slices, m_i, 1 / l_i, row sums per lane quarter
+constexpr int kMMiscBytes = 18432;      // epilogue: group records (two slots), m_i, 1 / l_i, row sums per lane quarter
 constexpr int kMSlots = 8;              // staging slots of the row copies
 constexpr int kBarEpi = 1;
-constexpr int kMRecBatch = 24;           // CTA records fetched per bulk copy by the statistics warp
-constexpr int kMRecBytes = kMRecBatch * 1024;
+// Tensor memory: three 64-column accumulators (one 60-key panel of a tile each, in rotation; the
+// second panel of a tile is computed on keys 56 .. 119 so that its operand starts on a swizzle-atom
+// boundary, and begins at column 4), and 320 columns of chunk partial sums: a ring that holds one
+// layer and two thirds of the next at c = 10, so the statistics of a layer have most of the next
+// layer's scoring time to travel before its contraction needs them.
+constexpr int kMAccN = 64;
+constexpr int kMAccBufs = 3;
+constexpr int kMAccSlots = 12;                     // (buffer, epilogue group) pairs: lcm(3 buffers, 4 groups)
+constexpr int kMAcc1Row = 56;
+constexpr int kMPartCol0 = kMAccBufs * kMAccN;
+constexpr int kMPartCols = 512 - kMPartCol0;
+constexpr int kMRingPanels10 = kMPartCols / 6;     // c = 10: 6 chunk columns per panel
+constexpr int kMRingPanels20 = 84;                 // c = 20: 3 per panel; more would only cost shared memory
+constexpr int kBarGroup = 2;                       // named barriers 2 .. 5: the four warps of an epilogue group
 
 struct ModelCtl {
     unsigned long long full[kRMaxStages];
     unsigned long long empty[kRMaxStages];
-    unsigned long long tfull[2];
-    unsigned long long tempty[2];
+    unsigned long long tfull[kMAccSlots];      // by panel number modulo 12: one (accumulator, epilogue group) pair each
+    unsigned long long tempty[kMAccSlots];
     unsigned long long qfull;
     unsigned long long qempty;
     unsigned long long gfull[kMSlots];
     unsigned long long sfull;          // a kept-chunk list has landed in shared memory (copy thread)
     unsigned long long stat_full[2];   // m_i and 1 / l_i of a slot are in shared memory (statistics warps -> epilogue)
-    unsigned long long rfull;          // a batch of CTA records has landed in shared memory (statistics warps)
     unsigned long long pub_done[2];    // every epilogue warp has stored its part of the slot's record (-> statistics warp)
     unsigned long long sc_done[2];     // every epilogue warp has stored its chunk scores of the slot (-> statistics warp)
     uint32_t tmem_base;
@@ -85,7 +100,6 @@ struct ModelParams {
     int sel_row_bytes;     // bytes of one kept-chunk list: 4 header ints + the kept chunk ids, padded to 16 bytes
     int sel_keys_fit;      // selector: the keys of a head fit its shared memory (many chunks per thread)
     int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes;
-    int off_rec;           // record staging buffer of the statistics warps, from off_tail
     float* cta_stat;       // [2 (slot parity)][grid][{max, sum}][128]
     float* scores;         // [n_compute][Hs][Cpad]
     unsigned* cnt_a;       // [Hs]
@@ -113,6 +127,51 @@ __device__ __forceinline__ void bulk_wait_read() {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Fold N (max, sum-of-exp2) records into (M, S), one row each of four rows at a time: the new maximum
+// first, then N independent exponentials (a short dependency chain, unlike N merges in sequence).
+template <int N>
+__device__ __forceinline__ void merge_batch(float (&M)[4], float (&S)[4], const float4 (&m)[N], const float4 (&l)[N], int n) {
+    const float ninf = -CUDART_INF_F;
+    float nm[4] = {M[0], M[1], M[2], M[3]};
+#pragma unroll
+    for (int j = 0; j < N; ++j)
+        if (j < n) {
+            nm[0] = fmaxf(nm[0], m[j].x);
+            nm[1] = fmaxf(nm[1], m[j].y);
+            nm[2] = fmaxf(nm[2], m[j].z);
+            nm[3] = fmaxf(nm[3], m[j].w);
+        }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) S[r] = (M[r] == ninf) ? 0.f : S[r] * ex2_approx(M[r] - nm[r]);
+#pragma unroll
+    for (int j = 0; j < N; ++j)
+        if (j < n) {
+            S[0] += (m[j].x == ninf) ? 0.f : l[j].x * ex2_approx(m[j].x - nm[0]);
+            S[1] += (m[j].y == ninf) ? 0.f : l[j].y * ex2_approx(m[j].y - nm[1]);
+            S[2] += (m[j].z == ninf) ? 0.f : l[j].z * ex2_approx(m[j].z - nm[2]);
+            S[3] += (m[j].w == ninf) ? 0.f : l[j].w * ex2_approx(m[j].w - nm[3]);
+        }
+#pragma unroll
+    for (int r = 0; r < 4; ++r) M[r] = nm[r];
+}
+
+// Bounded wait of a whole warp on a counter that only grows: every lane performs the acquire load, so
+// each lane's later loads are ordered behind the arrivals it has seen. Lane 0 keeps the time limit.
+__device__ __forceinline__ bool wait_counter_warp(const unsigned* counter, unsigned target, volatile int* abort_flag) {
+    const long long t0 = clock64();
+    for (;;) {
+        unsigned cur;
+        asm volatile("ld.acquire.gpu.u32 %0, [%1];" : "=r"(cur) : "l"(counter) : "memory");
+        if (__all_sync(0xffffffffu, cur >= target)) return true;
+        int bad = 0;
+        if ((threadIdx.x & 31) == 0) {
+            if (*abort_flag) bad = 1;
+            else if (clock64() - t0 > kWaitLimitClocks) { *abort_flag = 1; bad = 1; }
+        }
+        if (__shfl_sync(0xffffffffu, bad, 0)) return false;
+    }
+}
 
 // Bounded wait of one thread on a counter that only grows.
 __device__ __forceinline__ bool wait_counter(const unsigned* counter, unsigned target, volatile int* abort_flag,
@@ -203,7 +262,7 @@ template <int C_STATIC>
 __global__ void __launch_bounds__(kMThreads, 1)
 model_kernel(const __grid_constant__ ModelParams p) {
     constexpr int SPP = kRPanel / C_STATIC;
-    constexpr uint32_t IDESC = umma_idesc_bf16(128, kRUmmaN);
+    constexpr uint32_t IDESC = umma_idesc_bf16(128, kMAccN);
 
     extern __shared__ uint8_t smem_raw[];
     __shared__ ModelCtl ctl;
@@ -216,7 +275,7 @@ model_kernel(const __grid_constant__ ModelParams p) {
     const uint32_t k_base = smem_base + static_cast<uint32_t>(p.off_ring);
     float* pmax = reinterpret_cast<float*>(dyn + p.off_pmax);
     float* misc = reinterpret_cast<float*>(dyn + p.off_misc);
-    float* rec = misc;                 // [4 groups][{max, sum}][128]
+    float* rec = misc;                 // [4 groups][{max, sum}][128]; the odd slots' copy sits at misc + 3584
     float* gstat = misc + 1024;        // [2 (slot parity)][{m_i, 1 / l_i}][128]
     float* red = misc + 2304;          // [4 lane quarters][256 chunk slots]
     volatile int* abort_flag = &ctl.abort_flag;
@@ -244,7 +303,9 @@ model_kernel(const __grid_constant__ ModelParams p) {
     }
     const int hs = blockIdx.x / p.cph, part = blockIdx.x - hs * p.cph;
     const int hkv = hs >> p.kv_shift;
-    const int t_begin = p.n_tiles * part / p.cph, t_end = p.n_tiles * (part + 1) / p.cph;
+    // tiles are dealt out rounding up, so the head's last CTA - whose last panels take the slow, masked path -
+    // is never one of those that get an extra tile
+    const int t_begin = (p.n_tiles * part + p.cph - 1) / p.cph, t_end = (p.n_tiles * (part + 1) + p.cph - 1) / p.cph;
     const int nt = t_end - t_begin;
 
     if (threadIdx.x == 0) {
@@ -252,9 +313,9 @@ model_kernel(const __grid_constant__ ModelParams p) {
             mbar_init(smem_u32(&ctl.full[s]), 1);
             mbar_init(smem_u32(&ctl.empty[s]), 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kMAccSlots; ++b) {
             mbar_init(smem_u32(&ctl.tfull[b]), 1);
-            mbar_init(smem_u32(&ctl.tempty[b]), 8);
+            mbar_init(smem_u32(&ctl.tempty[b]), 4);
         }
         mbar_init(smem_u32(&ctl.qfull), 1);
         mbar_init(smem_u32(&ctl.qempty), 1);
@@ -262,7 +323,6 @@ model_kernel(const __grid_constant__ ModelParams p) {
         mbar_init(smem_u32(&ctl.sfull), 1);
         mbar_init(smem_u32(&ctl.stat_full[0]), 1);
         mbar_init(smem_u32(&ctl.stat_full[1]), 1);
-        mbar_init(smem_u32(&ctl.rfull), 1);
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&ctl.pub_done[b]), 16);
             mbar_init(smem_u32(&ctl.sc_done[b]), 16);
@@ -328,31 +388,47 @@ model_kernel(const __grid_constant__ ModelParams p) {
         // ------------------------------------------------------------------ UMMA issuer
         if (elect_one() && nt > 0) {
             uint32_t st = 0, st_par = 0;
-            int tg = 0;                  // tiles issued so far (all layers): buffer = tg & 1
+            int tg = 0;                  // tiles issued so far (all layers); the epilogue pair tg & 1 reads tile tg
             bool ok = true;
             for (int s = 0; s < p.n_compute && ok; ++s) {
                 ok = mbar_wait(smem_u32(&ctl.qfull), s & 1, abort_flag);
                 for (int ti = 0; ti < nt && ok; ++ti, ++tg) {
-                    const int buf = tg & 1, use = tg >> 1;
-                    ok = mbar_wait(smem_u32(&ctl.tempty[buf]), (use & 1) ^ 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t d_addr = tmem_base + static_cast<uint32_t>(buf * kRUmmaN);
+                    uint32_t st_kb[2] = {0u, 0u};
 #pragma unroll
                     for (int kb = 0; kb < 2; ++kb) {
                         if (kb >= KB || !ok) break;
                         ok = mbar_wait(smem_u32(&ctl.full[st]), st_par, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                        const uint64_t b_desc = umma_desc_sw128(k_base + st * kRStageBytes);
-                        const uint64_t a_desc = umma_desc_sw128(q_base + static_cast<uint32_t>(kb) * kRQTileBytes);
-#pragma unroll
-                        for (int k4 = 0; k4 < 4; ++k4)
-                            umma_bf16(d_addr, a_desc + 2u * k4, b_desc + 2u * k4, IDESC, (kb > 0 || k4 > 0) ? 1u : 0u);
-                        umma_commit(smem_u32(&ctl.empty[st]));
+                        st_kb[kb] = st;
                         if (++st == n_stages) { st = 0; st_par ^= 1u; }
                     }
-                    if (ok) umma_commit(smem_u32(&ctl.tfull[buf]));
+                    if (!ok) break;
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        // panel pc goes to accumulator pc % 3, which panel pc - 3 used last
+                        const int pc = 2 * tg + half;
+                        if (pc >= kMAccBufs) {
+                            const int prev = pc - kMAccBufs;
+                            ok = mbar_wait(smem_u32(&ctl.tempty[prev % kMAccSlots]), (prev / kMAccSlots) & 1, abort_flag);
+                        }
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t d_addr = tmem_base + static_cast<uint32_t>((pc % kMAccBufs) * kMAccN);
+#pragma unroll
+                        for (int kb = 0; kb < 2; ++kb) {
+                            if (kb >= KB) break;
+                            const uint64_t b_desc =
+                                umma_desc_sw128(k_base + st_kb[kb] * kRStageBytes + static_cast<uint32_t>(half * kMAcc1Row * 128));
+                            const uint64_t a_desc = umma_desc_sw128(q_base + static_cast<uint32_t>(kb) * kRQTileBytes);
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4)
+                                umma_bf16(d_addr, a_desc + 2u * k4, b_desc + 2u * k4, IDESC, (kb > 0 || k4 > 0) ? 1u : 0u);
+                        }
+                        umma_commit(smem_u32(&ctl.tfull[pc % kMAccSlots]));
+                    }
+                    if (!ok) break;
+#pragma unroll
+                    for (int kb = 0; kb < 2; ++kb)
+                        if (kb < KB) umma_commit(smem_u32(&ctl.empty[st_kb[kb]]));
                 }
                 if (ok) umma_commit(smem_u32(&ctl.qempty));       // every UMMA of this layer has read the Q tile
             }
@@ -364,35 +440,35 @@ model_kernel(const __grid_constant__ ModelParams p) {
         // thread only publishes the CTA's row records and goes straight on with the first `ahead`
         // tiles of layer s + 1; the chunk scores of layer s are formed after those, when the other
         // CTAs' records have long arrived and the statistics warp has merged them.
-        const int et = threadIdx.x - 64;                 // 0 .. 511
         const int grp = (warp - 2) >> 2, quarter = warp & 3;
+        const int gt = threadIdx.x - 64 - grp * 128;    // 0 .. 127 within the group
         const int pair = grp >> 1, half = grp & 1;
         const int row = quarter * 32 + lane;
         const bool active = row < p.R;
         const int last_visible = p.P + (row % p.w);
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const int n_pl = 2 * nt;
-        constexpr int PR = kRPartCols / 6 * 6 / SPP;     // panels in the rings (252 columns)
+        constexpr int PR = (C_STATIC == 10) ? kMRingPanels10 : kMRingPanels20;     // panels in the rings
         const int ahead = max(0, min(nt, (PR - n_pl) / 2));   // tiles of the next layer scored before the contraction
-        const int n_local = nt * (kRTile / C_STATIC);
         const int ch0 = t_begin * (kRTile / C_STATIC);
         bool ok = true;
         float run_m = -CUDART_INF_F, run_l = 0.f;
         // tiles [ti_lo, ti_hi) of slot s that belong to this thread's pair
         auto do_tiles = [&](int s, int ti_lo, int ti_hi) {
-            if (!ok) return;      // (a warp whose wait failed still joins the barriers below until all warps leave together)
+            if (!ok) return;
             const int tg0 = s * nt, pbase = (s * n_pl) % PR;
             for (int ti = ti_lo + ((pair - ((tg0 + ti_lo) & 1)) & 1); ti < ti_hi; ti += 2) {
-                const int tg = tg0 + ti, use = tg >> 1;
+                const int pc = 2 * (tg0 + ti) + half;        // panel number since the start of the launch
+                const int aslot = pc % kMAccSlots;
                 bool ready = true;
-                if (lane == 0) ready = mbar_wait(smem_u32(&ctl.tfull[pair]), use & 1, abort_flag);
+                if (lane == 0) ready = mbar_wait(smem_u32(&ctl.tfull[aslot]), (pc / kMAccSlots) & 1, abort_flag);
                 if (!__shfl_sync(0xffffffffu, ready, 0)) { ok = false; break; }
                 tc_fence_after();
                 float v[kRPanel];
-                load_panel<kRPanel>(lane_addr + static_cast<uint32_t>(pair * kRUmmaN + half * kRPanel), v);
+                load_panel<kRPanel>(lane_addr + static_cast<uint32_t>((pc % kMAccBufs) * kMAccN + half * (kRPanel - kMAcc1Row)), v);
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[pair]));
+                if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[aslot]));
                 const int pl = ti * 2 + half;
                 int slot = pbase + pl;
                 slot -= (slot >= PR) ? PR : 0;
@@ -403,7 +479,7 @@ model_kernel(const __grid_constant__ ModelParams p) {
                     panel_fast<C_STATIC, kRPanel>(v, p.sl2, emit, &m2, &l);
                 else
                     panel_static_tail<C_STATIC, kRPanel>(v, p.sl2, emit, j0, p.P, last_visible, &m2, &l);
-                part_store<SPP>(lane_addr + static_cast<uint32_t>(kRPartCol0 + slot * SPP), pr);
+                part_store<SPP>(lane_addr + static_cast<uint32_t>(kMPartCol0 + slot * SPP), pr);
                 pmax[slot * 128 + row] = m2;
                 const float nm = fmaxf(run_m, m2);
                 const float s_old = (run_m == -CUDART_INF_F) ? 0.f : ex2_approx(run_m - nm);
@@ -412,75 +488,66 @@ model_kernel(const __grid_constant__ ModelParams p) {
                 run_m = nm;
             }
         };
-        // end of slot s: this CTA's (max, sum) per row -> global memory, announced on the head's first counter
-        auto publish = [&](int s) -> bool {
-            tmem_st_wait();
-            rec[(grp * 2 + 0) * 128 + row] = active ? run_m : -CUDART_INF_F;
-            rec[(grp * 2 + 1) * 128 + row] = active ? run_l : 0.f;
+        // end of slot s: this group's (max, sum) per row -> shared memory; the statistics warp merges the four
+        // groups, stores the CTA's record and announces it (no block-wide barrier on the scoring warps' path)
+        auto publish = [&](int s) {
+            float* rc = rec + (s & 1) * 3584;
+            rc[(grp * 2 + 0) * 128 + row] = active ? run_m : -CUDART_INF_F;
+            rc[(grp * 2 + 1) * 128 + row] = active ? run_l : 0.f;
             run_m = -CUDART_INF_F;
             run_l = 0.f;
-            named_barrier(kBarEpi, kMEpiThreads);
-            if (ctl.abort_flag) return false;            // same answer in every epilogue thread
-            if (et < 128) {
-                float M = -CUDART_INF_F, Ls = 0.f;
-#pragma unroll
-                for (int g = 0; g < 4; ++g) merge_ml(M, Ls, rec[(g * 2) * 128 + et], rec[(g * 2 + 1) * 128 + et]);
-                float* dst = p.cta_stat + (static_cast<size_t>(s & 1) * gridDim.x + blockIdx.x) * 256;
-                dst[et] = M;
-                dst[128 + et] = Ls;
-            }
-            // the statistics warp announces the record once every epilogue warp has got here: no block-wide
-            // barrier and no memory fence on the scoring warps' path
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl.pub_done[s & 1]));
-            return true;
         };
-        // chunk scores of slot s from the partial sums in the rings (see layer_resident.cu)
+        // Chunk scores of slot s from the partial sums in the rings. A group contracts the panels it
+        // scored itself - every thread reads back the tensor-memory columns and panel maxima it wrote -
+        // so the only synchronisation is among the group's four warps (the four lane quarters of a sum).
         auto contract = [&](int s) -> bool {
-            const int pbase = (s * n_pl) % PR;
-            // m_i and 1 / l_i of the head, merged by the statistics warp
+            const int tg0 = s * nt, pbase = (s * n_pl) % PR;
+            // first panel of the slot that this group scored; its others follow every fourth panel
+            const int g1 = 2 * (((grp >> 1) - tg0) & 1) + half;
             bool ready = true;
             if (lane == 0) ready = mbar_wait(smem_u32(&ctl.stat_full[s & 1]), (s >> 1) & 1, abort_flag);
             if (!__shfl_sync(0xffffffffu, ready, 0)) ok = false;   // (the failed wait has raised the abort flag)
-            tc_fence_before();
-            named_barrier(kBarEpi, kMEpiThreads);        // every partial sum of the slot has been stored
-            tc_fence_after();
-            if (ctl.abort_flag) return false;            // same answer in every epilogue thread
+            tmem_st_wait();
+            // the group's previous sums have been read by all its warps; and a uniform decision to go on
+            if (named_barrier_or(kBarGroup + grp, 128, !ok || ctl.abort_flag != 0)) return false;
             const float* gm = gstat + (s & 1) * 256;
             const float mi = gm[row], li = gm[128 + row];
             constexpr int PPB = 30 / SPP;
-            for (int b0 = 0; grp + 4 * b0 < n_pl; b0 += PPB) {
+            for (int b0 = 0; g1 + 4 * b0 < n_pl; b0 += PPB) {
                 float v[32];
                 int slot_of[PPB];
 #pragma unroll
                 for (int u = 0; u < PPB; ++u) {
-                    const int pl = min(grp + 4 * (b0 + u), n_pl - 1);
+                    const int pl = min(g1 + 4 * (b0 + u), n_pl - 1);
                     int slot = pbase + pl;
                     slot -= (slot >= PR) ? PR : 0;
                     slot_of[u] = slot;
-                    part_load<SPP>(lane_addr + static_cast<uint32_t>(kRPartCol0 + slot * SPP), &v[u * SPP]);
+                    part_load<SPP>(lane_addr + static_cast<uint32_t>(kMPartCol0 + slot * SPP), &v[u * SPP]);
                 }
                 tmem_ld_wait();
                 v[30] = 0.f;
                 v[31] = 0.f;
 #pragma unroll
                 for (int u = 0; u < PPB; ++u) {
-                    const int pl = grp + 4 * (b0 + u);
+                    const int pl = g1 + 4 * (b0 + u);
                     const bool have = active && pl < n_pl;
                     const float f = have ? ex2_approx(pmax[slot_of[u] * 128 + row] - mi) * li : 0.f;
 #pragma unroll
                     for (int q = 0; q < SPP; ++q) v[u * SPP + q] = have ? v[u * SPP + q] * f : 0.f;
                 }
                 const float tot = warp_transpose_reduce(v, lane);
-                const int pl = grp + 4 * (b0 + lane / SPP);
+                const int pl = g1 + 4 * (b0 + lane / SPP);
                 if (lane < 30 && pl < n_pl) red[quarter * 256 + pl * SPP + lane % SPP] = tot;
             }
-            tc_fence_before();
-            named_barrier(kBarEpi, kMEpiThreads);
-            tc_fence_after();
+            named_barrier(kBarGroup + grp, 128);
             float* sc_out = p.scores + (static_cast<size_t>(s) * p.Hs + hs) * p.Cpad;
-            for (int lc = et; lc < n_local; lc += kMEpiThreads)
+            const int n_own = (n_pl - g1 + 3) / 4 * SPP;     // chunk slots of this group's panels
+            for (int i = gt; i < n_own; i += 128) {
+                const int lc = (g1 + 4 * (i / SPP)) * SPP + i % SPP;
                 if (ch0 + lc < p.C) sc_out[ch0 + lc] = (red[lc] + red[256 + lc]) + (red[512 + lc] + red[768 + lc]);
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl.sc_done[s & 1]));      // announced by the statistics warp
             return true;
@@ -490,7 +557,7 @@ model_kernel(const __grid_constant__ ModelParams p) {
             if (s > 0 && !contract(s - 1)) break;
             if (s < p.n_compute) {
                 do_tiles(s, ahead, nt);
-                if (!publish(s)) break;
+                publish(s);
             }
         }
         if (!ok && lane == 0) ctl.abort_flag = 1;
@@ -501,42 +568,46 @@ model_kernel(const __grid_constant__ ModelParams p) {
         // per copy), merge them into m_i and 1 / l_i - four rows per lane - and hand the result to
         // the epilogue.
         const int r0 = 4 * lane;
-        const float* recbuf = reinterpret_cast<const float*>(dyn + p.off_tail + p.off_rec);
-        uint32_t rc = 0;                                  // record copies completed so far
         bool ok = true;
         for (int s = 0; s < p.n_compute && ok; ++s) {
             bool w_ok = true;
-            if (lane == 0) {
-                // this CTA's record is complete (all epilogue warps arrived): announce it. release: the
-                // record stores, ordered before by the mbarrier, are visible to whoever sees the count
+            if (lane == 0)
                 w_ok = mbar_wait(smem_u32(&ctl.pub_done[s & 1]), static_cast<uint32_t>(s >> 1) & 1u, abort_flag);
-                if (w_ok) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt_a + hs) : "memory");
-                if (w_ok) w_ok = wait_counter(p.cnt_a + hs, static_cast<unsigned>(s + 1) * p.cph, abort_flag, 0);
-                asm volatile("fence.acq_rel.gpu;" ::: "memory");
-            }
             if (!__shfl_sync(0xffffffffu, w_ok, 0)) break;
+            {
+                // every epilogue warp has left its group's (max, sum) per row in shared memory: merge the
+                // four groups (this lane: rows 4 lane .. 4 lane + 3), store the CTA's record and announce it.
+                // release: the record stores of the whole warp, ordered by __syncwarp, are visible to whoever
+                // sees the count
+                const float* rc = rec + (s & 1) * 3584;
+                float Mo[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F}, So[4] = {0.f, 0.f, 0.f, 0.f};
+                float4 m[4], l[4];
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    m[g] = *reinterpret_cast<const float4*>(rc + (g * 2) * 128 + r0);
+                    l[g] = *reinterpret_cast<const float4*>(rc + (g * 2 + 1) * 128 + r0);
+                }
+                merge_batch<4>(Mo, So, m, l, 4);
+                float* dst = p.cta_stat + (static_cast<size_t>(s & 1) * gridDim.x + blockIdx.x) * 256;
+                *reinterpret_cast<float4*>(dst + r0) = make_float4(Mo[0], Mo[1], Mo[2], Mo[3]);
+                *reinterpret_cast<float4*>(dst + 128 + r0) = make_float4(So[0], So[1], So[2], So[3]);
+                __syncwarp();
+            }
+            if (lane == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.cnt_a + hs) : "memory");
+            if (!wait_counter_warp(p.cnt_a + hs, static_cast<unsigned>(s + 1) * p.cph, abort_flag)) break;
             const float* src = p.cta_stat + (static_cast<size_t>(s & 1) * gridDim.x + static_cast<size_t>(hs) * p.cph) * 256;
             float M[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F}, S[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int j0 = 0; j0 < p.cph; j0 += kMRecBatch, ++rc) {
-                const int n = min(kMRecBatch, p.cph - j0);
-                if (lane == 0) {
-                    const uint32_t bar = smem_u32(&ctl.rfull);
-                    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(n) * 1024u);
-                    // the records were written with ordinary stores by other CTAs
-                    asm volatile("fence.proxy.async.global;" ::: "memory");
-                    bulk_load(smem_u32(recbuf), src + static_cast<size_t>(j0) * 256, static_cast<uint32_t>(n) * 1024u, bar);
+            // the head's records straight from the L2 (they were written by other SMs; every lane has
+            // acquired the counter), six CTAs' worth of loads in flight per lane
+            for (int j0 = 0; j0 < p.cph; j0 += 6) {
+                float4 m[6], l[6];
+#pragma unroll
+                for (int j = 0; j < 6; ++j) {
+                    const int jj = min(j0 + j, p.cph - 1);
+                    m[j] = __ldcg(reinterpret_cast<const float4*>(src + static_cast<size_t>(jj) * 256 + r0));
+                    l[j] = __ldcg(reinterpret_cast<const float4*>(src + static_cast<size_t>(jj) * 256 + 128 + r0));
                 }
-                if (!mbar_wait(smem_u32(&ctl.rfull), rc & 1u, abort_flag)) { ok = false; break; }
-#pragma unroll 2
-                for (int j = 0; j < n; ++j) {
-                    const float4 m = *reinterpret_cast<const float4*>(recbuf + j * 256 + r0);
-                    const float4 l = *reinterpret_cast<const float4*>(recbuf + j * 256 + 128 + r0);
-                    merge_ml(M[0], S[0], m.x, l.x);
-                    merge_ml(M[1], S[1], m.y, l.y);
-                    merge_ml(M[2], S[2], m.z, l.z);
-                    merge_ml(M[3], S[3], m.w, l.w);
-                }
-                __syncwarp();                             // the buffer may be overwritten by the next copy
+                merge_batch<6>(M, S, m, l, p.cph - j0);
             }
             if (!ok) break;
             float* gm = gstat + (s & 1) * 256;
@@ -692,14 +763,15 @@ bool make_model_plan(int L, int Rs, int Hs, int kv_shift, int d, int c, int C, i
     p.grid = p.n_score + p.n_sel;
     p.n_tiles = (L + kRTile - 1) / kRTile;
     p.t_max = (p.n_tiles + p.cph - 1) / p.cph;
-    if (p.t_max * (kRTile / c) > 252) return false;          // a layer's chunk slots must fit the 252-column ring
+    const int ring_panels = c == 10 ? kMRingPanels10 : kMRingPanels20;
+    // a layer's chunk scores are summed in a 4 x 256-float buffer, its panels must fit the rings
+    if (p.t_max * (kRTile / c) > 252 || 2 * p.t_max > ring_panels) return false;
     const int KB = d / 64;
     const int q_bytes = KB * kRQTileBytes;
-    const int pmax_bytes = (252 / (kRPanel / c)) * 128 * 4;  // the panel-maxima ring: one row set per ring panel
+    const int pmax_bytes = ring_panels * 128 * 4;            // the panel-maxima ring: one row set per ring panel
     p.stage_slot_bytes = 2 * c * d * 2;                        // K rows and V rows of one chunk
     p.sel_row_bytes = ((4 + kk) * 4 + 127) & ~127;
-    p.off_rec = p.sel_row_bytes + kMSlots * p.stage_slot_bytes;
-    const int tail_bytes = p.off_rec + kMRecBytes + 128;
+    const int tail_bytes = p.sel_row_bytes + kMSlots * p.stage_slot_bytes + 128;
     const int fixed = 1024 + q_bytes + 1024 + pmax_bytes + kMMiscBytes + tail_bytes;
     int ns = (smem_limit - 512 - fixed) / kRStageBytes;           // (the control block is larger than the layer kernel's)
     if (ns > kRMaxStages) ns = kRMaxStages;
@@ -757,7 +829,6 @@ cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtenso
     p.sel_row_bytes = plan.sel_row_bytes; p.sel_keys_fit = plan.sel_keys_fit;
     p.off_ring = plan.off_ring; p.off_pmax = plan.off_pmax; p.off_misc = plan.off_misc; p.off_tail = plan.off_tail;
     p.stage_slot_bytes = plan.stage_slot_bytes;
-    p.off_rec = plan.off_rec;
     p.cta_stat = io.scratch;
     p.scores = io.scratch + static_cast<size_t>(2) * plan.grid * 256;
     p.sel_rows = reinterpret_cast<int*>(p.scores + static_cast<size_t>(n_compute) * io.Hs * p.Cpad);   // 16-byte aligned: Cpad % 4 == 0

@@ -97,15 +97,28 @@ __device__ __forceinline__ void panel_static_tail(const float (&v)[WP], float sl
                                                   int last_visible, float* out_m, float* out_l) {
     const int n_vis = last_visible - j0 + 1;     // columns u < n_vis are visible
     const int n_pre = P - j0;                    // columns u < n_pre belong to the prefix
-    float mx = -CUDART_INF_F;
+    if (n_vis <= 0) {                            // the row sees nothing of this panel (e.g. a panel past L)
 #pragma unroll
-    for (int u = 0; u < WP; ++u) mx = (u < n_vis) ? fmaxf(mx, v[u]) : mx;
+        for (int ch = 0; ch < WP / C; ++ch) emit(ch, 0.f);
+        *out_m = -CUDART_INF_F;
+        *out_l = 0.f;
+        return;
+    }
+    // two independent chains each for the maximum and the row sum
+    float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+#pragma unroll
+    for (int u = 0; u + 1 < WP; u += 2) {
+        mx0 = (u < n_vis) ? fmaxf(mx0, v[u]) : mx0;
+        mx1 = (u + 1 < n_vis) ? fmaxf(mx1, v[u + 1]) : mx1;
+    }
+    if constexpr (WP % 2 == 1) mx0 = (WP - 1 < n_vis) ? fmaxf(mx0, v[WP - 1]) : mx0;
+    const float mx = fmaxf(mx0, mx1);
     const float neg_m2 = (mx == -CUDART_INF_F) ? 0.f : -mx * sl2;
-    float l = 0.f, acc = 0.f;
+    float l0 = 0.f, l1 = 0.f, acc = 0.f;
 #pragma unroll
     for (int u = 0; u < WP; ++u) {
         const float e = (u < n_vis) ? ex2_approx(fmaf(v[u], sl2, neg_m2)) : 0.f;
-        l += e;
+        if (u & 1) l1 += e; else l0 += e;
         const float pe = (u < n_pre) ? e : 0.f;
         acc = (u % C == 0) ? pe : acc + pe;
         if ((u + 1) % C == 0) {
@@ -113,6 +126,7 @@ __device__ __forceinline__ void panel_static_tail(const float (&v)[WP], float sl
             emit((u + 1) / C - 1, ((u + 1 - C) < n_pre) ? acc : 0.f);
         }
     }
+    const float l = l0 + l1;
     *out_m = (mx == -CUDART_INF_F) ? -CUDART_INF_F : mx * sl2;
     *out_l = l;
 }
