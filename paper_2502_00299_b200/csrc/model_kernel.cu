@@ -54,8 +54,12 @@ constexpr int kMAccSlots = 12;                     // (buffer, epilogue group) p
 constexpr int kMAcc1Row = 56;
 constexpr int kMPartCol0 = kMAccBufs * kMAccN;
 constexpr int kMPartCols = 512 - kMPartCol0;
-constexpr int kMRingPanels10 = kMPartCols / 6;     // c = 10: 6 chunk columns per panel
-constexpr int kMRingPanels20 = 84;                 // c = 20: 3 per panel; more would only cost shared memory
+// Ring sizes are multiples of the four epilogue groups: a panel's ring slot is its number (since the
+// start of the launch) modulo the ring size and its group is that number modulo 4, so a ring slot
+// is only ever reused by the group that wrote and contracted its previous contents.
+constexpr int kMRingPanels10 = kMPartCols / 6 / 4 * 4;   // c = 10: 6 chunk columns per panel
+constexpr int kMRingPanels20 = 84;                       // c = 20: 3 per panel; more would only cost shared memory
+static_assert(kMRingPanels10 % 4 == 0 && kMRingPanels20 % 4 == 0 && kMRingPanels20 * 3 <= kMPartCols, "ring sizes");
 constexpr int kBarGroup = 2;                       // named barriers 2 .. 5: the four warps of an epilogue group
 
 struct ModelCtl {
@@ -563,10 +567,10 @@ model_kernel(const __grid_constant__ ModelParams p) {
         if (!ok && lane == 0) ctl.abort_flag = 1;
     } else if (warp == 19) {
         // ------------------------------------------------------------------ statistics warp
-        // Per slot: wait (bounded) until every CTA of the scoring head has published its records,
-        // fetch them with bulk copies (they are contiguous in global memory; up to 24 CTAs' records
-        // per copy), merge them into m_i and 1 / l_i - four rows per lane - and hand the result to
-        // the epilogue.
+        // Per slot: merge the groups' records into the CTA's record, store and announce it, wait (bounded)
+        // until every CTA of the scoring head has done the same, read their records from the L2, merge
+        // them into m_i and 1 / l_i - four rows per lane - and hand the result to the epilogue; then
+        // announce the CTA's chunk scores once the epilogue has stored them.
         const int r0 = 4 * lane;
         bool ok = true;
         for (int s = 0; s < p.n_compute && ok; ++s) {
