@@ -16,7 +16,7 @@ CSRC = os.path.join(PKG_DIR, "csrc")
 BUILD_DIR = os.path.join(PKG_DIR, "_build")
 LIB_PATH = os.path.join(PKG_DIR, "libchunkkv.so")
 INCLUDE_DIR = os.path.join(os.path.dirname(PKG_DIR), "include")
-SOURCES = ("api.cu", "score.cu", "layer_resident.cu", "model_kernel.cu", "token_kernel.cu", "select.cu", "gather.cu", "diagnostics.cu", "score_noalloc.cu")
+SOURCES = ("api.cu", "score.cu", "layer_resident.cu", "model_kernel.cu", "token_kernel.cu", "select.cu", "select_cluster.cu", "gather.cu", "diagnostics.cu", "score_noalloc.cu")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",

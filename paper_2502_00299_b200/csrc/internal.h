@@ -169,6 +169,10 @@ cudaError_t launch_finalize(const ScorePlan& plan, const ScoreArgs& args, int C,
                             int num_sms, cudaStream_t stream);
 
 // tok_cap: at most this many tokens of the kept chunks are emitted (lowest positions first)
+// Selection over a cluster of eight CTAs per head (select_cluster.cu): for heads with thousands of chunks.
+bool select_cluster_applies(int C, int k);
+cudaError_t launch_select_cluster(const float* scores, int L, int Hkv, int w, int c, int C, int k, int n_max,
+                                  int32_t* out_idx, cudaStream_t stream, int tok_cap);
 cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int C, int k, int n_max,
                           int32_t* out_idx, cudaStream_t stream, int tok_cap = 0x7fffffff);
 

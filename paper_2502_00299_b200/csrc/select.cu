@@ -31,6 +31,8 @@ select_kernel(const float* __restrict__ scores, int L, int w, int c, int C, int 
 
 cudaError_t launch_select(const float* scores, int L, int Hkv, int w, int c, int C, int k, int n_max,
                           int32_t* out_idx, cudaStream_t stream, int tok_cap) {
+    // thousands of chunks per head: eight CTAs per head
+    if (select_cluster_applies(C, k)) return launch_select_cluster(scores, L, Hkv, w, c, C, k, n_max, out_idx, stream, tok_cap);
     // a few keys per thread: registers (the fewest that hold every key)
     if (C <= kSelThreads * 4) {
         select_kernel<4><<<Hkv, kSelThreads, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx, 0, tok_cap);

@@ -74,7 +74,8 @@ def test_select_ties_go_to_lower_chunk_ids(ck):
         assert np.array_equal(idx, ora.select(s.astype(np.float64), L, w, c, budget))
 
 
-@pytest.mark.parametrize("L", [9000, 70000])      # keys in shared memory / recomputed from the scores
+# a cluster of eight CTAs per head with 512 / with 1024 threads each; one CTA, keys recomputed from the scores
+@pytest.mark.parametrize("L", [9000, 40000, 70000])
 def test_select_ties_with_many_chunks_per_thread(ck, L):
     w, c, Hkv = 8, 1, 4
     C = ora.num_chunks(L, w, c)
@@ -88,6 +89,25 @@ def test_select_ties_with_many_chunks_per_thread(ck, L):
     for budget in (w + 1, w + 37, w + C // 2, w + C - 1):
         idx = ck.select(torch.from_numpy(s).cuda(), L, w, c, budget).cpu().numpy()
         assert np.array_equal(idx, ora.select(s.astype(np.float64), L, w, c, budget))
+
+
+@pytest.mark.parametrize("L,c", [(50003, 4), (131072, 20), (65536, 10)])
+def test_select_over_a_cluster_with_chunks_of_several_tokens(ck, L, c):
+    # thousands of chunks per head (a cluster of CTAs selects), a clipped last chunk that is kept in
+    # head 0, ties across the slices of the cluster's CTAs, and Algorithm 1's token cap
+    w, Hkv = 64, 3
+    C = ora.num_chunks(L, w, c)
+    rng = np.random.default_rng(L + c)
+    s = rng.random((Hkv, C)).astype(np.float32)
+    s[0, C - 1] = 2.0
+    s[1] = rng.integers(0, 4, size=C).astype(np.float32)
+    s[2, :: C // 9] = 0.5
+    for budget in (w + c * 3, w + c * (C // 10), w + c * (C - 2)):
+        idx = ck.select(torch.from_numpy(s).cuda(), L, w, c, budget).cpu().numpy()
+        assert np.array_equal(idx, ora.select(s.astype(np.float64), L, w, c, budget))
+    budget = w + c * (C // 7) + 3
+    idx = ck.select_alg1(torch.from_numpy(s).cuda(), L, w, c, budget).cpu().numpy()
+    assert np.array_equal(idx, ora.select_alg1(s.astype(np.float64), L, w, c, budget))
 
 
 # ------------------------------------------------------------------------------ score
