@@ -112,8 +112,10 @@ token_scores_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
             int issued = 0;
             bool ok = true;
             for (int pass = 0; pass < 2 && ok; ++pass) {
-                const int te = t_begin + (pass == 0 ? nt : nt2);
-                for (int t = t_begin; t < te && ok; ++t) {
+                // pass 2 walks the tiles backwards: the keys read last in pass 1 are the ones still in L2
+                const int n_pass = pass == 0 ? nt : nt2;
+                for (int i = 0; i < n_pass && ok; ++i) {
+                    const int t = pass == 0 ? t_begin + i : t_begin + nt2 - 1 - i;
                     for (int kb = 0; kb < KB; ++kb) {
                         ok = mbar_wait(smem_u32(&ctl.empty[st]), st_par, abort_flag);
                         if (!ok) break;
@@ -292,7 +294,7 @@ token_scores_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                 named_barrier(2 + grp, 128);               // the four lane quarters of this panel are in shared memory
                 if (ctl.abort_flag) break;                 // same answer in the four warps of the group
                 const int gt = threadIdx.x - 64 - grp * 128;   // 0 .. 127 within the group
-                const int j = (t_begin + ti) * kRTile + half * kRPanel + gt;
+                const int j = (t_begin + nt2 - 1 - ti) * kRTile + half * kRPanel + gt;      // (pass 2 runs backwards)
                 if (gt < kRPanel && j < a.P) {
                     const float* q0 = qsum + ((grp * 2 + (mine & 1)) * 4) * 64 + gt;
                     out[j] = (q0[0] + q0[64]) + (q0[128] + q0[192]);
