@@ -18,13 +18,12 @@ namespace {
 
 constexpr int kCsCtas = 8;            // CTAs per cluster (the portable maximum)
 constexpr int kCsKpt = 8;             // keys per thread
-constexpr int kCsBinsPerCta = kSelBins / kCsCtas;
+constexpr int kCsCandCap = 512;       // at most this many keys are ranked against each other directly
 
 struct ClusterSel {
-    int hist[kSelBins];
-    uint32_t cand[kSelCandCap];
+    alignas(16) int hist[kSelBins];
+    uint32_t cand[kCsCandCap];
     unsigned long long minmax[kCsCtas];     // written by every CTA of the cluster
-    int slice_tot[kCsCtas];                 // keys in a CTA's 256 bins (all CTAs' histograms added)
     unsigned long long cta_cnt[kCsCtas];    // (#equal << 32 | #above) per CTA
     unsigned long long warp_sums[33];
     int warp_tot[32];
@@ -95,7 +94,6 @@ select_cluster_kernel(const float* __restrict__ scores, int L, int w, int c, int
         if (span == 0u) { thresh = base; need_eq = need; break; }
         const int shift = max(0, 21 - __clz(span));      // (span >> shift) < kSelBins
         if (round > 0) {
-            // every CTA has read this histogram (the cluster barriers of the previous round lie behind)
             for (int i = tid; i < kSelBins; i += kCsThreads) cs.hist[i] = 0;
             __syncthreads();
         }
@@ -105,15 +103,19 @@ select_cluster_kernel(const float* __restrict__ scores, int L, int w, int c, int
             if (c0 + u < c1 && keys[u] >= base && dlt <= span) atomicAdd(&cs.hist[dlt >> shift], 1);
         }
         cluster.sync();
-        // CTA r adds up bins [256 r, 256 r + 256) of the eight histograms; thread t < 256 takes bin
-        // 256 r + 255 - t, so a prefix over the threads counts from the top of the slice
-        int tot = 0;
-        if (tid < kCsBinsPerCta) {
-            const int b = kCsBinsPerCta * r + kCsBinsPerCta - 1 - tid;
+        // every CTA adds up the eight histograms itself (thread t < 512 takes bins 2047 - 4t .. 2044 - 4t,
+        // so a prefix over the threads counts from the top) and finds the bin of the need-th largest
+        // key on its own: same answer everywhere, no further exchange
+        int cnt[4] = {0, 0, 0, 0}, sum = 0;
+        if (tid < kSelBins / 4) {
 #pragma unroll
-            for (int q = 0; q < kCsCtas; ++q) tot += *cluster.map_shared_rank(&cs.hist[b], q);
+            for (int q = 0; q < kCsCtas; ++q) {
+                const int4 v = *reinterpret_cast<const int4*>(cluster.map_shared_rank(&cs.hist[kSelBins - 4 - 4 * tid], q));
+                cnt[0] += v.w; cnt[1] += v.z; cnt[2] += v.y; cnt[3] += v.x;
+            }
+            sum = (cnt[0] + cnt[1]) + (cnt[2] + cnt[3]);
         }
-        int inc = tot;
+        int inc = sum;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
             const int n = __shfl_up_sync(kFull, inc, off);
@@ -122,26 +124,18 @@ select_cluster_kernel(const float* __restrict__ scores, int L, int w, int c, int
         if (lane == 31) cs.warp_tot[warp] = inc;
         __syncthreads();
         int before = 0;
-        for (int wv = 0; wv < warp && wv < kCsBinsPerCta / 32; ++wv) before += cs.warp_tot[wv];
+        for (int wv = 0; wv < warp; ++wv) before += cs.warp_tot[wv];
         inc += before;
-        if (tid == kCsBinsPerCta - 1) {
+        if (tid < kSelBins / 4 && inc - sum < need && need <= inc) {     // exactly one thread of the CTA
+            int above = inc - sum, q = 0, cq = cnt[0];
 #pragma unroll
-            for (int q = 0; q < kCsCtas; ++q) *cluster.map_shared_rank(&cs.slice_tot[r], q) = inc;
+            for (int t = 0; t < 3; ++t)          // (unrolled: cnt stays in registers)
+                if (q == t && above + cnt[t] < need) { above += cnt[t]; q = t + 1; cq = cnt[t + 1]; }
+            cs.bin = static_cast<uint32_t>(kSelBins - 1 - 4 * tid - q);
+            cs.need = need - above;
+            cs.bin_count = cq;
         }
-        cluster.sync();
-        int above = 0;                   // keys in the bins above this CTA's slice
-        for (int q = r + 1; q < kCsCtas; ++q) above += cs.slice_tot[q];
-        if (tid < kCsBinsPerCta && above + inc - tot < need && need <= above + inc) {     // exactly one thread of the cluster
-            const uint32_t b = static_cast<uint32_t>(kCsBinsPerCta * r + kCsBinsPerCta - 1 - tid);
-            const int nd = need - (above + inc - tot);
-#pragma unroll
-            for (int q = 0; q < kCsCtas; ++q) {
-                *cluster.map_shared_rank(&cs.bin, q) = b;
-                *cluster.map_shared_rank(&cs.need, q) = nd;
-                *cluster.map_shared_rank(&cs.bin_count, q) = tot;
-            }
-        }
-        cluster.sync();
+        __syncthreads();
         const uint32_t bin = cs.bin;
         const int n_bin = cs.bin_count;
         need = cs.need;
@@ -149,29 +143,43 @@ select_cluster_kernel(const float* __restrict__ scores, int L, int w, int c, int
         const uint32_t width = (shift >= 32) ? 0xffffffffu : ((1u << shift) - 1u);
         base += sub;
         span = min(width, span - sub);
-        if (n_bin <= kSelCandCap) {
-            // few keys left: gather them in CTA 0, then every CTA ranks its own copy of them
-            ClusterSel* lead = cluster.map_shared_rank(&cs, 0);
+        if (n_bin <= kCsCandCap) {
+            // few keys left: every CTA gets a copy of all of them (positions handed out by a counter in
+            // CTA 0)
+            int* lead_count = cluster.map_shared_rank(&cs.n_cand, 0);
 #pragma unroll
             for (int u = 0; u < kCsKpt; ++u) {
                 const uint32_t dlt = keys[u] - base;
-                if (c0 + u < c1 && keys[u] >= base && dlt <= span) lead->cand[atomicAdd(&lead->n_cand, 1)] = keys[u];
+                if (c0 + u < c1 && keys[u] >= base && dlt <= span) {
+                    const int pos = atomicAdd(lead_count, 1);
+#pragma unroll
+                    for (int q = 0; q < kCsCtas; ++q) *cluster.map_shared_rank(&cs.cand[pos], q) = keys[u];
+                }
             }
             cluster.sync();
-            if (r != 0)
-                for (int j = tid; j < n_bin; j += kCsThreads) cs.cand[j] = lead->cand[j];
-            __syncthreads();
-            for (int j = tid; j < n_bin; j += kCsThreads) {
+            // the CTAs share the candidates out; a warp per candidate, its lanes striding over the others.
+            // The warp that holds the need-th largest tells every CTA.
+            for (int j = r + kCsCtas * warp; j < n_bin; j += kCsCtas * nwarps) {
                 const uint32_t v = cs.cand[j];
                 int gt = 0, ge = 0;
-                for (int i = 0; i < n_bin; ++i) { gt += cs.cand[i] > v; ge += cs.cand[i] >= v; }
-                if (gt < need && need <= ge) { cs.thresh = v; cs.need_eq = need - gt; }   // same values from every writer
+                for (int i = lane; i < n_bin; i += 32) {
+                    const uint32_t x = cs.cand[i];
+                    gt += x > v;
+                    ge += x >= v;
+                }
+                gt = __reduce_add_sync(kFull, gt);
+                ge = __reduce_add_sync(kFull, ge);
+                if (lane < kCsCtas && gt < need && need <= ge) {       // (same values from every writer)
+                    *cluster.map_shared_rank(&cs.thresh, lane) = v;
+                    *cluster.map_shared_rank(&cs.need_eq, lane) = need - gt;
+                }
             }
-            __syncthreads();
+            cluster.sync();
             thresh = cs.thresh;
             need_eq = cs.need_eq;
             break;
         }
+        cluster.sync();      // another round: every CTA has read this histogram before it is cleared
     }
 
     // ---- ordered sweep over the chunk ids
