@@ -40,6 +40,9 @@ LAYERS_PER_STEP = 32
 SHARED_SETS = 4
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes per layer of the persistent kernel, from the ncu capture summarised under profiles/ (4 layers, cfg2)
+NCU_DRAM_BYTES_PER_LAYER = 337.7e6 / 4
+NCU_TRAFFIC_WORKLOAD = "cfg2_llama3_8b_32k"
 FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 
 
@@ -406,8 +409,12 @@ def run_ours(args, wl):
         "kernel": "model_kernel<10>: the persistent kernel behind chunkkv_compress_model - 32 layers per launch; "
                   "scoring (TMA + tcgen05), chunk sums in tensor memory, top-k on selector CTAs, row copies by bulk copy",
         "bound": "hbm", "achieved": achieved, "peak": peak, "peak_source": peak_src, "unit": "GB/s",
-        "frac": achieved / peak, "frac_of_8TBps": achieved / NOMINAL_HBM_GBS, "traffic": None,
-        "traffic_note": "not captured for the 32-layer launch (ncu's size rule); see profiles/ for the layer kernel's DRAM counters",
+        "frac": achieved / peak, "frac_of_8TBps": achieved / NOMINAL_HBM_GBS,
+        "traffic": NCU_DRAM_BYTES_PER_LAYER * NL if wl.name == NCU_TRAFFIC_WORKLOAD else None,
+        "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one 4-layer launch of the same kernel on this "
+                          "workload (profiles/model_kernel_cfg2_4layers_ncu.txt: 337.7 MB), per layer x the 32 layers of a "
+                          "launch: every layer streams its own K once, so the traffic grows with the layers; the 32-layer "
+                          "launch itself is too large for a counter capture",
         "algorithmic_bytes_per_launch": nbytes["layer"] * NL, "avg_launch_us": ms_per_step * 1e3,
         "launches_per_step": 1, "layers_per_launch": NL,
         "isolated_launch_us": iso_us,
