@@ -17,6 +17,10 @@ __global__ void __launch_bounds__(THREADS)
 gather_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, const int32_t* __restrict__ idx,
               int L, int n_max, uint4* __restrict__ out_K, uint4* __restrict__ out_V,
               int32_t* __restrict__ idx_copy) {
+    // launched as a programmatic dependent of the preceding kernel: let the next kernel's CTAs be
+    // scheduled as this one's retire, and touch no global memory before the predecessor is complete
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int h = blockIdx.y;
     const uint4* Kh = K + static_cast<size_t>(h) * L * VPR;
     const uint4* Vh = V + static_cast<size_t>(h) * L * VPR;
@@ -146,16 +150,21 @@ static cudaError_t launch_gather_t(const void* K, const void* V, const int32_t* 
     const int cap = (max_blocks + Hkv - 1) / Hkv;
     if (bx > cap) bx = cap;
     if (bx < 1) bx = 1;
-    dim3 grid(bx, Hkv);
-    if (vpr == 16)
-        gather_kernel<16, THREADS><<<grid, THREADS, 0, stream>>>(
-            static_cast<const uint4*>(K), static_cast<const uint4*>(V), idx, L, n_max,
-            static_cast<uint4*>(out_K), static_cast<uint4*>(out_V), idx_copy_or_null);
-    else
-        gather_kernel<8, THREADS><<<grid, THREADS, 0, stream>>>(
-            static_cast<const uint4*>(K), static_cast<const uint4*>(V), idx, L, n_max,
-            static_cast<uint4*>(out_K), static_cast<uint4*>(out_V), idx_copy_or_null);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(bx, Hkv);
+    cfg.blockDim = dim3(THREADS);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint4* Kp = static_cast<const uint4*>(K);
+    const uint4* Vp = static_cast<const uint4*>(V);
+    uint4* oK = static_cast<uint4*>(out_K);
+    uint4* oV = static_cast<uint4*>(out_V);
+    if (vpr == 16) return cudaLaunchKernelEx(&cfg, gather_kernel<16, THREADS>, Kp, Vp, idx, L, n_max, oK, oV, idx_copy_or_null);
+    return cudaLaunchKernelEx(&cfg, gather_kernel<8, THREADS>, Kp, Vp, idx, L, n_max, oK, oV, idx_copy_or_null);
 }
 
 cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d,

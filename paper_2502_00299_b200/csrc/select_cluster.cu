@@ -43,6 +43,9 @@ select_cluster_kernel(const float* __restrict__ scores, int L, int w, int c, int
                       int32_t* __restrict__ out_idx, int tok_cap) {
     constexpr unsigned kFull = 0xffffffffu;
     __shared__ ClusterSel cs;
+    // (launched as a programmatic dependent of the kernel that wrote the scores)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     cg::cluster_group cluster = cg::this_cluster();
     const int r = static_cast<int>(cluster.block_rank());
     const int h = blockIdx.x / kCsCtas;
@@ -249,11 +252,18 @@ bool select_cluster_applies(int C, int k) {
 
 cudaError_t launch_select_cluster(const float* scores, int L, int Hkv, int w, int c, int C, int k, int n_max,
                                   int32_t* out_idx, cudaStream_t stream, int tok_cap) {
-    if (C <= kCsCtas * 512 * kCsKpt)
-        select_cluster_kernel<512><<<Hkv * kCsCtas, 512, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx, tok_cap);
-    else
-        select_cluster_kernel<1024><<<Hkv * kCsCtas, 1024, 0, stream>>>(scores, L, w, c, C, k, n_max, out_idx, tok_cap);
-    return cudaGetLastError();
+    const bool small = C <= kCsCtas * 512 * kCsKpt;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(Hkv * kCsCtas);
+    cfg.blockDim = dim3(small ? 512 : 1024);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (small) return cudaLaunchKernelEx(&cfg, select_cluster_kernel<512>, scores, L, w, c, C, k, n_max, out_idx, tok_cap);
+    return cudaLaunchKernelEx(&cfg, select_cluster_kernel<1024>, scores, L, w, c, C, k, n_max, out_idx, tok_cap);
 }
 
 }  // namespace chunkkv

@@ -97,6 +97,8 @@ token_scores_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
+    // the selection that follows is a programmatic dependent: its CTAs may be scheduled as this grid's retire
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: the key range, twice
