@@ -238,6 +238,17 @@ def test_compress_layer_config2_full_size(ck):
         assert set(x.planted.tolist()) <= set(got.tolist()) and 0 in got   # planted + sink chunk
 
 
+@pytest.mark.parametrize("cfg,L", [(2, 32768), (1, 65536)])
+def test_token_level_layer_full_size(ck, cfg, L):
+    # c = 1 at the benchmark's shape (two passes over the keys; selection of 3244 of 32736 tokens by
+    # a cluster of eight 512-thread CTAs per head, 32 tokens short of what it holds) and on a
+    # 64K-token sequence (1024-thread CTAs), whole layer against the oracle
+    wl = scaled(CONFIGS[cfg], L=L, c=1, budget=CONFIGS[cfg].w + L // 10)
+    x = make_layer(wl)
+    oK, oV, idx = _run_layer(ck, x, wl)
+    _check_layer(x, wl, oK, oV, idx)
+
+
 def test_reuse_layers_config3_scaled(ck):
     wl = scaled(CONFIGS[3], L=3000, budget=300, n_layers=5)
     layers = list(iter_layers(wl))
