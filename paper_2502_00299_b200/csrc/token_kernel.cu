@@ -97,8 +97,10 @@ token_scores_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
-    // the selection that follows is a programmatic dependent: its CTAs may be scheduled as this grid's retire
+    // the selection that follows is a programmatic dependent: its CTAs may be scheduled as this grid's retire;
+    // this grid itself touches no global memory before its predecessor is complete
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer: the key range, twice
@@ -260,11 +262,11 @@ token_scores_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
 #pragma unroll
                 for (int q = 0; q < 4; ++q) merge_ml(M2, L2, slice[(q * 2) * 128 + et], slice[(q * 2 + 1) * 128 + et]);
                 gm[et] = M2;
-                ginv[et] = 1.0f / L2;
+                ginv[et] = log2f(L2);          // the normaliser goes into the exponent: exp2(s - m_i - log2 l_i)
             }
             named_barrier(1, 512);
             // ---- pass 2: the same tiles again, normalised, summed over the rows
-            const float mi = gm[row], li = active ? ginv[row] : 0.f;
+            const float nm = active ? -(gm[row] + ginv[row]) : 0.f;
             float* out = a.token_scores + static_cast<size_t>(hs) * a.P;
             int mine = 0;                                  // tiles this group has taken in pass 2 (column-sum buffer = mine & 1)
             for (int ti = (pair - (nt & 1)) & 1; ti < nt2; ti += 2, ++mine) {
@@ -280,13 +282,12 @@ token_scores_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_const
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(smem_u32(&ctl.tempty[pair]));
-                    const float nm = -mi;
 #pragma unroll
                     for (int b = 0; b < 2; ++b) {
                         float x[32];
 #pragma unroll
                         for (int u = 0; u < 30; ++u)      // (an inactive row holds garbage: select, do not multiply)
-                            x[u] = active ? ex2_approx(fmaf(v[b * 30 + u], a.sl2, nm)) * li : 0.f;
+                            x[u] = active ? ex2_approx(fmaf(v[b * 30 + u], a.sl2, nm)) : 0.f;
                         x[30] = 0.f;
                         x[31] = 0.f;
                         const float tot = warp_transpose_reduce(x, lane);
@@ -370,9 +371,21 @@ cudaError_t launch_token_scores(const TokenPlan& plan, const CUtensorMap& tm_q, 
         if (dev >= 0 && dev < 64) smem_set[dev] = plan.smem_bytes;
     }
     void* params[] = {const_cast<CUtensorMap*>(&tm_q), const_cast<CUtensorMap*>(&tm_k), &a};
-    // the CTAs of a head wait for one another: all must be resident
-    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(token_scores_kernel), dim3(plan.grid), dim3(kTThreads),
-                                       params, static_cast<size_t>(plan.smem_bytes), stream);
+    // The CTAs of a head wait for one another, so all must be resident: the plan allows at most one CTA
+    // per SM (its shared memory) and no more CTAs than SMs, and this path is only taken with the whole
+    // GPU, so every CTA becomes resident without waiting for another CTA of this grid. Launched as a
+    // programmatic dependent of the preceding kernel, the set-up of this one overlaps the end of that one.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan.grid);
+    cfg.blockDim = dim3(kTThreads);
+    cfg.dynamicSmemBytes = static_cast<size_t>(plan.smem_bytes);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(token_scores_kernel), params);
 }
 
 }  // namespace chunkkv
