@@ -589,6 +589,7 @@ static int compress_impl(const void* q_obs, const void* K, const void* V, int L,
             io.chunk_scores = payload;
             io.C = C; io.k = k; io.n_max = n_max; io.Hkv_out = Hkv;
             io.bar_count = reinterpret_cast<unsigned long long*>(base + 64);
+            io.cooperative = lane != nullptr;
             {
                 Timer t(ctx, s, 0);
                 e = launch_layer_fused(plan, tm_q, tm_k, a, io, s);

@@ -71,6 +71,7 @@ struct FusedLayerIO {
     int C, k, n_max;
     int Hkv_out;           // KV heads (selection and gather), = scoring heads >> kv_shift
     unsigned long long* bar_count;   // grid barrier ticket counter in the scratch header
+    bool cooperative = true;         // lanes: cooperative launch; the whole GPU: programmatic dependent launch
 };
 
 // The whole layer in one cooperative launch (plan made with full_grid = true, C > 0, k > 0).

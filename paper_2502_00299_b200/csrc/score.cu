@@ -399,6 +399,7 @@ struct LayerArgs {
     int C, k, n_max;
     int Hkv_out;           // KV heads: selection and gather (scoring heads >> kv_shift)
     unsigned long long* bar_count;   // grid barrier counter (zero between launches); its exit counter 64 bytes on
+    int cooperative;                 // host side only: which kind of launch
 };
 
 // Grid-wide barrier for a cooperative launch (all CTAs co-resident). One 64-bit counter that
@@ -529,6 +530,10 @@ score_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl.tmem_base;
+    // (as a programmatic dependent: dependents may be scheduled as this grid retires; no global memory
+    // is touched before the predecessor is complete. Both are no-ops in any other launch.)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
@@ -998,8 +1003,23 @@ cudaError_t launch_variant(const ScorePlan& plan, const CUtensorMap& tm_q, const
         // together, which measured 9 % faster with 18 layers in flight than an ordinary launch.
         void* params[] = {const_cast<CUtensorMap*>(&tm_q), const_cast<CUtensorMap*>(&tm_k),
                           const_cast<ScoreArgs*>(&args), &g, const_cast<LayerArgs*>(&la)};
-        return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kern), dim3(plan.grid), dim3(kThreads),
-                                           params, static_cast<size_t>(plan.smem_bytes), stream);
+        if (la.cooperative)
+            return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(kern), dim3(plan.grid), dim3(kThreads),
+                                               params, static_cast<size_t>(plan.smem_bytes), stream);
+        // With the whole GPU to itself (no lanes) every CTA becomes resident anyway - at most one per SM, no
+        // more CTAs than SMs - and the kernel is launched as a programmatic dependent of its predecessor
+        // instead: its set-up overlaps the end of that one.
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(plan.grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = static_cast<size_t>(plan.smem_bytes);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelExC(&cfg, reinterpret_cast<const void*>(kern), params);
     } else {
         kern<<<plan.grid, kThreads, plan.smem_bytes, stream>>>(tm_q, tm_k, args, g, la);
         return cudaGetLastError();
@@ -1095,6 +1115,7 @@ cudaError_t launch_layer_fused(const ScorePlan& plan, const CUtensorMap& tm_q, c
     la.n_max = io.n_max;
     la.Hkv_out = io.Hkv_out;
     la.bar_count = io.bar_count;
+    la.cooperative = io.cooperative ? 1 : 0;
     return dispatch_variant<true>(plan, tm_q, tm_k, args, la, stream);
 }
 
