@@ -39,10 +39,8 @@ namespace {
 
 constexpr int kMThreads = 640;          // warp 0: TMA, warp 1: UMMA issue, warps 2..17: epilogue, warp 18: row copies, warp 19: row statistics
                                         // (five warps per scheduler: a sixth would cut every thread to 80 registers)
-constexpr int kMEpiThreads = 512;
 constexpr int kMMiscBytes = 18432;      // epilogue: group records (two slots), m_i, 1 / l_i, row sums per lane quarter
 constexpr int kMSlots = 8;              // staging slots of the row copies
-constexpr int kBarEpi = 1;
 // Tensor memory: three 64-column accumulators (one 60-key panel of a tile each, in rotation; the
 // second panel of a tile is computed on keys 56 .. 119 so that its operand starts on a swizzle-atom
 // boundary, and begins at column 4), and 320 columns of chunk partial sums: a ring that holds one
@@ -76,7 +74,6 @@ struct ModelCtl {
     unsigned long long sc_done[2];     // every epilogue warp has stored its chunk scores of the slot (-> statistics warp)
     uint32_t tmem_base;
     int abort_flag;
-    int epi_ok;
     int sel_flag[2];                   // selector CTAs: wait result, abort flag
 };
 
@@ -332,7 +329,6 @@ model_kernel(const __grid_constant__ ModelParams p) {
             mbar_init(smem_u32(&ctl.sc_done[b]), 16);
         }
         ctl.abort_flag = 0;
-        ctl.epi_ok = 1;
         fence_mbar_init();
         fence_proxy_async();
     }
