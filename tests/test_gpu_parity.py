@@ -301,6 +301,29 @@ def test_config3_full_size_reuse_depth_2(ck):
     assert 0.0 < float(ratio.min()) <= 1.0
 
 
+def test_model_call_32_computed_layers_at_benchmark_size(ck):
+    # the benchmark's step: 32 distinct 32K-token layers, every one computed, in one persistent launch
+    # (its tensor-memory rings wrap about twenty times). Every layer's rows are checked against its own
+    # inputs, three layers against the oracle, and a second call must reproduce the first bit for bit.
+    from concurrent.futures import ThreadPoolExecutor
+    wl = CONFIGS[2]
+    with ThreadPoolExecutor(8) as ex:
+        layers = list(ex.map(lambda i: make_layer(wl, layer=i), range(32)))
+    dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in layers]
+    outs = ck.compress_model(dev, wl.Hq, wl.w, wl.c, wl.budget, n_reuse=1)
+    _status_ok(ck)
+    first = [(o[0].clone(), o[1].clone(), o[2].clone()) for o in outs]
+    for l, (x, (oK, oV, idx)) in enumerate(zip(layers, outs)):
+        idx_np = idx.cpu().numpy()
+        assert_gather_exact(bits_of(oK), bits_of(oV), idx_np, x.K, x.V)
+        if l in (0, 13, 31):
+            _check_layer(x, wl, bits_of(oK), bits_of(oV), idx_np)
+    again = ck.compress_model(dev, wl.Hq, wl.w, wl.c, wl.budget, n_reuse=1)
+    _status_ok(ck)
+    for a, b in zip(first, again):
+        assert torch.equal(a[2], b[2]) and torch.equal(a[0], b[0]) and torch.equal(a[1], b[1])
+
+
 def test_config5_all_ragged_lengths_one_reuse_group(ck):
     # the batched workload: all eight sequences at their real lengths (8192..65536 tokens, 64 query
     # heads), one reuse group each (depth 3: one computed layer, two gather-only layers)
