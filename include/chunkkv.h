@@ -192,6 +192,14 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
  * chunkkv_compress_layer_paged: chunkkv_compress_layer (or, with reuse_idx, a layer that reuses
  *   indices) writing the kept rows to a paged cache instead of dense out_K / out_V; out_idx
  *   [Hkv, n_max] is still written. Runs as separate score / select / gather launches.
+ *
+ * chunkkv_compress_layer_strided: chunkkv_compress_layer (or, with reuse_idx, a layer that reuses
+ *   indices) on keys and values that are not packed [Hkv, L, d]: row l of head h of K starts at
+ *   element l * k_token_stride + h * k_head_stride of K (likewise V); a token-major prefill cache
+ *   [L, Hkv, d] has token stride Hkv * d and head stride d. Strides are in bf16 elements, multiples
+ *   of 8 and at least d; K and V 16-byte aligned. The outputs are packed as usual. With the packed
+ *   strides (d and L * d) this is chunkkv_compress_layer itself; otherwise separate score / select /
+ *   gather launches. Returns CHUNKKV_EINVAL_SHAPE for other strides.
  */
 CHUNKKV_API int chunkkv_window_queries(const void* qkv, long long row_elems, int T, int Hq, int Hkv, int d, int w,
                                        const float* cos_rows, const float* sin_rows, void* out_q_obs, void* stream);
@@ -202,6 +210,11 @@ CHUNKKV_API int chunkkv_compress_layer_paged(const void* q_obs, const void* K, c
                                              int d, int w, int c, int budget, const int32_t* reuse_idx_or_null,
                                              const int32_t* block_table, int page_size, int num_pages, void* cache_K,
                                              void* cache_V, int32_t* out_idx, void* stream);
+CHUNKKV_API int chunkkv_compress_layer_strided(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv,
+                                               int d, int w, int c, int budget, long long k_token_stride,
+                                               long long k_head_stride, long long v_token_stride,
+                                               long long v_head_stride, const int32_t* reuse_idx_or_null,
+                                               void* out_K, void* out_V, int32_t* out_idx, void* stream);
 
 /*
  * A whole model with layer-wise index reuse (Algorithm 2): layer l computes its indices iff

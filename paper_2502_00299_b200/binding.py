@@ -54,6 +54,8 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_window_queries.argtypes = [vp, ctypes.c_longlong] + [i32] * 5 + [vp, vp, vp, vp]
     L.chunkkv_gather_paged.restype = i32
     L.chunkkv_gather_paged.argtypes = [vp, vp, vp] + [i32] * 4 + [vp, i32, i32, vp, vp, vp]
+    L.chunkkv_compress_layer_strided.restype = i32
+    L.chunkkv_compress_layer_strided.argtypes = [vp, vp, vp] + [i32] * 7 + [ctypes.c_longlong] * 4 + [vp, vp, vp, vp, vp]
     L.chunkkv_compress_layer_paged.restype = i32
     L.chunkkv_compress_layer_paged.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, i32, i32, vp, vp, vp, vp]
     L.chunkkv_compress_layer_host.restype = i32
@@ -323,6 +325,39 @@ def gather_paged(K: torch.Tensor, V: torch.Tensor, idx: torch.Tensor, block_tabl
     _check(lib.chunkkv_gather_paged(K.data_ptr(), V.data_ptr(), idx.data_ptr(), L, Hkv, d, idx.shape[1],
                                     block_table.data_ptr(), cache_K.shape[1], cache_K.shape[0], cache_K.data_ptr(),
                                     cache_V.data_ptr(), _stream(stream)), "chunkkv_gather_paged")
+
+
+def compress_layer_strided(q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tensor, Hq: int, w: int, c: int,
+                           budget: int, reuse_idx: Optional[torch.Tensor] = None,
+                           out_K: Optional[torch.Tensor] = None, out_V: Optional[torch.Tensor] = None,
+                           out_idx: Optional[torch.Tensor] = None,
+                           stream: Optional[torch.cuda.Stream] = None) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """One layer on K / V given as [Hkv, L, d] *views* with arbitrary token and head strides (the last
+    dimension contiguous), e.g. ``cache.permute(1, 0, 2)`` of a token-major cache [L, Hkv, d]. Outputs
+    are packed [Hkv, n_max, d]."""
+    for t, name in ((K, "K"), (V, "V")):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.dim() == 3 and t.stride(2) == 1):
+            raise ValueError(f"{name}: a CUDA bf16 [Hkv, L, d] view with a contiguous last dimension is required")
+    if q_obs is not None:
+        _dev(q_obs, torch.bfloat16, "q_obs")
+    if reuse_idx is not None:
+        _dev(reuse_idx, torch.int32, "reuse_idx")
+    Hkv, L, d = K.shape
+    n_max = out_len(L, w, c, budget)
+    dev = K.device
+    if reuse_idx is None:
+        ensure_workspace(L, Hq, Hkv, d, w, c)
+    if out_K is None:
+        out_K = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
+    if out_V is None:
+        out_V = torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev)
+    if out_idx is None:
+        out_idx = torch.empty((Hkv, n_max), dtype=torch.int32, device=dev)
+    _check(lib.chunkkv_compress_layer_strided(_ptr(q_obs), K.data_ptr(), V.data_ptr(), L, Hq, Hkv, d, w, c, budget,
+                                              K.stride(1), K.stride(0), V.stride(1), V.stride(0), _ptr(reuse_idx),
+                                              out_K.data_ptr(), out_V.data_ptr(), out_idx.data_ptr(), _stream(stream)),
+           "chunkkv_compress_layer_strided")
+    return out_K, out_V, out_idx
 
 
 def compress_layer_paged(q_obs: Optional[torch.Tensor], K: torch.Tensor, V: torch.Tensor, Hq: int, w: int, c: int,

@@ -120,11 +120,14 @@ int check_sizes(int L, int w, int c, int budget) {
     return CHUNKKV_OK;
 }
 
+// row_elems / head_elems: elements between consecutive rows of a head and between heads; 0 = packed [heads, rows, d]
 int encode_bf16_3d(CUtensorMap* tm, const void* base, int d, long long rows, int heads, int box_rows,
-                   CUtensorMapL2promotion promo) {
+                   CUtensorMapL2promotion promo, long long row_elems = 0, long long head_elems = 0) {
     cuuint64_t dims[3] = {static_cast<cuuint64_t>(d), static_cast<cuuint64_t>(rows),
                           static_cast<cuuint64_t>(heads)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(d) * 2, static_cast<cuuint64_t>(rows) * d * 2};
+    if (row_elems == 0) row_elems = d;
+    if (head_elems == 0) head_elems = rows * d;
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(row_elems) * 2, static_cast<cuuint64_t>(head_elems) * 2};
     cuuint32_t box[3] = {64, static_cast<cuuint32_t>(box_rows), 1};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides,
@@ -163,7 +166,7 @@ struct Timer {
 // address used. Caller holds g_mu and has validated the arguments.
 int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, int Hkv, int d, int w,
               int c, float* out_scores, size_t extra_payload_floats, float** resolved,
-              cudaStream_t stream) {
+              cudaStream_t stream, long long k_row_elems = 0, long long k_head_elems = 0) {
     const int P = L - w;
     const int C = (P + c - 1) / c;
     if (C <= 0) return CHUNKKV_OK;
@@ -184,7 +187,7 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
         CUtensorMap tq, tk;
         st2 = encode_bf16_3d(&tq, q_obs, d, R, sh.Hs, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
         if (st2 != CHUNKKV_OK) return st2;
-        st2 = encode_bf16_3d(&tk, K, d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+        st2 = encode_bf16_3d(&tk, K, d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, k_row_elems, k_head_elems);
         if (st2 != CHUNKKV_OK) return st2;
         TokenIO io;
         io.L = L; io.w = w; io.Rs = R; io.Hs = sh.Hs; io.d = d; io.kv_shift = sh.shift;
@@ -220,7 +223,7 @@ int run_score(DeviceCtx& ctx, const void* q_obs, const void* K, int L, int Hq, i
     st = encode_bf16_3d(&tm_q, q_obs, d, R, sh.Hs, R < 128 ? R : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (st != CHUNKKV_OK) return st;
     st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < plan.n_tile ? L : plan.n_tile,
-                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, k_row_elems, k_head_elems);
     if (st != CHUNKKV_OK) return st;
     cudaError_t e;
     {
@@ -632,6 +635,56 @@ int chunkkv_compress_layer(const void* q_obs, const void* K, const void* V, int 
                            void* out_K, void* out_V, int32_t* out_idx, void* stream) {
     return compress_impl(q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_idx, out_K, out_V, out_idx, nullptr, 0, 0,
                          stream);
+}
+
+// The whole layer on keys and values that are not packed [Hkv, L, d]: e.g. a token-major cache [L, Hkv, d]
+// (token stride Hkv * d, head stride d). Scores through tensor maps with those strides, selection, and a
+// gather that reads rows by stride and writes packed outputs: separate launches.
+int chunkkv_compress_layer_strided(const void* q_obs, const void* K, const void* V, int L, int Hq, int Hkv, int d,
+                                   int w, int c, int budget, long long k_token_stride, long long k_head_stride,
+                                   long long v_token_stride, long long v_head_stride, const int32_t* reuse_idx,
+                                   void* out_K, void* out_V, int32_t* out_idx, void* stream) {
+    if (k_token_stride == d && v_token_stride == d && k_head_stride == static_cast<long long>(L) * d &&
+        v_head_stride == static_cast<long long>(L) * d)
+        return chunkkv_compress_layer(q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_idx, out_K, out_V, out_idx, stream);
+    int st = check_heads(L, Hq, Hkv, d, w);
+    if (st != CHUNKKV_OK) return st;
+    st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    if (K == nullptr || V == nullptr || out_K == nullptr || out_V == nullptr || out_idx == nullptr) return CHUNKKV_EINVAL_NULL;
+    if (reuse_idx == nullptr && q_obs == nullptr) return CHUNKKV_EINVAL_NULL;
+    // rows are moved and loaded 16 bytes at a time; a row may not overlap the next one
+    const long long strides[4] = {k_token_stride, k_head_stride, v_token_stride, v_head_stride};
+    for (long long sdv : strides)
+        if (sdv < d || (sdv & 7) != 0) return CHUNKKV_EINVAL_SHAPE;
+    if (!aligned16(q_obs) || !aligned16(K) || !aligned16(V) || !aligned16(out_K) || !aligned16(out_V))
+        return CHUNKKV_EINVAL_ALIGN;
+    const int C = chunkkv_num_chunks(L, w, c);
+    const int k = chunkkv_num_kept_chunks(L, w, c, budget);
+    const int n_max = chunkkv_out_len(L, w, c, budget);
+    if (n_max < 0) return n_max;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    std::lock_guard<std::mutex> lk(g_mu);
+    DeviceCtx* ctx = nullptr;
+    st = get_ctx(&ctx);
+    if (st != CHUNKKV_OK) return st;
+    cudaError_t e;
+    const int32_t* idx = reuse_idx;
+    if (reuse_idx == nullptr) {
+        float* chunk_scores = nullptr;
+        if (C > 0 && k > 0) {
+            st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, round64(static_cast<size_t>(Hkv) * C), &chunk_scores, s,
+                           k_token_stride, k_head_stride);
+            if (st != CHUNKKV_OK) return st;
+        }
+        e = launch_select(chunk_scores, L, Hkv, w, c, C, k, n_max, out_idx, s);
+        if (e != cudaSuccess) return cuda_fail(e);
+        idx = out_idx;
+    }
+    e = launch_gather_strided(K, V, idx, L, Hkv, d, n_max, k_token_stride, k_head_stride, v_token_stride, v_head_stride,
+                              out_K, out_V, idx == out_idx ? nullptr : out_idx, ctx->num_sms, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return CHUNKKV_OK;
 }
 
 // ---- Adapters to the steps either side of the path: window queries out of a fused QKV activation

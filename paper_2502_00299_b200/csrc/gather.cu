@@ -140,6 +140,27 @@ cudaError_t launch_window_queries(const void* qkv, long long row_elems, int T, i
     return cudaGetLastError();
 }
 
+// The same gather from keys and values that are not packed [Hkv, L, d]: source rows are found by a token
+// stride and a head stride (in 16-byte vectors); the outputs are packed.
+template <int VPR>
+__global__ void __launch_bounds__(kGatherThreads)
+gather_strided_kernel(const uint4* __restrict__ K, const uint4* __restrict__ V, const int32_t* __restrict__ idx,
+                      int L, int n_max, long long k_tok, long long k_head, long long v_tok, long long v_head,
+                      uint4* __restrict__ out_K, uint4* __restrict__ out_V, int32_t* __restrict__ idx_copy) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int h = blockIdx.y;
+    const uint4* Kh = K + static_cast<size_t>(h) * k_head;
+    const uint4* Vh = V + static_cast<size_t>(h) * v_head;
+    const int32_t* ih = idx + static_cast<size_t>(h) * n_max;
+    uint4* oK = out_K + static_cast<size_t>(h) * n_max * VPR;
+    uint4* oV = out_V + static_cast<size_t>(h) * n_max * VPR;
+    int32_t* ic = idx_copy ? idx_copy + static_cast<size_t>(h) * n_max : nullptr;
+    const int rows_per_block = (kGatherThreads / VPR) * kGatherRowsPerThread;
+    for (int n0 = blockIdx.x * rows_per_block; n0 < n_max; n0 += gridDim.x * rows_per_block)
+        gather_rows<VPR, false>(Kh, Vh, ih, L, n_max, n0, threadIdx.x, kGatherThreads, oK, oV, ic, k_tok, v_tok);
+}
+
 template <int THREADS>
 static cudaError_t launch_gather_t(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d, int n_max,
                                    void* out_K, void* out_V, int32_t* idx_copy_or_null, int max_blocks,
@@ -173,6 +194,37 @@ cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int 
     if (n_max <= 0 || Hkv <= 0) return cudaSuccess;
     return launch_gather_t<kGatherThreads>(K, V, idx, L, Hkv, d, n_max, out_K, out_V, idx_copy_or_null, 16 * num_sms,
                                            stream);
+}
+
+cudaError_t launch_gather_strided(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d, int n_max,
+                                  long long k_token_stride, long long k_head_stride, long long v_token_stride,
+                                  long long v_head_stride, void* out_K, void* out_V, int32_t* idx_copy_or_null,
+                                  int num_sms, cudaStream_t stream) {
+    if (n_max <= 0 || Hkv <= 0) return cudaSuccess;
+    const int vpr = d / 8;
+    const int rows_per_block = (kGatherThreads / vpr) * kGatherRowsPerThread;
+    int bx = (n_max + rows_per_block - 1) / rows_per_block;
+    const int cap = (16 * num_sms + Hkv - 1) / Hkv;
+    if (bx > cap) bx = cap;
+    if (bx < 1) bx = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(bx, Hkv);
+    cfg.blockDim = dim3(kGatherThreads);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const uint4* Kp = static_cast<const uint4*>(K);
+    const uint4* Vp = static_cast<const uint4*>(V);
+    uint4* oK = static_cast<uint4*>(out_K);
+    uint4* oV = static_cast<uint4*>(out_V);
+    // strides in 16-byte vectors (8 bf16 elements)
+    const long long kt = k_token_stride / 8, kh = k_head_stride / 8, vt = v_token_stride / 8, vh = v_head_stride / 8;
+    if (vpr == 16)
+        return cudaLaunchKernelEx(&cfg, gather_strided_kernel<16>, Kp, Vp, idx, L, n_max, kt, kh, vt, vh, oK, oV, idx_copy_or_null);
+    return cudaLaunchKernelEx(&cfg, gather_strided_kernel<8>, Kp, Vp, idx, L, n_max, kt, kh, vt, vh, oK, oV, idx_copy_or_null);
 }
 
 // The same gather in CTAs of 64 threads spread over the whole GPU: such a CTA fits on an SM

@@ -34,11 +34,13 @@ __device__ __forceinline__ void gather_st(uint4* p, const uint4& v) {
 // Work item `item` of `n_items` (a CTA-sized slab of rows of one head); threads = nthreads
 // (a multiple of VPR). VPR = 16-byte vectors per row: 8 (d = 64) or 16 (d = 128).
 // FRESH_IDX: the indices were written earlier in the same kernel launch, so they must not be
-// read through the non-coherent path.
+// read through the non-coherent path. k_row_vecs / v_row_vecs: 16-byte vectors between consecutive
+// source rows of a head (VPR for packed rows; more for a token-major cache).
 template <int VPR, bool FRESH_IDX>
 __device__ __forceinline__ void gather_rows(const uint4* __restrict__ Kh, const uint4* __restrict__ Vh,
                                             const int32_t* ih, int L, int n_max, int n0, int tid, int nthreads,
-                                            uint4* __restrict__ oK, uint4* __restrict__ oV, int32_t* idx_copy) {
+                                            uint4* __restrict__ oK, uint4* __restrict__ oV, int32_t* idx_copy,
+                                            long long k_row_vecs = VPR, long long v_row_vecs = VPR) {
     const int rows_per_pass = nthreads / VPR;
     const int vec = tid % VPR, sub = tid / VPR;
     const unsigned long long policy = gather_policy();
@@ -53,8 +55,8 @@ __device__ __forceinline__ void gather_rows(const uint4* __restrict__ Kh, const 
 #pragma unroll
     for (int u = 0; u < kGatherRowsPerThread; ++u) {
         const bool ok = static_cast<unsigned>(src[u]) < static_cast<unsigned>(L);
-        kv[u] = ok ? gather_ld(Kh + static_cast<size_t>(src[u]) * VPR + vec, policy) : make_uint4(0, 0, 0, 0);
-        vv[u] = ok ? gather_ld(Vh + static_cast<size_t>(src[u]) * VPR + vec, policy) : make_uint4(0, 0, 0, 0);
+        kv[u] = ok ? gather_ld(Kh + static_cast<size_t>(src[u]) * k_row_vecs + vec, policy) : make_uint4(0, 0, 0, 0);
+        vv[u] = ok ? gather_ld(Vh + static_cast<size_t>(src[u]) * v_row_vecs + vec, policy) : make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
     for (int u = 0; u < kGatherRowsPerThread; ++u) {

@@ -181,6 +181,10 @@ cudaError_t launch_gather(const void* K, const void* V, const int32_t* idx, int 
                           int n_max, void* out_K, void* out_V, int32_t* idx_copy_or_null,
                           int num_sms, cudaStream_t stream);
 // The gather into a paged cache [page, slot, head, d] through a block table (device int32).
+cudaError_t launch_gather_strided(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d, int n_max,
+                                  long long k_token_stride, long long k_head_stride, long long v_token_stride,
+                                  long long v_head_stride, void* out_K, void* out_V, int32_t* idx_copy_or_null,
+                                  int num_sms, cudaStream_t stream);
 cudaError_t launch_gather_paged(const void* K, const void* V, const int32_t* idx, int L, int Hkv, int d, int n_max,
                                 const int32_t* block_table, int page_size, int num_pages, void* cache_K, void* cache_V,
                                 int num_sms, cudaStream_t stream);

@@ -764,3 +764,54 @@ def test_paged_cache_outputs_match_oracle(ck, cfg, L, budget, page):
     ck.gather_paged(to_dev(x0.K), to_dev(x0.V), idx, torch.from_numpy(bad).cuda(), cK.t, cV.t)
     torch.cuda.synchronize()
     assert np.array_equal(bits_of(cK.t), before)
+
+
+@pytest.mark.parametrize("cfg,L,budget,c,pad", [(2, 4000, 400, 10, 0), (1, 2048, 256, 10, 24), (5, 3000, 300, 10, 0),
+                                               (2, 5000, 532, 1, 8), (4, 9000, 900, 20, 0)])
+def test_token_major_cache_inputs_match_oracle(ck, cfg, L, budget, c, pad):
+    # keys and values handed over as a token-major cache [L, Hkv, d (+ padding)], i.e. [Hkv, L, d] views with
+    # token stride Hkv * (d + pad) and head stride d + pad: same results as on packed inputs (the oracle's),
+    # then a layer that reuses the indices; the packed strides take the ordinary path
+    wl = scaled(CONFIGS[cfg], L=L, budget=budget, c=c)
+    x0, x1 = make_layer(wl, layer=0), make_layer(wl, layer=1)
+
+    def token_major(bits):
+        t = to_dev(bits)                                       # [Hkv, L, d]
+        buf = torch.zeros((L, wl.Hkv, wl.d + pad), dtype=torch.bfloat16, device="cuda")
+        buf[:, :, :wl.d] = t.permute(1, 0, 2)
+        return buf, buf[:, :, :wl.d].permute(1, 0, 2)          # the cache and the [Hkv, L, d] view of it
+
+    bK, vK = token_major(x0.K)
+    bV, vV = token_major(x0.V)
+    assert not vK.is_contiguous()
+    gK, gV, gI = guarded_outputs(wl.Hkv, ck.out_len(L, wl.w, c, budget), wl.d)
+    oK, oV, idx = ck.compress_layer_strided(to_dev(x0.q_obs), vK, vV, wl.Hq, wl.w, c, budget,
+                                            out_K=gK.t, out_V=gV.t, out_idx=gI.t)
+    _status_ok(ck)
+    for g, name in ((gK, "out_K"), (gV, "out_V"), (gI, "out_idx")):
+        g.check(name)
+    idx_np = idx.cpu().numpy()
+    _check_layer(x0, wl, bits_of(oK), bits_of(oV), idx_np, budget=budget)
+    b1K, v1K = token_major(x1.K)
+    b1V, v1V = token_major(x1.V)
+    rK, rV, ridx = ck.compress_layer_strided(None, v1K, v1V, wl.Hq, wl.w, c, budget, reuse_idx=idx)
+    assert torch.equal(ridx, idx)
+    assert_gather_exact(bits_of(rK), bits_of(rV), idx_np, x1.K, x1.V)
+    # packed views go to the ordinary layer call
+    dK, dV, didx = ck.compress_layer_strided(to_dev(x0.q_obs), to_dev(x0.K), to_dev(x0.V), wl.Hq, wl.w, c, budget)
+    pK, pV, pidx = ck.compress_layer(to_dev(x0.q_obs), to_dev(x0.K), to_dev(x0.V), wl.Hq, wl.w, c, budget)
+    assert torch.equal(didx, pidx) and torch.equal(dK, pK) and torch.equal(dV, pV)
+
+
+def test_strided_inputs_refused_when_rows_overlap_or_are_misaligned(ck):
+    wl = scaled(CONFIGS[1], L=512, budget=64)
+    x = make_layer(wl)
+    q, K, V = to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)
+    n_max = ck.out_len(512, wl.w, wl.c, 64)
+    oK = torch.empty((wl.Hkv, n_max, wl.d), dtype=torch.bfloat16, device="cuda")
+    oI = torch.empty((wl.Hkv, n_max), dtype=torch.int32, device="cuda")
+    for strides in ((wl.d - 8, 512 * wl.d, wl.d, 512 * wl.d), (wl.d + 4, 512 * (wl.d + 4), wl.d, 512 * wl.d)):
+        st = ck.lib.chunkkv_compress_layer_strided(q.data_ptr(), K.data_ptr(), V.data_ptr(), 512, wl.Hq, wl.Hkv, wl.d, wl.w,
+                                                   wl.c, 64, *strides, None, oK.data_ptr(), oK.data_ptr(), oI.data_ptr(), None)
+        assert st == -2
+
