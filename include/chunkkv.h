@@ -198,8 +198,9 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
  *   element l * k_token_stride + h * k_head_stride of K (likewise V); a token-major prefill cache
  *   [L, Hkv, d] has token stride Hkv * d and head stride d. Strides are in bf16 elements, multiples
  *   of 8 and at least d; K and V 16-byte aligned. The outputs are packed as usual. With the packed
- *   strides (d and L * d) this is chunkkv_compress_layer itself; otherwise separate score / select /
- *   gather launches. Returns CHUNKKV_EINVAL_SHAPE for other strides.
+ *   strides (d and L * d) this is chunkkv_compress_layer itself; otherwise the one-launch layer kernel
+ *   where the shape fits it (chunk sizes 10 and 20, up to 128 score rows per scoring head), else separate
+ *   score / select / gather launches. Returns CHUNKKV_EINVAL_SHAPE for other strides.
  */
 CHUNKKV_API int chunkkv_window_queries(const void* qkv, long long row_elems, int T, int Hq, int Hkv, int d, int w,
                                        const float* cos_rows, const float* sin_rows, void* out_q_obs, void* stream);

@@ -670,6 +670,36 @@ int chunkkv_compress_layer_strided(const void* q_obs, const void* K, const void*
     if (st != CHUNKKV_OK) return st;
     cudaError_t e;
     const int32_t* idx = reuse_idx;
+    if (reuse_idx == nullptr && C > 0 && k > 0) {
+        // the one-launch layer kernel takes strided keys and values as they are (tensor map and gather strides)
+        const ScoreShape sh = score_shape(Hq, Hkv, w);
+        ResidentPlan rplan;
+        if (make_resident_plan(L, sh.Rs, sh.Hs, sh.shift, d, c, C, n_max, ctx->num_sms, smem_budget(*ctx), &rplan)) {
+            st = ensure_workspace(*ctx, resident_scratch_floats(rplan, sh.Hs, C) * sizeof(float));
+            if (st != CHUNKKV_OK) return st;
+            char* base = static_cast<char*>(ctx->ws);
+            CUtensorMap tm_q, tm_k;
+            st = encode_bf16_3d(&tm_q, q_obs, d, sh.Rs, sh.Hs, sh.Rs < 128 ? sh.Rs : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+            if (st != CHUNKKV_OK) return st;
+            st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, k_token_stride,
+                                k_head_stride);
+            if (st != CHUNKKV_OK) return st;
+            ResidentIO io;
+            io.L = L; io.w = w; io.Rs = sh.Rs; io.Hs = sh.Hs; io.d = d; io.kv_shift = sh.shift;
+            io.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
+            io.C = C; io.k = k; io.n_max = n_max;
+            io.K = K; io.V = V; io.out_K = out_K; io.out_V = out_V; io.out_idx = out_idx;
+            io.scratch = reinterpret_cast<float*>(base + kHeaderBytes);
+            io.counters = reinterpret_cast<unsigned*>(base + kResidentCountersOffset);
+            io.status = reinterpret_cast<int*>(base);
+            io.cooperative = false;
+            io.k_row_elems = k_token_stride; io.k_head_elems = k_head_stride;
+            io.v_row_elems = v_token_stride; io.v_head_elems = v_head_stride;
+            e = launch_layer_resident(rplan, tm_q, tm_k, io, s);
+            if (e != cudaSuccess) return cuda_fail(e);
+            return CHUNKKV_OK;
+        }
+    }
     if (reuse_idx == nullptr) {
         float* chunk_scores = nullptr;
         if (C > 0 && k > 0) {

@@ -103,6 +103,8 @@ struct ResidentIO {
     unsigned* counters;   // header + kResidentCountersOffset
     int* status;
     bool cooperative;     // cooperative launch (lanes: several launches share the GPU) instead of a programmatic dependent one
+    // elements between consecutive rows of a head and between heads of K and of V; 0 = packed [Hkv, L, d]
+    long long k_row_elems = 0, k_head_elems = 0, v_row_elems = 0, v_head_elems = 0;
 };
 
 // false when the shape does not fit this kernel (chunk size other than 10 / 20, more than 128 rows

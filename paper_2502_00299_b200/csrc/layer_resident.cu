@@ -61,6 +61,7 @@ struct ResArgs {
     int off_ring, ring_bytes, off_pmax, off_misc;   // dynamic shared memory layout (bytes from the aligned base)
     const uint4* K;
     const uint4* V;
+    long long k_row, k_head, v_row, v_head;   // 16-byte vectors between rows of a head / between heads
     uint4* out_K;
     uint4* out_V;
     int32_t* out_idx;
@@ -410,15 +411,15 @@ layer_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const int rows_per_pass = (kRThreads / vpr) * kGatherRowsPerThread;
         for (int n0 = r_begin; n0 < r_end; n0 += rows_per_pass) {
             if (vpr == 16)
-                gather_rows<16, false>(a.K + static_cast<size_t>(hkv) * a.L * 16, a.V + static_cast<size_t>(hkv) * a.L * 16,
+                gather_rows<16, false>(a.K + static_cast<size_t>(hkv) * a.k_head, a.V + static_cast<size_t>(hkv) * a.v_head,
                                        sidx, a.L, r_end, n0, threadIdx.x, kRThreads,
                                        a.out_K + static_cast<size_t>(hkv) * a.n_max * 16,
-                                       a.out_V + static_cast<size_t>(hkv) * a.n_max * 16, nullptr);
+                                       a.out_V + static_cast<size_t>(hkv) * a.n_max * 16, nullptr, a.k_row, a.v_row);
             else
-                gather_rows<8, false>(a.K + static_cast<size_t>(hkv) * a.L * 8, a.V + static_cast<size_t>(hkv) * a.L * 8,
+                gather_rows<8, false>(a.K + static_cast<size_t>(hkv) * a.k_head, a.V + static_cast<size_t>(hkv) * a.v_head,
                                       sidx, a.L, r_end, n0, threadIdx.x, kRThreads,
                                       a.out_K + static_cast<size_t>(hkv) * a.n_max * 8,
-                                      a.out_V + static_cast<size_t>(hkv) * a.n_max * 8, nullptr);
+                                      a.out_V + static_cast<size_t>(hkv) * a.n_max * 8, nullptr, a.k_row, a.v_row);
         }
     }
     // tensor memory has not been read since the barrier after the contraction (or after scoring)
@@ -489,6 +490,13 @@ cudaError_t launch_layer_resident(const ResidentPlan& plan, const CUtensorMap& t
     a.C = io.C; a.k = io.k; a.n_max = io.n_max; a.Hkv = io.Hs >> io.kv_shift;
     a.off_ring = plan.off_ring; a.ring_bytes = plan.ring_bytes; a.off_pmax = plan.off_pmax; a.off_misc = plan.off_misc;
     a.K = static_cast<const uint4*>(io.K); a.V = static_cast<const uint4*>(io.V);
+    {
+        const long long vpr = io.d / 8;
+        a.k_row = io.k_row_elems ? io.k_row_elems / 8 : vpr;
+        a.v_row = io.v_row_elems ? io.v_row_elems / 8 : vpr;
+        a.k_head = io.k_head_elems ? io.k_head_elems / 8 : static_cast<long long>(io.L) * vpr;
+        a.v_head = io.v_head_elems ? io.v_head_elems / 8 : static_cast<long long>(io.L) * vpr;
+    }
     a.out_K = static_cast<uint4*>(io.out_K); a.out_V = static_cast<uint4*>(io.out_V); a.out_idx = io.out_idx;
     a.cta_stat = io.scratch;
     a.scores = io.scratch + static_cast<size_t>(plan.grid) * 256;
