@@ -495,6 +495,60 @@ def run_ours(args, wl):
             note="32 chunkkv_compress_layer calls with c = 1 on the 32 distinct layers, back to back, as a graph (the way "
                  "single_layer is timed); us_eager = the same calls issued directly")
         del o1, g_token
+
+        # ---- the adapters either side of the path and Algorithm 1's budget rule, on the same layers
+        #      (one call at a time, issued directly; the bindings' output allocations are outside the loop)
+        ad = {}
+        oA = alloc_outs(ck, wl, 1, dev)[0]
+        qi, Ki, Vi = layers[0]
+        tmK = Ki.permute(1, 0, 2).contiguous()                  # a token-major cache [L, Hkv, d]
+        tmV = Vi.permute(1, 0, 2).contiguous()
+        vK, vV = tmK.permute(1, 0, 2), tmV.permute(1, 0, 2)
+
+        def strided_layer():
+            ck.compress_layer_strided(qi, vK, vV, wl.Hq, wl.w, wl.c, wl.budget, out_K=oA[0], out_V=oA[1], out_idx=oA[2],
+                                      stream=stream)
+
+        page = 16
+        n_blk = (n_max + page - 1) // page
+        table = torch.randperm(n_blk, device=dev).to(torch.int32)
+        cK = torch.empty((n_blk, page, wl.Hkv, wl.d), dtype=torch.bfloat16, device=dev)
+        cV = torch.empty_like(cK)
+
+        def paged_layer():
+            ck.compress_layer_paged(qi, Ki, Vi, wl.Hq, wl.w, wl.c, wl.budget, table, cK, cV, out_idx=oA[2], stream=stream)
+
+        n1 = ck.out_len_alg1(wl.L, wl.w, wl.c, wl.budget)
+        o1a = (torch.empty((wl.Hkv, n1, wl.d), dtype=torch.bfloat16, device=dev),
+               torch.empty((wl.Hkv, n1, wl.d), dtype=torch.bfloat16, device=dev),
+               torch.empty((wl.Hkv, n1), dtype=torch.int32, device=dev))
+
+        def alg1_layer():
+            ck.compress_layer_alg1(qi, Ki, Vi, wl.Hq, wl.w, wl.c, wl.budget, out_K=o1a[0], out_V=o1a[1], out_idx=o1a[2],
+                                   stream=stream)
+
+        T = 4 * wl.w
+        row = (wl.Hq + 2 * wl.Hkv) * wl.d
+        qkv = torch.randn((T, row), device=dev).to(torch.bfloat16)
+        ang = torch.rand((wl.w, wl.d // 2), device=dev) * 6.28
+        cos_r, sin_r = torch.cos(ang), torch.sin(ang)
+
+        def window_q():
+            ck.window_queries(qkv, wl.Hq, wl.Hkv, wl.d, wl.w, cos_r, sin_r, stream=stream)
+
+        with torch.cuda.stream(stream):
+            for name, fn, nb in (("compress_layer_strided", strided_layer, nbytes["layer"]),
+                                 ("compress_layer_paged", paged_layer, nbytes["layer"]),
+                                 ("compress_layer_alg1", alg1_layer, nbytes["layer"]),
+                                 ("window_queries", window_q, None)):
+                us_a = time_calls(fn)
+                ad[name] = {"us": us_a} if nb is None else frac_row(nb, us_a)
+        ad["note"] = ("cfg2 layer: keys and values read from a token-major cache [L, Hkv, d]; kept rows written to a paged cache "
+                      "(16 tokens per page, shuffled block table); Algorithm 1's budget rule; the last w rows of a fused QKV "
+                      "activation rotated into q_obs (includes the binding's output allocation)")
+        extra_roof["adapters"] = ad
+        del tmK, tmV, cK, cV, o1a, qkv
+        check_status()
         check_status()
 
     del g_model, g_shared, g_reuse2, g_single, g_reuse, model, model_shared, model_reuse2
