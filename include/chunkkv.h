@@ -191,7 +191,8 @@ CHUNKKV_API int chunkkv_compress_layer(const void* q_obs, const void* K, const v
  *
  * chunkkv_compress_layer_paged: chunkkv_compress_layer (or, with reuse_idx, a layer that reuses
  *   indices) writing the kept rows to a paged cache instead of dense out_K / out_V; out_idx
- *   [Hkv, n_max] is still written. Runs as separate score / select / gather launches.
+ *   [Hkv, n_max] is still written. The one-launch layer kernel places the rows through the block table
+ *   where the shape fits it; otherwise separate score / select / gather launches.
  *
  * chunkkv_compress_layer_strided: chunkkv_compress_layer (or, with reuse_idx, a layer that reuses
  *   indices) on keys and values that are not packed [Hkv, L, d]: row l of head h of K starts at

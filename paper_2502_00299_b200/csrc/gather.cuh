@@ -31,6 +31,14 @@ __device__ __forceinline__ void gather_st(uint4* p, const uint4& v) {
                  : "memory");
 }
 
+// Destination rows in a paged cache [num_pages, page_size, Hkv, d]: compacted position n of head h goes to
+// page block_table[n / page_size], slot n % page_size; pages outside [0, num_pages) are skipped.
+// block_table == nullptr: packed outputs.
+struct PagedDst {
+    const int32_t* block_table;
+    int page_size, num_pages, Hkv, h;
+};
+
 // Work item `item` of `n_items` (a CTA-sized slab of rows of one head); threads = nthreads
 // (a multiple of VPR). VPR = 16-byte vectors per row: 8 (d = 64) or 16 (d = 128).
 // FRESH_IDX: the indices were written earlier in the same kernel launch, so they must not be
@@ -40,7 +48,8 @@ template <int VPR, bool FRESH_IDX>
 __device__ __forceinline__ void gather_rows(const uint4* __restrict__ Kh, const uint4* __restrict__ Vh,
                                             const int32_t* ih, int L, int n_max, int n0, int tid, int nthreads,
                                             uint4* __restrict__ oK, uint4* __restrict__ oV, int32_t* idx_copy,
-                                            long long k_row_vecs = VPR, long long v_row_vecs = VPR) {
+                                            long long k_row_vecs = VPR, long long v_row_vecs = VPR,
+                                            PagedDst pg = PagedDst{nullptr, 0, 0, 0, 0}) {
     const int rows_per_pass = nthreads / VPR;
     const int vec = tid % VPR, sub = tid / VPR;
     const unsigned long long policy = gather_policy();
@@ -62,8 +71,17 @@ __device__ __forceinline__ void gather_rows(const uint4* __restrict__ Kh, const 
     for (int u = 0; u < kGatherRowsPerThread; ++u) {
         const int n = n0 + u * rows_per_pass + sub;
         if (n < n_max) {
-            gather_st(oK + static_cast<size_t>(n) * VPR + vec, kv[u]);
-            gather_st(oV + static_cast<size_t>(n) * VPR + vec, vv[u]);
+            if (pg.block_table == nullptr) {
+                gather_st(oK + static_cast<size_t>(n) * VPR + vec, kv[u]);
+                gather_st(oV + static_cast<size_t>(n) * VPR + vec, vv[u]);
+            } else {                                    // (oK / oV are the bases of the paged caches)
+                const int page = pg.block_table[n / pg.page_size];
+                if (static_cast<unsigned>(page) < static_cast<unsigned>(pg.num_pages)) {
+                    const size_t row = (static_cast<size_t>(page) * pg.page_size + n % pg.page_size) * pg.Hkv + pg.h;
+                    gather_st(oK + row * VPR + vec, kv[u]);
+                    gather_st(oV + row * VPR + vec, vv[u]);
+                }
+            }
             if (idx_copy != nullptr && vec == 0) idx_copy[n] = src[u];
         }
     }

@@ -105,6 +105,9 @@ struct ResidentIO {
     bool cooperative;     // cooperative launch (lanes: several launches share the GPU) instead of a programmatic dependent one
     // elements between consecutive rows of a head and between heads of K and of V; 0 = packed [Hkv, L, d]
     long long k_row_elems = 0, k_head_elems = 0, v_row_elems = 0, v_head_elems = 0;
+    // out_K / out_V are paged caches [num_pages, page_size, Hkv, d] addressed through this block table (else packed)
+    const int32_t* block_table = nullptr;
+    int page_size = 0, num_pages = 0;
 };
 
 // false when the shape does not fit this kernel (chunk size other than 10 / 20, more than 128 rows

@@ -62,6 +62,8 @@ struct ResArgs {
     const uint4* K;
     const uint4* V;
     long long k_row, k_head, v_row, v_head;   // 16-byte vectors between rows of a head / between heads
+    const int32_t* block_table;              // non-null: out_K / out_V are paged caches
+    int page_size, num_pages;
     uint4* out_K;
     uint4* out_V;
     int32_t* out_idx;
@@ -409,17 +411,18 @@ layer_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const int r_end = static_cast<int>(static_cast<long long>(a.n_max) * (q + 1) / Q);
         const int vpr = a.d >> 3;
         const int rows_per_pass = (kRThreads / vpr) * kGatherRowsPerThread;
+        // packed outputs: this head's block; paged outputs: the cache base (rows are placed through the block table)
+        const PagedDst pg{a.block_table, a.page_size, a.num_pages, a.Hkv, hkv};
+        const size_t head_out = a.block_table ? 0 : static_cast<size_t>(hkv) * a.n_max;
         for (int n0 = r_begin; n0 < r_end; n0 += rows_per_pass) {
             if (vpr == 16)
                 gather_rows<16, false>(a.K + static_cast<size_t>(hkv) * a.k_head, a.V + static_cast<size_t>(hkv) * a.v_head,
-                                       sidx, a.L, r_end, n0, threadIdx.x, kRThreads,
-                                       a.out_K + static_cast<size_t>(hkv) * a.n_max * 16,
-                                       a.out_V + static_cast<size_t>(hkv) * a.n_max * 16, nullptr, a.k_row, a.v_row);
+                                       sidx, a.L, r_end, n0, threadIdx.x, kRThreads, a.out_K + head_out * 16,
+                                       a.out_V + head_out * 16, nullptr, a.k_row, a.v_row, pg);
             else
                 gather_rows<8, false>(a.K + static_cast<size_t>(hkv) * a.k_head, a.V + static_cast<size_t>(hkv) * a.v_head,
-                                      sidx, a.L, r_end, n0, threadIdx.x, kRThreads,
-                                      a.out_K + static_cast<size_t>(hkv) * a.n_max * 8,
-                                      a.out_V + static_cast<size_t>(hkv) * a.n_max * 8, nullptr, a.k_row, a.v_row);
+                                      sidx, a.L, r_end, n0, threadIdx.x, kRThreads, a.out_K + head_out * 8,
+                                      a.out_V + head_out * 8, nullptr, a.k_row, a.v_row, pg);
         }
     }
     // tensor memory has not been read since the barrier after the contraction (or after scoring)
@@ -490,6 +493,7 @@ cudaError_t launch_layer_resident(const ResidentPlan& plan, const CUtensorMap& t
     a.C = io.C; a.k = io.k; a.n_max = io.n_max; a.Hkv = io.Hs >> io.kv_shift;
     a.off_ring = plan.off_ring; a.ring_bytes = plan.ring_bytes; a.off_pmax = plan.off_pmax; a.off_misc = plan.off_misc;
     a.K = static_cast<const uint4*>(io.K); a.V = static_cast<const uint4*>(io.V);
+    a.block_table = io.block_table; a.page_size = io.page_size; a.num_pages = io.num_pages;
     {
         const long long vpr = io.d / 8;
         a.k_row = io.k_row_elems ? io.k_row_elems / 8 : vpr;
