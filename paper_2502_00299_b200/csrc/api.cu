@@ -1041,6 +1041,34 @@ int chunkkv_compress_layer_alg1(const void* q_obs, const void* K, const void* V,
     st = get_ctx(&ctx);
     if (st != CHUNKKV_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (C > 0 && k > 0) {
+        // the one-launch layer kernel with Algorithm 1's chunk count and token cap
+        const ScoreShape sh = score_shape(Hq, Hkv, w);
+        ResidentPlan rplan;
+        if (make_resident_plan(L, sh.Rs, sh.Hs, sh.shift, d, c, C, n_max, ctx->num_sms, smem_budget(*ctx), &rplan)) {
+            st = ensure_workspace(*ctx, resident_scratch_floats(rplan, sh.Hs, C) * sizeof(float));
+            if (st != CHUNKKV_OK) return st;
+            char* base = static_cast<char*>(ctx->ws);
+            CUtensorMap tm_q, tm_k;
+            st = encode_bf16_3d(&tm_q, q_obs, d, sh.Rs, sh.Hs, sh.Rs < 128 ? sh.Rs : 128, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
+            if (st != CHUNKKV_OK) return st;
+            st = encode_bf16_3d(&tm_k, K, d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+            if (st != CHUNKKV_OK) return st;
+            ResidentIO io;
+            io.L = L; io.w = w; io.Rs = sh.Rs; io.Hs = sh.Hs; io.d = d; io.kv_shift = sh.shift;
+            io.sl2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(d)));
+            io.C = C; io.k = k; io.n_max = n_max;
+            io.K = K; io.V = V; io.out_K = out_K; io.out_V = out_V; io.out_idx = out_idx;
+            io.scratch = reinterpret_cast<float*>(base + kHeaderBytes);
+            io.counters = reinterpret_cast<unsigned*>(base + kResidentCountersOffset);
+            io.status = reinterpret_cast<int*>(base);
+            io.cooperative = false;
+            io.tok_cap = budget - w;
+            cudaError_t e2 = launch_layer_resident(rplan, tm_q, tm_k, io, s);
+            if (e2 != cudaSuccess) return cuda_fail(e2);
+            return CHUNKKV_OK;
+        }
+    }
     float* chunk_scores = nullptr;
     if (C > 0 && k > 0) {
         st = run_score(*ctx, q_obs, K, L, Hq, Hkv, d, w, c, nullptr, round64(static_cast<size_t>(Hkv) * C), &chunk_scores, s);

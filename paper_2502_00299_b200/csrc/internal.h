@@ -108,6 +108,8 @@ struct ResidentIO {
     // out_K / out_V are paged caches [num_pages, page_size, Hkv, d] addressed through this block table (else packed)
     const int32_t* block_table = nullptr;
     int page_size = 0, num_pages = 0;
+    // Algorithm 1's budget rule: at most this many tokens of the kept chunks are emitted (lowest positions first)
+    int tok_cap = 0x7fffffff;
 };
 
 // false when the shape does not fit this kernel (chunk size other than 10 / 20, more than 128 rows

@@ -64,6 +64,7 @@ struct ResArgs {
     long long k_row, k_head, v_row, v_head;   // 16-byte vectors between rows of a head / between heads
     const int32_t* block_table;              // non-null: out_K / out_V are paged caches
     int page_size, num_pages;
+    int tok_cap;                             // Algorithm 1: tokens of the kept chunks that are emitted
     uint4* out_K;
     uint4* out_V;
     int32_t* out_idx;
@@ -391,13 +392,13 @@ layer_resident_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
         const float* sc = a.scores + (static_cast<size_t>(hkv) << a.kv_shift) * a.C;
         const float* sc2 = a.kv_shift ? sc + a.C : nullptr;
         if (a.C <= kRThreads * 6) {
-            select_head_regs<6>(sc, sc2, a.L, a.w, C_STATIC, a.C, a.k, a.n_max, sidx, ss);
+            select_head_regs<6>(sc, sc2, a.L, a.w, C_STATIC, a.C, a.k, a.n_max, sidx, ss, a.tok_cap);
         } else {
             const size_t idx_bytes = (static_cast<size_t>(a.n_max) * 4 + 127) & ~size_t(127);
             uint32_t* kbuf = reinterpret_cast<uint32_t*>(ring + kSelBytes + idx_bytes);
             const bool fits = kSelBytes + idx_bytes + static_cast<size_t>(a.C) * 4 <= static_cast<size_t>(a.ring_bytes);
             if (fits)
-                select_head_smem(sc, sc2, a.L, a.w, C_STATIC, a.C, a.k, a.n_max, sidx, ss, kbuf);
+                select_head_smem(sc, sc2, a.L, a.w, C_STATIC, a.C, a.k, a.n_max, sidx, ss, kbuf, a.tok_cap);
             else
                 select_head_rows(sc, sc2, a.L, a.w, C_STATIC, a.C, a.k, a.n_max, sidx, ss, nullptr);
         }
@@ -494,6 +495,7 @@ cudaError_t launch_layer_resident(const ResidentPlan& plan, const CUtensorMap& t
     a.off_ring = plan.off_ring; a.ring_bytes = plan.ring_bytes; a.off_pmax = plan.off_pmax; a.off_misc = plan.off_misc;
     a.K = static_cast<const uint4*>(io.K); a.V = static_cast<const uint4*>(io.V);
     a.block_table = io.block_table; a.page_size = io.page_size; a.num_pages = io.num_pages;
+    a.tok_cap = io.tok_cap;
     {
         const long long vpr = io.d / 8;
         a.k_row = io.k_row_elems ? io.k_row_elems / 8 : vpr;
