@@ -243,6 +243,20 @@ CHUNKKV_API int chunkkv_compress_model(int n_layers, const void* const* q_obs, c
                                        int32_t* const* out_idx, void* stream);
 
 /*
+ * chunkkv_compress_model on keys and values that are not packed [Hkv, L, d] (the same strides, in bf16
+ * elements, for every layer: see chunkkv_compress_layer_strided; a token-major cache [L, Hkv, d] has
+ * token stride Hkv * d and head stride d). Outputs are packed. The persistent kernel scores through
+ * tensor maps with those strides and copies the kept rows one row at a time; shapes it does not take
+ * run layer by layer. No counterpart in the paper: it is Algorithm 2 on another memory layout.
+ */
+CHUNKKV_API int chunkkv_compress_model_strided(int n_layers, const void* const* q_obs, const void* const* K,
+                                               const void* const* V, int L, int Hq, int Hkv, int d, int w, int c,
+                                               int budget, int reuse_depth, long long k_token_stride,
+                                               long long k_head_stride, long long v_token_stride,
+                                               long long v_head_stride, void* const* out_K, void* const* out_V,
+                                               int32_t* const* out_idx, void* stream);
+
+/*
  * Algorithm 1's budget rule, as an alternative to Algorithm 3's (which the calls above follow):
  * k = floor(L_max / c) chunks are selected (at most the C that exist), their tokens are taken in
  * ascending order and cut to the first L_max - w ("K'[0 : L_max - w]"), and the observe window

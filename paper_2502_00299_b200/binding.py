@@ -48,6 +48,8 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_compress_layer.argtypes = [vp, vp, vp] + [i32] * 7 + [vp, vp, vp, vp, vp]
     L.chunkkv_model_workspace_bytes.restype = sz
     L.chunkkv_model_workspace_bytes.argtypes = [i32] * 9
+    L.chunkkv_compress_model_strided.restype = i32
+    L.chunkkv_compress_model_strided.argtypes = [i32, vp, vp, vp] + [i32] * 8 + [ctypes.c_longlong] * 4 + [vp, vp, vp, vp]
     L.chunkkv_compress_model.restype = i32
     L.chunkkv_compress_model.argtypes = [i32, vp, vp, vp] + [i32] * 8 + [vp, vp, vp, vp]
     L.chunkkv_window_queries.restype = i32
@@ -567,6 +569,44 @@ def compress_model(layers: Sequence[Tuple[Optional[torch.Tensor], torch.Tensor, 
     oia = arr(*[o[2].data_ptr() for o in outs])
     _check(lib.chunkkv_compress_model(n, qa, ka, va, L, Hq, Hkv, d, w, c, budget, n_reuse, oka, ova, oia,
                                       _stream(stream)), "chunkkv_compress_model")
+    return [tuple(o) for o in outs]
+
+
+def compress_model_strided(layers: Sequence[Tuple[Optional[torch.Tensor], torch.Tensor, torch.Tensor]], Hq: int, w: int,
+                           c: int, budget: int, n_reuse: int = 1,
+                           stream: Optional[torch.cuda.Stream] = None,
+                           outs: Optional[Sequence[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]]] = None,
+                           ) -> List[Tuple[torch.Tensor, torch.Tensor, torch.Tensor]]:
+    """compress_model on K / V given as [Hkv, L, d] views that share one set of token and head strides
+    (last dimension contiguous), e.g. ``cache.permute(1, 0, 2)`` of token-major caches [L, Hkv, d]."""
+    n = len(layers)
+    K0, V0 = layers[0][1], layers[0][2]
+    Hkv, L, d = K0.shape
+    ks, vs = (K0.stride(1), K0.stride(0)), (V0.stride(1), V0.stride(0))
+    for q, K, V in layers:
+        for t, name, st in ((K, "K", ks), (V, "V", vs)):
+            if not (t.is_cuda and t.dtype == torch.bfloat16 and tuple(t.shape) == (Hkv, L, d) and t.stride(2) == 1
+                    and (t.stride(1), t.stride(0)) == st):
+                raise ValueError(f"{name}: CUDA bf16 [Hkv, L, d] views with the same strides in every layer are required")
+        if q is not None:
+            _dev(q, torch.bfloat16, "q_obs")
+    n_max = out_len(L, w, c, budget)
+    dev = K0.device
+    if outs is None:
+        outs = [(torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev),
+                 torch.empty((Hkv, n_max, d), dtype=torch.bfloat16, device=dev),
+                 torch.empty((Hkv, n_max), dtype=torch.int32, device=dev)) for _ in range(n)]
+    _ensure_bytes(max(int(lib.chunkkv_model_workspace_bytes(n, L, Hq, Hkv, d, w, c, budget, n_reuse)),
+                      workspace_bytes(L, Hq, Hkv, d, w, c)))
+    arr = ctypes.c_void_p * n
+    qa = arr(*[None if t[0] is None else t[0].data_ptr() for t in layers])
+    ka = arr(*[t[1].data_ptr() for t in layers])
+    va = arr(*[t[2].data_ptr() for t in layers])
+    oka = arr(*[o[0].data_ptr() for o in outs])
+    ova = arr(*[o[1].data_ptr() for o in outs])
+    oia = arr(*[o[2].data_ptr() for o in outs])
+    _check(lib.chunkkv_compress_model_strided(n, qa, ka, va, L, Hq, Hkv, d, w, c, budget, n_reuse, ks[0], ks[1], vs[0], vs[1],
+                                              oka, ova, oia, _stream(stream)), "chunkkv_compress_model_strided")
     return [tuple(o) for o in outs]
 
 

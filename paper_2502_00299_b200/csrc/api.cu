@@ -863,9 +863,12 @@ size_t chunkkv_model_workspace_bytes(int n_layers, int L, int Hq, int Hkv, int d
     return need;
 }
 
-int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* const* K, const void* const* V,
-                           int L, int Hq, int Hkv, int d, int w, int c, int budget, int reuse_depth,
-                           void* const* out_K, void* const* out_V, int32_t* const* out_idx, void* stream) {
+// kt / kh / vt / vh: elements between consecutive rows of a head and between heads of K and of V; 0 = packed
+static int compress_model_impl(int n_layers, const void* const* q_obs, const void* const* K, const void* const* V,
+                               int L, int Hq, int Hkv, int d, int w, int c, int budget, int reuse_depth,
+                               void* const* out_K, void* const* out_V, int32_t* const* out_idx, void* stream,
+                               long long kt, long long kh, long long vt, long long vh) {
+    const bool strided = kt != 0;
     int st = model_args_ok(n_layers, reuse_depth);
     if (st != CHUNKKV_OK) return st;
     st = check_sizes(L, w, c, budget);
@@ -903,7 +906,12 @@ int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* c
         // layer by layer: Algorithm 2's call sequence over chunkkv_compress_layer
         for (int l = 0; l < n_layers; ++l) {
             const int src = (l / reuse_depth) * reuse_depth;
-            st = chunkkv_compress_layer(l == src ? q_obs[l] : nullptr, K[l], V[l], L, Hq, Hkv, d, w, c, budget,
+            if (strided)
+                st = chunkkv_compress_layer_strided(l == src ? q_obs[l] : nullptr, K[l], V[l], L, Hq, Hkv, d, w, c, budget, kt, kh,
+                                                    vt, vh, l == src ? nullptr : out_idx[src], out_K[l], out_V[l], out_idx[l],
+                                                    stream);
+            else
+                st = chunkkv_compress_layer(l == src ? q_obs[l] : nullptr, K[l], V[l], L, Hq, Hkv, d, w, c, budget,
                                         l == src ? nullptr : out_idx[src], out_K[l], out_V[l], out_idx[l], stream);
             if (st != CHUNKKV_OK) return st;
         }
@@ -942,7 +950,7 @@ int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* c
                 st = encode_bf16_3d(&tm_q[nc], q_obs[l], d, sh.Rs, sh.Hs, sh.Rs < 128 ? sh.Rs : 128,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
                 if (st != CHUNKKV_OK) return st;
-                st = encode_bf16_3d(&tm_k[nc], K[l], d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+                st = encode_bf16_3d(&tm_k[nc], K[l], d, L, Hkv, L < 120 ? L : 120, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, kt, kh);
                 if (st != CHUNKKV_OK) return st;
                 ++nc;
             }
@@ -953,8 +961,10 @@ int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* c
             int i = 0;
             for (; i < n && !lay[i].computes; ++i) {
                 const int l = l0 + i, src = (l / reuse_depth) * reuse_depth;
-                cudaError_t e = launch_gather(K[l], V[l], out_idx[src], L, Hkv, d, n_max, out_K[l], out_V[l], out_idx[l],
-                                              ctx->num_sms, s);
+                cudaError_t e = strided ? launch_gather_strided(K[l], V[l], out_idx[src], L, Hkv, d, n_max, kt, kh, vt, vh, out_K[l],
+                                                                out_V[l], out_idx[l], ctx->num_sms, s)
+                                        : launch_gather(K[l], V[l], out_idx[src], L, Hkv, d, n_max, out_K[l], out_V[l], out_idx[l],
+                                                        ctx->num_sms, s);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
             l0 += i;
@@ -967,6 +977,7 @@ int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* c
         io.scratch = reinterpret_cast<float*>(base + kHeaderBytes);
         io.counters = reinterpret_cast<unsigned*>(base + kResidentCountersOffset);
         io.status = reinterpret_cast<int*>(base);
+        io.k_row_elems = kt; io.k_head_elems = kh; io.v_row_elems = vt; io.v_head_elems = vh;
         cudaError_t e;
         {
             Timer t(ctx, s, 0);
@@ -976,6 +987,29 @@ int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* c
         l0 = l1;
     }
     return CHUNKKV_OK;
+}
+
+int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* const* K, const void* const* V,
+                           int L, int Hq, int Hkv, int d, int w, int c, int budget, int reuse_depth,
+                           void* const* out_K, void* const* out_V, int32_t* const* out_idx, void* stream) {
+    return compress_model_impl(n_layers, q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_depth, out_K, out_V, out_idx, stream,
+                               0, 0, 0, 0);
+}
+
+int chunkkv_compress_model_strided(int n_layers, const void* const* q_obs, const void* const* K, const void* const* V,
+                                   int L, int Hq, int Hkv, int d, int w, int c, int budget, int reuse_depth,
+                                   long long k_token_stride, long long k_head_stride, long long v_token_stride,
+                                   long long v_head_stride, void* const* out_K, void* const* out_V,
+                                   int32_t* const* out_idx, void* stream) {
+    if (k_token_stride == d && v_token_stride == d && k_head_stride == static_cast<long long>(L) * d &&
+        v_head_stride == static_cast<long long>(L) * d)
+        return chunkkv_compress_model(n_layers, q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_depth, out_K, out_V, out_idx,
+                                      stream);
+    const long long strides[4] = {k_token_stride, k_head_stride, v_token_stride, v_head_stride};
+    for (long long sdv : strides)
+        if (sdv < d || (sdv & 7) != 0) return CHUNKKV_EINVAL_SHAPE;
+    return compress_model_impl(n_layers, q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_depth, out_K, out_V, out_idx, stream,
+                               k_token_stride, k_head_stride, v_token_stride, v_head_stride);
 }
 
 // ---- Algorithm 1's budget rule: k = floor(L_max / c) chunks, their tokens cut to the first

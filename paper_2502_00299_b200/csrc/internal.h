@@ -139,6 +139,8 @@ struct ModelIO {
     float* scratch;       // model_scratch_floats() floats
     unsigned* counters;   // header + kResidentCountersOffset
     int* status;
+    // elements between consecutive rows of a head and between heads of K and of V (all layers); 0 = packed
+    long long k_row_elems = 0, k_head_elems = 0, v_row_elems = 0, v_head_elems = 0;
 };
 
 struct ModelLayerIO {

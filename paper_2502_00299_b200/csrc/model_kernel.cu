@@ -101,6 +101,8 @@ struct ModelParams {
     int sel_row_bytes;     // bytes of one kept-chunk list: 4 header ints + the kept chunk ids, padded to 16 bytes
     int sel_keys_fit;      // selector: the keys of a head fit its shared memory (many chunks per thread)
     int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes;
+    // bytes between consecutive rows of a head and between heads of K and of V (packed: d * 2 and L * d * 2)
+    long long k_row_bytes, k_head_bytes, v_row_bytes, v_head_bytes;
     float* cta_stat;       // [2 (slot parity)][grid][{max, sum}][128]
     float* scores;         // [n_compute][Hs][Cpad]
     unsigned* cnt_a;       // [Hs]
@@ -259,7 +261,9 @@ __device__ __forceinline__ bool selector_loop(const ModelParams& p, uint8_t* dyn
     return true;
 }
 
-template <int C_STATIC>
+// STRIDED: the rows of a head are not adjacent in memory (e.g. token-major caches): the copy thread moves
+// kept rows one at a time. A variant of its own, so that the packed kernel's code is exactly what it was.
+template <int C_STATIC, bool STRIDED>
 __global__ void __launch_bounds__(kMThreads, 1)
 model_kernel(const __grid_constant__ ModelParams p) {
     constexpr int SPP = kRPanel / C_STATIC;
@@ -629,8 +633,9 @@ model_kernel(const __grid_constant__ ModelParams p) {
         // One thread: waits until the selector CTA has published the head's kept-chunk list of a
         // slot, fetches the list, and moves this CTA's share of the rows - whole chunks and window
         // pieces - through the staging slots with bulk copies, for the computed layer and for every
-        // layer that reuses its indices.
-        if (lane == 0) {
+        // layer that reuses its indices. (Strided variant: the whole warp runs this loop in step - lane 0 waits,
+        // stores and keeps the books, every lane issues the copy of one source row.)
+        if (STRIDED || lane == 0) {
             uint8_t* tbase = dyn + p.off_tail;
             int* row = reinterpret_cast<int*>(tbase);        // [4 + kkpad]: n_tok, -, -, -, kept chunk ids
             const uint32_t stage0 = smem_u32(tbase + p.sel_row_bytes);
@@ -649,19 +654,23 @@ model_kernel(const __grid_constant__ ModelParams p) {
             bool ok = true;
             for (int li = 0; li < p.n_layers && ok;) {
                 const int s = p.layer[li].slot;
-                ok = wait_counter(p.cnt_c + hkv, static_cast<unsigned>(s + 1), abort_flag, 200);
-                if (!ok) break;
-                asm volatile("fence.acq_rel.gpu;" ::: "memory");
-                {
-                    const uint32_t bar = smem_u32(&ctl.sfull);
-                    mbar_arrive_expect_tx(bar, static_cast<uint32_t>(p.sel_row_bytes));
-                    // the list was written with ordinary stores by the selector CTA
-                    asm volatile("fence.proxy.async.global;" ::: "memory");
-                    bulk_load(smem_u32(row), p.sel_rows + (static_cast<size_t>(s) * p.Hkv + hkv) * (p.sel_row_bytes / 4),
-                              static_cast<uint32_t>(p.sel_row_bytes), bar);
-                    ok = mbar_wait(bar, static_cast<uint32_t>(s) & 1u, abort_flag);
-                    if (!ok) break;
+                if (lane == 0) {
+                    ok = wait_counter(p.cnt_c + hkv, static_cast<unsigned>(s + 1), abort_flag, 200);
+                    if (ok) {
+                        asm volatile("fence.acq_rel.gpu;" ::: "memory");
+                        const uint32_t bar = smem_u32(&ctl.sfull);
+                        mbar_arrive_expect_tx(bar, static_cast<uint32_t>(p.sel_row_bytes));
+                        // the list was written with ordinary stores by the selector CTA
+                        asm volatile("fence.proxy.async.global;" ::: "memory");
+                        bulk_load(smem_u32(row), p.sel_rows + (static_cast<size_t>(s) * p.Hkv + hkv) * (p.sel_row_bytes / 4),
+                                  static_cast<uint32_t>(p.sel_row_bytes), bar);
+                    }
                 }
+                if constexpr (STRIDED) ok = __shfl_sync(0xffffffffu, ok, 0);
+                // (every lane that reads the list waits for it itself)
+                if (ok) ok = mbar_wait(smem_u32(&ctl.sfull), static_cast<uint32_t>(s) & 1u, abort_flag);
+                if constexpr (STRIDED) ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
                 const int n_tok = row[0];
                 auto unit = [&](int u, int& src_row, int& dst_row, int& rows) {
                     if (u < kk) {
@@ -678,8 +687,10 @@ model_kernel(const __grid_constant__ ModelParams p) {
                 int lj = li;
                 do {
                     const ModelLayer& ly = p.layer[lj];
-                    const char* Kh = reinterpret_cast<const char*>(ly.K) + static_cast<size_t>(hkv) * p.L * row_bytes;
-                    const char* Vh = reinterpret_cast<const char*>(ly.V) + static_cast<size_t>(hkv) * p.L * row_bytes;
+                    const char* Kh = reinterpret_cast<const char*>(ly.K) +
+                                     (STRIDED ? static_cast<size_t>(hkv) * p.k_head_bytes : static_cast<size_t>(hkv) * p.L * row_bytes);
+                    const char* Vh = reinterpret_cast<const char*>(ly.V) +
+                                     (STRIDED ? static_cast<size_t>(hkv) * p.v_head_bytes : static_cast<size_t>(hkv) * p.L * row_bytes);
                     char* oK = reinterpret_cast<char*>(ly.out_K) + static_cast<size_t>(hkv) * p.n_max * row_bytes;
                     char* oV = reinterpret_cast<char*>(ly.out_V) + static_cast<size_t>(hkv) * p.n_max * row_bytes;
                     int loaded = 0;
@@ -689,38 +700,54 @@ model_kernel(const __grid_constant__ ModelParams p) {
                         const uint32_t slot = (g_issued + idx) % kMSlots;
                         const uint32_t bytes = static_cast<uint32_t>(rows) * row_bytes;
                         const uint32_t bar = smem_u32(&ctl.gfull[slot]);
-                        mbar_arrive_expect_tx(bar, 2u * bytes);
-                        bulk_load(stage0 + slot * p.stage_slot_bytes, Kh + static_cast<size_t>(sr) * row_bytes, bytes, bar);
-                        bulk_load(stage0 + slot * p.stage_slot_bytes + half_slot, Vh + static_cast<size_t>(sr) * row_bytes, bytes, bar);
+                        if (lane == 0) mbar_arrive_expect_tx(bar, 2u * bytes);
+                        if constexpr (!STRIDED) {
+                            bulk_load(stage0 + slot * p.stage_slot_bytes, Kh + static_cast<size_t>(sr) * row_bytes, bytes, bar);
+                            bulk_load(stage0 + slot * p.stage_slot_bytes + half_slot, Vh + static_cast<size_t>(sr) * row_bytes, bytes, bar);
+                        } else {
+                            // rows of a chunk are not adjacent in memory (e.g. a token-major cache): lane r copies row r
+                            __syncwarp();             // the byte count is on the barrier before any copy can complete
+                            if (lane < rows) {
+                                bulk_load(stage0 + slot * p.stage_slot_bytes + static_cast<uint32_t>(lane) * row_bytes,
+                                          Kh + static_cast<size_t>(sr + lane) * p.k_row_bytes, row_bytes, bar);
+                                bulk_load(stage0 + slot * p.stage_slot_bytes + half_slot + static_cast<uint32_t>(lane) * row_bytes,
+                                          Vh + static_cast<size_t>(sr + lane) * p.v_row_bytes, row_bytes, bar);
+                            }
+                        }
                     };
                     // loads run kMSlots - 1 units ahead of the stores
                     for (; loaded < n_units && loaded < kMSlots - 1; ++loaded) issue_load(loaded);
                     for (int idx = 0; idx < n_units && ok; ++idx) {
                         const uint32_t gi = g_issued + idx;
                         const uint32_t slot = gi % kMSlots;
-                        ok = mbar_wait(smem_u32(&ctl.gfull[slot]), (gi / kMSlots) & 1u, abort_flag);
+                        if (lane == 0) ok = mbar_wait(smem_u32(&ctl.gfull[slot]), (gi / kMSlots) & 1u, abort_flag);
+                        if constexpr (STRIDED) ok = __shfl_sync(0xffffffffu, ok, 0);
                         if (!ok) break;
                         int sr, dr, rows;
                         unit(u_begin + idx, sr, dr, rows);
                         const uint32_t bytes = static_cast<uint32_t>(rows) * row_bytes;
-                        bulk_store(oK + static_cast<size_t>(dr) * row_bytes, stage0 + slot * p.stage_slot_bytes, bytes);
-                        bulk_store(oV + static_cast<size_t>(dr) * row_bytes, stage0 + slot * p.stage_slot_bytes + half_slot, bytes);
-                        bulk_commit();
+                        if (lane == 0) {
+                            bulk_store(oK + static_cast<size_t>(dr) * row_bytes, stage0 + slot * p.stage_slot_bytes, bytes);
+                            bulk_store(oV + static_cast<size_t>(dr) * row_bytes, stage0 + slot * p.stage_slot_bytes + half_slot, bytes);
+                            bulk_commit();
+                        }
                         if (loaded < n_units) {
                             // the slot the next load takes was stored one unit ago: all but the newest group have been read
-                            bulk_wait_read<1>();
+                            if (lane == 0) bulk_wait_read<1>();
+                            if constexpr (STRIDED) __syncwarp();
                             issue_load(loaded);
                             ++loaded;
                         }
                     }
-                    bulk_wait_read<0>();          // the slots are reused by the next layer's first loads
+                    if (lane == 0) bulk_wait_read<0>();          // the slots are reused by the next layer's first loads
+                    if constexpr (STRIDED) __syncwarp();
                     g_issued += static_cast<uint32_t>(n_units);
                     ++lj;
                 } while (ok && lj < p.n_layers && !p.layer[lj].computes);
                 li = lj;
             }
-            bulk_wait_all();
-            if (!ok) ctl.abort_flag = 1;
+            if (lane == 0) bulk_wait_all();
+            if (!ok && lane == 0) ctl.abort_flag = 1;
         }
     }
 
@@ -820,6 +847,10 @@ cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtenso
     p.n_compute = n_compute;
     p.L = io.L; p.P = io.L - io.w; p.w = io.w; p.R = io.Rs; p.Hs = io.Hs; p.d = io.d; p.kv_shift = io.kv_shift;
     p.sl2 = io.sl2;
+    p.k_row_bytes = 2 * (io.k_row_elems ? io.k_row_elems : io.d);
+    p.v_row_bytes = 2 * (io.v_row_elems ? io.v_row_elems : io.d);
+    p.k_head_bytes = 2 * (io.k_head_elems ? io.k_head_elems : static_cast<long long>(io.L) * io.d);
+    p.v_head_bytes = 2 * (io.v_head_elems ? io.v_head_elems : static_cast<long long>(io.L) * io.d);
     p.cph = plan.cph; p.n_tiles = plan.n_tiles; p.n_stages = plan.n_stages;
     p.q_box_rows = io.Rs < 128 ? io.Rs : 128;
     p.k_box_rows = io.L < kRTile ? io.L : kRTile;
@@ -837,12 +868,14 @@ cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtenso
     p.cnt_b = io.counters + 16 + kResidentMaxHeads;
     p.cnt_c = io.counters + 16 + 2 * kResidentMaxHeads;
     p.status = io.status;
-    const void* kern = plan.c_static == 10 ? reinterpret_cast<const void*>(model_kernel<10>)
-                                           : reinterpret_cast<const void*>(model_kernel<20>);
-    static int smem_set[2][64] = {{0}};
+    const bool strided = io.k_row_elems != 0 || io.v_row_elems != 0 || io.k_head_elems != 0 || io.v_head_elems != 0;
+    const void* kern = plan.c_static == 10
+                           ? (strided ? reinterpret_cast<const void*>(model_kernel<10, true>) : reinterpret_cast<const void*>(model_kernel<10, false>))
+                           : (strided ? reinterpret_cast<const void*>(model_kernel<20, true>) : reinterpret_cast<const void*>(model_kernel<20, false>));
+    static int smem_set[4][64] = {{0}};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
-    const int v = plan.c_static == 10 ? 0 : 1;
+    const int v = (plan.c_static == 10 ? 0 : 1) + (strided ? 2 : 0);
     if (e == cudaSuccess && (dev < 0 || dev >= 64 || smem_set[v][dev] < plan.smem_bytes)) {
         e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, plan.smem_bytes);
         if (e == cudaSuccess && dev >= 0 && dev < 64) smem_set[v][dev] = plan.smem_bytes;

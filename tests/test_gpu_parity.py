@@ -815,3 +815,35 @@ def test_strided_inputs_refused_when_rows_overlap_or_are_misaligned(ck):
                                                    wl.c, 64, *strides, None, oK.data_ptr(), oK.data_ptr(), oI.data_ptr(), None)
         assert st == -2
 
+
+
+
+@pytest.mark.parametrize("cfg,L,budget,n_layers,n_reuse,pad", [(2, 6000, 600, 5, 2, 0), (1, 2048, 256, 3, 1, 16),
+                                                                (5, 5000, 500, 4, 3, 0), (2, 32768, 3276, 4, 2, 0)])
+def test_model_call_on_token_major_caches_matches_packed_call(ck, cfg, L, budget, n_layers, n_reuse, pad):
+    # chunkkv_compress_model_strided on token-major caches [L, Hkv, d (+ padding)]: the persistent kernel scores
+    # through strided tensor maps and copies kept rows one by one; results equal the packed call's bit for
+    # bit (same kernel, same arithmetic), and the first layer is checked against the oracle
+    wl = scaled(CONFIGS[cfg], L=L, budget=budget)
+    xs = [make_layer(wl, layer=i) for i in range(n_layers)]
+    packed = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in xs]
+
+    def token_major(t):
+        buf = torch.zeros((L, wl.Hkv, wl.d + pad), dtype=torch.bfloat16, device="cuda")
+        buf[:, :, :wl.d] = t.permute(1, 0, 2)
+        return buf[:, :, :wl.d].permute(1, 0, 2)
+
+    views = [(q, token_major(K), token_major(V)) for q, K, V in packed]
+    n_max = ck.out_len(L, wl.w, wl.c, budget)
+    guards = [guarded_outputs(wl.Hkv, n_max, wl.d) for _ in range(n_layers)]
+    outs = ck.compress_model_strided(views, wl.Hq, wl.w, wl.c, budget, n_reuse=n_reuse,
+                                     outs=[(g[0].t, g[1].t, g[2].t) for g in guards])
+    _status_ok(ck)
+    for g in guards:
+        for t, name in zip(g, ("out_K", "out_V", "out_idx")):
+            t.check(name)
+    ref = ck.compress_model(packed, wl.Hq, wl.w, wl.c, budget, n_reuse=n_reuse)
+    _status_ok(ck)
+    for (oK, oV, oI), (rK, rV, rI) in zip(outs, ref):
+        assert torch.equal(oI, rI) and torch.equal(oK, rK) and torch.equal(oV, rV)
+    _check_layer(xs[0], wl, bits_of(outs[0][0]), bits_of(outs[0][1]), outs[0][2].cpu().numpy(), budget=budget)
