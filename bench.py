@@ -543,9 +543,17 @@ def run_ours(args, wl):
                                  ("window_queries", window_q, None)):
                 us_a = time_calls(fn)
                 ad[name] = {"us": us_a} if nb is None else frac_row(nb, us_a)
+            tm8 = []
+            for q8, K8, V8 in layers[:8]:
+                tm8.append((q8, K8.permute(1, 0, 2).contiguous().permute(1, 0, 2), V8.permute(1, 0, 2).contiguous().permute(1, 0, 2)))
+            us_m = time_calls(lambda: ck.compress_model_strided(tm8, wl.Hq, wl.w, wl.c, wl.budget, n_reuse=1, outs=outs[:8],
+                                                                stream=stream), n=10) / 8
+            ad["compress_model_strided"] = frac_row(nbytes["layer"], us_m, layers_per_call=8)
+            del tm8
         ad["note"] = ("cfg2 layer: keys and values read from a token-major cache [L, Hkv, d]; kept rows written to a paged cache "
                       "(16 tokens per page, shuffled block table); Algorithm 1's budget rule; the last w rows of a fused QKV "
-                      "activation rotated into q_obs (includes the binding's output allocation)")
+                      "activation rotated into q_obs (includes the binding's output allocation); compress_model_strided: 8 token-major "
+                      "layers per call, us per layer")
         extra_roof["adapters"] = ad
         del tmK, tmV, cK, cV, o1a, qkv
         check_status()
