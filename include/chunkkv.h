@@ -257,6 +257,19 @@ CHUNKKV_API int chunkkv_compress_model_strided(int n_layers, const void* const* 
                                                int32_t* const* out_idx, void* stream);
 
 /*
+ * chunkkv_compress_model writing every layer's kept rows into that layer's paged decode cache
+ * (cache_K[l] / cache_V[l] [num_pages, page_size, Hkv, d] through block_tables[l], as in
+ * chunkkv_gather_paged; one page_size and num_pages for all layers); out_idx[l] [Hkv, n_max] is still
+ * written. The persistent kernel places the rows itself (one row per lane of its copy warp); shapes it
+ * does not take run layer by layer through chunkkv_compress_layer_paged.
+ */
+CHUNKKV_API int chunkkv_compress_model_paged(int n_layers, const void* const* q_obs, const void* const* K,
+                                             const void* const* V, int L, int Hq, int Hkv, int d, int w, int c,
+                                             int budget, int reuse_depth, const int32_t* const* block_tables,
+                                             int page_size, int num_pages, void* const* cache_K, void* const* cache_V,
+                                             int32_t* const* out_idx, void* stream);
+
+/*
  * Algorithm 1's budget rule, as an alternative to Algorithm 3's (which the calls above follow):
  * k = floor(L_max / c) chunks are selected (at most the C that exist), their tokens are taken in
  * ascending order and cut to the first L_max - w ("K'[0 : L_max - w]"), and the observe window

@@ -8,7 +8,7 @@ so that the build module itself can be imported before the library exists.
 """
 _EXPORTS = (
     "ChunkKVError", "LIB_PATH", "Lane", "Pipe", "budget_from_ratio", "compress_layer", "compress_layer_alg1",
-    "compress_layer_host", "compress_layer_paged", "compress_layer_strided", "compress_model", "compress_model_strided", "gather_paged", "window_queries", "out_len_alg1", "select_alg1",
+    "compress_layer_host", "compress_layer_paged", "compress_layer_strided", "compress_model", "compress_model_paged", "compress_model_strided", "gather_paged", "window_queries", "out_len_alg1", "select_alg1",
     "device_status", "ensure_workspace", "gather", "jaccard", "lib", "num_chunks", "num_kept_chunks", "out_len", "profile_enable",
     "profile_read", "score", "select", "set_workspace", "strerror", "workspace_bytes",
 )

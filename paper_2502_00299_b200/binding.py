@@ -50,6 +50,8 @@ def _load() -> ctypes.CDLL:
     L.chunkkv_model_workspace_bytes.argtypes = [i32] * 9
     L.chunkkv_compress_model_strided.restype = i32
     L.chunkkv_compress_model_strided.argtypes = [i32, vp, vp, vp] + [i32] * 8 + [ctypes.c_longlong] * 4 + [vp, vp, vp, vp]
+    L.chunkkv_compress_model_paged.restype = i32
+    L.chunkkv_compress_model_paged.argtypes = [i32, vp, vp, vp] + [i32] * 8 + [vp, i32, i32, vp, vp, vp, vp]
     L.chunkkv_compress_model.restype = i32
     L.chunkkv_compress_model.argtypes = [i32, vp, vp, vp] + [i32] * 8 + [vp, vp, vp, vp]
     L.chunkkv_window_queries.restype = i32
@@ -608,6 +610,43 @@ def compress_model_strided(layers: Sequence[Tuple[Optional[torch.Tensor], torch.
     _check(lib.chunkkv_compress_model_strided(n, qa, ka, va, L, Hq, Hkv, d, w, c, budget, n_reuse, ks[0], ks[1], vs[0], vs[1],
                                               oka, ova, oia, _stream(stream)), "chunkkv_compress_model_strided")
     return [tuple(o) for o in outs]
+
+
+def compress_model_paged(layers: Sequence[Tuple[Optional[torch.Tensor], torch.Tensor, torch.Tensor]], Hq: int, w: int,
+                         c: int, budget: int, block_tables: Sequence[torch.Tensor], caches: Sequence[Tuple[torch.Tensor, torch.Tensor]],
+                         n_reuse: int = 1, stream: Optional[torch.cuda.Stream] = None,
+                         out_idx: Optional[Sequence[torch.Tensor]] = None) -> List[torch.Tensor]:
+    """compress_model with every layer's kept rows written to that layer's paged cache
+    (caches[l] = (cache_K, cache_V) [num_pages, page_size, Hkv, d], block_tables[l] int32); returns the
+    layers' idx [Hkv, n_max]."""
+    n = len(layers)
+    Hkv, L, d = layers[0][1].shape
+    for q, K, V in layers:
+        _dev(K, torch.bfloat16, "K"); _dev(V, torch.bfloat16, "V")
+        if q is not None:
+            _dev(q, torch.bfloat16, "q_obs")
+    page_size, num_pages = caches[0][0].shape[1], caches[0][0].shape[0]
+    for (cK, cV), bt in zip(caches, block_tables):
+        _dev(cK, torch.bfloat16, "cache_K"); _dev(cV, torch.bfloat16, "cache_V"); _dev(bt, torch.int32, "block_table")
+        if cK.shape[0] != num_pages or cK.shape[1] != page_size:
+            raise ValueError("all layers' caches must share page_size and num_pages")
+    n_max = out_len(L, w, c, budget)
+    dev = layers[0][1].device
+    if out_idx is None:
+        out_idx = [torch.empty((Hkv, n_max), dtype=torch.int32, device=dev) for _ in range(n)]
+    _ensure_bytes(max(int(lib.chunkkv_model_workspace_bytes(n, L, Hq, Hkv, d, w, c, budget, n_reuse)),
+                      workspace_bytes(L, Hq, Hkv, d, w, c)))
+    arr = ctypes.c_void_p * n
+    qa = arr(*[None if t[0] is None else t[0].data_ptr() for t in layers])
+    ka = arr(*[t[1].data_ptr() for t in layers])
+    va = arr(*[t[2].data_ptr() for t in layers])
+    bta = arr(*[t.data_ptr() for t in block_tables])
+    cka = arr(*[t[0].data_ptr() for t in caches])
+    cva = arr(*[t[1].data_ptr() for t in caches])
+    oia = arr(*[t.data_ptr() for t in out_idx])
+    _check(lib.chunkkv_compress_model_paged(n, qa, ka, va, L, Hq, Hkv, d, w, c, budget, n_reuse, bta, page_size, num_pages,
+                                            cka, cva, oia, _stream(stream)), "chunkkv_compress_model_paged")
+    return list(out_idx)
 
 
 def profile_enable(on: bool) -> None:

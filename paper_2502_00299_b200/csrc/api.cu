@@ -867,8 +867,10 @@ size_t chunkkv_model_workspace_bytes(int n_layers, int L, int Hq, int Hkv, int d
 static int compress_model_impl(int n_layers, const void* const* q_obs, const void* const* K, const void* const* V,
                                int L, int Hq, int Hkv, int d, int w, int c, int budget, int reuse_depth,
                                void* const* out_K, void* const* out_V, int32_t* const* out_idx, void* stream,
-                               long long kt, long long kh, long long vt, long long vh) {
+                               long long kt, long long kh, long long vt, long long vh,
+                               const int32_t* const* block_tables = nullptr, int page_size = 0, int num_pages = 0) {
     const bool strided = kt != 0;
+    const bool paged = page_size > 0;      // out_K / out_V are then the layers' paged caches
     int st = model_args_ok(n_layers, reuse_depth);
     if (st != CHUNKKV_OK) return st;
     st = check_sizes(L, w, c, budget);
@@ -906,7 +908,11 @@ static int compress_model_impl(int n_layers, const void* const* q_obs, const voi
         // layer by layer: Algorithm 2's call sequence over chunkkv_compress_layer
         for (int l = 0; l < n_layers; ++l) {
             const int src = (l / reuse_depth) * reuse_depth;
-            if (strided)
+            if (paged)
+                st = chunkkv_compress_layer_paged(l == src ? q_obs[l] : nullptr, K[l], V[l], L, Hq, Hkv, d, w, c, budget,
+                                                  l == src ? nullptr : out_idx[src], block_tables[l], page_size, num_pages,
+                                                  out_K[l], out_V[l], out_idx[l], stream);
+            else if (strided)
                 st = chunkkv_compress_layer_strided(l == src ? q_obs[l] : nullptr, K[l], V[l], L, Hq, Hkv, d, w, c, budget, kt, kh,
                                                     vt, vh, l == src ? nullptr : out_idx[src], out_K[l], out_V[l], out_idx[l],
                                                     stream);
@@ -946,6 +952,7 @@ static int compress_model_impl(int n_layers, const void* const* q_obs, const voi
             const bool computes = (l % reuse_depth) == 0;
             lay[i].K = K[l]; lay[i].V = V[l]; lay[i].out_K = out_K[l]; lay[i].out_V = out_V[l]; lay[i].out_idx = out_idx[l];
             lay[i].computes = computes;
+            lay[i].block_table = paged ? block_tables[l] : nullptr;
             if (computes) {
                 st = encode_bf16_3d(&tm_q[nc], q_obs[l], d, sh.Rs, sh.Hs, sh.Rs < 128 ? sh.Rs : 128,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
@@ -961,11 +968,18 @@ static int compress_model_impl(int n_layers, const void* const* q_obs, const voi
             int i = 0;
             for (; i < n && !lay[i].computes; ++i) {
                 const int l = l0 + i, src = (l / reuse_depth) * reuse_depth;
-                cudaError_t e = strided ? launch_gather_strided(K[l], V[l], out_idx[src], L, Hkv, d, n_max, kt, kh, vt, vh, out_K[l],
+                cudaError_t e = paged   ? launch_gather_paged(K[l], V[l], out_idx[src], L, Hkv, d, n_max, block_tables[l], page_size,
+                                                              num_pages, out_K[l], out_V[l], ctx->num_sms, s)
+                                : strided ? launch_gather_strided(K[l], V[l], out_idx[src], L, Hkv, d, n_max, kt, kh, vt, vh, out_K[l],
                                                                 out_V[l], out_idx[l], ctx->num_sms, s)
                                         : launch_gather(K[l], V[l], out_idx[src], L, Hkv, d, n_max, out_K[l], out_V[l], out_idx[l],
                                                         ctx->num_sms, s);
                 if (e != cudaSuccess) return cuda_fail(e);
+                if (paged && out_idx[l] != out_idx[src]) {      // (the paged gather does not copy the indices)
+                    e = cudaMemcpyAsync(out_idx[l], out_idx[src], static_cast<size_t>(Hkv) * n_max * sizeof(int32_t),
+                                        cudaMemcpyDeviceToDevice, s);
+                    if (e != cudaSuccess) return cuda_fail(e);
+                }
             }
             l0 += i;
             continue;
@@ -978,6 +992,7 @@ static int compress_model_impl(int n_layers, const void* const* q_obs, const voi
         io.counters = reinterpret_cast<unsigned*>(base + kResidentCountersOffset);
         io.status = reinterpret_cast<int*>(base);
         io.k_row_elems = kt; io.k_head_elems = kh; io.v_row_elems = vt; io.v_head_elems = vh;
+        io.page_size = page_size; io.num_pages = num_pages;
         cudaError_t e;
         {
             Timer t(ctx, s, 0);
@@ -994,6 +1009,25 @@ int chunkkv_compress_model(int n_layers, const void* const* q_obs, const void* c
                            void* const* out_K, void* const* out_V, int32_t* const* out_idx, void* stream) {
     return compress_model_impl(n_layers, q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_depth, out_K, out_V, out_idx, stream,
                                0, 0, 0, 0);
+}
+
+int chunkkv_compress_model_paged(int n_layers, const void* const* q_obs, const void* const* K, const void* const* V,
+                                 int L, int Hq, int Hkv, int d, int w, int c, int budget, int reuse_depth,
+                                 const int32_t* const* block_tables, int page_size, int num_pages, void* const* cache_K,
+                                 void* const* cache_V, int32_t* const* out_idx, void* stream) {
+    int st = model_args_ok(n_layers, reuse_depth);
+    if (st != CHUNKKV_OK) return st;
+    st = check_sizes(L, w, c, budget);
+    if (st != CHUNKKV_OK) return st;
+    if (block_tables == nullptr || cache_K == nullptr || cache_V == nullptr) return CHUNKKV_EINVAL_NULL;
+    const int n_max = chunkkv_out_len(L, w, c, budget);
+    if (n_max < 0) return n_max;
+    for (int l = 0; l < n_layers; ++l) {
+        st = check_paged(n_max, page_size, num_pages, block_tables[l], cache_K[l], cache_V[l]);
+        if (st != CHUNKKV_OK) return st;
+    }
+    return compress_model_impl(n_layers, q_obs, K, V, L, Hq, Hkv, d, w, c, budget, reuse_depth, cache_K, cache_V, out_idx, stream,
+                               0, 0, 0, 0, block_tables, page_size, num_pages);
 }
 
 int chunkkv_compress_model_strided(int n_layers, const void* const* q_obs, const void* const* K, const void* const* V,

@@ -847,3 +847,43 @@ def test_model_call_on_token_major_caches_matches_packed_call(ck, cfg, L, budget
     for (oK, oV, oI), (rK, rV, rI) in zip(outs, ref):
         assert torch.equal(oI, rI) and torch.equal(oK, rK) and torch.equal(oV, rV)
     _check_layer(xs[0], wl, bits_of(outs[0][0]), bits_of(outs[0][1]), outs[0][2].cpu().numpy(), budget=budget)
+
+
+@pytest.mark.parametrize("cfg,L,budget,n_layers,n_reuse,page", [(2, 6000, 600, 5, 2, 16), (1, 2048, 256, 3, 1, 7),
+                                                                 (2, 2595 + 32, 5000, 3, 2, 16), (5, 5000, 500, 4, 3, 32),
+                                                                 (2, 32768, 3276, 3, 1, 16)])
+def test_model_call_into_paged_caches_matches_oracle(ck, cfg, L, budget, n_layers, n_reuse, page):
+    # chunkkv_compress_model_paged: every layer's kept rows go to that layer's paged cache through its own
+    # (shuffled) block table, inside the persistent kernel; indices equal the dense call's, cache contents
+    # equal the oracle's paged gather, untouched pages and the margins keep their fill pattern. The third
+    # case keeps a clipped last chunk: zero rows behind the kept rows are placed through the table too.
+    wl = scaled(CONFIGS[cfg], L=L, budget=budget)
+    xs = [make_layer(wl, layer=i) for i in range(n_layers)]
+    dev = [(to_dev(x.q_obs), to_dev(x.K), to_dev(x.V)) for x in xs]
+    n_max = ck.out_len(L, wl.w, wl.c, budget)
+    n_blk = (n_max + page - 1) // page
+    n_pages = n_blk + 3
+    rng = np.random.default_rng(L + page)
+    tables = [rng.permutation(n_pages).astype(np.int32)[:n_blk].copy() for _ in range(n_layers)]
+    caches = []
+    for _ in range(n_layers):
+        cK, cV = Guarded((n_pages, page, wl.Hkv, wl.d), torch.bfloat16), Guarded((n_pages, page, wl.Hkv, wl.d), torch.bfloat16)
+        cK.t.view(torch.int16).fill_(0x1111)
+        cV.t.view(torch.int16).fill_(0x2222)
+        caches.append((cK, cV))
+    idxs = ck.compress_model_paged(dev, wl.Hq, wl.w, wl.c, budget, [torch.from_numpy(t).cuda() for t in tables],
+                                   [(a.t, b.t) for a, b in caches], n_reuse=n_reuse)
+    _status_ok(ck)
+    ref = ck.compress_model(dev, wl.Hq, wl.w, wl.c, budget, n_reuse=n_reuse)
+    for l, x in enumerate(xs):
+        idx_np = idxs[l].cpu().numpy()
+        assert np.array_equal(idx_np, ref[l][2].cpu().numpy())
+        caches[l][0].check("cache_K")
+        caches[l][1].check("cache_V")
+        refK = np.full((n_pages, page, wl.Hkv, wl.d), 0x1111, dtype=np.uint16)
+        refV = np.full((n_pages, page, wl.Hkv, wl.d), 0x2222, dtype=np.uint16)
+        ora.gather_paged(x.K, x.V, idx_np, tables[l], page, refK, refV)
+        assert np.array_equal(bits_of(caches[l][0].t), refK) and np.array_equal(bits_of(caches[l][1].t), refV)
+    s0 = ora.chunk_scores(ora.token_scores(xs[0].q_obs, xs[0].K, wl.Hq, wl.Hkv, wl.w), wl.c)
+    assert_selection_matches(idxs[0].cpu().numpy(), s0, L, wl.w, wl.c, budget)
+
