@@ -550,10 +550,17 @@ def run_ours(args, wl):
                                                                 stream=stream), n=10) / 8
             ad["compress_model_strided"] = frac_row(nbytes["layer"], us_m, layers_per_call=8)
             del tm8
+            tabs8 = [torch.randperm(n_blk, device=dev).to(torch.int32) for _ in range(8)]
+            caches8 = [(torch.empty_like(cK), torch.empty_like(cV)) for _ in range(8)]
+            idx8 = [o[2] for o in outs[:8]]
+            us_p = time_calls(lambda: ck.compress_model_paged(layers[:8], wl.Hq, wl.w, wl.c, wl.budget, tabs8, caches8, n_reuse=1,
+                                                              stream=stream, out_idx=idx8), n=10) / 8
+            ad["compress_model_paged"] = frac_row(nbytes["layer"], us_p, layers_per_call=8)
+            del caches8
         ad["note"] = ("cfg2 layer: keys and values read from a token-major cache [L, Hkv, d]; kept rows written to a paged cache "
                       "(16 tokens per page, shuffled block table); Algorithm 1's budget rule; the last w rows of a fused QKV "
-                      "activation rotated into q_obs (includes the binding's output allocation); compress_model_strided: 8 token-major "
-                      "layers per call, us per layer")
+                      "activation rotated into q_obs (includes the binding's output allocation); compress_model_strided / _paged: 8 layers "
+                      "per call (token-major inputs / paged outputs), us per layer")
         extra_roof["adapters"] = ad
         del tmK, tmV, cK, cV, o1a, qkv
         check_status()

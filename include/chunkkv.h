@@ -260,8 +260,8 @@ CHUNKKV_API int chunkkv_compress_model_strided(int n_layers, const void* const* 
  * chunkkv_compress_model writing every layer's kept rows into that layer's paged decode cache
  * (cache_K[l] / cache_V[l] [num_pages, page_size, Hkv, d] through block_tables[l], as in
  * chunkkv_gather_paged; one page_size and num_pages for all layers); out_idx[l] [Hkv, n_max] is still
- * written. The persistent kernel places the rows itself (one row per lane of its copy warp); shapes it
- * does not take run layer by layer through chunkkv_compress_layer_paged.
+ * written. Runs layer by layer through chunkkv_compress_layer_paged (the one-launch layer kernel places
+ * the rows through the block table with all its threads), in Algorithm 2's order.
  */
 CHUNKKV_API int chunkkv_compress_model_paged(int n_layers, const void* const* q_obs, const void* const* K,
                                              const void* const* V, int L, int Hq, int Hkv, int d, int w, int c,

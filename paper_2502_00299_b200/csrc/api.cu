@@ -901,7 +901,9 @@ static int compress_model_impl(int n_layers, const void* const* q_obs, const voi
         std::lock_guard<std::mutex> lk(g_mu);
         st = get_ctx(&ctx);
         if (st != CHUNKKV_OK) return st;
-        persistent = C > 0 && k > 0 &&
+        // paged outputs run layer by layer: the one-launch layer kernel places rows through the block table with all
+        // its threads, which measured faster (35 us per layer) than the persistent kernel's copy warp doing it (41 us)
+        persistent = !paged && C > 0 && k > 0 &&
                      make_model_plan(L, sh.Rs, sh.Hs, sh.shift, d, c, C, k, ctx->num_sms, smem_budget(*ctx), &mp);
     }
     if (!persistent) {
@@ -952,7 +954,6 @@ static int compress_model_impl(int n_layers, const void* const* q_obs, const voi
             const bool computes = (l % reuse_depth) == 0;
             lay[i].K = K[l]; lay[i].V = V[l]; lay[i].out_K = out_K[l]; lay[i].out_V = out_V[l]; lay[i].out_idx = out_idx[l];
             lay[i].computes = computes;
-            lay[i].block_table = paged ? block_tables[l] : nullptr;
             if (computes) {
                 st = encode_bf16_3d(&tm_q[nc], q_obs[l], d, sh.Rs, sh.Hs, sh.Rs < 128 ? sh.Rs : 128,
                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
@@ -992,7 +993,6 @@ static int compress_model_impl(int n_layers, const void* const* q_obs, const voi
         io.counters = reinterpret_cast<unsigned*>(base + kResidentCountersOffset);
         io.status = reinterpret_cast<int*>(base);
         io.k_row_elems = kt; io.k_head_elems = kh; io.v_row_elems = vt; io.v_head_elems = vh;
-        io.page_size = page_size; io.num_pages = num_pages;
         cudaError_t e;
         {
             Timer t(ctx, s, 0);

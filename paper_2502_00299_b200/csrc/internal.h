@@ -141,8 +141,6 @@ struct ModelIO {
     int* status;
     // elements between consecutive rows of a head and between heads of K and of V (all layers); 0 = packed
     long long k_row_elems = 0, k_head_elems = 0, v_row_elems = 0, v_head_elems = 0;
-    // > 0: out_K / out_V of every layer are paged caches [num_pages, page_size, Hkv, d]
-    int page_size = 0, num_pages = 0;
 };
 
 struct ModelLayerIO {
@@ -152,7 +150,6 @@ struct ModelLayerIO {
     void* out_V;
     int32_t* out_idx;
     bool computes;        // false: gather with the indices of the nearest computed layer before it
-    const int32_t* block_table = nullptr;   // paged outputs (ModelIO::page_size > 0): this layer's block table
 };
 
 bool make_model_plan(int L, int Rs, int Hs, int kv_shift, int d, int c, int C, int k, int max_ctas, int smem_limit,

@@ -83,7 +83,6 @@ struct ModelLayer {
     uint4* out_K;
     uint4* out_V;
     int32_t* out_idx;
-    const int32_t* block_table;   // paged outputs: this layer's block table
     int slot;          // computed layer: its slot (0 .. n_compute - 1); reuse layer: the slot of its source layer
     int computes;      // 1: scored and selected here; 0: gathered with the slot's indices
 };
@@ -104,7 +103,6 @@ struct ModelParams {
     int off_ring, off_pmax, off_misc, off_tail, stage_slot_bytes;
     // bytes between consecutive rows of a head and between heads of K and of V (packed: d * 2 and L * d * 2)
     long long k_row_bytes, k_head_bytes, v_row_bytes, v_head_bytes;
-    int page_size, num_pages;   // > 0: outputs are paged caches [num_pages, page_size, Hkv, d] (strided variant only)
     float* cta_stat;       // [2 (slot parity)][grid][{max, sum}][128]
     float* scores;         // [n_compute][Hs][Cpad]
     unsigned* cnt_a;       // [Hs]
@@ -247,22 +245,10 @@ __device__ __forceinline__ bool selector_loop(const ModelParams& p, uint8_t* dyn
                 const ModelLayer& ly = p.layer[lj];
                 int32_t* dst = ly.out_idx + static_cast<size_t>(hkv) * p.n_max;
                 for (int n = threadIdx.x; n < p.n_max; n += kMThreads) dst[n] = sidx[n];
+                uint4* zk = ly.out_K + (static_cast<size_t>(hkv) * p.n_max + n_tok + p.w) * vpr;
+                uint4* zv = ly.out_V + (static_cast<size_t>(hkv) * p.n_max + n_tok + p.w) * vpr;
                 const int nz = (p.n_max - n_tok - p.w) * vpr;
-                if (p.page_size == 0) {
-                    uint4* zk = ly.out_K + (static_cast<size_t>(hkv) * p.n_max + n_tok + p.w) * vpr;
-                    uint4* zv = ly.out_V + (static_cast<size_t>(hkv) * p.n_max + n_tok + p.w) * vpr;
-                    for (int i = threadIdx.x; i < nz; i += kMThreads) { zk[i] = make_uint4(0, 0, 0, 0); zv[i] = make_uint4(0, 0, 0, 0); }
-                } else {
-                    for (int i = threadIdx.x; i < nz; i += kMThreads) {       // (a paged cache: through the block table)
-                        const int n = n_tok + p.w + i / vpr;
-                        const int page = ly.block_table[n / p.page_size];
-                        if (static_cast<unsigned>(page) < static_cast<unsigned>(p.num_pages)) {
-                            const size_t rowi = (static_cast<size_t>(page) * p.page_size + n % p.page_size) * p.Hkv + hkv;
-                            ly.out_K[rowi * vpr + i % vpr] = make_uint4(0, 0, 0, 0);
-                            ly.out_V[rowi * vpr + i % vpr] = make_uint4(0, 0, 0, 0);
-                        }
-                    }
-                }
+                for (int i = threadIdx.x; i < nz; i += kMThreads) { zk[i] = make_uint4(0, 0, 0, 0); zv[i] = make_uint4(0, 0, 0, 0); }
             }
             __syncthreads();
             if (threadIdx.x == 0) {
@@ -707,11 +693,6 @@ model_kernel(const __grid_constant__ ModelParams p) {
                                      (STRIDED ? static_cast<size_t>(hkv) * p.v_head_bytes : static_cast<size_t>(hkv) * p.L * row_bytes);
                     char* oK = reinterpret_cast<char*>(ly.out_K) + static_cast<size_t>(hkv) * p.n_max * row_bytes;
                     char* oV = reinterpret_cast<char*>(ly.out_V) + static_cast<size_t>(hkv) * p.n_max * row_bytes;
-                    if constexpr (STRIDED) {
-                        // the layer's block table (a few cache lines) on its way into L1 before the first store needs it
-                        if (p.page_size > 0 && lane * 32 * p.page_size < p.n_max)
-                            asm volatile("prefetch.global.L1 [%0];" ::"l"(ly.block_table + lane * 32));
-                    }
                     int loaded = 0;
                     auto issue_load = [&](int idx) {
                         int sr, dr, rows;
@@ -745,45 +726,27 @@ model_kernel(const __grid_constant__ ModelParams p) {
                         int sr, dr, rows;
                         unit(u_begin + idx, sr, dr, rows);
                         const uint32_t bytes = static_cast<uint32_t>(rows) * row_bytes;
-                        bool paged = false;
-                        if constexpr (STRIDED) paged = p.page_size > 0;
-                        if (paged) {
-                            // lane r places row r through the block table (bulk-copy groups belong to the issuing thread:
-                            // every lane commits and waits for its own)
-                            if (lane < rows) {
-                                const int n = dr + lane;
-                                const int page = __ldg(ly.block_table + n / p.page_size);
-                                if (static_cast<unsigned>(page) < static_cast<unsigned>(p.num_pages)) {
-                                    const size_t rowi = (static_cast<size_t>(page) * p.page_size + n % p.page_size) * p.Hkv + hkv;
-                                    bulk_store(reinterpret_cast<char*>(ly.out_K) + rowi * row_bytes,
-                                               stage0 + slot * p.stage_slot_bytes + static_cast<uint32_t>(lane) * row_bytes, row_bytes);
-                                    bulk_store(reinterpret_cast<char*>(ly.out_V) + rowi * row_bytes,
-                                               stage0 + slot * p.stage_slot_bytes + half_slot + static_cast<uint32_t>(lane) * row_bytes,
-                                               row_bytes);
-                                }
-                            }
-                            bulk_commit();
-                        } else if (lane == 0) {
+                        if (lane == 0) {
                             bulk_store(oK + static_cast<size_t>(dr) * row_bytes, stage0 + slot * p.stage_slot_bytes, bytes);
                             bulk_store(oV + static_cast<size_t>(dr) * row_bytes, stage0 + slot * p.stage_slot_bytes + half_slot, bytes);
                             bulk_commit();
                         }
                         if (loaded < n_units) {
                             // the slot the next load takes was stored one unit ago: all but the newest group have been read
-                            if (paged || lane == 0) bulk_wait_read<1>();
+                            if (lane == 0) bulk_wait_read<1>();
                             if constexpr (STRIDED) __syncwarp();
                             issue_load(loaded);
                             ++loaded;
                         }
                     }
-                    if (STRIDED || lane == 0) bulk_wait_read<0>();          // the slots are reused by the next layer's first loads
+                    if (lane == 0) bulk_wait_read<0>();          // the slots are reused by the next layer's first loads
                     if constexpr (STRIDED) __syncwarp();
                     g_issued += static_cast<uint32_t>(n_units);
                     ++lj;
                 } while (ok && lj < p.n_layers && !p.layer[lj].computes);
                 li = lj;
             }
-            if (STRIDED || lane == 0) bulk_wait_all();
+            if (lane == 0) bulk_wait_all();
             if (!ok && lane == 0) ctl.abort_flag = 1;
         }
     }
@@ -873,7 +836,6 @@ cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtenso
         ly.out_V = static_cast<uint4*>(layers[i].out_V);
         ly.out_idx = layers[i].out_idx;
         ly.computes = layers[i].computes ? 1 : 0;
-        ly.block_table = layers[i].block_table;
         if (ly.computes) {
             p.tm_q[n_compute] = tm_q[n_compute];
             p.tm_k[n_compute] = tm_k[n_compute];
@@ -885,7 +847,6 @@ cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtenso
     p.n_compute = n_compute;
     p.L = io.L; p.P = io.L - io.w; p.w = io.w; p.R = io.Rs; p.Hs = io.Hs; p.d = io.d; p.kv_shift = io.kv_shift;
     p.sl2 = io.sl2;
-    p.page_size = io.page_size; p.num_pages = io.num_pages;
     p.k_row_bytes = 2 * (io.k_row_elems ? io.k_row_elems : io.d);
     p.v_row_bytes = 2 * (io.v_row_elems ? io.v_row_elems : io.d);
     p.k_head_bytes = 2 * (io.k_head_elems ? io.k_head_elems : static_cast<long long>(io.L) * io.d);
@@ -907,8 +868,7 @@ cudaError_t launch_model(const ModelPlan& plan, const ModelIO& io, const CUtenso
     p.cnt_b = io.counters + 16 + kResidentMaxHeads;
     p.cnt_c = io.counters + 16 + 2 * kResidentMaxHeads;
     p.status = io.status;
-    const bool strided = io.k_row_elems != 0 || io.v_row_elems != 0 || io.k_head_elems != 0 || io.v_head_elems != 0 ||
-                         io.page_size > 0;      // (the variant whose copy warp moves rows one by one also places them in pages)
+    const bool strided = io.k_row_elems != 0 || io.v_row_elems != 0 || io.k_head_elems != 0 || io.v_head_elems != 0;
     const void* kern = plan.c_static == 10
                            ? (strided ? reinterpret_cast<const void*>(model_kernel<10, true>) : reinterpret_cast<const void*>(model_kernel<10, false>))
                            : (strided ? reinterpret_cast<const void*>(model_kernel<20, true>) : reinterpret_cast<const void*>(model_kernel<20, false>));

@@ -854,7 +854,7 @@ def test_model_call_on_token_major_caches_matches_packed_call(ck, cfg, L, budget
                                                                  (2, 32768, 3276, 3, 1, 16)])
 def test_model_call_into_paged_caches_matches_oracle(ck, cfg, L, budget, n_layers, n_reuse, page):
     # chunkkv_compress_model_paged: every layer's kept rows go to that layer's paged cache through its own
-    # (shuffled) block table, inside the persistent kernel; indices equal the dense call's, cache contents
+    # (shuffled) block table; indices equal the dense call's, cache contents
     # equal the oracle's paged gather, untouched pages and the margins keep their fill pattern. The third
     # case keeps a clipped last chunk: zero rows behind the kept rows are placed through the table too.
     wl = scaled(CONFIGS[cfg], L=L, budget=budget)
