@@ -41,7 +41,7 @@ SHARED_SETS = 4
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes per layer of the persistent kernel, from the ncu capture summarised under profiles/ (4 layers, cfg2)
-NCU_DRAM_BYTES_PER_LAYER = 337.7e6 / 4
+NCU_DRAM_BYTES_PER_LAYER = 338.2e6 / 4
 NCU_TRAFFIC_WORKLOAD = "cfg2_llama3_8b_32k"
 FALLBACK_BF16_SUSTAINED_TFLOPS = 1400.0
 
@@ -412,7 +412,7 @@ def run_ours(args, wl):
         "frac": achieved / peak, "frac_of_8TBps": achieved / NOMINAL_HBM_GBS,
         "traffic": NCU_DRAM_BYTES_PER_LAYER * NL if wl.name == NCU_TRAFFIC_WORKLOAD else None,
         "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one 4-layer launch of the same kernel on this "
-                          "workload (profiles/model_kernel_cfg2_4layers_ncu.txt: 337.7 MB), per layer x the 32 layers of a "
+                          "workload (profiles/model_kernel_cfg2_4layers_ncu.txt: 338.2 MB), per layer x the 32 layers of a "
                           "launch: every layer streams its own K once, so the traffic grows with the layers; the 32-layer "
                           "launch itself is too large for a counter capture",
         "algorithmic_bytes_per_launch": nbytes["layer"] * NL, "avg_launch_us": ms_per_step * 1e3,
